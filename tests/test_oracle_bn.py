@@ -1,0 +1,58 @@
+"""Pins for the oracle's BN fold and fused BN + binarize + re-pack (Section 2.1.1, last sentence)."""
+from decimal import Decimal, getcontext
+from fractions import Fraction
+
+import numpy as np
+
+
+def test_fold_matches_batchnorm_definition(oracle_mod):
+    """scale*x + shift equals gamma*(x-mean)/sqrt(var+eps)+beta, evaluated with 50-digit decimals."""
+    o = oracle_mod
+    getcontext().prec = 50
+    rng = np.random.default_rng(2)
+    O = 64
+    gamma = rng.uniform(0.5, 1.5, O).astype(np.float32)
+    gamma[:4] *= -1  # negative scales too
+    beta = rng.normal(0, 0.1, O).astype(np.float32)
+    mean = rng.normal(0, 0.1, O).astype(np.float32)
+    var = rng.uniform(0.5, 1.5, O).astype(np.float32)
+    scale, shift = o.bn_fold(gamma, beta, mean, var, 1e-5)
+    assert scale.dtype == np.float32 and shift.dtype == np.float32
+    eps = Decimal(1e-5)  # the double nearest to 1e-5, exactly
+    for i in range(O):
+        sd = Decimal(float(gamma[i])) / (Decimal(float(var[i])) + eps).sqrt()
+        sh = Decimal(float(beta[i])) - Decimal(float(mean[i])) * sd
+        # one rounding to fp32 each: relative error <= 2^-24 (plus the double rounding underneath)
+        assert abs(Decimal(float(scale[i])) - sd) <= abs(sd) * Decimal(2) ** -23
+        assert abs(Decimal(float(shift[i])) - sh) <= max(abs(sh), Decimal(1e-30)) * Decimal(2) ** -22
+        for x in (-576, -3, 0, 7, 4608):
+            bn = Decimal(float(gamma[i])) * (Decimal(x) - Decimal(float(mean[i]))) / (Decimal(float(var[i])) + eps).sqrt() + Decimal(float(beta[i]))
+            folded = Decimal(float(scale[i])) * Decimal(x) + Decimal(float(shift[i]))
+            assert abs(bn - folded) <= Decimal(1e-6) * (abs(bn) + 1)
+
+
+def test_sign_decision_is_the_sign_of_the_exact_value(oracle_mod):
+    """fmaf rounds the exact scale*acc+shift once, so y<0 iff the exact rational value is <0
+    (no underflow in this range).  Checked with exact fractions for every acc of a K=576 layer."""
+    o = oracle_mod
+    rng = np.random.default_rng(4)
+    O, K = 70, 576
+    scale = rng.normal(0, 0.05, O).astype(np.float32)
+    shift = rng.normal(0, 1.0, O).astype(np.float32)
+    scale[0], shift[0] = 0.0, -1.0   # constant negative
+    scale[1], shift[1] = 0.0, 2.0    # constant positive
+    scale[2], shift[2] = 0.5, -3.0   # exact zero at acc = 6 -> +1
+    scale[3], shift[3] = -0.25, 0.0  # exact zero at acc = 0 -> +1
+    accs = np.arange(-K, K + 1, 2, dtype=np.int32)
+    acc = np.repeat(accs[:, None], O, axis=1)  # [npix][O]
+    P = o.bn_sign_pack(acc, scale, shift)
+    assert P.shape == (len(accs), 2)
+    for ch in range(O):
+        fs, fb = Fraction(float(scale[ch])), Fraction(float(shift[ch]))
+        bits = (P[:, ch >> 6] >> np.uint64(ch & 63)) & np.uint64(1)
+        want = [1 if fs * int(a) + fb < 0 else 0 for a in accs]
+        assert bits.astype(int).tolist() == want, ch
+        # monotone in acc: at most one change of sign along the sorted acc values
+        assert int(np.count_nonzero(np.diff(bits.astype(int)))) <= 1
+    # tail bits of the last word are zero
+    assert not np.any(P[:, 1] >> np.uint64(O - 64))

@@ -1,0 +1,77 @@
+"""Pins for the oracle's binarize + pack (Section 2.1.1), independent of the oracle itself."""
+import numpy as np
+import pytest
+
+
+def unpack_words(P, C):
+    """uint64 [..., Cw] -> {0,1} array [..., C] by shifting, written here independently."""
+    Cw = P.shape[-1]
+    bits = np.zeros(P.shape[:-1] + (Cw * 64,), dtype=np.uint8)
+    for c in range(Cw * 64):
+        bits[..., c] = ((P[..., c >> 6] >> np.uint64(c & 63)) & np.uint64(1)).astype(np.uint8)
+    return bits[..., :C], bits[..., C:]
+
+
+def test_hand_vectors(oracle_mod):
+    o = oracle_mod
+    C = 130  # three words, tail of 2 valid bits in the last
+    def one(vals):
+        x = np.asarray(vals, dtype=np.float32).reshape(1, C, 1, 1)
+        return [int(v) for v in o.pack(x, o.NCHW).reshape(-1)]
+    assert one([1.0] * C) == [0, 0, 0]
+    assert one([-1.0] * C) == [0xFFFFFFFFFFFFFFFF, 0xFFFFFFFFFFFFFFFF, 0x3]
+    alt = [(-1.0 if c % 2 else 1.0) for c in range(C)]  # odd channels negative
+    assert one(alt) == [0xAAAAAAAAAAAAAAAA, 0xAAAAAAAAAAAAAAAA, 0x2]
+    for c, want in ((0, [1, 0, 0]), (63, [1 << 63, 0, 0]), (64, [0, 1, 0]), (127, [0, 1 << 63, 0]),
+                    (128, [0, 0, 1]), (129, [0, 0, 2])):
+        v = [0.5] * C
+        v[c] = -0.5
+        assert one(v) == want, c
+
+
+def test_special_floats(oracle_mod):
+    o = oracle_mod
+    neg_nan = np.frombuffer(np.uint32(0xFFC00000).tobytes(), dtype=np.float32)[0]
+    pos_nan = np.frombuffer(np.uint32(0x7FC00000).tobytes(), dtype=np.float32)[0]
+    vals = [0.0, -0.0, 1e-45, -1e-45, np.inf, -np.inf, pos_nan, neg_nan, 1.17549435e-38, -1.17549435e-38]
+    want = [0, 0, 0, 1, 0, 1, 0, 0, 0, 1]  # only values that compare below zero give bit 1
+    x = np.asarray(vals, dtype=np.float32).reshape(1, len(vals), 1, 1)
+    word = int(o.pack(x, o.NCHW).reshape(-1)[0])
+    assert [(word >> i) & 1 for i in range(len(vals))] == want
+
+
+@pytest.mark.parametrize("shape", [(2, 70, 5, 7), (1, 64, 3, 3), (3, 1, 2, 2), (1, 200, 4, 1)])
+def test_unpack_matches_comparison(oracle_mod, shape):
+    o = oracle_mod
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal(shape).astype(np.float32)
+    x[rng.random(shape) < 0.05] = 0.0
+    P = o.pack(x, o.NCHW)
+    N, C, H, W = shape
+    assert P.shape == (N, H, W, (C + 63) // 64) and P.dtype == np.uint64
+    bits, tail = unpack_words(P, C)
+    assert np.array_equal(bits, (np.transpose(x, (0, 2, 3, 1)) < 0).astype(np.uint8))
+    assert not tail.any()  # tail bits are zero
+    # NHWC input gives the same words
+    P2 = o.pack(np.ascontiguousarray(np.transpose(x, (0, 2, 3, 1))), o.NHWC)
+    assert np.array_equal(P, P2)
+
+
+def test_size_is_32x_smaller(oracle_mod):
+    # one bit per fp32 element (Section 3: packed weights are 32x smaller)
+    o = oracle_mod
+    x = np.ones((2, 256, 4, 4), dtype=np.float32)
+    assert o.pack(x).nbytes * 32 == x.nbytes
+    w = np.ones((8, 128, 3, 3), dtype=np.float32)
+    assert o.pack_weights(w).nbytes * 32 == w.nbytes
+
+
+def test_pack_weights_layout(oracle_mod):
+    o = oracle_mod
+    rng = np.random.default_rng(5)
+    w = rng.standard_normal((5, 70, 3, 2)).astype(np.float32)
+    Wp = o.pack_weights(w)
+    assert Wp.shape == (5, 3, 2, 2)
+    bits, tail = unpack_words(Wp, 70)
+    assert np.array_equal(bits, (np.transpose(w, (0, 2, 3, 1)) < 0).astype(np.uint8))
+    assert not tail.any()
