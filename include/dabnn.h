@@ -1,0 +1,133 @@
+/*
+ * dabnn.h -- C ABI of libdabnn_b200: binarized convolution on NVIDIA B200 (sm_100a).
+ *
+ * The operations are those of daBNN (arXiv 1908.05858): sign-binarize + bit-pack along the
+ * channel axis (Section 2.1.1), binary convolution on the packed words (Section 2.1.2, Eq. 1)
+ * and the fused BN + binarize + re-pack that feeds the next binary layer (Section 2.1.1, last
+ * sentence), plus a Bi-Real Net 18 forward built from them (Section 2.3, Table 2).
+ *
+ * Conventions shared by every entry point
+ *   - Every data pointer is DEVICE memory owned by the caller unless its name ends in _host.
+ *     The library allocates nothing, frees nothing and keeps no pointer after the call's work
+ *     on the stream has completed.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *     enqueue work; they do not synchronise.
+ *   - Binarization: v = (x < 0) ? -1 : +1 as an IEEE comparison (+0.0, -0.0 and NaN give +1).
+ *     A packed bit is 1 for -1.  Words are 64-bit; channel c lives in word c>>6 at bit c&63;
+ *     bits beyond C in the last word are 0.
+ *   - Packed activations: uint64 [N][H][W][Cw], Cw = ceil(C/64).
+ *     Packed weights:     uint64 [O][kh][kw][Cw].
+ *   - Convolution is cross-correlation, dilation 1, groups 1;
+ *     OH = floor((H + 2*pad_h - kh)/stride_h) + 1, likewise OW.  Spatial padding holds the
+ *     declared value pad_value (+1 or -1), so every output sums K = C*kh*kw terms and
+ *     out = K - 2*popcount(xor) lies in [-K, K] with the parity of K.
+ *   - Errors: argument problems are reported synchronously, before anything is launched
+ *     (DABNN_ERR_NULL / _SHAPE / _ALIGNMENT / _WORKSPACE); a failed launch gives DABNN_ERR_CUDA.
+ *     Nothing throws; kernels never trap.
+ *   - Alignment: packed buffers 8 bytes; fp32 buffers 4 bytes (16 bytes enables vector paths,
+ *     chosen automatically).
+ */
+#ifndef DABNN_H_
+#define DABNN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DABNN_OK = 0,
+  DABNN_ERR_NULL = 1,        /* a required pointer is NULL */
+  DABNN_ERR_SHAPE = 2,       /* non-positive dimension, empty output, bad stride / pad_value / layout */
+  DABNN_ERR_UNSUPPORTED = 3, /* a size beyond what the index arithmetic supports (>= 2^31 elements per axis product) */
+  DABNN_ERR_ALIGNMENT = 4,
+  DABNN_ERR_WORKSPACE = 5,   /* workspace too small */
+  DABNN_ERR_CUDA = 6         /* the CUDA runtime reported an error at launch */
+} dabnn_status;
+
+typedef enum { DABNN_NCHW = 0, DABNN_NHWC = 1 } dabnn_layout;
+
+/* Logical (unpacked) shape of an activation tensor. */
+typedef struct { int N, C, H, W; } dabnn_shape;
+
+/* Convolution geometry.  pad_value is the value (+1 or -1) every padded position holds. */
+typedef struct { int kh, kw, stride_h, stride_w, pad_h, pad_w, pad_value; } dabnn_conv;
+
+const char* dabnn_status_string(dabnn_status s);
+
+/* ceil(C/64): 64-bit words per pixel (or per weight tap). */
+size_t dabnn_words_per_pixel(int C);
+/* floor((in + 2*pad - k)/stride) + 1 (may be <= 0: no output). */
+int dabnn_out_dim(int in, int k, int stride, int pad);
+
+/* Section 2.1.1 -- binarize + pack activations.
+ * x: fp32, N*C*H*W elements in `in_layout`.  packed: uint64 [N][H][W][Cw], fully overwritten. */
+dabnn_status dabnn_pack(const float* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed, void* stream);
+
+/* Section 3 (weights are binarized and packed once, 32x smaller).
+ * w_oihw: fp32 [O][C][kh][kw].  wpacked: uint64 [O][kh][kw][Cw], fully overwritten. */
+dabnn_status dabnn_pack_weights(const float* w_oihw, int O, int C, int kh, int kw, uint64_t* wpacked, void* stream);
+
+/* Section 2.1.2, Eq. 1 -- binary convolution, int32 result.
+ * a_packed: [N][H][W][Cw] for in = {N,C,H,W}; w_packed: [O][kh][kw][Cw];
+ * out: int32, N*OH*OW*O elements in `out_layout` ([N][OH][OW][O] or [N][O][OH][OW]). */
+dabnn_status dabnn_bconv2d(const uint64_t* a_packed, dabnn_shape in, const uint64_t* w_packed, int O, dabnn_conv cv,
+                           int32_t* out, dabnn_layout out_layout, void* stream);
+
+/* Section 2.1.1 (fused BN-binarization) on top of Eq. 1: the int32 result never leaves the chip.
+ * y = fmaf((float)acc, scale[o], shift[o]); bit = (y < 0); out_packed: uint64 [N][OH][OW][ceil(O/64)]. */
+dabnn_status dabnn_bconv2d_bn_sign_pack(const uint64_t* a_packed, dabnn_shape in, const uint64_t* w_packed, int O,
+                                        dabnn_conv cv, const float* scale, const float* shift, uint64_t* out_packed,
+                                        void* stream);
+
+/* The Bi-Real block epilogue (Section 2.3): y = fmaf((float)acc, scale[o], shift[o]) + residual, one rounded
+ * add.  residual and y_out are fp32 [N][OH][OW][O] (may alias each other); out_packed as above holds the sign
+ * bits of y_out.  out_packed may be NULL when the packed signs are not needed. */
+dabnn_status dabnn_bconv2d_bn_add_sign_pack(const uint64_t* a_packed, dabnn_shape in, const uint64_t* w_packed, int O,
+                                            dabnn_conv cv, const float* scale, const float* shift,
+                                            const float* residual, float* y_out, uint64_t* out_packed, void* stream);
+
+/* BN parameters -> per-channel (scale, shift), evaluated in double on the device with IEEE-rounded operations:
+ * sd = gamma/sqrt(var+eps); scale = (float)sd; shift = (float)(beta - mean*sd).  All arrays hold O floats. */
+dabnn_status dabnn_bn_fold(const float* gamma, const float* beta, const float* mean, const float* var, double eps,
+                           int O, float* scale, float* shift, void* stream);
+
+/* Section 2.3 / Table 2 -- Bi-Real Net 18 (binary ResNet-18; 7x7 stem conv and the final fc in fp32).
+ * Stages of 64/128/256/512 channels at 56/28/14/7 pixels, four blocks each; block b:
+ * out = BN_b(bconv3x3(sign(x))) + shortcut(x), pad value -1; the first block of stages 2..4 has stride 2
+ * and shortcut(x) = BN(conv1x1_fp32(avgpool2x2(x))).  No activation function other than sign.
+ * Every fp32 operation is a single IEEE-rounded operation in a fixed order, so results are reproducible. */
+typedef struct {
+  const float* stem_w;           /* fp32 [64][3][7][7] */
+  const float* stem_scale;       /* folded BN, [64] */
+  const float* stem_shift;
+  const uint64_t* block_w[16];   /* packed [O][3][3][Cw] (dabnn_pack_weights) */
+  const float* block_scale[16];  /* folded BN, [O] */
+  const float* block_shift[16];
+  const float* down_w[3];        /* fp32 [O][C] 1x1 weights for the first block of stages 2, 3, 4 */
+  const float* down_scale[3];
+  const float* down_shift[3];
+  const float* fc_w;             /* fp32 [1000][512] */
+  const float* fc_b;             /* fp32 [1000] */
+} dabnn_bireal18_params;
+
+/* Bytes of device workspace dabnn_bireal18_forward needs for a batch of N images (0 if N <= 0). */
+size_t dabnn_bireal18_workspace_bytes(int N);
+
+/* p: HOST struct of device pointers.  images: fp32 NCHW [N][3][224][224].  logits: fp32 [N][1000].
+ * workspace: device memory, 256-byte aligned, at least dabnn_bireal18_workspace_bytes(N) bytes; its contents
+ * are scratch (activations between layers) and are undefined afterwards. */
+dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float* images, int N, float* logits,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/* Selects the convolution inner loop for measurement runs: 0 = automatic (default),
+ * 1 = one POPC per 32-bit word pair, 2 = carry-save (one POPC per two word pairs).  All give identical results.
+ * Returns the previous setting.  Not thread-safe against concurrent calls into the library. */
+int dabnn_set_conv_variant(int variant);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DABNN_H_ */

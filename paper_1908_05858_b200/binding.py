@@ -1,0 +1,263 @@
+"""Thin ctypes binding over the C ABI of ``libdabnn_b200.so`` (see ``include/dabnn.h``).
+
+Argument marshalling only: every function checks dtypes / devices, allocates the output tensor with
+torch (torch owns device memory and the stream) and calls the entry point of the same name.  There
+is no CPU path: without the compiled library, or with a tensor that is not on a CUDA device, the
+functions raise.
+
+Packed tensors are ``torch.int64`` on the device (the bit pattern of the library's ``uint64`` words).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+NCHW = 0
+NHWC = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdabnn_b200.so")
+
+EXPORTS = (
+    "dabnn_status_string", "dabnn_words_per_pixel", "dabnn_out_dim", "dabnn_pack", "dabnn_pack_weights",
+    "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack", "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold",
+    "dabnn_bireal18_workspace_bytes", "dabnn_bireal18_forward", "dabnn_set_conv_variant",
+)
+
+
+class DabnnError(RuntimeError):
+    pass
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [("N", ctypes.c_int), ("C", ctypes.c_int), ("H", ctypes.c_int), ("W", ctypes.c_int)]
+
+
+class Conv(ctypes.Structure):
+    _fields_ = [("kh", ctypes.c_int), ("kw", ctypes.c_int), ("stride_h", ctypes.c_int), ("stride_w", ctypes.c_int),
+                ("pad_h", ctypes.c_int), ("pad_w", ctypes.c_int), ("pad_value", ctypes.c_int)]
+
+
+class Bireal18Params(ctypes.Structure):
+    _fields_ = [
+        ("stem_w", ctypes.c_void_p), ("stem_scale", ctypes.c_void_p), ("stem_shift", ctypes.c_void_p),
+        ("block_w", ctypes.c_void_p * 16), ("block_scale", ctypes.c_void_p * 16), ("block_shift", ctypes.c_void_p * 16),
+        ("down_w", ctypes.c_void_p * 3), ("down_scale", ctypes.c_void_p * 3), ("down_shift", ctypes.c_void_p * 3),
+        ("fc_w", ctypes.c_void_p), ("fc_b", ctypes.c_void_p),
+    ]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise DabnnError("libdabnn_b200.so is missing: run `python -m paper_1908_05858_b200.build` "
+                             "(or __graft_entry__.build()) first; there is no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci = ctypes.c_void_p, ctypes.c_int
+        L.dabnn_status_string.restype = ctypes.c_char_p
+        L.dabnn_status_string.argtypes = [ci]
+        L.dabnn_words_per_pixel.restype = ctypes.c_size_t
+        L.dabnn_words_per_pixel.argtypes = [ci]
+        L.dabnn_out_dim.restype = ci
+        L.dabnn_out_dim.argtypes = [ci, ci, ci, ci]
+        L.dabnn_pack.argtypes = [vp, ci, Shape, vp, vp]
+        L.dabnn_pack_weights.argtypes = [vp, ci, ci, ci, ci, vp, vp]
+        L.dabnn_bconv2d.argtypes = [vp, Shape, vp, ci, Conv, vp, ci, vp]
+        L.dabnn_bconv2d_bn_sign_pack.argtypes = [vp, Shape, vp, ci, Conv, vp, vp, vp, vp]
+        L.dabnn_bconv2d_bn_add_sign_pack.argtypes = [vp, Shape, vp, ci, Conv, vp, vp, vp, vp, vp, vp]
+        L.dabnn_bn_fold.argtypes = [vp, vp, vp, vp, ctypes.c_double, ci, vp, vp, vp]
+        L.dabnn_bireal18_workspace_bytes.restype = ctypes.c_size_t
+        L.dabnn_bireal18_workspace_bytes.argtypes = [ci]
+        L.dabnn_bireal18_forward.argtypes = [ctypes.POINTER(Bireal18Params), vp, ci, vp, vp, ctypes.c_size_t, vp]
+        L.dabnn_set_conv_variant.restype = ci
+        L.dabnn_set_conv_variant.argtypes = [ci]
+        for name in ("dabnn_pack", "dabnn_pack_weights", "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack",
+                     "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold", "dabnn_bireal18_forward"):
+            getattr(L, name).restype = ci
+        _lib = L
+    return _lib
+
+
+def _check(status: int) -> None:
+    if status != 0:
+        raise DabnnError("dabnn status %d: %s" % (status, lib().dabnn_status_string(status).decode()))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype, name: str) -> torch.Tensor:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise DabnnError("%s must be a CUDA tensor (there is no CPU path)" % name)
+    if t.dtype != dtype:
+        raise DabnnError("%s must have dtype %s, got %s" % (name, dtype, t.dtype))
+    return t.contiguous()
+
+
+def words_per_pixel(C: int) -> int:
+    return int(lib().dabnn_words_per_pixel(C))
+
+
+def out_dim(size: int, k: int, stride: int, pad: int) -> int:
+    return int(lib().dabnn_out_dim(size, k, stride, pad))
+
+
+def _conv(kh, kw, stride, pad, pad_value) -> Conv:
+    return Conv(kh, kw, stride[0], stride[1], pad[0], pad[1], pad_value)
+
+
+def pack(x: torch.Tensor, layout: int = NCHW, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_pack: fp32 NCHW or NHWC -> packed int64 [N][H][W][Cw]."""
+    x = _dev(x, torch.float32, "x")
+    if layout == NCHW:
+        N, C, H, W = x.shape
+    else:
+        N, H, W, C = x.shape
+    if out is None:
+        out = torch.empty((N, H, W, words_per_pixel(C)), dtype=torch.int64, device=x.device)
+    _check(lib().dabnn_pack(x.data_ptr(), layout, Shape(N, C, H, W), out.data_ptr(), _stream()))
+    return out
+
+
+def pack_weights(w_oihw: torch.Tensor) -> torch.Tensor:
+    """dabnn_pack_weights: fp32 OIHW -> packed int64 [O][kh][kw][Cw]."""
+    w = _dev(w_oihw, torch.float32, "w")
+    O, C, kh, kw = w.shape
+    out = torch.empty((O, kh, kw, words_per_pixel(C)), dtype=torch.int64, device=w.device)
+    _check(lib().dabnn_pack_weights(w.data_ptr(), O, C, kh, kw, out.data_ptr(), _stream()))
+    return out
+
+
+def _geom(a_packed, C, w_packed, stride, pad):
+    a = _dev(a_packed, torch.int64, "a_packed")
+    w = _dev(w_packed, torch.int64, "w_packed")
+    N, H, W, Cw = a.shape
+    O, kh, kw, Cw2 = w.shape
+    if Cw != Cw2 or Cw != (C + 63) // 64:
+        raise DabnnError("packed word counts do not match C")
+    OH, OW = out_dim(H, kh, stride[0], pad[0]), out_dim(W, kw, stride[1], pad[1])
+    return a, w, N, H, W, O, kh, kw, OH, OW
+
+
+def bconv2d(a_packed, C: int, w_packed, stride=(1, 1), pad=(0, 0), pad_value: int = -1, out_layout: int = NHWC,
+            out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_bconv2d: int32 result, NHWC [N][OH][OW][O] or NCHW [N][O][OH][OW]."""
+    a, w, N, H, W, O, kh, kw, OH, OW = _geom(a_packed, C, w_packed, stride, pad)
+    if out is None:
+        shape = (N, max(OH, 0), max(OW, 0), O) if out_layout == NHWC else (N, O, max(OH, 0), max(OW, 0))
+        out = torch.empty(shape, dtype=torch.int32, device=a.device)
+    _check(lib().dabnn_bconv2d(a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O, _conv(kh, kw, stride, pad, pad_value),
+                               out.data_ptr(), out_layout, _stream()))
+    return out
+
+
+def bconv2d_bn_sign_pack(a_packed, C: int, w_packed, scale, shift, stride=(1, 1), pad=(0, 0), pad_value: int = -1,
+                         out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_bconv2d_bn_sign_pack: packed int64 [N][OH][OW][ceil(O/64)]."""
+    a, w, N, H, W, O, kh, kw, OH, OW = _geom(a_packed, C, w_packed, stride, pad)
+    scale = _dev(scale, torch.float32, "scale")
+    shift = _dev(shift, torch.float32, "shift")
+    if out is None:
+        out = torch.empty((N, max(OH, 0), max(OW, 0), words_per_pixel(O)), dtype=torch.int64, device=a.device)
+    _check(lib().dabnn_bconv2d_bn_sign_pack(a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O,
+                                            _conv(kh, kw, stride, pad, pad_value), scale.data_ptr(), shift.data_ptr(),
+                                            out.data_ptr(), _stream()))
+    return out
+
+
+def bconv2d_bn_add_sign_pack(a_packed, C: int, w_packed, scale, shift, residual, stride=(1, 1), pad=(0, 0),
+                             pad_value: int = -1, want_bits: bool = True):
+    """dabnn_bconv2d_bn_add_sign_pack: returns (y fp32 NHWC, packed signs of y or None)."""
+    a, w, N, H, W, O, kh, kw, OH, OW = _geom(a_packed, C, w_packed, stride, pad)
+    scale = _dev(scale, torch.float32, "scale")
+    shift = _dev(shift, torch.float32, "shift")
+    residual = _dev(residual, torch.float32, "residual")
+    if tuple(residual.shape) != (N, OH, OW, O):
+        raise DabnnError("residual must be NHWC [N][OH][OW][O]")
+    y = torch.empty_like(residual)
+    bits = torch.empty((N, OH, OW, words_per_pixel(O)), dtype=torch.int64, device=a.device) if want_bits else None
+    _check(lib().dabnn_bconv2d_bn_add_sign_pack(a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O,
+                                                _conv(kh, kw, stride, pad, pad_value), scale.data_ptr(),
+                                                shift.data_ptr(), residual.data_ptr(), y.data_ptr(),
+                                                bits.data_ptr() if want_bits else None, _stream()))
+    return y, bits
+
+
+def bn_fold(gamma, beta, mean, var, eps: float = 1e-5):
+    """dabnn_bn_fold: (scale, shift) fp32 device tensors."""
+    g, b, m, v = (_dev(t, torch.float32, "bn") for t in (gamma, beta, mean, var))
+    O = g.numel()
+    scale = torch.empty(O, dtype=torch.float32, device=g.device)
+    shift = torch.empty(O, dtype=torch.float32, device=g.device)
+    _check(lib().dabnn_bn_fold(g.data_ptr(), b.data_ptr(), m.data_ptr(), v.data_ptr(), float(eps), O,
+                               scale.data_ptr(), shift.data_ptr(), _stream()))
+    return scale, shift
+
+
+def bireal18_workspace_bytes(N: int) -> int:
+    return int(lib().dabnn_bireal18_workspace_bytes(N))
+
+
+class Bireal18:
+    """Device-resident Bi-Real Net 18 parameters, prepared once with the library's own kernels
+    (weights packed by dabnn_pack_weights, BN folded by dabnn_bn_fold)."""
+
+    def __init__(self, params: dict, device="cuda"):
+        dev = torch.device(device)
+
+        def up(a):
+            return torch.as_tensor(a, dtype=torch.float32).contiguous().to(dev)
+
+        eps = float(params.get("bn_eps", 1e-5))
+        self.keep = []
+        P = Bireal18Params()
+        self.stem_w = up(params["stem_w"])
+        self.stem_scale, self.stem_shift = bn_fold(*[up(t) for t in params["stem_bn"]], eps=eps)
+        P.stem_w, P.stem_scale, P.stem_shift = self.stem_w.data_ptr(), self.stem_scale.data_ptr(), self.stem_shift.data_ptr()
+        for b in range(16):
+            wp = pack_weights(up(params["block_w"][b]))
+            sc, sh = bn_fold(*[up(t) for t in params["block_bn"][b]], eps=eps)
+            self.keep += [wp, sc, sh]
+            P.block_w[b], P.block_scale[b], P.block_shift[b] = wp.data_ptr(), sc.data_ptr(), sh.data_ptr()
+        for d in range(3):
+            w = up(params["down_w"][d])
+            sc, sh = bn_fold(*[up(t) for t in params["down_bn"][d]], eps=eps)
+            self.keep += [w, sc, sh]
+            P.down_w[d], P.down_scale[d], P.down_shift[d] = w.data_ptr(), sc.data_ptr(), sh.data_ptr()
+        self.fc_w, self.fc_b = up(params["fc_w"]), up(params["fc_b"])
+        P.fc_w, P.fc_b = self.fc_w.data_ptr(), self.fc_b.data_ptr()
+        self.P = P
+        self.device = dev
+        self._ws = None
+
+    def workspace(self, N: int) -> torch.Tensor:
+        need = bireal18_workspace_bytes(N)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    def forward(self, images: torch.Tensor, logits: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """dabnn_bireal18_forward: images fp32 NCHW [N][3][224][224] -> logits fp32 [N][1000]."""
+        images = _dev(images, torch.float32, "images")
+        N = images.shape[0]
+        if tuple(images.shape[1:]) != (3, 224, 224):
+            raise DabnnError("images must be [N][3][224][224]")
+        ws = self.workspace(N)
+        if logits is None:
+            logits = torch.empty((N, 1000), dtype=torch.float32, device=images.device)
+        _check(lib().dabnn_bireal18_forward(ctypes.byref(self.P), images.data_ptr(), N, logits.data_ptr(),
+                                            ws.data_ptr(), ws.numel(), _stream()))
+        return logits
+
+
+def set_conv_variant(variant: int) -> int:
+    return int(lib().dabnn_set_conv_variant(int(variant)))

@@ -1,0 +1,340 @@
+// Bi-Real Net 18 forward (Section 2.3, Table 2 of the paper): fp32 stem and head around sixteen binary
+// 3x3 convolutions whose BN + shortcut + sign + re-pack run in the convolution's epilogue.
+//
+// All activations between layers are NHWC.  Every fp32 value is produced by single IEEE-rounded
+// operations in a fixed order (explicit fmaf chains, ascending channel / tap order), never by tensor
+// cores or split sums, because the next binary layer takes the SIGN of these values: a different
+// rounding order could flip a bit and change integer results downstream.
+#include "common.cuh"
+
+namespace dabnn {
+
+namespace {
+
+// ---- BN fold, in double ---------------------------------------------------------------------------
+__global__ void bn_fold_kernel(const float* gamma, const float* beta, const float* mean, const float* var, double eps,
+                               int O, float* scale, float* shift) {
+  const int o = blockIdx.x * blockDim.x + threadIdx.x;
+  if (o >= O) return;
+  const double sd = __ddiv_rn((double)gamma[o], __dsqrt_rn(__dadd_rn((double)var[o], eps)));
+  scale[o] = (float)sd;
+  shift[o] = (float)__dsub_rn((double)beta[o], __dmul_rn((double)mean[o], sd));
+}
+
+// ---- stem: conv 7x7 / 2, 3 -> 64, zero pad 3, then BN ----------------------------------------------
+// A CTA computes a TS x TS tile of output pixels for all 64 channels.  The input patch sits in shared
+// memory with even and odd columns apart, so that lanes walking along ow (input stride 2) read
+// consecutive words.  A thread owns PPT pixels (rows TS/PPT apart... see below) x 16 channels and runs one fmaf
+// chain per output over (c, kh, kw) in that order.  Zero padding is held as zeros in the patch:
+// fmaf(0, w, acc) returns acc.
+constexpr int STEM_K = 147;
+
+template <int TS, int PPT>
+__global__ void __launch_bounds__((TS * TS / PPT) * 4) stem_conv_bn(const float* __restrict__ img,
+                                                                    const float* __restrict__ w,
+                                                                    const float* __restrict__ scale,
+                                                                    const float* __restrict__ shift,
+                                                                    float* __restrict__ out /*[N][112][112][64]*/) {
+  constexpr int IH = 224, IW = 224, OHW = 112;
+  constexpr int PS = 2 * TS + 5;         // patch side
+  constexpr int HALF = (PS + 1) / 2 + 1; // columns per parity, padded
+  constexpr int PGROUPS = TS * TS / PPT; // pixel groups = threads per channel group
+  constexpr int THREADS = PGROUPS * 4;
+  constexpr int RSTEP = TS / PPT;        // a thread's pixels are RSTEP rows apart
+  extern __shared__ __align__(16) float sm[];
+  float* w_s = sm;                       // [147][64]
+  float* x_s = sm + STEM_K * 64;         // [3][PS][2][HALF]
+  const int tid = threadIdx.x;
+  const int n = blockIdx.z, oh0 = blockIdx.y * TS, ow0 = blockIdx.x * TS;
+  for (int t = tid; t < STEM_K * 64; t += THREADS) {
+    const int o = t % 64, k = t / 64;    // w is [64][147]
+    w_s[k * 64 + o] = w[o * STEM_K + k];
+  }
+  const int ih_base = 2 * oh0 - 3, iw_base = 2 * ow0 - 3;
+  for (int t = tid; t < 3 * PS * PS; t += THREADS) {
+    const int lw = t % PS, lh = (t / PS) % PS, c = t / (PS * PS);
+    const int ih = ih_base + lh, iw = iw_base + lw;
+    float v = 0.0f;
+    if (ih >= 0 && ih < IH && iw >= 0 && iw < IW) v = img[(((size_t)n * 3 + c) * IH + ih) * IW + iw];
+    x_s[((c * PS + lh) * 2 + (lw & 1)) * HALF + (lw >> 1)] = v;
+  }
+  __syncthreads();
+  const int cg = tid / PGROUPS;          // channel group: 16 channels
+  const int pg = tid % PGROUPS;
+  const int low = pg % TS, lohb = pg / TS;  // pixels (lohb + RSTEP*i, low)
+  float acc[PPT][16];
+#pragma unroll
+  for (int i = 0; i < PPT; i++)
+#pragma unroll
+    for (int j = 0; j < 16; j++) acc[i][j] = 0.0f;
+  for (int c = 0; c < 3; c++)
+    for (int ki = 0; ki < 7; ki++) {
+#pragma unroll
+      for (int kj = 0; kj < 7; kj++) {
+        const int k = (c * 7 + ki) * 7 + kj;
+        float wv[16];
+#pragma unroll
+        for (int q = 0; q < 4; q++) {
+          const float4 t4 = *reinterpret_cast<const float4*>(w_s + k * 64 + cg * 16 + 4 * q);
+          wv[4 * q] = t4.x; wv[4 * q + 1] = t4.y; wv[4 * q + 2] = t4.z; wv[4 * q + 3] = t4.w;
+        }
+#pragma unroll
+        for (int i = 0; i < PPT; i++) {
+          const int lh = 2 * (lohb + RSTEP * i) + ki;
+          const float xv = x_s[((c * PS + lh) * 2 + (kj & 1)) * HALF + low + (kj >> 1)];
+#pragma unroll
+          for (int j = 0; j < 16; j++) acc[i][j] = __fmaf_rn(xv, wv[j], acc[i][j]);
+        }
+      }
+    }
+  float sc[16], sf[16];
+#pragma unroll
+  for (int j = 0; j < 16; j++) {
+    sc[j] = scale[cg * 16 + j];
+    sf[j] = shift[cg * 16 + j];
+  }
+#pragma unroll
+  for (int i = 0; i < PPT; i++) {
+    const int oh = oh0 + lohb + RSTEP * i, ow = ow0 + low;
+    if (oh >= OHW || ow >= OHW) continue;
+    float* dst = out + (((size_t)n * OHW + oh) * OHW + ow) * 64 + cg * 16;
+#pragma unroll
+    for (int j = 0; j < 16; j += 4)
+      *reinterpret_cast<float4*>(dst + j) =
+          make_float4(__fmaf_rn(acc[i][j], sc[j], sf[j]), __fmaf_rn(acc[i][j + 1], sc[j + 1], sf[j + 1]),
+                      __fmaf_rn(acc[i][j + 2], sc[j + 2], sf[j + 2]), __fmaf_rn(acc[i][j + 3], sc[j + 3], sf[j + 3]));
+  }
+}
+
+// ---- maxpool 3x3 / 2, pad 1 (64 channels) -> fp32 residual stream + packed signs -------------------
+// A thread handles 4 channels of one output pixel; 16 lanes make one 64-bit word.
+__global__ void __launch_bounds__(256) maxpool_pack(const float* __restrict__ x /*[N][112][112][64]*/, long long npix,
+                                                    float* __restrict__ y /*[N][56][56][64]*/,
+                                                    uint64_t* __restrict__ bits /*[N][56][56][1]*/) {
+  const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  const long long pix = t >> 4;
+  const int c4 = (int)(t & 15);
+  const bool live = pix < npix;
+  float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+  if (live) {
+    const int ow = (int)(pix % 56), oh = (int)((pix / 56) % 56);
+    const long long n = pix / (56 * 56);
+#pragma unroll
+    for (int i = 0; i < 3; i++)
+#pragma unroll
+      for (int j = 0; j < 3; j++) {
+        const int ih = 2 * oh + i - 1, iw = 2 * ow + j - 1;
+        if (ih < 0 || ih >= 112 || iw < 0 || iw >= 112) continue;
+        const float4 v = *reinterpret_cast<const float4*>(x + ((n * 112 + ih) * 112 + iw) * 64 + c4 * 4);
+        m.x = fmaxf(m.x, v.x); m.y = fmaxf(m.y, v.y); m.z = fmaxf(m.z, v.z); m.w = fmaxf(m.w, v.w);
+      }
+    *reinterpret_cast<float4*>(y + pix * 64 + c4 * 4) = m;
+  }
+  unsigned nib = 0;
+  if (live) nib = (unsigned)(m.x < 0.0f) | ((unsigned)(m.y < 0.0f) << 1) | ((unsigned)(m.z < 0.0f) << 2) | ((unsigned)(m.w < 0.0f) << 3);
+  const unsigned gmask = 0xFFu << (lane & 24);
+  const unsigned half = __reduce_or_sync(gmask, nib << (4 * (lane & 7)));
+  const unsigned other = __shfl_xor_sync(0xFFFFFFFFu, half, 8);
+  if (live && (lane & 15) == 0) bits[pix] = (uint64_t)half | ((uint64_t)other << 32);
+}
+
+// ---- downsample shortcut: avgpool 2x2 / 2 -> fp32 conv 1x1 (C -> O) -> BN ---------------------------
+// CTA tile: 32 output pixels x 64 output channels; a thread owns 8 consecutive pixels x 2 channels (o, o+32).
+// One fmaf chain per output over c ascending.
+__global__ void __launch_bounds__(128) shortcut_down(const float* __restrict__ x /*[N][HW][HW][C]*/, int HW, int C,
+                                                     const float* __restrict__ w /*[O][C]*/, int O,
+                                                     const float* __restrict__ scale, const float* __restrict__ shift,
+                                                     long long npix_out, float* __restrict__ y /*[N][HW/2][HW/2][O]*/) {
+  __shared__ __align__(16) float p_s[32][36];   // [c in chunk][pixel], padded
+  __shared__ float w_s[64][33];                 // [o in tile][c in chunk]
+  const int tid = threadIdx.x;
+  const long long p0 = (long long)blockIdx.x * 32;
+  const int o0 = blockIdx.y * 64;
+  const int OHW = HW / 2;
+  const int ol = tid % 32, pgp = tid / 32;      // pixels pgp*8 .. pgp*8+7
+  float acc[8][2];
+#pragma unroll
+  for (int i = 0; i < 8; i++) acc[i][0] = acc[i][1] = 0.0f;
+  for (int c0 = 0; c0 < C; c0 += 32) {
+    __syncthreads();
+    for (int t = tid; t < 32 * 32; t += 128) {
+      const int cc = t % 32, pp = t / 32;
+      const long long p = p0 + pp;
+      float v = 0.0f;
+      if (p < npix_out && c0 + cc < C) {
+        const int ow = (int)(p % OHW), oh = (int)((p / OHW) % OHW);
+        const long long n = p / ((long long)OHW * OHW);
+        const float* q = x + ((n * HW + 2 * oh) * HW + 2 * ow) * C + c0 + cc;
+        float s = __fadd_rn(q[0], q[C]);
+        s = __fadd_rn(s, q[(size_t)HW * C]);
+        s = __fadd_rn(s, q[(size_t)HW * C + C]);
+        v = __fmul_rn(s, 0.25f);
+      }
+      p_s[cc][pp] = v;
+    }
+    for (int t = tid; t < 64 * 32; t += 128) {
+      const int cc = t % 32, oo = t / 32;
+      w_s[oo][cc] = (o0 + oo < O && c0 + cc < C) ? w[(size_t)(o0 + oo) * C + c0 + cc] : 0.0f;
+    }
+    __syncthreads();
+    const int cn = min(32, C - c0);
+    for (int cc = 0; cc < cn; cc++) {
+      const float w0 = w_s[ol][cc], w1 = w_s[ol + 32][cc];
+      const float4 pa = *reinterpret_cast<const float4*>(&p_s[cc][pgp * 8]);
+      const float4 pb = *reinterpret_cast<const float4*>(&p_s[cc][pgp * 8 + 4]);
+      const float pv[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+#pragma unroll
+      for (int i = 0; i < 8; i++) {
+        acc[i][0] = __fmaf_rn(pv[i], w0, acc[i][0]);
+        acc[i][1] = __fmaf_rn(pv[i], w1, acc[i][1]);
+      }
+    }
+  }
+#pragma unroll
+  for (int h = 0; h < 2; h++) {
+    const int o = o0 + ol + 32 * h;
+    if (o >= O) continue;
+    const float sc = scale[o], sf = shift[o];
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+      const long long p = p0 + pgp * 8 + i;
+      if (p < npix_out) y[p * O + o] = __fmaf_rn(acc[i][h], sc, sf);
+    }
+  }
+}
+
+// ---- head: global average over 7x7 (sequential sum, then /49), fc 512 -> 1000 -----------------------
+__global__ void __launch_bounds__(256) gap_fc(const float* __restrict__ x /*[N][7][7][512]*/,
+                                              const float* __restrict__ fw /*[1000][512]*/,
+                                              const float* __restrict__ fb, float* __restrict__ logits) {
+  __shared__ __align__(16) float g[512];
+  const int n = blockIdx.y;
+  for (int c = threadIdx.x; c < 512; c += blockDim.x) {
+    float s = 0.0f;
+    for (int q = 0; q < 49; q++) s = __fadd_rn(s, x[((size_t)n * 49 + q) * 512 + c]);
+    g[c] = __fdiv_rn(s, 49.0f);
+  }
+  __syncthreads();
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= 1000) return;
+  const float4* wr = reinterpret_cast<const float4*>(fw + (size_t)j * 512);
+  float a = 0.0f;
+  for (int k4 = 0; k4 < 128; k4++) {
+    const float4 wv = __ldg(wr + k4);
+    const float4 gv = *reinterpret_cast<const float4*>(g + 4 * k4);
+    a = __fmaf_rn(gv.x, wv.x, a);
+    a = __fmaf_rn(gv.y, wv.y, a);
+    a = __fmaf_rn(gv.z, wv.z, a);
+    a = __fmaf_rn(gv.w, wv.w, a);
+  }
+  logits[(size_t)n * 1000 + j] = __fadd_rn(a, fb[j]);
+}
+
+constexpr int kStageC[4] = {64, 128, 256, 512};
+constexpr int kStageHW[4] = {56, 28, 14, 7};
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Workspace {
+  size_t stem_out, res_a, res_b, bits_a, bits_b, total;
+};
+
+Workspace plan(int N) {
+  Workspace ws;
+  size_t off = 0;
+  ws.stem_out = off; off = align_up(off + (size_t)N * 112 * 112 * 64 * 4, 256);
+  ws.res_a = off;    off = align_up(off + (size_t)N * 56 * 56 * 64 * 4, 256);
+  ws.res_b = off;    off = align_up(off + (size_t)N * 28 * 28 * 128 * 4, 256);
+  ws.bits_a = off;   off = align_up(off + (size_t)N * 56 * 56 * 8, 256);
+  ws.bits_b = off;   off = align_up(off + (size_t)N * 56 * 56 * 8, 256);
+  ws.total = off;
+  return ws;
+}
+
+template <int TS, int PPT>
+dabnn_status launch_stem(const dabnn_bireal18_params* p, const float* images, int N, float* out, cudaStream_t st) {
+  constexpr int PS = 2 * TS + 5, HALF = (PS + 1) / 2 + 1;
+  constexpr size_t SMEM = (size_t)(STEM_K * 64 + 3 * PS * 2 * HALF) * 4;
+  auto kern = stem_conv_bn<TS, PPT>;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) {
+      cudaGetLastError();
+      return DABNN_ERR_CUDA;
+    }
+    configured = true;
+  }
+  const int tiles = (112 + TS - 1) / TS;
+  kern<<<dim3(tiles, tiles, N), (TS * TS / PPT) * 4, SMEM, st>>>(images, p->stem_w, p->stem_scale, p->stem_shift, out);
+  return launch_status();
+}
+
+}  // namespace
+
+}  // namespace dabnn
+
+using namespace dabnn;
+
+extern "C" dabnn_status dabnn_bn_fold(const float* gamma, const float* beta, const float* mean, const float* var,
+                                      double eps, int O, float* scale, float* shift, void* stream) {
+  if (!gamma || !beta || !mean || !var || !scale || !shift) return DABNN_ERR_NULL;
+  if (O <= 0 || !(eps >= 0.0)) return DABNN_ERR_SHAPE;
+  bn_fold_kernel<<<ceil_div(O, 128), 128, 0, as_stream(stream)>>>(gamma, beta, mean, var, eps, O, scale, shift);
+  return launch_status();
+}
+
+extern "C" size_t dabnn_bireal18_workspace_bytes(int N) { return N <= 0 ? 0 : plan(N).total; }
+
+extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float* images, int N,
+                                               float* logits, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!p || !images || !logits || !workspace) return DABNN_ERR_NULL;
+  if (N <= 0 || N > 65535) return DABNN_ERR_SHAPE;
+  if (!p->stem_w || !p->stem_scale || !p->stem_shift || !p->fc_w || !p->fc_b) return DABNN_ERR_NULL;
+  for (int b = 0; b < 16; b++)
+    if (!p->block_w[b] || !p->block_scale[b] || !p->block_shift[b]) return DABNN_ERR_NULL;
+  for (int d = 0; d < 3; d++)
+    if (!p->down_w[d] || !p->down_scale[d] || !p->down_shift[d]) return DABNN_ERR_NULL;
+  if (!aligned(workspace, 256) || !aligned(images, 4) || !aligned(logits, 4) || !aligned(p->fc_w, 16))
+    return DABNN_ERR_ALIGNMENT;
+  const Workspace ws = plan(N);
+  if (workspace_bytes < ws.total) return DABNN_ERR_WORKSPACE;
+  cudaStream_t st = as_stream(stream);
+  char* base = static_cast<char*>(workspace);
+  float* stem_out = reinterpret_cast<float*>(base + ws.stem_out);
+  float* cur = reinterpret_cast<float*>(base + ws.res_a);
+  float* other = reinterpret_cast<float*>(base + ws.res_b);
+  uint64_t* bits_in = reinterpret_cast<uint64_t*>(base + ws.bits_a);
+  uint64_t* bits_out = reinterpret_cast<uint64_t*>(base + ws.bits_b);
+
+  dabnn_status s = (N * 49 >= 2 * sm_count()) ? launch_stem<16, 4>(p, images, N, stem_out, st)
+                                               : launch_stem<8, 1>(p, images, N, stem_out, st);
+  if (s != DABNN_OK) return s;
+  {
+    const long long npix = (long long)N * 56 * 56;
+    maxpool_pack<<<ceil_div(npix * 16, 256), 256, 0, st>>>(stem_out, npix, cur, bits_in);
+    if ((s = launch_status()) != DABNN_OK) return s;
+  }
+  int C = 64, HW = 56;
+  for (int b = 0; b < 16; b++) {
+    const int stage = b / 4, O = kStageC[stage], OHW = kStageHW[stage];
+    const bool down = stage > 0 && b % 4 == 0;
+    if (down) {
+      const long long npo = (long long)N * OHW * OHW;
+      shortcut_down<<<dim3(ceil_div(npo, 32), ceil_div(O, 64)), 128, 0, st>>>(
+          cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
+      if ((s = launch_status()) != DABNN_OK) return s;
+      float* t = cur; cur = other; other = t;
+    }
+    const dabnn_shape in = {N, C, HW, HW};
+    const int stride = down ? 2 : 1;
+    const dabnn_conv cv = {3, 3, stride, stride, 1, 1, -1};
+    s = dabnn_bconv2d_bn_add_sign_pack(bits_in, in, p->block_w[b], O, cv, p->block_scale[b], p->block_shift[b], cur, cur,
+                                       b == 15 ? nullptr : bits_out, st);
+    if (s != DABNN_OK) return s;
+    uint64_t* tb = bits_in; bits_in = bits_out; bits_out = tb;
+    C = O; HW = OHW;
+  }
+  gap_fc<<<dim3(4, N), 256, 0, st>>>(cur, p->fc_w, p->fc_b, logits);
+  return launch_status();
+}

@@ -1,0 +1,219 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded
+inputs.  Integer and bit results must be identical; fp32 results of the Bi-Real path are produced by
+the same IEEE operations in the same order on both sides, so they are compared bit for bit as well,
+and the logits additionally within the stated tolerance (max-abs 1e-3 of the logit scale, same argmax)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_1908_05858_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_1908_05858_b200 import binding
+
+    assert torch.cuda.is_available(), "the parity tests need a CUDA device"
+    binding.lib()  # raises if the CUDA library is missing: no fallback
+    return binding
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def u64(t):
+    return t.cpu().numpy().view(np.uint64)
+
+
+# ---- pack ---------------------------------------------------------------------------------------------
+PACK_SHAPES = [
+    (2, 64, 14, 14),    # vector path, one word
+    (3, 256, 56, 56),   # vector path, four warps per pixel group, ragged last tile (3136 = 24.5 * 128)
+    (2, 128, 28, 28),   # vector path, two words
+    (1, 192, 12, 12),   # three words
+    (2, 70, 7, 5),      # generic path (H*W not a multiple of 4), channel tail
+    (1, 1, 1, 1),
+    (1, 1000, 2, 2),    # 16 words, tail of 40 bits
+    (5, 3, 224, 8),
+]
+
+
+@pytest.mark.parametrize("shape", PACK_SHAPES)
+def test_pack_nchw(B, oracle_mod, shape):
+    rng = np.random.default_rng(sum(shape))
+    x = rng.standard_normal(shape).astype(np.float32)
+    x[rng.random(shape) < 0.01] = 0.0
+    flat = x.reshape(-1)
+    flat[:6] = [0.0, -0.0, np.nan, -np.inf, 1e-45, -1e-45][: min(6, flat.size)]
+    got = u64(B.pack(dev(x), B.NCHW))
+    assert np.array_equal(got, oracle_mod.pack(x, oracle_mod.NCHW))
+
+
+@pytest.mark.parametrize("shape", [(2, 14, 14, 64), (3, 9, 7, 256), (2, 5, 5, 70), (1, 3, 3, 4), (4, 31, 17, 128)])
+def test_pack_nhwc(B, oracle_mod, shape):
+    rng = np.random.default_rng(sum(shape) + 1)
+    x = rng.standard_normal(shape).astype(np.float32)
+    x[rng.random(shape) < 0.02] = -0.0
+    got = u64(B.pack(dev(x), B.NHWC))
+    assert np.array_equal(got, oracle_mod.pack(x, oracle_mod.NHWC))
+
+
+def test_pack_unaligned_input_takes_the_generic_path(B, oracle_mod):
+    rng = np.random.default_rng(8)
+    buf = rng.standard_normal(1 + 2 * 64 * 8 * 8).astype(np.float32)
+    d = dev(buf)
+    x = d[1:].view(2, 64, 8, 8)  # 4-byte aligned only
+    got = u64(B.pack(x, B.NCHW))
+    assert np.array_equal(got, oracle_mod.pack(buf[1:].reshape(2, 64, 8, 8)))
+
+
+@pytest.mark.parametrize("shape", [(64, 64, 3, 3), (9, 70, 3, 3), (2048, 512, 1, 1), (5, 130, 5, 2)])
+def test_pack_weights(B, oracle_mod, shape):
+    w = np.random.default_rng(shape[0]).standard_normal(shape).astype(np.float32)
+    assert np.array_equal(u64(B.pack_weights(dev(w))), oracle_mod.pack_weights(w))
+
+
+# ---- binary convolution ---------------------------------------------------------------------------------
+CONV_CASES = [
+    # N, C, H, W, O, kh, kw, stride, pad, pad_value
+    (1, 64, 14, 14, 64, 3, 3, (1, 1), (1, 1), -1),      # BASELINE config 1
+    (2, 70, 7, 5, 9, 3, 3, (1, 1), (1, 1), -1),         # channel tail, tiny O
+    (2, 70, 7, 5, 9, 3, 3, (1, 1), (1, 1), +1),
+    (1, 130, 9, 8, 37, 3, 3, (2, 2), (1, 1), -1),       # three words (8-byte copy units), stride 2
+    (3, 128, 13, 11, 100, 3, 3, (1, 1), (1, 1), -1),    # 16-byte copy units, ragged pixel and channel tiles
+    (1, 3, 12, 12, 5, 5, 5, (1, 2), (2, 2), -1),
+    (2, 128, 6, 6, 130, 1, 1, (1, 1), (0, 0), -1),      # 1x1
+    (1, 17, 6, 7, 3, 2, 3, (2, 1), (0, 1), +1),
+    (1, 256, 14, 14, 256, 3, 3, (1, 1), (1, 1), -1),    # several K chunks
+    (1, 512, 7, 7, 512, 3, 3, (1, 1), (1, 1), -1),      # K = 4608 bits, 5 chunks
+    (1, 64, 56, 56, 64, 3, 3, (1, 1), (1, 1), -1),
+    (4, 64, 30, 30, 128, 7, 7, (2, 2), (3, 3), -1),     # 49 taps
+    (40, 192, 20, 20, 192, 3, 3, (1, 1), (1, 1), -1),   # large enough for the 128x128 tile
+]
+
+
+def conv_inputs(case):
+    N, C, H, W, O, kh, kw, stride, pad, pv = case
+    rng = np.random.default_rng(abs(hash(case)) % (2**32))
+    x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+    w = rng.standard_normal((O, C, kh, kw)).astype(np.float32)
+    return x, w
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_bconv2d_matches_oracle(B, oracle_mod, case, variant):
+    N, C, H, W, O, kh, kw, stride, pad, pv = case
+    x, w = conv_inputs(case)
+    o = oracle_mod
+    want = o.bconv_bits(o.pack(x), C, o.pack_weights(w), stride, pad, pv, o.NHWC)
+    prev = B.set_conv_variant(variant)
+    try:
+        a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
+        got = B.bconv2d(a, C, wp, stride, pad, pv, B.NHWC).cpu().numpy()
+        got_nchw = B.bconv2d(a, C, wp, stride, pad, pv, B.NCHW).cpu().numpy()
+        again = B.bconv2d(a, C, wp, stride, pad, pv, B.NHWC).cpu().numpy()
+    finally:
+        B.set_conv_variant(prev)
+    assert np.array_equal(got, want)
+    assert np.array_equal(got_nchw, np.transpose(want, (0, 3, 1, 2)))
+    assert np.array_equal(again, got)  # a second run gives the same bits (no race)
+    if N * O * want.shape[1] * want.shape[2] * C * kh * kw < 3e8:  # the definition itself, where it is quick
+        assert np.array_equal(want, o.bconv_pm1(x, w, stride, pad, pv, o.NHWC))
+
+
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_fused_bn_sign_pack_matches_oracle(B, oracle_mod, case):
+    N, C, H, W, O, kh, kw, stride, pad, pv = case
+    x, w = conv_inputs(case)
+    o = oracle_mod
+    rng = np.random.default_rng(O)
+    gamma, beta, mean, var = synth.bn_params(rng, O)
+    gamma[::5] *= -1.0
+    mean *= 30.0  # thresholds spread over the range of the integer results
+    scale_o, shift_o = o.bn_fold(gamma, beta, mean, var)
+    scale_g, shift_g = B.bn_fold(dev(gamma), dev(beta), dev(mean), dev(var))
+    assert np.array_equal(scale_g.cpu().numpy().view(np.uint32), scale_o.view(np.uint32))
+    assert np.array_equal(shift_g.cpu().numpy().view(np.uint32), shift_o.view(np.uint32))
+    acc = o.bconv_bits(o.pack(x), C, o.pack_weights(w), stride, pad, pv, o.NHWC)
+    want = o.bn_sign_pack(acc, scale_o, shift_o)
+    a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
+    got = u64(B.bconv2d_bn_sign_pack(a, C, wp, scale_g, shift_g, stride, pad, pv))
+    assert np.array_equal(got, want)
+    assert 0 < np.count_nonzero(got) < got.size * 64 or O < 4
+
+
+@pytest.mark.parametrize("case", [CONV_CASES[0], CONV_CASES[3], CONV_CASES[4], CONV_CASES[8], CONV_CASES[12]])
+def test_bireal_block_epilogue_matches_oracle(B, oracle_mod, case):
+    N, C, H, W, O, kh, kw, stride, pad, pv = case
+    x, w = conv_inputs(case)
+    o = oracle_mod
+    rng = np.random.default_rng(O + 1)
+    scale_o, shift_o = o.bn_fold(*synth.bn_params(rng, O))
+    acc = o.bconv_bits(o.pack(x), C, o.pack_weights(w), stride, pad, pv, o.NHWC)
+    res = rng.standard_normal(acc.shape).astype(np.float32) * 20
+    # y = fmaf(acc, scale, shift) + r: fp64 product-sum is exact here, so rounding it once gives fmaf
+    y = (acc.astype(np.float64) * scale_o.astype(np.float64) + shift_o.astype(np.float64)).astype(np.float32) + res
+    want_bits = o.pack(y, o.NHWC)
+    a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
+    got_y, got_bits = B.bconv2d_bn_add_sign_pack(a, C, wp, dev(scale_o), dev(shift_o), dev(res), stride, pad, pv)
+    assert np.array_equal(got_y.cpu().numpy().view(np.uint32), y.view(np.uint32))
+    assert np.array_equal(u64(got_bits), want_bits)
+
+
+# ---- full-size configurations, sampled ---------------------------------------------------------------------
+def sample_coords(rng, N, O, OH, OW, n):
+    c = np.stack([rng.integers(0, N, n), rng.integers(0, O, n), rng.integers(0, OH, n), rng.integers(0, OW, n)], axis=1)
+    # always include the corners and edges, where padding matters
+    fixed = [(0, 0, 0, 0), (N - 1, O - 1, OH - 1, OW - 1), (N - 1, 0, 0, OW - 1), (0, O - 1, OH - 1, 0), (N // 2, O // 2, 0, OW // 2)]
+    return np.concatenate([np.array(fixed), c]).astype(np.int32)
+
+
+FULL = [(64, C, HW, C, 3, 1) for C, HW in synth.SWEEP_SHAPES] + [(256, 256, 28, 256, 3, 1), (256, 512, 14, 2048, 1, 0)]
+
+
+@pytest.mark.parametrize("cfg", FULL)
+def test_full_size_configs_on_sampled_outputs(B, oracle_mod, cfg):
+    N, C, HW, O, k, pad = cfg
+    x, w = synth.conv_case(2 if N == 64 else 5, N, C, HW, HW, O, k, k, salt=C)
+    a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
+    got = B.bconv2d(a, C, wp, (1, 1), (pad, pad), -1, B.NHWC)
+    K = C * k * k
+    # properties that hold for every output
+    assert int(got.min()) >= -K and int(got.max()) <= K
+    assert bool(((got - K) % 2 == 0).all())
+    g = got.cpu().numpy()
+    rng = np.random.default_rng(C + N)
+    coords = sample_coords(rng, N, O, HW, HW, 100000)
+    want = oracle_mod.bconv_pm1_at(x, w, coords, (1, 1), (pad, pad), -1)  # the definition, output by output
+    assert np.array_equal(g[coords[:, 0], coords[:, 2], coords[:, 3], coords[:, 1]], want)
+    # packed operands too, bit for bit
+    assert np.array_equal(u64(a), oracle_mod.pack(x))
+
+
+def test_full_size_pack_config(B, oracle_mod):
+    x = synth.pack_case(N=128, C=256, H=56, W=56)
+    assert abs(float((x == 0).mean()) - 0.01) < 1e-3
+    got = u64(B.pack(dev(x)))
+    assert got.shape == (128, 56, 56, 4)
+    assert np.array_equal(got, oracle_mod.pack(x))
+
+
+# ---- Bi-Real Net 18 ---------------------------------------------------------------------------------------------
+def test_bireal18_forward_matches_oracle(B, oracle_mod):
+    p = synth.bireal18_params()
+    img = synth.bireal18_images(3)
+    want, taps = oracle_mod.bireal18_forward(p, img, conv_form=1, want_taps=True)
+    net = B.Bireal18(p)
+    got = net.forward(dev(img)).cpu().numpy()
+    scale = np.max(np.abs(want))
+    assert np.max(np.abs(got - want)) <= 1e-3 * scale
+    assert np.array_equal(got.argmax(axis=1), want.argmax(axis=1))
+    # the pinned evaluation order makes the two sides agree to the last bit
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    # batch 1 gives the same logits for the same image
+    got1 = net.forward(dev(img[:1])).cpu().numpy()
+    assert np.array_equal(got1, got[:1])
