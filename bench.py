@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the binarized-convolution hot path on B200.
+
+One "step" is one pass of the whole path over one batch of synthetic input: for each of the four
+ResNet-18 stage shapes (C = 64/128/256/512 at 56/28/14/7 pixels, 3x3, stride 1, pad 1 with value -1)
+at batch 64: binarize + pack the fp32 activations, binary convolution with int32 output, and binary
+convolution with the fused BN + sign + re-pack epilogue.  The headline value is the convolutions'
+bit-operations (2 per bit pair) divided by the time of the whole step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
+
+Prints ONE JSON line (rank 0).  Under torchrun every rank runs the same per-GPU work on its own
+seeded batch (weak scaling, no data-path collective); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_1908_05858_b200 import synth  # noqa: E402
+
+BATCH = 64
+METRIC = "binary conv Gbit-ops/s"
+UNIT = "Gbit-ops/s"
+WORKLOAD = "binary 3x3 conv sweep, batch 64, (C,HW) in (64,56),(128,28),(256,14),(512,7): pack + bconv(int32) + bconv(bn,sign,pack)"
+
+
+def conv_bitops(N, C, HW, O, k):
+    return 2.0 * N * HW * HW * O * C * k * k
+
+
+def step_bitops(batch):
+    return sum(2 * conv_bitops(batch, C, HW, C, 3) for C, HW in synth.SWEEP_SHAPES)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+
+
+def bitop_peak_tbitops(sm_count, sm_mhz):
+    """Carry-save bound of sum popcount(a xor w) on the B200 integer pipes: with one POPC (XU pipe, 16 lanes/clk/SM)
+    and four logic ops (ALU pipe, 64 lanes/clk/SM) per two 32-bit word pairs both pipes are full at 32 word pairs
+    per clock per SM; 32 bit pairs per word pair, 2 bit-ops per bit pair."""
+    return sm_count * 32 * 32 * 2 * sm_mhz * 1e6 / 1e12
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        # samples under load: the top half of the clock samples (idle samples before/after are low)
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw), "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: each step is a bounded sample (batch 2 per shape) of the
+    workload, timed with the wall clock."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    cores = oracle.max_threads()
+    oracle.set_threads(cores)
+    nb = 2
+    cases = []
+    for C, HW in synth.SWEEP_SHAPES:
+        x, w = synth.conv_case(2, nb, C, HW, HW, C, 3, 3, salt=C)
+        scale, shift = oracle.bn_fold(*synth.bn_params(synth.rng(2, 900 + C), C))
+        cases.append((C, x, oracle.pack_weights(w), scale, shift))
+
+    def step():
+        for C, x, wp, scale, shift in cases:
+            a = oracle.pack(x)
+            oracle.bconv_bits(a, C, wp, (1, 1), (1, 1), -1)
+            acc = oracle.bconv_bits(a, C, wp, (1, 1), (1, 1), -1)
+            oracle.bn_sign_pack(acc, scale, shift)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = step_bitops(nb) * args.steps / dt / 1e9
+    sample = "batch %d of each of the four shapes per step (the workload's batch is %d)" % (nb, BATCH)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u64 words / int32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---------------------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the per-config extra measurements")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_1908_05858_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()
+    dev = torch.device("cuda", local)
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    peaks = measured_peaks()
+    warmup = max(args.warmup, 3)
+
+    # ---- inputs: seeded, drawn on the host, resident in HBM before the timed region ------------------------------
+    layers = []
+    for C, HW in synth.SWEEP_SHAPES:
+        x, w = synth.conv_case(2, BATCH, C, HW, HW, C, 3, 3, salt=C + 1000 * rank)
+        g = synth.rng(2, 900 + C)
+        bn = [torch.from_numpy(t).to(dev) for t in synth.bn_params(g, C)]
+        scale, shift = B.bn_fold(*bn)
+        xh = torch.from_numpy(x).pin_memory()
+        L = {
+            "C": C, "HW": HW, "x_host": xh, "x": xh.to(dev), "w": B.pack_weights(torch.from_numpy(w).to(dev)),
+            "scale": scale, "shift": shift,
+            "a": torch.empty((BATCH, HW, HW, (C + 63) // 64), dtype=torch.int64, device=dev),
+            "out": torch.empty((BATCH, HW, HW, C), dtype=torch.int32, device=dev),
+            "bits": torch.empty((BATCH, HW, HW, (C + 63) // 64), dtype=torch.int64, device=dev),
+            "bitops": conv_bitops(BATCH, C, HW, C, 3),
+        }
+        L["out_host"] = torch.empty(L["out"].shape, dtype=torch.int32).pin_memory()
+        L["bits_host"] = torch.empty(L["bits"].shape, dtype=torch.int64).pin_memory()
+        ws_bytes = B.binary_layer_host_workspace_bytes(BATCH, C, HW, HW, C, 3, 3, (1, 1), (1, 1), -1)
+        L["ws"] = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        layers.append(L)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)  # larger than the 126 MB L2
+
+    conv_events = []  # (start, end, bitops) of every convolution launch in the timed region
+
+    def step(record):
+        for L in layers:
+            B.pack(L["x"], B.NCHW, out=L["a"])
+            for fused in (False, True):
+                if record:
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                if fused:
+                    B.bconv2d_bn_sign_pack(L["a"], L["C"], L["w"], L["scale"], L["shift"], (1, 1), (1, 1), -1, out=L["bits"])
+                else:
+                    B.bconv2d(L["a"], L["C"], L["w"], (1, 1), (1, 1), -1, B.NHWC, out=L["out"])
+                if record:
+                    e1.record()
+                    conv_events.append((e0, e1, L["bitops"], fused))
+    launches_per_step = 3 * len(layers)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        step(False)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    barrier()
+    for k in range(args.steps):
+        flush.zero_()  # evict the previous step's data from L2 (outside the step's event pair)
+        starts[k].record()
+        step(True)
+        ends[k].record()
+    barrier()
+    clocks = sampler.stop()
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
+    total_ms = float(total_ms.item())
+    value = world * step_bitops(BATCH) * args.steps / (total_ms * 1e-3) / 1e9
+
+    # dominant kernel: the convolution launches, timed one by one inside the timed region
+    conv_ms = sum(e0.elapsed_time(e1) for e0, e1, _, _ in conv_events)
+    conv_ops = sum(b for _, _, b, _ in conv_events)
+    achieved = conv_ops / (conv_ms * 1e-3) / 1e12
+    peak = bitop_peak_tbitops(sm_count, peaks["sm_max_mhz"])
+    roofline = {
+        "bound": "alu", "kernel": "bconv_kernel (all 8 launches of a step)", "achieved": achieved, "peak": peak,
+        "unit": "Tbit-ops/s", "frac": achieved / peak,
+        "peak_is": "ALU+XU carry-save bound at %d SMs x %.0f MHz (derived, see DESIGN.md); one-POPC-per-word-pair bound is half of it"
+                   % (sm_count, peaks["sm_max_mhz"]),
+        "traffic": None, "avg_launch_ms": conv_ms / max(1, len(conv_events)),
+        "conv_share_of_step": conv_ms / sum(step_ms),
+    }
+
+    # ---- end to end through the host-buffer entry point ----------------------------------------------------------
+    def e2e_step():
+        for L in layers:
+            B.binary_layer_host(L["x_host"], L["w"], L["ws"], (1, 1), (1, 1), -1, L["scale"], L["shift"],
+                                out_host=L["out_host"], bits_host=L["bits_host"])
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e = {
+        "value": world * step_bitops(BATCH) * e2e_steps / (float(e2e_ms.item()) * 1e-3) / 1e9, "unit": UNIT,
+        "h2d_bytes_per_step": int(sum(L["x_host"].numel() * 4 for L in layers)),
+        "d2h_bytes_per_step": int(sum(L["out_host"].numel() * 4 + L["bits_host"].numel() * 8 for L in layers)),
+        "steps": e2e_steps, "api": "dabnn_binary_layer_host (pinned host buffers in and out)",
+    }
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u64 words / int32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "l2": "flushed between timed steps (256 MB write)",
+                   "parallelism": "replicas" if world > 1 else "single GPU"},
+        "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+    }
+
+    if rank == 0 and world == 1:
+        if not args.no_cpu_baseline:
+            result["cpu_baseline"] = cpu_baseline()
+        if not args.no_extras:
+            result["extras"] = extras(B, torch, dev, peaks, sm_count)
+    if rank == 0:
+        print(json.dumps(result))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline():
+    """The oracle on the host cores, on a bounded sample of the same workload: whole steps at batch 32
+    (half the workload's batch), repeated until about 10 s of wall time have passed."""
+    import oracle
+    cores = oracle.max_threads()
+    oracle.set_threads(cores)
+    nb = 32
+    cases = []
+    for C, HW in synth.SWEEP_SHAPES:
+        x, w = synth.conv_case(2, nb, C, HW, HW, C, 3, 3, salt=C)
+        scale, shift = oracle.bn_fold(*synth.bn_params(synth.rng(2, 900 + C), C))
+        cases.append((C, x, oracle.pack_weights(w), scale, shift))
+    t, reps = 0.0, 0
+    while t < 10.0 and reps < 50:
+        t0 = time.perf_counter()
+        for C, x, wp, scale, shift in cases:
+            a = oracle.pack(x)
+            oracle.bconv_bits(a, C, wp, (1, 1), (1, 1), -1)
+            acc = oracle.bconv_bits(a, C, wp, (1, 1), (1, 1), -1)
+            oracle.bn_sign_pack(acc, scale, shift)
+        t += time.perf_counter() - t0
+        reps += 1
+    return {"value": step_bitops(nb) * reps / t / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d steps at batch %d instead of %d (%.1f s of wall time on %d threads)" % (reps, nb, BATCH, t, cores)}
+
+
+def extras(B, torch, dev, peaks, sm_count):
+    """Per-configuration measurements beside the headline (each a few launches; CUDA events)."""
+    out = {}
+
+    def time_fn(fn, iters, flush=None):
+        fn(); fn(); fn()
+        torch.cuda.synchronize()
+        ms = []
+        for _ in range(iters):
+            if flush is not None:
+                flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+        return statistics.median(ms), min(ms)
+
+    # bit-pack alone: fp32 NCHW 128x256x56x56 with ~1 % exact zeros (input 411 MB: cold by construction)
+    x = torch.from_numpy(synth.pack_case()).to(dev)
+    packed = torch.empty((128, 56, 56, 4), dtype=torch.int64, device=dev)
+    med, best = time_fn(lambda: B.pack(x, B.NCHW, out=packed), 10)
+    nbytes = x.numel() * 4 + packed.numel() * 8
+    out["pack_128x256x56x56"] = {"ms": med, "GB/s": nbytes / med / 1e6, "frac_of_hbm_peak": nbytes / med / 1e6 / peaks["hbm_gbs"],
+                                 "peak_GB/s": peaks["hbm_gbs"], "peak_source": peaks["source"], "bytes": nbytes}
+    del x, packed
+
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    peak = bitop_peak_tbitops(sm_count, peaks["sm_max_mhz"])
+    for name, (N, C, HW, O, k, pad) in {"conv_256x256x28x28_3x3": (256, 256, 28, 256, 3, 1),
+                                        "conv_256x512x14x14_1x1_to_2048": (256, 512, 14, 2048, 1, 0)}.items():
+        g = torch.Generator(device=dev); g.manual_seed(5)
+        a = torch.randint(-2**62, 2**62, (N, HW, HW, (C + 63) // 64), dtype=torch.int64, device=dev, generator=g)
+        w = torch.randint(-2**62, 2**62, (O, k, k, (C + 63) // 64), dtype=torch.int64, device=dev, generator=g)
+        o = torch.empty((N, HW, HW, O), dtype=torch.int32, device=dev)
+        med, best = time_fn(lambda: B.bconv2d(a, C, w, (1, 1), (pad, pad), -1, B.NHWC, out=o), 10, flush)
+        ops = conv_bitops(N, C, HW, O, k)
+        out[name] = {"ms": med, "Tbit-ops/s": ops / med / 1e9, "frac_of_bitop_peak": ops / med / 1e9 / peak}
+        del a, w, o
+
+    # batch-1 latency of the four sweep shapes (CUDA-graph replay of 50 launches)
+    for C, HW in synth.SWEEP_SHAPES:
+        g = torch.Generator(device=dev); g.manual_seed(7)
+        a = torch.randint(-2**62, 2**62, (1, HW, HW, C // 64), dtype=torch.int64, device=dev, generator=g)
+        w = torch.randint(-2**62, 2**62, (C, 3, 3, C // 64), dtype=torch.int64, device=dev, generator=g)
+        o = torch.empty((1, HW, HW, C), dtype=torch.int32, device=dev)
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            for _ in range(3):
+                B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC, out=o)
+            s.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=s):
+                for _ in range(50):
+                    B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC, out=o)
+            med, best = time_fn(graph.replay, 5)
+        out["conv_batch1_C%d_%dx%d" % (C, HW, HW)] = {"us_per_conv": med * 1e3 / 50, "Tbit-ops/s": conv_bitops(1, C, HW, C, 3) / (med / 50) / 1e9}
+
+    # Bi-Real Net 18: batch 128 (eager launches) and batch 1 (CUDA-graph replay)
+    net = B.Bireal18(synth.bireal18_params())
+    img = torch.from_numpy(synth.bireal18_images(128)).to(dev)
+    logits = torch.empty((128, 1000), dtype=torch.float32, device=dev)
+    med, best = time_fn(lambda: net.forward(img, logits), 5)
+    out["bireal18_batch128"] = {"ms": med, "images/s": 128 / med * 1e3}
+    img1, logits1 = img[:1].contiguous(), torch.empty((1, 1000), dtype=torch.float32, device=dev)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        for _ in range(3):
+            net.forward(img1, logits1)
+        s.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            net.forward(img1, logits1)
+        med, best = time_fn(graph.replay, 20)
+    out["bireal18_batch1"] = {"ms": med, "images/s": 1e3 / med, "launch": "CUDA graph replay of the 22 kernels"}
+    return out
+
+
+if __name__ == "__main__":
+    main()

@@ -122,6 +122,19 @@ size_t dabnn_bireal18_workspace_bytes(int N);
 dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float* images, int N, float* logits,
                                     void* workspace, size_t workspace_bytes, void* stream);
 
+/* One binary layer with HOST buffers (Section 2.1.1 + 2.1.2 end to end): copies x_host (fp32 NCHW, in.N*in.C*in.H*in.W
+ * elements; pinned memory makes the copies asynchronous) to the device, packs it, and then
+ *   - if out_host  != NULL: runs dabnn_bconv2d and copies the int32 NHWC result [N][OH][OW][O] to out_host;
+ *   - if bits_host != NULL: runs dabnn_bconv2d_bn_sign_pack (scale, shift: DEVICE, required then) and copies the
+ *     packed result [N][OH][OW][ceil(O/64)] to bits_host.
+ * w_packed, scale, shift and workspace are DEVICE pointers; workspace must be 256-byte aligned and hold at least
+ * dabnn_binary_layer_host_workspace_bytes(in, O, cv) bytes (0 is returned for an invalid geometry).
+ * Everything is enqueued on `stream`; the host results are complete once the stream has been synchronised. */
+size_t dabnn_binary_layer_host_workspace_bytes(dabnn_shape in, int O, dabnn_conv cv);
+dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const uint64_t* w_packed, int O, dabnn_conv cv,
+                                     const float* scale, const float* shift, int32_t* out_host, uint64_t* bits_host,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
 /* Selects the convolution inner loop for measurement runs: 0 = automatic (default),
  * 1 = one POPC per 32-bit word pair, 2 = carry-save (one POPC per two word pairs).  All give identical results.
  * Returns the previous setting.  Not thread-safe against concurrent calls into the library. */

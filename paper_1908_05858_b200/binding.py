@@ -25,6 +25,7 @@ EXPORTS = (
     "dabnn_status_string", "dabnn_words_per_pixel", "dabnn_out_dim", "dabnn_pack", "dabnn_pack_weights",
     "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack", "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold",
     "dabnn_bireal18_workspace_bytes", "dabnn_bireal18_forward", "dabnn_set_conv_variant",
+    "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host",
 )
 
 
@@ -77,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.dabnn_bireal18_workspace_bytes.restype = ctypes.c_size_t
         L.dabnn_bireal18_workspace_bytes.argtypes = [ci]
         L.dabnn_bireal18_forward.argtypes = [ctypes.POINTER(Bireal18Params), vp, ci, vp, vp, ctypes.c_size_t, vp]
+        L.dabnn_binary_layer_host_workspace_bytes.restype = ctypes.c_size_t
+        L.dabnn_binary_layer_host_workspace_bytes.argtypes = [Shape, ci, Conv]
+        L.dabnn_binary_layer_host.argtypes = [vp, Shape, vp, ci, Conv, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.dabnn_binary_layer_host.restype = ci
         L.dabnn_set_conv_variant.restype = ci
         L.dabnn_set_conv_variant.argtypes = [ci]
         for name in ("dabnn_pack", "dabnn_pack_weights", "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack",
@@ -257,6 +262,30 @@ class Bireal18:
         _check(lib().dabnn_bireal18_forward(ctypes.byref(self.P), images.data_ptr(), N, logits.data_ptr(),
                                             ws.data_ptr(), ws.numel(), _stream()))
         return logits
+
+
+def binary_layer_host_workspace_bytes(N, C, H, W, O, kh, kw, stride=(1, 1), pad=(0, 0), pad_value=-1) -> int:
+    return int(lib().dabnn_binary_layer_host_workspace_bytes(Shape(N, C, H, W), O, _conv(kh, kw, stride, pad, pad_value)))
+
+
+def binary_layer_host(x_host: torch.Tensor, w_packed: torch.Tensor, workspace: torch.Tensor, stride=(1, 1), pad=(0, 0),
+                      pad_value: int = -1, scale=None, shift=None, out_host: Optional[torch.Tensor] = None,
+                      bits_host: Optional[torch.Tensor] = None):
+    """dabnn_binary_layer_host: x_host / out_host / bits_host are HOST tensors (pin them for asynchronous
+    copies); w_packed, scale, shift, workspace are device tensors.  Work is enqueued on the current stream."""
+    if x_host.is_cuda or x_host.dtype != torch.float32 or not x_host.is_contiguous():
+        raise DabnnError("x_host must be a contiguous fp32 host tensor")
+    w = _dev(w_packed, torch.int64, "w_packed")
+    N, C, H, W = x_host.shape
+    O, kh, kw, _ = w.shape
+    for t, dt in ((out_host, torch.int32), (bits_host, torch.int64)):
+        if t is not None and (t.is_cuda or t.dtype != dt or not t.is_contiguous()):
+            raise DabnnError("host outputs must be contiguous host tensors of the right dtype")
+    _check(lib().dabnn_binary_layer_host(
+        x_host.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O, _conv(kh, kw, stride, pad, pad_value),
+        scale.data_ptr() if scale is not None else None, shift.data_ptr() if shift is not None else None,
+        out_host.data_ptr() if out_host is not None else None, bits_host.data_ptr() if bits_host is not None else None,
+        workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()))
 
 
 def set_conv_variant(variant: int) -> int:
