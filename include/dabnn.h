@@ -44,7 +44,8 @@ typedef enum {
   DABNN_ERR_UNSUPPORTED = 3, /* a size beyond what the index arithmetic supports (>= 2^31 elements per axis product) */
   DABNN_ERR_ALIGNMENT = 4,
   DABNN_ERR_WORKSPACE = 5,   /* workspace too small */
-  DABNN_ERR_CUDA = 6         /* the CUDA runtime reported an error at launch */
+  DABNN_ERR_CUDA = 6,        /* the CUDA runtime reported an error at launch */
+  DABNN_ERR_STATIC_LIMIT = 7 /* the request is larger than the library's built-in scratch area */
 } dabnn_status;
 
 typedef enum { DABNN_NCHW = 0, DABNN_NHWC = 1 } dabnn_layout;
@@ -121,6 +122,27 @@ size_t dabnn_bireal18_workspace_bytes(int N);
  * are scratch (activations between layers) and are undefined afterwards. */
 dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float* images, int N, float* logits,
                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* (No counterpart in the paper: a packaging convenience of this library.)
+ * dabnn_bireal18_forward for callers that must not allocate device memory.  Some hosts of this library cannot call
+ * cudaMalloc: a plug-in inside a server whose framework has reserved the whole device for its own pool, a
+ * latency-critical loop that may not take cudaMalloc's implicit device synchronisation, or code running where any
+ * allocation is forbidden by policy.  For them the activations between layers live in a scratch area that is part
+ * of the library image itself, so the caller passes only inputs and outputs.
+ *   - Limit: N <= DABNN_STATIC_MAX_BATCH images per call; a larger N returns DABNN_ERR_STATIC_LIMIT and nothing runs.
+ *   - Cost: the scratch area (DABNN_STATIC_SCRATCH_BYTES, about 8.5 MiB) is reserved on every GPU on which the
+ *     library is loaded, from load until the process exits, whether or not this entry point is ever called.
+ *   - The first call on each device looks up the area's device address (no allocation, but a runtime query);
+ *     make that first call outside any stream capture.  Later calls on that device reuse the address.
+ *   - The call itself performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ *   - All calls share the one area and it keeps whatever the previous call left in it.  Nothing in it has to start
+ *     at zero (every region is fully written before it is read), so no clearing is done.  Two calls whose work
+ *     overlaps on the GPU (different streams, or different threads) race on the area: serialise them.
+ * Arguments and results are otherwise exactly those of dabnn_bireal18_forward. */
+#define DABNN_STATIC_MAX_BATCH 2
+#define DABNN_STATIC_SCRATCH_BYTES 8931328
+dabnn_status dabnn_bireal18_forward_static(const dabnn_bireal18_params* p, const float* images, int N, float* logits,
+                                           void* stream);
 
 /* One binary layer with HOST buffers (Section 2.1.1 + 2.1.2 end to end): copies x_host (fp32 NCHW, in.N*in.C*in.H*in.W
  * elements; pinned memory makes the copies asynchronous) to the device, packs it, and then

@@ -25,7 +25,7 @@ EXPORTS = (
     "dabnn_status_string", "dabnn_words_per_pixel", "dabnn_out_dim", "dabnn_pack", "dabnn_pack_weights",
     "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack", "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold",
     "dabnn_bireal18_workspace_bytes", "dabnn_bireal18_forward", "dabnn_set_conv_variant",
-    "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host",
+    "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host", "dabnn_bireal18_forward_static",
 )
 
 
@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.dabnn_binary_layer_host.restype = ci
         L.dabnn_set_conv_variant.restype = ci
         L.dabnn_set_conv_variant.argtypes = [ci]
+        L.dabnn_bireal18_forward_static.restype = ci
+        L.dabnn_bireal18_forward_static.argtypes = [ctypes.POINTER(Bireal18Params), vp, ci, vp, vp]
         for name in ("dabnn_pack", "dabnn_pack_weights", "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack",
                      "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold", "dabnn_bireal18_forward"):
             getattr(L, name).restype = ci
@@ -286,6 +288,23 @@ def binary_layer_host(x_host: torch.Tensor, w_packed: torch.Tensor, workspace: t
         scale.data_ptr() if scale is not None else None, shift.data_ptr() if shift is not None else None,
         out_host.data_ptr() if out_host is not None else None, bits_host.data_ptr() if bits_host is not None else None,
         workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()))
+
+
+STATIC_MAX_BATCH = 2
+
+
+def bireal18_forward_static(net: "Bireal18", images: torch.Tensor, logits: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_bireal18_forward_static: the same forward pass for callers that may not allocate device memory
+    (the library's built-in scratch area replaces the workspace; at most STATIC_MAX_BATCH images per call).
+    Only `logits` is allocated here, by torch, when the caller does not pass it."""
+    images = _dev(images, torch.float32, "images")
+    N = images.shape[0]
+    if tuple(images.shape[1:]) != (3, 224, 224):
+        raise DabnnError("images must be [N][3][224][224]")
+    if logits is None:
+        logits = torch.empty((N, 1000), dtype=torch.float32, device=images.device)
+    _check(lib().dabnn_bireal18_forward_static(ctypes.byref(net.P), images.data_ptr(), N, logits.data_ptr(), _stream()))
+    return logits
 
 
 def set_conv_variant(variant: int) -> int:

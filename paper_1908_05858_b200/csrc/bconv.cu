@@ -444,6 +444,7 @@ extern "C" const char* dabnn_status_string(dabnn_status s) {
     case DABNN_ERR_ALIGNMENT: return "misaligned pointer";
     case DABNN_ERR_WORKSPACE: return "workspace too small";
     case DABNN_ERR_CUDA: return "CUDA launch error";
+    case DABNN_ERR_STATIC_LIMIT: return "request exceeds the library's built-in scratch area (see DABNN_STATIC_MAX_BATCH)";
   }
   return "unknown status";
 }

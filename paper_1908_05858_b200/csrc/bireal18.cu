@@ -5,6 +5,8 @@
 // operations in a fixed order (explicit fmaf chains, ascending channel / tap order), never by tensor
 // cores or split sums, because the next binary layer takes the SIGN of these values: a different
 // rounding order could flip a bit and change integer results downstream.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace dabnn {
@@ -337,4 +339,42 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
   }
   gap_fc<<<dim3(4, N), 256, 0, st>>>(cur, p->fc_w, p->fc_b, logits);
   return launch_status();
+}
+
+// ---- allocation-free variant ---------------------------------------------------------------------------
+// Scratch for dabnn_bireal18_forward_static: part of the library image, present on every device that loads
+// it.  In host code the symbol below is only a handle; its device address is looked up per device.
+static __device__ __align__(256) unsigned char g_static_scratch[DABNN_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_addr[kMaxDevices] = {};  // device address of g_static_scratch, per device ordinal
+}  // namespace
+
+extern "C" dabnn_status dabnn_bireal18_forward_static(const dabnn_bireal18_params* p, const float* images, int N,
+                                                      float* logits, void* stream) {
+  if (N > DABNN_STATIC_MAX_BATCH) return DABNN_ERR_STATIC_LIMIT;
+  if (N <= 0) return DABNN_ERR_SHAPE;
+  if (dabnn_bireal18_workspace_bytes(N) > (size_t)DABNN_STATIC_SCRATCH_BYTES) return DABNN_ERR_STATIC_LIMIT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return DABNN_ERR_CUDA;
+  }
+  if (dev < 0 || dev >= kMaxDevices) return DABNN_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    scratch = g_static_addr[dev];
+    if (scratch == nullptr) {
+      // once per device, with that device current: the symbol's address in this device's memory
+      if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess || scratch == nullptr) {
+        cudaGetLastError();
+        return DABNN_ERR_CUDA;
+      }
+      g_static_addr[dev] = scratch;
+    }
+  }
+  return dabnn_bireal18_forward(p, images, N, logits, scratch, (size_t)DABNN_STATIC_SCRATCH_BYTES, stream);
 }
