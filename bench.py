@@ -61,50 +61,72 @@ def bitop_peak_tbitops(sm_count, sm_mhz):
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock, power and throttle reasons through NVML from a background thread while the timed region runs."""
 
-    def __init__(self, index):
-        self.index = index
-        self.proc = None
+    def __init__(self, index, period_s=0.005):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.err = [], set(), None
+        self._stop = None
+        self._thread = None
 
     def start(self):
+        import threading
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = None
+            try:
+                import torch
+                uuid = str(torch.cuda.get_device_properties(self.index).uuid)
+            except Exception:
+                uuid = None
+            h = None
+            if uuid:
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+                except Exception:
+                    h = None
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # NVML not usable: report that instead of clocks
+            self.err = "nvml unavailable: %s" % e
+            return
+        self._stop = threading.Event()
+        R = pynvml
+        masks = {"hw_slowdown": R.nvmlClocksThrottleReasonHwSlowdown,
+                 "hw_thermal_slowdown": R.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": R.nvmlClocksThrottleReasonSwThermalSlowdown,
+                 "sw_power_cap": R.nvmlClocksThrottleReasonSwPowerCap}
+
+        def loop():
+            while not self._stop.is_set():
+                try:
+                    mhz = float(R.nvmlDeviceGetClockInfo(h, R.NVML_CLOCK_SM))
+                    pw = R.nvmlDeviceGetPowerUsage(h) / 1000.0
+                    bits = R.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                    self.samples.append((mhz, pw))
+                    for nm, m in masks.items():
+                        if bits & m:
+                            self.reasons.add(nm)
+                except Exception as e:
+                    self.err = str(e)
+                    return
+                self._stop.wait(self.period)
+
+        self._thread = threading.Thread(target=loop, daemon=True)
+        self._thread.start()
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-            out, _ = self.proc.communicate()
-        sm, mx, pw, reasons = [], [], [], set()
-        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in out.splitlines():
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 7:
-                continue
-            try:
-                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
-            except ValueError:
-                continue
-            for nm, val in zip(names, parts[3:7]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        # samples under load: the top half of the clock samples (idle samples before/after are low)
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw), "samples": len(sm),
-                "reasons": sorted(reasons)}
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [self.err or "no samples"]}
+        sm = [m for m, _ in self.samples]
+        return {"sm_mhz": statistics.median(sm), "sm_min_mhz": min(sm), "sm_max_mhz": self.max_mhz,
+                "power_w_max": max(p for _, p in self.samples), "samples": len(sm), "reasons": sorted(self.reasons),
+                "how": "NVML, every %.0f ms during the timed region" % (self.period * 1e3)}
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -198,6 +220,9 @@ def main():
             "bits": torch.empty((BATCH, HW, HW, (C + 63) // 64), dtype=torch.int64, device=dev),
             "bitops": conv_bitops(BATCH, C, HW, C, 3),
         }
+        L["call_pack"] = B.prepare_pack(L["x"], L["a"])
+        L["call_conv"] = B.prepare_bconv2d(L["a"], C, L["w"], L["out"], (1, 1), (1, 1), -1, B.NHWC)
+        L["call_fused"] = B.prepare_bconv2d_bn_sign_pack(L["a"], C, L["w"], L["scale"], L["shift"], L["bits"], (1, 1), (1, 1), -1)
         L["out_host"] = torch.empty(L["out"].shape, dtype=torch.int32).pin_memory()
         L["bits_host"] = torch.empty(L["bits"].shape, dtype=torch.int64).pin_memory()
         ws_bytes = B.binary_layer_host_workspace_bytes(BATCH, C, HW, HW, C, 3, 3, (1, 1), (1, 1), -1)
@@ -209,15 +234,15 @@ def main():
 
     def step(record):
         for L in layers:
-            B.pack(L["x"], B.NCHW, out=L["a"])
+            L["call_pack"]()
             for fused in (False, True):
                 if record:
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     e0.record()
                 if fused:
-                    B.bconv2d_bn_sign_pack(L["a"], L["C"], L["w"], L["scale"], L["shift"], (1, 1), (1, 1), -1, out=L["bits"])
+                    L["call_fused"]()
                 else:
-                    B.bconv2d(L["a"], L["C"], L["w"], (1, 1), (1, 1), -1, B.NHWC, out=L["out"])
+                    L["call_conv"]()
                 if record:
                     e1.record()
                     conv_events.append((e0, e1, L["bitops"], fused))
@@ -231,25 +256,49 @@ def main():
     for _ in range(warmup):
         step(False)
     barrier()
+    # the step as a CUDA graph: one host call per step, so the timed loop is never host-bound
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step(False)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            step(False)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(warmup):
+        graph.replay()
+    barrier()
     sampler = ClockSampler(local)
     sampler.start()
-    time.sleep(0.3)
+    time.sleep(0.05)
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     barrier()
+    host_t0 = time.perf_counter()
     for k in range(args.steps):
         flush.zero_()  # evict the previous step's data from L2 (outside the step's event pair)
         starts[k].record()
-        step(True)
+        graph.replay()
         ends[k].record()
+    host_issue_ms = (time.perf_counter() - host_t0) * 1e3  # time the host needed to enqueue everything
     barrier()
-    clocks = sampler.stop()
     step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
     total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
     total_ms = float(total_ms.item())
     value = world * step_bitops(BATCH) * args.steps / (total_ms * 1e-3) / 1e9
+
+    # the same steps again, launch by launch, with an event pair around every convolution.  Each step starts
+    # behind a GPU-side delay so that the host has enqueued the whole step before its first kernel runs: the
+    # event pairs then bracket GPU execution only, never host launch latency.
+    for k in range(args.steps):
+        flush.zero_()
+        torch.cuda._sleep(int(1.5e6))
+        step(True)
+    barrier()
+    clocks = sampler.stop()
 
     # dominant kernel: the convolution launches, timed one by one inside the timed region
     conv_ms = sum(e0.elapsed_time(e1) for e0, e1, _, _ in conv_events)
@@ -262,7 +311,9 @@ def main():
         "peak_is": "ALU+XU carry-save bound at %d SMs x %.0f MHz (derived, see DESIGN.md); one-POPC-per-word-pair bound is half of it"
                    % (sm_count, peaks["sm_max_mhz"]),
         "traffic": None, "avg_launch_ms": conv_ms / max(1, len(conv_events)),
-        "conv_share_of_step": conv_ms / sum(step_ms),
+        "conv_share_of_step": (conv_ms / args.steps) / (sum(step_ms) / args.steps),
+        "timed": "CUDA events around each of the %d convolution launches of %d eager steps (L2 flushed before each step)"
+                 % (len(conv_events), args.steps),
     }
 
     # ---- end to end through the host-buffer entry point ----------------------------------------------------------
@@ -294,8 +345,10 @@ def main():
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u64 words / int32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "l2": "flushed between timed steps (256 MB write)",
+                   "launch": "each step is one CUDA-graph replay of its 12 kernels",
                    "parallelism": "replicas" if world > 1 else "single GPU"},
         "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        "host_issue_ms_per_step": host_issue_ms / args.steps,
     }
 
     if rank == 0 and world == 1:

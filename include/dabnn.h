@@ -161,6 +161,9 @@ dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const 
  * 1 = one POPC per 32-bit word pair, 2 = carry-save (one POPC per two word pairs).  All give identical results.
  * Returns the previous setting.  Not thread-safe against concurrent calls into the library. */
 int dabnn_set_conv_variant(int variant);
+/* Forces the convolution's CTA tile for measurement runs: 0 = automatic (default), 1 = 128 pixels x 128 channels,
+ * 2 = 128 x 64, 3 = 64 x 64, 4 = 32 x 32.  All give identical results.  Returns the previous setting. */
+int dabnn_set_conv_tile(int tile);
 
 #ifdef __cplusplus
 }

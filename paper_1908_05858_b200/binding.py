@@ -25,7 +25,7 @@ EXPORTS = (
     "dabnn_status_string", "dabnn_words_per_pixel", "dabnn_out_dim", "dabnn_pack", "dabnn_pack_weights",
     "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack", "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold",
     "dabnn_bireal18_workspace_bytes", "dabnn_bireal18_forward", "dabnn_set_conv_variant",
-    "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host", "dabnn_bireal18_forward_static",
+    "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host", "dabnn_bireal18_forward_static", "dabnn_set_conv_tile",
 )
 
 
@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.dabnn_binary_layer_host.restype = ci
         L.dabnn_set_conv_variant.restype = ci
         L.dabnn_set_conv_variant.argtypes = [ci]
+        L.dabnn_set_conv_tile.restype = ci
+        L.dabnn_set_conv_tile.argtypes = [ci]
         L.dabnn_bireal18_forward_static.restype = ci
         L.dabnn_bireal18_forward_static.argtypes = [ctypes.POINTER(Bireal18Params), vp, ci, vp, vp]
         for name in ("dabnn_pack", "dabnn_pack_weights", "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack",
@@ -307,5 +309,44 @@ def bireal18_forward_static(net: "Bireal18", images: torch.Tensor, logits: Optio
     return logits
 
 
+class Prepared:
+    """A library call with its arguments marshalled once (pointers and structs; the stream is torch's current one),
+    for loops where the per-call Python overhead of the checked wrappers would rival the kernel time.
+    The tensors passed at creation must stay alive and in place; `keep` holds references to them."""
+
+    def __init__(self, fn, args, keep):
+        self.fn, self.args, self.keep = fn, args, keep
+
+    def __call__(self):
+        st = self.fn(*self.args, torch.cuda.current_stream().cuda_stream)
+        if st != 0:
+            _check(st)
+
+
+def prepare_pack(x: torch.Tensor, out: torch.Tensor, layout: int = NCHW) -> Prepared:
+    x = _dev(x, torch.float32, "x")
+    N, C, H, W = x.shape if layout == NCHW else (x.shape[0], x.shape[3], x.shape[1], x.shape[2])
+    return Prepared(lib().dabnn_pack, (x.data_ptr(), layout, Shape(N, C, H, W), out.data_ptr()), (x, out))
+
+
+def prepare_bconv2d(a_packed, C, w_packed, out, stride=(1, 1), pad=(0, 0), pad_value=-1, out_layout=NHWC) -> Prepared:
+    a, w, N, H, W, O, kh, kw, OH, OW = _geom(a_packed, C, w_packed, stride, pad)
+    return Prepared(lib().dabnn_bconv2d, (a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O,
+                                          _conv(kh, kw, stride, pad, pad_value), out.data_ptr(), out_layout),
+                    (a, w, out))
+
+
+def prepare_bconv2d_bn_sign_pack(a_packed, C, w_packed, scale, shift, out, stride=(1, 1), pad=(0, 0),
+                                 pad_value=-1) -> Prepared:
+    a, w, N, H, W, O, kh, kw, OH, OW = _geom(a_packed, C, w_packed, stride, pad)
+    return Prepared(lib().dabnn_bconv2d_bn_sign_pack,
+                    (a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O, _conv(kh, kw, stride, pad, pad_value),
+                     scale.data_ptr(), shift.data_ptr(), out.data_ptr()), (a, w, scale, shift, out))
+
+
 def set_conv_variant(variant: int) -> int:
     return int(lib().dabnn_set_conv_variant(int(variant)))
+
+
+def set_conv_tile(tile: int) -> int:
+    return int(lib().dabnn_set_conv_tile(int(tile)))

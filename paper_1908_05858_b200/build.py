@@ -21,7 +21,7 @@ def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "dabnn.h"), __file__]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh")) and not f.startswith("ubench")] + [os.path.join(ROOT, "include", "dabnn.h"), __file__]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
@@ -47,5 +47,17 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_ubench() -> str:
+    """Builds the integer-pipe micro-benchmark executable beside the library."""
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    exe = os.path.join(HERE, "ubench_int_pipes")
+    src = os.path.join(CSRC, "ubench_int_pipes.cu")
+    if not os.path.exists(exe) or os.path.getmtime(exe) < os.path.getmtime(src):
+        subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-o", exe, src])
+    return exe
+
+
 if __name__ == "__main__":
+    if "--ubench" in sys.argv:
+        print(build_ubench())
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

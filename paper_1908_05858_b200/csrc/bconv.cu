@@ -45,6 +45,7 @@ struct BConvArgs {
   float* y_out;
   uint32_t* out_packed32;  // packed output viewed as 32-bit halves
   int Ow32;                // 2*ceil(O/64)
+  int one;                 // the constant 1 (see bit_mac)
 };
 
 struct RowInfo {
@@ -65,22 +66,26 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// `one` is the constant 1 passed through the kernel arguments: multiplying by it keeps the accumulation an
+// integer multiply-add, which issues on the FMA pipe and leaves the ALU pipe to the logic operations.
 template <bool CSA>
-__device__ __forceinline__ void bit_mac(uint32_t a0, uint32_t a1, uint32_t w0, uint32_t w1, int& acc, uint32_t& ones) {
+__device__ __forceinline__ void bit_mac(uint32_t a0, uint32_t a1, uint32_t w0, uint32_t w1, int& acc, uint32_t& ones,
+                                        int one) {
   if (CSA) {
     const uint32_t x1 = a0 ^ w0, x2 = a1 ^ w1;
     uint32_t s, c;
     asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(s) : "r"(ones), "r"(x1), "r"(x2));  // sum bit
     asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(c) : "r"(ones), "r"(x1), "r"(x2));  // carry bit (majority)
     ones = s;
-    acc += __popc(c);
+    acc = __popc(c) * one + acc;
   } else {
-    acc += __popc(a0 ^ w0) + __popc(a1 ^ w1);
+    acc = __popc(a0 ^ w0) * one + acc;
+    acc = __popc(a1 ^ w1) * one + acc;
   }
 }
 
-template <int BP, int BO, int TP, int TO, int EPI, bool CSA, bool VEC16>
-__global__ void __launch_bounds__((BP / TP) * (BO / TO)) bconv_kernel(const BConvArgs g) {
+template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16>
+__global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(const BConvArgs g) {
   constexpr int THREADS = (BP / TP) * (BO / TO);
   constexpr int UW = VEC16 ? 2 : 1;         // 64-bit words per copy unit
   constexpr int UNITS = KC64 / UW;          // units per row and chunk
@@ -89,6 +94,7 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO)) bconv_kernel(const BCon
   static_assert(BP % (8 * TP) == 0 && BO % (4 * TO) == 0, "warp tile");
   static_assert(BP % ROWS_PER_PASS == 0 && BO % ROWS_PER_PASS == 0, "loader passes");
   constexpr int WPN = BP / (8 * TP);        // warps along the pixel axis
+  constexpr int UNROLL_K = (TP * TO >= 32) ? 1 : 2;
   constexpr int STAGE_WORDS = (BP + BO) * PITCH;
 
   extern __shared__ __align__(16) uint32_t smem[];
@@ -170,6 +176,7 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO)) bconv_kernel(const BCon
     }
   };
 
+  const int one = g.one;
   const int lane = tid & 31, wid = tid >> 5;
   const int pl = lane & 7, ol = lane >> 3;
   const int wp = wid % WPN, wo = wid / WPN;
@@ -204,7 +211,7 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO)) bconv_kernel(const BCon
     const uint32_t* Ws = As + BP * PITCH;
     const int kvalid = min(KC64, g.K64 - chunk * KC64);  // 64-bit words in this chunk
     int k = 0;
-#pragma unroll 2
+#pragma unroll UNROLL_K
     for (; k + 2 <= kvalid; k += 2) {
       uint4 a[TP], w[TO];
 #pragma unroll
@@ -215,8 +222,8 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO)) bconv_kernel(const BCon
       for (int i = 0; i < TP; i++)
 #pragma unroll
         for (int j = 0; j < TO; j++) {
-          bit_mac<CSA>(a[i].x, a[i].y, w[j].x, w[j].y, acc[i][j], ones[i][j]);
-          bit_mac<CSA>(a[i].z, a[i].w, w[j].z, w[j].w, acc[i][j], ones[i][j]);
+          bit_mac<CSA>(a[i].x, a[i].y, w[j].x, w[j].y, acc[i][j], ones[i][j], one);
+          bit_mac<CSA>(a[i].z, a[i].w, w[j].z, w[j].w, acc[i][j], ones[i][j], one);
         }
     }
     if (k < kvalid) {  // odd tail: one 64-bit word
@@ -228,7 +235,7 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO)) bconv_kernel(const BCon
 #pragma unroll
       for (int i = 0; i < TP; i++)
 #pragma unroll
-        for (int j = 0; j < TO; j++) bit_mac<CSA>(a[i].x, a[i].y, w[j].x, w[j].y, acc[i][j], ones[i][j]);
+        for (int j = 0; j < TO; j++) bit_mac<CSA>(a[i].x, a[i].y, w[j].x, w[j].y, acc[i][j], ones[i][j], one);
     }
   }
   cp_async_wait<0>();
@@ -335,12 +342,13 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO)) bconv_kernel(const BCon
 // ---- host side -----------------------------------------------------------------------------------
 
 int g_conv_variant = 0;
+int g_conv_tile = 0;
 
-template <int BP, int BO, int TP, int TO, int EPI, bool CSA, bool VEC16>
+template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16>
 dabnn_status launch_one(const BConvArgs& g, cudaStream_t st) {
   constexpr int THREADS = (BP / TP) * (BO / TO);
   constexpr size_t SMEM = (size_t)STAGES * (BP + BO) * PITCH * 4 + (size_t)BP * sizeof(RowInfo);
-  auto kern = bconv_kernel<BP, BO, TP, TO, EPI, CSA, VEC16>;
+  auto kern = bconv_kernel<BP, BO, TP, TO, MINB, EPI, CSA, VEC16>;
   static bool configured = false;  // one attribute call per instantiation (idempotent if raced)
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) {
@@ -357,11 +365,14 @@ dabnn_status launch_one(const BConvArgs& g, cudaStream_t st) {
   return launch_status();
 }
 
-template <int BP, int BO, int TP, int TO, int EPI>
+template <int BP, int BO, int TP, int TO, int MINB, int EPI>
 dabnn_status launch_tile(const BConvArgs& g, bool csa, cudaStream_t st) {
   const bool vec16 = (g.Cw % 2 == 0) && aligned(g.a, 16) && aligned(g.w, 16);
-  if (csa) return vec16 ? launch_one<BP, BO, TP, TO, EPI, true, true>(g, st) : launch_one<BP, BO, TP, TO, EPI, true, false>(g, st);
-  return vec16 ? launch_one<BP, BO, TP, TO, EPI, false, true>(g, st) : launch_one<BP, BO, TP, TO, EPI, false, false>(g, st);
+  if (csa)
+    return vec16 ? launch_one<BP, BO, TP, TO, MINB, EPI, true, true>(g, st)
+                 : launch_one<BP, BO, TP, TO, MINB, EPI, true, false>(g, st);
+  return vec16 ? launch_one<BP, BO, TP, TO, MINB, EPI, false, true>(g, st)
+               : launch_one<BP, BO, TP, TO, MINB, EPI, false, false>(g, st);
 }
 
 template <int EPI>
@@ -370,9 +381,19 @@ dabnn_status launch_epi(const BConvArgs& g, cudaStream_t st) {
   const int sms = sm_count();
   const int ochan = (EPI == EPI_I32) ? g.O : g.Ow32 * 32;
   auto ctas = [&](int bp, int bo) { return ((g.M + bp - 1) / bp) * ((ochan + bo - 1) / bo); };
-  if (ctas(128, 128) >= 2LL * sms) return launch_tile<128, 128, 8, 8, EPI>(g, csa, st);
-  if (ctas(64, 64) >= 2LL * sms) return launch_tile<64, 64, 4, 4, EPI>(g, csa, st);
-  return launch_tile<32, 32, 2, 4, EPI>(g, csa, st);
+  int tile = g_conv_tile;
+  if (tile == 0) {
+    if (ochan > 64 && ctas(128, 128) >= 2LL * sms) tile = 1;
+    else if (ctas(128, 64) >= 4LL * sms) tile = 2;
+    else if (ctas(64, 64) >= 2LL * sms) tile = 3;
+    else tile = 4;
+  }
+  switch (tile) {
+    case 1: return launch_tile<128, 128, 8, 8, 1, EPI>(g, csa, st);
+    case 2: return launch_tile<128, 64, 8, 4, 2, EPI>(g, csa, st);
+    case 3: return launch_tile<64, 64, 4, 4, 2, EPI>(g, csa, st);
+    default: return launch_tile<32, 32, 2, 4, 4, EPI>(g, csa, st);
+  }
 }
 
 dabnn_status fill_args(BConvArgs& g, const uint64_t* a, dabnn_shape in, const uint64_t* w, int O, dabnn_conv cv) {
@@ -397,7 +418,7 @@ dabnn_status fill_args(BConvArgs& g, const uint64_t* a, dabnn_shape in, const ui
   g.pad_neg = cv.pad_value < 0;
   g.tail_mask = (in.C % 64 == 0) ? ~0ull : ((1ull << (in.C % 64)) - 1);
   g.out = nullptr; g.out_nchw = 0; g.scale = g.shift = g.residual = nullptr; g.y_out = nullptr;
-  g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64);
+  g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64); g.one = 1;
   return DABNN_OK;
 }
 
@@ -423,6 +444,12 @@ using namespace dabnn;
 extern "C" int dabnn_set_conv_variant(int variant) {
   const int prev = g_conv_variant;
   if (variant >= 0 && variant <= 2) g_conv_variant = variant;
+  return prev;
+}
+
+extern "C" int dabnn_set_conv_tile(int tile) {
+  const int prev = g_conv_tile;
+  if (tile >= 0 && tile <= 4) g_conv_tile = tile;
   return prev;
 }
 

@@ -14,64 +14,64 @@ namespace {
 
 constexpr int kPackThreads = 128;
 
-// NCHW, H*W a multiple of 4, 16-byte aligned input.  A CTA covers `pix_per_cta` = 128 * (4 / wc)
-// consecutive pixels of one image; wc warps share a 128-pixel group and split its channel words.
-// Each lane owns 4 consecutive pixels (one float4 per channel) and walks 64 channels per word.
-template <int WC>  // warps per pixel group: 1, 2 or 4
+// Streaming 16-byte load.  Written as volatile asm so that a batch of them is issued back to back, in program
+// order, before the first result is consumed (memory-level parallelism is what an HBM-bound kernel lives on).
+__device__ __forceinline__ float4 ld_stream_f4(const float4* p) {
+  float4 v;
+  asm volatile("ld.global.cs.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+
+// NCHW, H*W a multiple of 4, 16-byte aligned input.  A CTA covers 128 consecutive pixels of one image and all
+// channels.  Each lane owns 4 consecutive pixels (one float4 per channel); the four warps split every word's 64
+// channels into quarters of 16, so a thread has 16 independent 16-byte loads in flight per word, and the 16-bit
+// quarters are placed side by side in shared memory, which assembles the 64-bit words without any exchange.
 __global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const float* __restrict__ x, int C, int HW, int Cw,
                                                                uint64_t* __restrict__ packed) {
-  extern __shared__ uint64_t s_words[];  // [pix_per_cta][Cw]
-  constexpr int GROUPS = 4 / WC;
+  extern __shared__ __align__(16) uint64_t s_words[];  // [128][Cw]
+  uint16_t* s_q = reinterpret_cast<uint16_t*>(s_words);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int group = warp / WC, wsel = warp % WC;
   const int n = blockIdx.y;
-  const int pix0 = blockIdx.x * (128 * GROUPS);
-  const int p = pix0 + group * 128 + lane * 4;  // first of this lane's 4 pixels
-  const bool live = p < HW;                     // HW % 4 == 0, so all 4 pixels are live together
+  const int pix0 = blockIdx.x * 128;
+  const int p = pix0 + lane * 4;  // first of this lane's 4 pixels
+  const bool live = p < HW;       // HW % 4 == 0, so all 4 pixels are live together
   const float* xn = x + (size_t)n * C * HW;
-  for (int cw = wsel; cw < Cw; cw += WC) {
-    uint64_t w0 = 0, w1 = 0, w2 = 0, w3 = 0;
-    const int c0 = cw * 64;
-    const int cn = min(64, C - c0);
-    if (live) {
+  const size_t cstride = (size_t)HW / 4;
+  for (int cw = 0; cw < Cw; cw++) {
+    const int c0 = cw * 64 + warp * 16;
+    unsigned b0 = 0, b1 = 0, b2 = 0, b3 = 0;  // 16 channels of each of the 4 pixels
+    if (live && c0 < C) {
       const float4* src = reinterpret_cast<const float4*>(xn + (size_t)c0 * HW + p);
-      const size_t cstride = (size_t)HW / 4;
-      int c = 0;
-#pragma unroll 1
-      for (; c + 8 <= cn; c += 8) {
-        float4 v[8];
+      if (c0 + 16 <= C) {
+        float4 v[16];
 #pragma unroll
-        for (int u = 0; u < 8; u++) v[u] = __ldcs(src + (size_t)(c + u) * cstride);
-        unsigned b0 = 0, b1 = 0, b2 = 0, b3 = 0;  // 8 channels of each of the 4 pixels
+        for (int u = 0; u < 16; u++) v[u] = ld_stream_f4(src + (size_t)u * cstride);
 #pragma unroll
-        for (int u = 0; u < 8; u++) {
+        for (int u = 0; u < 16; u++) {
           b0 |= (unsigned)(v[u].x < 0.0f) << u;
           b1 |= (unsigned)(v[u].y < 0.0f) << u;
           b2 |= (unsigned)(v[u].z < 0.0f) << u;
           b3 |= (unsigned)(v[u].w < 0.0f) << u;
         }
-        w0 |= (uint64_t)b0 << c;
-        w1 |= (uint64_t)b1 << c;
-        w2 |= (uint64_t)b2 << c;
-        w3 |= (uint64_t)b3 << c;
-      }
-      for (; c < cn; c++) {
-        float4 v = __ldcs(src + (size_t)c * cstride);
-        w0 |= (uint64_t)(v.x < 0.0f) << c;
-        w1 |= (uint64_t)(v.y < 0.0f) << c;
-        w2 |= (uint64_t)(v.z < 0.0f) << c;
-        w3 |= (uint64_t)(v.w < 0.0f) << c;
+      } else {
+        for (int u = 0; u < C - c0; u++) {
+          const float4 v = __ldcs(src + (size_t)u * cstride);
+          b0 |= (unsigned)(v.x < 0.0f) << u;
+          b1 |= (unsigned)(v.y < 0.0f) << u;
+          b2 |= (unsigned)(v.z < 0.0f) << u;
+          b3 |= (unsigned)(v.w < 0.0f) << u;
+        }
       }
     }
-    const int lp = group * 128 + lane * 4;
-    s_words[(size_t)(lp + 0) * Cw + cw] = w0;
-    s_words[(size_t)(lp + 1) * Cw + cw] = w1;
-    s_words[(size_t)(lp + 2) * Cw + cw] = w2;
-    s_words[(size_t)(lp + 3) * Cw + cw] = w3;
+    const int lp = lane * 4;
+    s_q[((lp + 0) * Cw + cw) * 4 + warp] = (uint16_t)b0;
+    s_q[((lp + 1) * Cw + cw) * 4 + warp] = (uint16_t)b1;
+    s_q[((lp + 2) * Cw + cw) * 4 + warp] = (uint16_t)b2;
+    s_q[((lp + 3) * Cw + cw) * 4 + warp] = (uint16_t)b3;
   }
   __syncthreads();
   // contiguous in global memory: pixels pix0 .. pix0+npix-1, all words
-  const int npix = min(128 * GROUPS, HW - pix0);
+  const int npix = min(128, HW - pix0);
   if (npix <= 0) return;
   uint64_t* dst = packed + ((size_t)n * HW + pix0) * Cw;
   const int total = npix * Cw;
@@ -83,6 +83,36 @@ __global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const float* __re
     if ((total & 1) && threadIdx.x == 0) dst[total - 1] = s_words[total - 1];
   } else {
     for (int i = threadIdx.x; i < total; i += kPackThreads) dst[i] = s_words[i];
+  }
+}
+
+// NCHW, any H*W and alignment: a CTA takes 128 consecutive pixels of one image and one 64-channel word.  The
+// 64 x 128 sign flags are gathered with coalesced scalar loads (lanes along pixels) into shared memory; each
+// thread then assembles 32 channel bits of one pixel and stores that half word.
+__global__ void __launch_bounds__(256) pack_nchw_tile(const float* __restrict__ x, int C, int HW, int Cw,
+                                                      uint64_t* __restrict__ packed) {
+  __shared__ unsigned char s_sign[64 * 128];
+  const int tid = threadIdx.x, lane = tid & 31, ty = tid >> 5;
+  const int n = blockIdx.y, p0 = blockIdx.x * 128, cw = blockIdx.z;
+  const int npix = min(128, HW - p0);
+  const float* xn = x + (size_t)n * C * HW + p0;
+  const int c0 = cw * 64, cn = min(64, C - c0);
+#pragma unroll
+  for (int c = ty; c < 64; c += 8) {
+    const float* row = xn + (size_t)(c0 + c) * HW;
+#pragma unroll
+    for (int q = 0; q < 4; q++) {
+      const int p = lane + 32 * q;
+      s_sign[c * 128 + p] = (c < cn && p < npix) ? (unsigned char)(__ldcs(row + p) < 0.0f) : (unsigned char)0;
+    }
+  }
+  __syncthreads();
+  const int p = tid & 127, half = tid >> 7;
+  if (p < npix) {
+    uint32_t bits = 0;
+#pragma unroll
+    for (int c = 0; c < 32; c++) bits |= (uint32_t)s_sign[(half * 32 + c) * 128 + p] << c;
+    reinterpret_cast<uint32_t*>(packed)[(((size_t)n * HW + p0 + p) * Cw + cw) * 2 + half] = bits;
   }
 }
 
@@ -167,15 +197,12 @@ extern "C" dabnn_status dabnn_pack(const float* x, dabnn_layout in_layout, dabnn
   if (HW > 0x7FFFFFFF || (long long)s.N * HW > 0x7FFFFFFFFFFLL) return DABNN_ERR_UNSUPPORTED;
   const long long total_words = (long long)s.N * HW * Cw;
   cudaStream_t st = as_stream(stream);
-  if (in_layout == DABNN_NCHW && HW % 4 == 0 && aligned(x, 16) && ((long long)s.C * HW) % 4 == 0 && s.N <= 65535 &&
-      Cw * 512 * 8 <= 48 * 1024) {
-    const int wc = Cw >= 4 ? 4 : (Cw >= 2 ? 2 : 1);
-    const int pix_per_cta = 128 * (4 / wc);
-    dim3 grid(ceil_div(HW, pix_per_cta), s.N);
-    const size_t smem = (size_t)pix_per_cta * Cw * 8;
-    if (wc == 4) pack_nchw_vec4<4><<<grid, kPackThreads, smem, st>>>(x, s.C, (int)HW, (int)Cw, packed);
-    else if (wc == 2) pack_nchw_vec4<2><<<grid, kPackThreads, smem, st>>>(x, s.C, (int)HW, (int)Cw, packed);
-    else pack_nchw_vec4<1><<<grid, kPackThreads, smem, st>>>(x, s.C, (int)HW, (int)Cw, packed);
+  if (in_layout == DABNN_NCHW && HW % 4 == 0 && aligned(x, 16) && s.N <= 65535 && Cw * 128 * 8 <= 48 * 1024) {
+    dim3 grid(ceil_div(HW, 128), s.N);
+    pack_nchw_vec4<<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, packed);
+  } else if (in_layout == DABNN_NCHW && s.N <= 65535 && Cw <= 65535) {
+    dim3 grid(ceil_div(HW, 128), s.N, (unsigned)Cw);
+    pack_nchw_tile<<<grid, 256, 0, st>>>(x, s.C, (int)HW, (int)Cw, packed);
   } else if (in_layout == DABNN_NHWC && s.C % 64 == 0 && aligned(x, 16)) {
     const long long warps_needed = (total_words + 7) / 8;
     long long blocks = (warps_needed + 7) / 8;

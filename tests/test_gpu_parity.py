@@ -38,6 +38,9 @@ PACK_SHAPES = [
     (1, 1, 1, 1),
     (1, 1000, 2, 2),    # 16 words, tail of 40 bits
     (5, 3, 224, 8),
+    (4, 512, 7, 7),     # tile path: H*W = 49
+    (2, 100, 15, 13),   # tile path, two pixel tiles, channel tail
+    (1, 2100, 3, 3),    # more than 32 words: generic path
 ]
 
 
@@ -217,3 +220,23 @@ def test_bireal18_forward_matches_oracle(B, oracle_mod):
     # batch 1 gives the same logits for the same image
     got1 = net.forward(dev(img[:1])).cpu().numpy()
     assert np.array_equal(got1, got[:1])
+
+
+@pytest.mark.parametrize("tile", [1, 2, 3, 4])
+@pytest.mark.parametrize("case", [CONV_CASES[1], CONV_CASES[4], CONV_CASES[9]])
+def test_every_conv_tile_gives_the_same_integers(B, oracle_mod, case, tile):
+    N, C, H, W, O, kh, kw, stride, pad, pv = case
+    x, w = conv_inputs(case)
+    o = oracle_mod
+    want = o.bconv_bits(o.pack(x), C, o.pack_weights(w), stride, pad, pv, o.NHWC)
+    scale_o, shift_o = o.bn_fold(*synth.bn_params(np.random.default_rng(tile), O))
+    want_bits = o.bn_sign_pack(want, scale_o, shift_o)
+    prev = B.set_conv_tile(tile)
+    try:
+        a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
+        got = B.bconv2d(a, C, wp, stride, pad, pv, B.NHWC).cpu().numpy()
+        got_bits = u64(B.bconv2d_bn_sign_pack(a, C, wp, dev(scale_o), dev(shift_o), stride, pad, pv))
+    finally:
+        B.set_conv_tile(prev)
+    assert np.array_equal(got, want)
+    assert np.array_equal(got_bits, want_bits)
