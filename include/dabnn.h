@@ -157,6 +157,27 @@ dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const 
                                      const float* scale, const float* shift, int32_t* out_host, uint64_t* bits_host,
                                      void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- tensor-core engine -------------------------------------------------------------------------------------------
+ * The same convolutions (Section 2.1.2, Eq. 1 read as a +-1 dot product) computed on the tcgen05 tensor cores with
+ * int8 {+1,-1} operands expanded on chip from the packed bits.  Results are identical to dabnn_bconv2d* bit for bit.
+ * Covered: stride 1, C a multiple of 32, filters whose expanded weights fit the resident budget (dabnn_tc_weights_bytes
+ * returns 0 otherwise); other cases return DABNN_ERR_UNSUPPORTED and are served by dabnn_bconv2d*.
+ *   dabnn_tc_weights_bytes    bytes of the expanded weight buffer for a filter bank (0 = not covered)
+ *   dabnn_tc_prepare_weights  w_packed [O][kh][kw][Cw] -> w_tc (device, 16-byte aligned, that many bytes); once per model
+ *   dabnn_tc_bconv2d*         as dabnn_bconv2d*, with w_tc in place of w_packed
+ *   dabnn_tc_error_flag       synchronises nothing itself; copies the device-side error flag (1 if a bounded wait inside
+ *                             a kernel ran out, else 0; -1 if it cannot be read).  Call after synchronising the stream. */
+size_t dabnn_tc_weights_bytes(int O, int C, int kh, int kw);
+dabnn_status dabnn_tc_prepare_weights(const uint64_t* w_packed, int O, int C, int kh, int kw, void* w_tc, void* stream);
+dabnn_status dabnn_tc_bconv2d(const uint64_t* a_packed, dabnn_shape in, const void* w_tc, int O, dabnn_conv cv,
+                              int32_t* out, dabnn_layout out_layout, void* stream);
+dabnn_status dabnn_tc_bconv2d_bn_sign_pack(const uint64_t* a_packed, dabnn_shape in, const void* w_tc, int O, dabnn_conv cv,
+                                           const float* scale, const float* shift, uint64_t* out_packed, void* stream);
+dabnn_status dabnn_tc_bconv2d_bn_add_sign_pack(const uint64_t* a_packed, dabnn_shape in, const void* w_tc, int O,
+                                               dabnn_conv cv, const float* scale, const float* shift, const float* residual,
+                                               float* y_out, uint64_t* out_packed, void* stream);
+int dabnn_tc_error_flag(void);
+
 /* Selects the convolution inner loop for measurement runs: 0 = automatic (default),
  * 1 = one POPC per 32-bit word pair, 2 = carry-save (one POPC per two word pairs).  All give identical results.
  * Returns the previous setting.  Not thread-safe against concurrent calls into the library. */

@@ -26,6 +26,8 @@ EXPORTS = (
     "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack", "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold",
     "dabnn_bireal18_workspace_bytes", "dabnn_bireal18_forward", "dabnn_set_conv_variant",
     "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host", "dabnn_bireal18_forward_static", "dabnn_set_conv_tile",
+    "dabnn_tc_weights_bytes", "dabnn_tc_prepare_weights", "dabnn_tc_bconv2d", "dabnn_tc_bconv2d_bn_sign_pack",
+    "dabnn_tc_bconv2d_bn_add_sign_pack", "dabnn_tc_error_flag",
 )
 
 
@@ -84,6 +86,15 @@ def lib() -> ctypes.CDLL:
         L.dabnn_binary_layer_host.restype = ci
         L.dabnn_set_conv_variant.restype = ci
         L.dabnn_set_conv_variant.argtypes = [ci]
+        L.dabnn_tc_weights_bytes.restype = ctypes.c_size_t
+        L.dabnn_tc_weights_bytes.argtypes = [ci, ci, ci, ci]
+        L.dabnn_tc_prepare_weights.argtypes = [vp, ci, ci, ci, ci, vp, vp]
+        L.dabnn_tc_bconv2d.argtypes = [vp, Shape, vp, ci, Conv, vp, ci, vp]
+        L.dabnn_tc_bconv2d_bn_sign_pack.argtypes = [vp, Shape, vp, ci, Conv, vp, vp, vp, vp]
+        L.dabnn_tc_bconv2d_bn_add_sign_pack.argtypes = [vp, Shape, vp, ci, Conv, vp, vp, vp, vp, vp, vp]
+        for name in ("dabnn_tc_prepare_weights", "dabnn_tc_bconv2d", "dabnn_tc_bconv2d_bn_sign_pack",
+                     "dabnn_tc_bconv2d_bn_add_sign_pack", "dabnn_tc_error_flag"):
+            getattr(L, name).restype = ci
         L.dabnn_set_conv_tile.restype = ci
         L.dabnn_set_conv_tile.argtypes = [ci]
         L.dabnn_bireal18_forward_static.restype = ci
@@ -307,6 +318,78 @@ def bireal18_forward_static(net: "Bireal18", images: torch.Tensor, logits: Optio
         logits = torch.empty((N, 1000), dtype=torch.float32, device=images.device)
     _check(lib().dabnn_bireal18_forward_static(ctypes.byref(net.P), images.data_ptr(), N, logits.data_ptr(), _stream()))
     return logits
+
+
+# ---- tensor-core engine ---------------------------------------------------------------------------------------------
+class TcWeights:
+    """Expanded int8 weights for the tensor-core engine (dabnn_tc_prepare_weights), with the filter geometry."""
+
+    def __init__(self, w_packed: torch.Tensor, C: int):
+        w = _dev(w_packed, torch.int64, "w_packed")
+        self.O, self.kh, self.kw, Cw = w.shape
+        self.C = C
+        nbytes = int(lib().dabnn_tc_weights_bytes(self.O, C, self.kh, self.kw))
+        if nbytes == 0:
+            raise DabnnError("this filter bank is not covered by the tensor-core engine")
+        self.buf = torch.empty(nbytes, dtype=torch.uint8, device=w.device)
+        _check(lib().dabnn_tc_prepare_weights(w.data_ptr(), self.O, C, self.kh, self.kw, self.buf.data_ptr(), _stream()))
+
+
+def tc_supported(O: int, C: int, kh: int, kw: int, stride=(1, 1)) -> bool:
+    return tuple(stride) == (1, 1) and int(lib().dabnn_tc_weights_bytes(O, C, kh, kw)) > 0
+
+
+def _tc_geom(a_packed, wt: TcWeights, stride, pad):
+    a = _dev(a_packed, torch.int64, "a_packed")
+    N, H, W, Cw = a.shape
+    if Cw != (wt.C + 63) // 64:
+        raise DabnnError("packed word count does not match C")
+    OH, OW = out_dim(H, wt.kh, stride[0], pad[0]), out_dim(W, wt.kw, stride[1], pad[1])
+    return a, N, H, W, OH, OW
+
+
+def tc_bconv2d(a_packed, wt: TcWeights, stride=(1, 1), pad=(0, 0), pad_value: int = -1, out_layout: int = NHWC,
+               out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_tc_bconv2d."""
+    a, N, H, W, OH, OW = _tc_geom(a_packed, wt, stride, pad)
+    if out is None:
+        shape = (N, OH, OW, wt.O) if out_layout == NHWC else (N, wt.O, OH, OW)
+        out = torch.empty(shape, dtype=torch.int32, device=a.device)
+    _check(lib().dabnn_tc_bconv2d(a.data_ptr(), Shape(N, wt.C, H, W), wt.buf.data_ptr(), wt.O,
+                                  _conv(wt.kh, wt.kw, stride, pad, pad_value), out.data_ptr(), out_layout, _stream()))
+    return out
+
+
+def tc_bconv2d_bn_sign_pack(a_packed, wt: TcWeights, scale, shift, stride=(1, 1), pad=(0, 0), pad_value: int = -1,
+                            out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_tc_bconv2d_bn_sign_pack."""
+    a, N, H, W, OH, OW = _tc_geom(a_packed, wt, stride, pad)
+    scale, shift = _dev(scale, torch.float32, "scale"), _dev(shift, torch.float32, "shift")
+    if out is None:
+        out = torch.empty((N, OH, OW, words_per_pixel(wt.O)), dtype=torch.int64, device=a.device)
+    _check(lib().dabnn_tc_bconv2d_bn_sign_pack(a.data_ptr(), Shape(N, wt.C, H, W), wt.buf.data_ptr(), wt.O,
+                                               _conv(wt.kh, wt.kw, stride, pad, pad_value), scale.data_ptr(),
+                                               shift.data_ptr(), out.data_ptr(), _stream()))
+    return out
+
+
+def tc_bconv2d_bn_add_sign_pack(a_packed, wt: TcWeights, scale, shift, residual, stride=(1, 1), pad=(0, 0),
+                                pad_value: int = -1, want_bits: bool = True):
+    """dabnn_tc_bconv2d_bn_add_sign_pack."""
+    a, N, H, W, OH, OW = _tc_geom(a_packed, wt, stride, pad)
+    scale, shift = _dev(scale, torch.float32, "scale"), _dev(shift, torch.float32, "shift")
+    residual = _dev(residual, torch.float32, "residual")
+    y = torch.empty_like(residual)
+    bits = torch.empty((N, OH, OW, words_per_pixel(wt.O)), dtype=torch.int64, device=a.device) if want_bits else None
+    _check(lib().dabnn_tc_bconv2d_bn_add_sign_pack(a.data_ptr(), Shape(N, wt.C, H, W), wt.buf.data_ptr(), wt.O,
+                                                   _conv(wt.kh, wt.kw, stride, pad, pad_value), scale.data_ptr(),
+                                                   shift.data_ptr(), residual.data_ptr(), y.data_ptr(),
+                                                   bits.data_ptr() if want_bits else None, _stream()))
+    return y, bits
+
+
+def tc_error_flag() -> int:
+    return int(lib().dabnn_tc_error_flag())
 
 
 class Prepared:

@@ -28,6 +28,7 @@ def main():
     ap.add_argument("--reps", type=int, default=1, help="launches per timed event pair")
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--tile", type=int, default=0)
+    ap.add_argument("--engine", default="popc", choices=["popc", "tc"])
     a = ap.parse_args()
     O = a.O or a.C
     dev = torch.device("cuda", 0)
@@ -50,6 +51,16 @@ def main():
             out = torch.empty_like(ap_)
             fn = lambda: B.pack(xd, B.NCHW, out=out)
             work = ("GB/s", (xd.numel() * 4 + out.numel() * 8) / 1e9)
+        elif a.case == "conv" and a.engine == "tc":
+            out = torch.empty((a.N, a.HW, a.HW, O), dtype=torch.int32, device=dev)
+            wt = B.TcWeights(wp, a.C)
+            fn = lambda: B.tc_bconv2d(ap_, wt, (1, 1), (pad, pad), -1, B.NHWC, out=out)
+            work = ("Tbit-ops/s", 2.0 * a.N * a.HW * a.HW * O * a.C * a.k * a.k / 1e12)
+        elif a.case == "fused" and a.engine == "tc":
+            out = torch.empty((a.N, a.HW, a.HW, (O + 63) // 64), dtype=torch.int64, device=dev)
+            wt = B.TcWeights(wp, a.C)
+            fn = lambda: B.tc_bconv2d_bn_sign_pack(ap_, wt, scale, shift, (1, 1), (pad, pad), -1, out=out)
+            work = ("Tbit-ops/s", 2.0 * a.N * a.HW * a.HW * O * a.C * a.k * a.k / 1e12)
         elif a.case == "conv":
             out = torch.empty((a.N, a.HW, a.HW, O), dtype=torch.int32, device=dev)
             fn = lambda: B.bconv2d(ap_, a.C, wp, (1, 1), (pad, pad), -1, B.NHWC, out=out)

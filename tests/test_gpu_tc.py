@@ -1,0 +1,110 @@
+"""GPU parity of the tensor-core engine (dabnn_tc_*): identical integers, bits and fp32 values as the CPU oracle,
+through every epilogue, on shapes that cover several channel tiles, ragged tiles, channel tails and pad values."""
+import numpy as np
+import pytest
+import torch
+
+from paper_1908_05858_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_1908_05858_b200 import binding
+
+    assert torch.cuda.is_available()
+    binding.lib()
+    return binding
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def u64(t):
+    return t.cpu().numpy().view(np.uint64)
+
+
+TC_CASES = [
+    # N, C, H, W, O, k, pad, pad_value
+    (1, 64, 14, 14, 64, 3, 1, -1),      # BASELINE config 1
+    (2, 128, 9, 11, 100, 3, 1, +1),     # O not a multiple of 16, pad +1
+    (3, 256, 14, 14, 256, 3, 1, -1),    # four channel tiles of 64
+    (2, 512, 7, 7, 512, 3, 1, -1),      # channel tiles of 32, K = 4608
+    (2, 512, 14, 14, 300, 1, 0, -1),    # 1x1, ragged channel tile
+    (1, 64, 56, 56, 64, 3, 1, -1),
+    (2, 96, 10, 10, 70, 5, 2, -1),      # C = 96: half-used last word, 5x5
+    (5, 32, 6, 7, 33, 3, 1, -1),        # smallest C, O just over a tile
+    (9, 128, 28, 28, 128, 3, 1, -1),    # many pixel tiles per CTA? (persistent loop over tiles)
+    (300, 64, 8, 8, 64, 3, 0, -1),      # no padding, many images per tile
+]
+
+
+def inputs(case):
+    N, C, H, W, O, k, pad, pv = case
+    rng = np.random.default_rng(abs(hash(case)) % (2**32))
+    return rng.standard_normal((N, C, H, W)).astype(np.float32), rng.standard_normal((O, C, k, k)).astype(np.float32)
+
+
+@pytest.mark.parametrize("case", TC_CASES)
+def test_tc_conv_and_epilogues_match_oracle(B, oracle_mod, case):
+    N, C, H, W, O, k, pad, pv = case
+    x, w = inputs(case)
+    o = oracle_mod
+    acc = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (1, 1), (pad, pad), pv, o.NHWC)
+    a = B.pack(dev(x))
+    wp = B.pack_weights(dev(w))
+    assert B.tc_supported(O, C, k, k)
+    wt = B.TcWeights(wp, C)
+    got = B.tc_bconv2d(a, wt, (1, 1), (pad, pad), pv, B.NHWC).cpu().numpy()
+    assert np.array_equal(got, acc)
+    got_nchw = B.tc_bconv2d(a, wt, (1, 1), (pad, pad), pv, B.NCHW).cpu().numpy()
+    assert np.array_equal(got_nchw, np.transpose(acc, (0, 3, 1, 2)))
+    # the xor/popcount kernel gives the same integers
+    assert np.array_equal(B.bconv2d(a, C, wp, (1, 1), (pad, pad), pv, B.NHWC).cpu().numpy(), acc)
+    # fused BN + sign + pack
+    rng = np.random.default_rng(O)
+    gamma, beta, mean, var = synth.bn_params(rng, O)
+    gamma[::5] *= -1.0
+    mean *= 30.0
+    scale, shift = o.bn_fold(gamma, beta, mean, var)
+    want_bits = o.bn_sign_pack(acc, scale, shift)
+    got_bits = u64(B.tc_bconv2d_bn_sign_pack(a, wt, dev(scale), dev(shift), (1, 1), (pad, pad), pv))
+    assert np.array_equal(got_bits, want_bits)
+    # Bi-Real block epilogue
+    res = rng.standard_normal(acc.shape).astype(np.float32) * 20
+    y = (acc.astype(np.float64) * scale.astype(np.float64) + shift.astype(np.float64)).astype(np.float32) + res
+    got_y, got_ybits = B.tc_bconv2d_bn_add_sign_pack(a, wt, dev(scale), dev(shift), dev(res), (1, 1), (pad, pad), pv)
+    assert np.array_equal(got_y.cpu().numpy().view(np.uint32), y.view(np.uint32))
+    assert np.array_equal(u64(got_ybits), o.pack(y, o.NHWC))
+    torch.cuda.synchronize()
+    assert B.tc_error_flag() == 0
+
+
+def test_tc_declines_what_it_does_not_cover(B):
+    assert not B.tc_supported(64, 64, 3, 3, stride=(2, 2))
+    assert not B.tc_supported(64, 70, 3, 3)          # C not a multiple of 32
+    assert not B.tc_supported(64, 1024, 7, 7)        # expanded weights larger than the resident budget
+    a = torch.zeros((1, 8, 8, 1), dtype=torch.int64, device="cuda")
+    wt = B.TcWeights(torch.zeros((64, 3, 3, 1), dtype=torch.int64, device="cuda"), 64)
+    with pytest.raises(B.DabnnError, match="supported"):
+        B.tc_bconv2d(a, wt, (2, 2), (1, 1), -1)
+
+
+@pytest.mark.parametrize("cfg", [(64, 64, 56, 64, 3, 1), (64, 512, 7, 512, 3, 1), (256, 256, 28, 256, 3, 1), (256, 512, 14, 2048, 1, 0)])
+def test_tc_full_size_configs_on_sampled_outputs(B, oracle_mod, cfg):
+    N, C, HW, O, k, pad = cfg
+    x, w = synth.conv_case(2 if N == 64 else 5, N, C, HW, HW, O, k, k, salt=C)
+    a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
+    got = B.tc_bconv2d(a, B.TcWeights(wp, C), (1, 1), (pad, pad), -1, B.NHWC)
+    K = C * k * k
+    assert int(got.min()) >= -K and int(got.max()) <= K and bool(((got - K) % 2 == 0).all())
+    # the whole tensor against the xor/popcount kernel (itself checked against the oracle), and samples against the definition
+    assert bool((got == B.bconv2d(a, C, wp, (1, 1), (pad, pad), -1, B.NHWC)).all())
+    g = got.cpu().numpy()
+    rng = np.random.default_rng(C + N)
+    coords = np.stack([rng.integers(0, N, 20000), rng.integers(0, O, 20000), rng.integers(0, HW, 20000), rng.integers(0, HW, 20000)], axis=1).astype(np.int32)
+    want = oracle_mod.bconv_pm1_at(x, w, coords, (1, 1), (pad, pad), -1)
+    assert np.array_equal(g[coords[:, 0], coords[:, 2], coords[:, 3], coords[:, 1]], want)
+    assert B.tc_error_flag() == 0
