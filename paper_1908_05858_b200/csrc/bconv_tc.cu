@@ -1,24 +1,27 @@
-// Binary convolution on the 5th-generation tensor cores (tcgen05, kind::i8) -- the same integers as the xor/popcount
-// kernel (Section 2.1.2, Eq. 1 of the paper, read as a +-1 dot product), computed as a dense int8 contraction.
+// Binary convolution on the 5th-generation tensor cores (tcgen05) -- the same integers as the xor/popcount kernel
+// (Section 2.1.2, Eq. 1 of the paper, read as a +-1 dot product), computed as a dense low-precision contraction.
 //
 // sm_100a has no native 1-bit MMA (mma.sync ... b1 is emulated and tcgen05 has no 1-bit kind), so the +-1 values
-// are expanded to int8 on chip: HBM still holds one bit per activation and per weight use.
+// are expanded on chip to the narrowest type the tensor core takes: 4-bit e2m1 (+1.0 = 0x2, -1.0 = 0xA), used through
+// the block-scaled kind::mxf4 with every scale factor set to 1.0 (ue8m0 127).  Products are +-1 and the fp32
+// accumulator adds at most K < 2^24 of them, so the result is the exact integer.  HBM still holds one bit per value.
 //
-//   * Weights: expanded once (dabnn_tc_prepare_weights) to int8 {+1,-1} in the UMMA K-major, no-swizzle core-matrix
-//     layout, one contiguous block per tile of NT output channels; a persistent CTA copies its block to shared
-//     memory once and keeps it for all its pixel tiles.
+//   * Weights: expanded once (dabnn_tc_prepare_weights) to e2m1 in the UMMA K-major, no-swizzle core-matrix layout
+//     (rows of 16 bytes = 32 channels), one contiguous block per tile of NT output channels; a persistent CTA copies
+//     its block to shared memory once and keeps it for all its pixel tiles.
 //   * Activations: a tile is 128 consecutive "slots" q of the padded image grid (slot pitch SP = W + 2*pad_w,
 //     H + 2*pad_h slot rows per image).  The CTA reads the packed bits of the 128 + (kh-1)*SP + (kw-1) slots it
-//     needs, expands them to int8 rows of 16 channels ([C/16][slots][16 B]) -- padded slots get the declared pad
+//     needs, expands them to e2m1 rows of 32 channels ([C/32][slots][16 B]) -- padded slots get the declared pad
 //     value -- and every filter tap (i, j) is the SAME array read from a start address shifted by (i*SP + j) rows:
 //     with a 16-byte row pitch a shift by one slot is a 16-byte step of the matrix descriptor, so no im2col copy
 //     is ever materialised.  Rows that fall on padding columns / rows compute garbage that is never stored.
-//   * One thread issues kh*kw*(C/32) tcgen05.mma (M = 128, N = NT, K = 32) per tile into a TMEM accumulator
-//     (two buffers), commits to an mbarrier, and the CTA's warps read the previous tile's accumulator with
-//     tcgen05.ld while the tensor core works on the current one.
+//   * Warp-specialised and mbarrier-driven: four producer warps prefetch the next tile's bits, expand them through a
+//     256-entry table (8 bits -> 8 nibbles) into one of up to two A buffers and arrive on `a_full`; one thread of a
+//     ninth warp waits for it, issues kh*kw*(C/64) tcgen05.mma (M = 128, N = NT, K = 64) into one of two TMEM
+//     accumulators and commits to `mma_done`; four epilogue warps wait for that, read the accumulator with
+//     tcgen05.ld, write the output form, and hand the accumulator back through `tmem_free`.
 //
-// Every wait on an mbarrier is bounded: on expiry the kernel records an error flag, skips the remaining work,
-// frees its TMEM and returns.
+// Every wait on an mbarrier is bounded: on expiry the kernel records an error flag, stops, frees its TMEM and returns.
 #include "common.cuh"
 
 namespace dabnn {
@@ -27,12 +30,22 @@ namespace {
 
 enum { EPI_I32 = 0, EPI_BNPACK = 1, EPI_BIREAL = 2 };
 
-constexpr int TC_THREADS = 256;
+constexpr int TC_THREADS = 288;           // 4 epilogue warps, 4 producer warps, 1 MMA-issue warp
 constexpr int TC_SMEM_LIMIT = 232448;     // 227 KB opt-in maximum per CTA
-constexpr int TC_SMEM_MISC = 1024;        // barriers, TMEM base, alignment slack
+constexpr int TC_SMEM_MISC = 2048;        // barriers, TMEM base, flags, this CTA's scale / shift
 constexpr int TC_WEIGHT_BUDGET = 147456;  // 144 KB of resident weights at most
+constexpr int TC_MAX_CW = 8;              // C <= 512
+constexpr int TC_MAX_SLOTS = 256;         // two slots per producer thread
+constexpr int TC_TMEM_COLS = 512;         // 2 accumulators (<= 128 columns each) + the scale-factor columns
+constexpr int TC_SF_COL = 256;            // columns [256, 512) hold scale factors (all 1.0)
 
 __device__ int g_tc_error = 0;  // 1: an mbarrier wait ran out
+#ifdef TC_TIMING
+__device__ unsigned long long g_tc_prof[24];
+#define TC_T(i) do { long long t_ = clock64(); prof[i] += t_ - tlast; tlast = t_; } while (0)
+#else
+#define TC_T(i) do {} while (0)
+#endif
 
 struct TcArgs {
   const uint64_t* a;
@@ -42,6 +55,7 @@ struct TcArgs {
   int SP, HP;          // slot pitch and slot rows per image
   long long total_q;   // N * HP * SP
   int slots;           // slots per tile, multiple of 8
+  int abufs;           // A buffers in shared memory (1 or 2)
   int ntile, n_ntiles; // output channels per tile, number of channel tiles
   long long m_tiles;
   int pad_neg;
@@ -64,14 +78,17 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 
 // Bounded wait for the given phase parity; false if it ran out.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (int tries = 0; tries < (1 << 22); tries++) {
+  for (int tries = 0; tries < (1 << 20); tries++) {  // about a second at most, then give up
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 0x10000;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, 0x400;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done)
         : "r"(bar), "r"(parity)
@@ -92,236 +109,369 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, uint32_t lbo, 
   return d;                // base offset 0, layout type 0 (no swizzle)
 }
 
-// 16 sign bits -> 16 bytes of {+1 (bit 0), -1 (bit 1)}.
-__device__ __forceinline__ uint32_t expand4(uint32_t nib) {
-  const uint32_t t = (nib * 0x00204081u) & 0x01010101u;  // bit k of the nibble -> byte k
-  return (t * 0xFFu) | 0x01010101u;                      // 1 -> 0xFF (-1), 0 -> 0x01 (+1)
+// 16 sign bits -> 16 e2m1 nibbles (8 bytes): +1.0 = 0x2 (bit 0), -1.0 = 0xA (bit 1).
+// A byte permute whose source register holds the four possible bytes 0x22, 0x2A, 0xA2, 0xAA maps a 2-bit pair value
+// to its byte; `h & 0x3333` and `(h >> 2) & 0x3333` already are four valid selector nibbles each, so the expansion is
+// three logic ops and two PRMTs, with no table.  Channels land in a permuted order inside their 16-byte row
+// (pairs 0,2,4,6 then 1,3,5,7): activations and weights go through this same function, and a dot product does not
+// care about the order of its terms.
+__device__ __forceinline__ uint2 expand16(uint32_t h) {
+  return make_uint2(__byte_perm(0xAAA22A22u, 0u, h & 0x3333u), __byte_perm(0xAAA22A22u, 0u, (h >> 2) & 0x3333u));
 }
-__device__ __forceinline__ uint4 expand16(uint32_t bits) {
-  return make_uint4(expand4(bits & 0xF), expand4((bits >> 4) & 0xF), expand4((bits >> 8) & 0xF),
-                    expand4((bits >> 12) & 0xF));
+__device__ __forceinline__ uint4 expand32(uint32_t w) {
+  const uint2 lo = expand16(w & 0xFFFFu), hi = expand16(w >> 16);
+  return make_uint4(lo.x, lo.y, hi.x, hi.y);
+}
+
+// 256-bit global store / load (32-byte aligned): a lane writes a whole 32-byte sector of its output row at once.
+__device__ __forceinline__ void st_global_v8(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e, uint32_t f,
+                                             uint32_t g2, uint32_t h) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d), "r"(e),
+               "r"(f), "r"(g2), "r"(h)
+               : "memory");
+}
+__device__ __forceinline__ void ld_global_v8(const void* p, float (&r)[8]) {
+  asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=f"(r[0]), "=f"(r[1]), "=f"(r[2]), "=f"(r[3]), "=f"(r[4]), "=f"(r[5]), "=f"(r[6]), "=f"(r[7])
+               : "l"(p));
 }
 
 template <int NT, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int K = g.kh * g.kw * g.C;  // bytes per weight row
-  uint8_t* w_s = smem;                                   // [taps][C/16][NT][16]
-  uint8_t* a_s = smem + (size_t)NT * K;                  // [C/16][slots][16]
-  uint8_t* misc = a_s + (size_t)g.slots * g.C;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(misc);    // 2 mbarriers
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 16);
-  int* s_fail = reinterpret_cast<int*>(misc + 24);
-  constexpr int TMEM_COLS = (2 * NT < 32) ? 32 : 2 * NT;
+  const int Kb = g.kh * g.kw * (g.C >> 1);               // bytes per weight row
+  const int a_bytes = g.slots * (g.C >> 1);              // bytes of one A buffer
+  uint8_t* w_s = smem;                                   // [taps][C/32][NT][16]
+  uint8_t* a_s = smem + (size_t)NT * Kb;                 // [abufs][C/32][slots][16]
+  uint8_t* misc = a_s + (size_t)g.abufs * a_bytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(misc);    // [0,1] mma_done  [2,3] tmem_free  [4,5] a_full
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 64);
+  volatile int* s_fail = reinterpret_cast<volatile int*>(misc + 72);
+  float* s_scale = reinterpret_cast<float*>(misc + 128);     // [NT] this CTA's channels
+  float* s_shift = s_scale + NT;                             // [NT]
 
   const int nt = blockIdx.x % g.n_ntiles;
   const long long mt_first = blockIdx.x / g.n_ntiles;
   const long long mt_step = gridDim.x / g.n_ntiles;
 
+  if (EPI != EPI_I32 && tid < NT) {
+    const int o = nt * NT + tid;
+    s_scale[tid] = (o < g.O) ? g.scale[o] : 0.0f;
+    s_shift[tid] = (o < g.O) ? g.shift[o] : 0.0f;
+  }
   if (tid == 0) {
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
+    mbar_init(smem_u32(&bars[2]), 128);
+    mbar_init(smem_u32(&bars[3]), 128);
+    mbar_init(smem_u32(&bars[4]), 128);
+    mbar_init(smem_u32(&bars[5]), 128);
     *s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"((uint32_t)TMEM_COLS)
+                 "r"((uint32_t)TC_TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // resident weights: one contiguous block per channel tile
   {
-    const uint8_t* src = g.w_tc + (size_t)nt * NT * K;
-    const int units = NT * K / 16;
+    const uint8_t* src = g.w_tc + (size_t)nt * NT * Kb;
+    const int units = NT * Kb / 16;
     for (int u = tid; u < units; u += TC_THREADS) cp_async16(smem_u32(w_s + (size_t)u * 16), src + (size_t)u * 16);
     asm volatile("cp.async.commit_group;" ::: "memory");
     asm volatile("cp.async.wait_group 0;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
-
-  const uint32_t idesc = (2u << 4)                      // accumulator: s32
-                         | (1u << 7) | (1u << 10)       // A, B: signed 8-bit
-                         | ((uint32_t)(NT >> 3) << 17)  // N
-                         | ((uint32_t)(128 >> 4) << 24);  // M = 128; both operands K-major
-  const int cgroups = g.C >> 4;  // 16-channel groups
-  const uint32_t a_lbo = (uint32_t)g.slots * 16, w_lbo = (uint32_t)NT * 16;
-  const uint32_t pad_word4 = g.pad_neg ? 0xFFFFFFFFu : 0x01010101u;
-
-  // ---- epilogue of one finished tile --------------------------------------------------------------------------
-  auto epilogue = [&](long long mt, int buf) {
-    const int row = 32 * (warp & 3) + lane;      // TMEM lane = slot row of the tile
-    const int half = warp >> 2;                  // which half of the NT columns this warp reads
-    constexpr int COLS = NT / 2;                 // columns per warp
-    const long long Q = mt * 128 + row;
-    const int col = (int)(Q % g.SP);
-    const long long rr = Q / g.SP;
-    const int r = (int)(rr % g.HP);
-    const long long n = rr / g.HP;
-    const bool valid = n < g.N && r < g.OH && col < g.OW;
-    const long long m = (n * g.OH + r) * g.OW + col;
-    const int o_base = nt * NT + half * COLS;
-#pragma unroll
-    for (int c0 = 0; c0 < COLS; c0 += 16) {
-      uint32_t v[16];
-      const uint32_t taddr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(buf * NT + half * COLS + c0);
+  if (warp < 4) {
+    // scale factors: every byte of the scale-factor columns is ue8m0 127 = 1.0, whatever their layout
+    const uint32_t one = 0x7F7F7F7Fu;
+    for (int c = TC_SF_COL; c < TC_TMEM_COLS; c += 16) {
+      const uint32_t taddr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)c;
       asm volatile(
-          "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-          : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-            "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-          : "r"(taddr));
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      const int o = o_base + c0;
-      if (!valid) continue;
-      if (EPI == EPI_I32 ? (o >= g.O) : (o >= g.Ow32 * 32)) continue;  // sign words are written whole, tail bits 0
-      if (EPI == EPI_I32) {
-        if (!g.out_nchw) {
-          int32_t* dst = g.out + m * g.O + o;
-          if (o + 16 <= g.O && (g.O & 3) == 0 && (reinterpret_cast<uintptr_t>(g.out) & 15) == 0) {
+          "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr),
+          "r"(one)
+          : "memory");
+    }
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+
+  if (warp == 8) {
+    // ================= MMA issue: one thread ======================================================================
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 7) | (1u << 10)          // A, B: e2m1
+                             | ((uint32_t)(NT >> 3) << 17)   // N
+                             | (1u << 23)                    // scale factors: ue8m0
+                             | ((uint32_t)(128 >> 4) << 24); // M = 128; both operands K-major; K = 64
+      const uint32_t tsfa = tmem_base + TC_SF_COL, tsfb = tmem_base + TC_SF_COL + 128;
+      const int cgroups = g.C >> 5;  // 32-channel groups (16-byte rows)
+      const uint64_t bdesc0 = make_desc(smem_u32(w_s), (uint32_t)NT * 16, 128);
+      const uint64_t a_step = (uint64_t)(2u * (uint32_t)g.slots), b_step = (uint64_t)(2u * NT);  // one K = 64 block
+      const int kblocks = g.C >> 6;
+#ifdef TC_TIMING
+      long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      long long tlast = clock64();
+#endif
+      int it = 0;
+      for (long long mt = mt_first; mt < g.m_tiles; mt += mt_step, it++) {
+        const int ab = it % g.abufs;
+        TC_T(0);
+        if (!mbar_wait(smem_u32(&bars[4 + ab]), (uint32_t)(it / g.abufs) & 1)) { *s_fail = 1; break; }      // rows written
+        TC_T(1);
+        if (it >= 2 && !mbar_wait(smem_u32(&bars[2 + (it & 1)]), ((it - 2) >> 1) & 1)) { *s_fail = 1; break; }  // accumulator drained
+        TC_T(2);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t d_tmem = tmem_base + (uint32_t)((it & 1) * NT);
+        const uint64_t adesc0 = make_desc(smem_u32(a_s + (size_t)ab * a_bytes), (uint32_t)g.slots * 16, 128);
+        uint32_t accumulate = 0;
+        uint64_t bdesc = bdesc0;  // weights are laid out in issue order: [tap][C/32][NT][16]
+        for (int ti = 0; ti < g.kh; ti++) {
+          uint64_t arow = adesc0 + (uint64_t)(uint32_t)(ti * g.SP);  // start addresses are in 16-byte units
+          for (int tj = 0; tj < g.kw; tj++, arow += 1) {
+            uint64_t adesc = arow;
+#pragma unroll 4
+            for (int kb = 0; kb < kblocks; kb++, adesc += a_step, bdesc += b_step) {
+              asm volatile(
+                  "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                  "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+                  : "memory");
+              accumulate = 1;
+            }
+          }
+        }
+        (void)cgroups;
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                         smem_u32(&bars[it & 1]))
+                     : "memory");
+        TC_T(3);
+      }
+#ifdef TC_TIMING
+      if (blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[16 + i] = prof[i]; }
+#endif
+    }
+  } else if (warp >= 4) {
+    // ================= producer warps: packed bits -> e2m1 rows ===================================================
+    const int ptid = tid - 128;
+    const int cgroups = g.C >> 5;
+    const uint32_t pad_word4 = g.pad_neg ? 0xAAAAAAAAu : 0x22222222u;
+    uint64_t words[2][TC_MAX_CW];
+    int kind[2];  // 0: inside the image (words valid), 1: padding, 2: beyond the batch, 3: no such slot
+    auto prefetch = [&](long long mt) {
 #pragma unroll
-            for (int j = 0; j < 16; j += 4)
-              *reinterpret_cast<int4*>(dst + j) = make_int4((int)v[j], (int)v[j + 1], (int)v[j + 2], (int)v[j + 3]);
+      for (int h = 0; h < 2; h++) {
+        const int s = ptid + 128 * h;
+        kind[h] = 3;
+        if (s < g.slots) {
+          const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)s;  // total_q < 2^31 is checked on the host
+          const uint32_t rr = Q / (uint32_t)g.SP;
+          const int col = (int)(Q - rr * (uint32_t)g.SP);
+          const uint32_t n = rr / (uint32_t)g.HP;
+          const int r = (int)(rr - n * (uint32_t)g.HP);
+          const int ih = r - g.ph, iw = col - g.pw;
+          if (n >= (uint32_t)g.N) kind[h] = 2;
+          else if (ih < 0 || ih >= g.H || iw < 0 || iw >= g.W) kind[h] = 1;
+          else {
+            kind[h] = 0;
+            const uint64_t* src = g.a + (((long long)n * g.H + ih) * g.W + iw) * g.Cw;
+#pragma unroll
+            for (int cw = 0; cw < TC_MAX_CW; cw++)
+              if (cw < g.Cw) words[h][cw] = __ldg(src + cw);
+          }
+        }
+      }
+    };
+    auto expand = [&](uint8_t* abuf) {
+#pragma unroll
+      for (int h = 0; h < 2; h++) {
+        if (kind[h] == 3) continue;
+        const int s = ptid + 128 * h;
+#pragma unroll
+        for (int cw = 0; cw < TC_MAX_CW; cw++) {
+          if (cw >= g.Cw) break;
+#pragma unroll
+          for (int q2 = 0; q2 < 2; q2++) {  // a 64-bit word = two 32-channel rows
+            const int grp = cw * 2 + q2;
+            if (grp >= cgroups) break;
+            uint4 bytes;
+            if (kind[h] == 0) {
+              const uint32_t half = (uint32_t)(words[h][cw] >> (32 * q2));
+              bytes = expand32(half);
+            } else if (kind[h] == 2) bytes = make_uint4(0, 0, 0, 0);
+            else bytes = make_uint4(pad_word4, pad_word4, pad_word4, pad_word4);
+            *reinterpret_cast<uint4*>(abuf + ((size_t)grp * g.slots + s) * 16) = bytes;
+          }
+        }
+      }
+    };
+
+    int it = 0;
+#ifdef TC_TIMING
+    long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long tlast = clock64();
+#endif
+    if (mt_first < g.m_tiles) prefetch(mt_first);
+    for (long long mt = mt_first; mt < g.m_tiles; mt += mt_step, it++) {
+      const int ab = it % g.abufs;
+      TC_T(0);
+      const int j = it - g.abufs;  // the tile whose MMAs last read this A buffer
+      if (j >= 0 && !mbar_wait(smem_u32(&bars[j & 1]), (uint32_t)(j >> 1) & 1)) { *s_fail = 1; break; }
+      TC_T(1);
+      expand(a_s + (size_t)ab * a_bytes);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+      mbar_arrive(smem_u32(&bars[4 + ab]));
+      TC_T(2);
+      if (mt + mt_step < g.m_tiles) prefetch(mt + mt_step);  // in flight while the tensor core works
+      if (*s_fail != 0) break;
+    }
+#ifdef TC_TIMING
+    if (ptid == 0 && blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[i] = prof[i]; g_tc_prof[15] = it; }
+#endif
+  } else {
+    // ================= epilogue warps: TMEM accumulator -> output ===============================================
+    int it = 0;
+#ifdef TC_TIMING
+    long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long tlast = clock64();
+#endif
+    for (long long mt = mt_first; mt < g.m_tiles; mt += mt_step, it++) {
+      const int buf = it & 1;
+      TC_T(0);
+      if (!mbar_wait(smem_u32(&bars[buf]), (it >> 1) & 1)) {
+        *s_fail = 1;
+        break;
+      }
+      TC_T(1);
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int row = 32 * warp + lane;  // TMEM lane = slot row of the tile
+      const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)row;
+      const uint32_t rr = Q / (uint32_t)g.SP;
+      const int col = (int)(Q - rr * (uint32_t)g.SP);
+      const uint32_t n = rr / (uint32_t)g.HP;
+      const int r = (int)(rr - n * (uint32_t)g.HP);
+      const int my_valid = (n < (uint32_t)g.N && r < g.OH && col < g.OW) ? 1 : 0;
+      const int my_m = (int)((n * (uint32_t)g.OH + (uint32_t)r) * (uint32_t)g.OW + (uint32_t)col);  // < 2^31 (host check)
+      const long long m = my_m;
+      // wide outputs: 256-bit accesses when rows are 32-byte multiples at 32-byte aligned addresses
+      const bool wide_i32 = EPI == EPI_I32 && !g.out_nchw && (g.O & 7) == 0 && (reinterpret_cast<uintptr_t>(g.out) & 31) == 0;
+      const bool wide_y = EPI == EPI_BIREAL && (g.O & 7) == 0 &&
+                          ((reinterpret_cast<uintptr_t>(g.residual) | reinterpret_cast<uintptr_t>(g.y_out)) & 31) == 0;
+#pragma unroll 1
+      for (int c0 = 0; c0 < NT; c0 += 32) {
+        __syncwarp();  // the TMEM load is warp-wide: rejoin lanes that took different paths below
+        uint32_t v[32];
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)(buf * NT + c0);
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+            "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+              "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+              "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+              "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+            : "r"(taddr));
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        const int o = nt * NT + c0;  // first of the 32 channels of this chunk; the lane owns them all for its row
+        if (!my_valid) continue;
+        const int nch = min(32, g.O - o);  // channels of this chunk that exist (<= 0: none)
+        if (EPI == EPI_I32) {
+          if (nch <= 0) continue;
+          if (wide_i32) {
+            int32_t* dst = g.out + m * g.O + o;
+#pragma unroll
+            for (int q = 0; q < 4; q++)
+              if (8 * q < nch)  // nch is a multiple of 8 here
+                st_global_v8(dst + 8 * q, (uint32_t)__float2int_rn(__uint_as_float(v[8 * q])),
+                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 1])),
+                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 2])),
+                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 3])),
+                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 4])),
+                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 5])),
+                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 6])),
+                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 7])));
+          } else if (!g.out_nchw) {
+            int32_t* dst = g.out + m * g.O + o;
+#pragma unroll
+            for (int j = 0; j < 32; j++)
+              if (j < nch) dst[j] = __float2int_rn(__uint_as_float(v[j]));
           } else {
+            const long long ohw = (long long)g.OH * g.OW;
+            const long long nn = m / ohw, q = m - nn * ohw;
 #pragma unroll
-            for (int j = 0; j < 16; j++)
-              if (o + j < g.O) dst[j] = (int)v[j];
+            for (int j = 0; j < 32; j++)
+              if (j < nch) g.out[(nn * g.O + o + j) * ohw + q] = __float2int_rn(__uint_as_float(v[j]));
           }
         } else {
-          const long long ohw = (long long)g.OH * g.OW, q = (long long)r * g.OW + col;
+          if (o >= g.Ow32 * 32) continue;  // sign words are written whole (tail bits 0), nothing beyond them
+          float y[32];
 #pragma unroll
-          for (int j = 0; j < 16; j++)
-            if (o + j < g.O) g.out[(n * g.O + o + j) * ohw + q] = (int)v[j];
-        }
-      } else {
-        float y[16];
+          for (int q = 0; q < 8; q++) {  // channels beyond O have scale = shift = 0: y = +0
+            const float4 sc = *reinterpret_cast<const float4*>(s_scale + c0 + 4 * q);
+            const float4 sh = *reinterpret_cast<const float4*>(s_shift + c0 + 4 * q);
+            y[4 * q] = __fmaf_rn(__uint_as_float(v[4 * q]), sc.x, sh.x);
+            y[4 * q + 1] = __fmaf_rn(__uint_as_float(v[4 * q + 1]), sc.y, sh.y);
+            y[4 * q + 2] = __fmaf_rn(__uint_as_float(v[4 * q + 2]), sc.z, sh.z);
+            y[4 * q + 3] = __fmaf_rn(__uint_as_float(v[4 * q + 3]), sc.w, sh.w);
+          }
+          if (EPI == EPI_BIREAL && nch > 0) {
+            const float* rs = g.residual + m * g.O + o;
+            float* yd = g.y_out + m * g.O + o;
+            if (wide_y) {
 #pragma unroll
-        for (int j = 0; j < 16; j++)
-          y[j] = (o + j < g.O) ? __fmaf_rn((float)(int)v[j], g.scale[o + j], g.shift[o + j]) : 0.0f;
-        if (EPI == EPI_BIREAL) {
-          const float* rs = g.residual + m * g.O + o;
-          float* yd = g.y_out + m * g.O + o;
-          if (o + 16 <= g.O && (g.O & 3) == 0 &&
-              ((reinterpret_cast<uintptr_t>(g.residual) | reinterpret_cast<uintptr_t>(g.y_out)) & 15) == 0) {
+              for (int q = 0; q < 4; q++)
+                if (8 * q < nch) {  // nch is a multiple of 8 here
+                  float r8[8];
+                  ld_global_v8(rs + 8 * q, r8);
 #pragma unroll
-            for (int j = 0; j < 16; j += 4) {
-              const float4 r4 = *reinterpret_cast<const float4*>(rs + j);
-              y[j] = __fadd_rn(y[j], r4.x);
-              y[j + 1] = __fadd_rn(y[j + 1], r4.y);
-              y[j + 2] = __fadd_rn(y[j + 2], r4.z);
-              y[j + 3] = __fadd_rn(y[j + 3], r4.w);
-              *reinterpret_cast<float4*>(yd + j) = make_float4(y[j], y[j + 1], y[j + 2], y[j + 3]);
+                  for (int j = 0; j < 8; j++) y[8 * q + j] = __fadd_rn(y[8 * q + j], r8[j]);
+                  st_global_v8(yd + 8 * q, __float_as_uint(y[8 * q]), __float_as_uint(y[8 * q + 1]), __float_as_uint(y[8 * q + 2]),
+                               __float_as_uint(y[8 * q + 3]), __float_as_uint(y[8 * q + 4]), __float_as_uint(y[8 * q + 5]),
+                               __float_as_uint(y[8 * q + 6]), __float_as_uint(y[8 * q + 7]));
+                }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j++)
+                if (j < nch) {
+                  y[j] = __fadd_rn(y[j], rs[j]);
+                  yd[j] = y[j];
+                }
             }
-          } else {
+          }
+          if (g.out_packed32 != nullptr) {
+            uint32_t word = 0;
 #pragma unroll
-            for (int j = 0; j < 16; j++)
-              if (o + j < g.O) {
-                y[j] = __fadd_rn(y[j], rs[j]);
-                yd[j] = y[j];
-              }
+            for (int j = 0; j < 32; j++) word |= (uint32_t)(j < nch && y[j] < 0.0f) << j;
+            g.out_packed32[m * g.Ow32 + (o >> 5)] = word;
           }
         }
-        if (g.out_packed32 != nullptr) {
-          uint32_t field = 0;
-#pragma unroll
-          for (int j = 0; j < 16; j++) field |= (uint32_t)((o + j < g.O) && (y[j] < 0.0f)) << j;
-          // 16 channels = half of a 32-bit sign word
-          reinterpret_cast<uint16_t*>(g.out_packed32)[(m * g.Ow32 + (o >> 5)) * 2 + ((o >> 4) & 1)] = (uint16_t)field;
-        }
       }
+      // this accumulator buffer may be overwritten by the tile after next
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      mbar_arrive(smem_u32(&bars[2 + buf]));
+      TC_T(2);
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  };
-
-  int it = 0;
-  long long prev_mt = -1;
-  bool failed = false;
-  for (long long mt = mt_first; mt < g.m_tiles; mt += mt_step, it++) {
-    if (it > 0) {
-      // the previous tile's MMAs must be complete before its A rows are overwritten
-      if (!mbar_wait(smem_u32(&bars[(it - 1) & 1]), ((it - 1) >> 1) & 1)) *s_fail = 1;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    }
-    // ---- expand this tile's slots: bits -> int8 rows ------------------------------------------------------------
-    const long long q0 = mt * 128;
-    for (int s = tid; s < g.slots; s += TC_THREADS) {
-      const long long Q = q0 + s;
-      const int col = (int)(Q % g.SP);
-      const long long rr = Q / g.SP;
-      const int r = (int)(rr % g.HP);
-      const long long n = rr / g.HP;
-      const int ih = r - g.ph, iw = col - g.pw;
-      const bool beyond = n >= g.N;
-      const bool inside = !beyond && ih >= 0 && ih < g.H && iw >= 0 && iw < g.W;
-      const uint64_t* src = g.a + ((n * g.H + ih) * g.W + iw) * g.Cw;
-      for (int cw = 0; cw < g.Cw; cw++) {
-        uint64_t word = 0;
-        if (inside) word = src[cw];
-#pragma unroll
-        for (int q4 = 0; q4 < 4; q4++) {
-          const int grp = cw * 4 + q4;
-          if (grp >= cgroups) break;
-          uint4 bytes;
-          if (inside) bytes = expand16((uint32_t)(word >> (16 * q4)) & 0xFFFFu);
-          else if (beyond) bytes = make_uint4(0, 0, 0, 0);
-          else bytes = make_uint4(pad_word4, pad_word4, pad_word4, pad_word4);
-          *reinterpret_cast<uint4*>(a_s + ((size_t)grp * g.slots + s) * 16) = bytes;
-        }
-      }
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    failed = *s_fail != 0;
-    if (failed) break;
-    if (tid == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t d_tmem = tmem_base + (uint32_t)((it & 1) * NT);
-      const uint32_t a_base = smem_u32(a_s), w_base = smem_u32(w_s);
-      uint32_t accumulate = 0;
-      for (int ti = 0; ti < g.kh; ti++)
-        for (int tj = 0; tj < g.kw; tj++) {
-          const int tap = ti * g.kw + tj;
-          const uint32_t shift = (uint32_t)(ti * g.SP + tj);
-          for (int kb = 0; kb < (g.C >> 5); kb++) {
-            const uint64_t adesc = make_desc(a_base + ((uint32_t)(2 * kb) * g.slots + shift) * 16, a_lbo, 128);
-            const uint64_t bdesc = make_desc(w_base + (uint32_t)((tap * cgroups + 2 * kb) * NT) * 16, w_lbo, 128);
-            asm volatile(
-                "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-                ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-                : "memory");
-            accumulate = 1;
-          }
-        }
-      asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                       smem_u32(&bars[it & 1]))
-                   : "memory");
-    }
-    if (it > 0) epilogue(prev_mt, (it - 1) & 1);  // overlaps the tensor core working on this tile
-    prev_mt = mt;
-  }
-  if (!failed && it > 0) {
-    if (mbar_wait(smem_u32(&bars[(it - 1) & 1]), ((it - 1) >> 1) & 1)) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      epilogue(prev_mt, (it - 1) & 1);
-    } else {
-      *s_fail = 1;
-    }
+#ifdef TC_TIMING
+    if (tid == 0 && blockIdx.x == 0) { for (int i = 0; i < 4; i++) g_tc_prof[8 + i] = prof[i]; }
+#endif
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (*s_fail != 0 && tid == 0) atomicExch(&g_tc_error, 1);
   if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TC_TMEM_COLS)
                  : "memory");
   }
 }
 
-// Weights: packed bits [O][taps][Cw] -> int8 [n_ntiles][taps][C/16][NT][16].
+// Weights: packed bits [O][taps][Cw] -> e2m1 [n_ntiles][taps][C/32][NT][16 bytes = 32 channels].
 __global__ void tc_prepare_weights_kernel(const uint64_t* __restrict__ wp, int O, int taps, int Cw, int cgroups, int NT,
                                           long long units, uint4* __restrict__ out) {
   const long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -333,18 +483,18 @@ __global__ void tc_prepare_weights_kernel(const uint64_t* __restrict__ wp, int O
   const int tap = (int)(t % taps);
   const int nt = (int)(t / taps);
   const int o = nt * NT + n;
-  uint4 bytes = make_uint4(0, 0, 0, 0);  // channels beyond O contribute nothing
+  uint4 bytes = make_uint4(0, 0, 0, 0);  // channels beyond O contribute nothing (e2m1 zero)
   if (o < O) {
-    const uint64_t word = wp[((long long)o * taps + tap) * Cw + (grp >> 2)];
-    bytes = expand16((uint32_t)(word >> (16 * (grp & 3))) & 0xFFFFu);
+    const uint32_t half = (uint32_t)(wp[((long long)o * taps + tap) * Cw + (grp >> 1)] >> (32 * (grp & 1)));
+    bytes = expand32(half);
   }
   out[u] = bytes;
 }
 
 int tc_ntile(int O, int C, int taps) {
-  const long long K = (long long)C * taps;
+  const long long Kb = (long long)C / 2 * taps;  // bytes per weight row
   for (int nt = 128; nt >= 32; nt >>= 1) {
-    if (nt * K > TC_WEIGHT_BUDGET) continue;
+    if (nt * Kb > TC_WEIGHT_BUDGET) continue;
     if (nt > 32 && nt / 2 >= O) continue;  // do not pad a small O to a wide tile
     return nt;
   }
@@ -375,7 +525,9 @@ dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
 
 template <int EPI>
 dabnn_status tc_dispatch(TcArgs& g, cudaStream_t st) {
-  const size_t smem = (size_t)g.ntile * g.kh * g.kw * g.C + (size_t)g.slots * g.C + TC_SMEM_MISC;
+  const size_t wbytes = (size_t)g.ntile * g.kh * g.kw * (g.C / 2), abytes = (size_t)g.slots * (g.C / 2);
+  g.abufs = (wbytes + 2 * abytes + TC_SMEM_MISC <= (size_t)TC_SMEM_LIMIT) ? 2 : 1;
+  const size_t smem = wbytes + g.abufs * abytes + TC_SMEM_MISC;
   if (smem > (size_t)TC_SMEM_LIMIT) return DABNN_ERR_UNSUPPORTED;
   switch (g.ntile) {
     case 128: return tc_launch<128, EPI>(g, smem, st);
@@ -395,7 +547,7 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   const int OH = dabnn_out_dim(in.H, cv.kh, cv.stride_h, cv.pad_h), OW = dabnn_out_dim(in.W, cv.kw, cv.stride_w, cv.pad_w);
   if (OH <= 0 || OW <= 0) return DABNN_ERR_SHAPE;
   // what this engine covers; everything else is served by the xor/popcount kernel
-  if (cv.stride_h != 1 || cv.stride_w != 1 || in.C % 32 != 0) return DABNN_ERR_UNSUPPORTED;
+  if (cv.stride_h != 1 || cv.stride_w != 1 || in.C % 64 != 0) return DABNN_ERR_UNSUPPORTED;
   const int nt = tc_ntile(O, in.C, cv.kh * cv.kw);
   if (nt == 0) return DABNN_ERR_UNSUPPORTED;
   g.a = a; g.w_tc = static_cast<const uint8_t*>(w_tc);
@@ -404,10 +556,10 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   g.SP = in.W + 2 * cv.pad_w; g.HP = in.H + 2 * cv.pad_h;
   g.total_q = (long long)in.N * g.HP * g.SP;
   g.slots = (128 + (cv.kh - 1) * g.SP + (cv.kw - 1) + 7) / 8 * 8;
-  if (g.slots > 16383) return DABNN_ERR_UNSUPPORTED;
+  if (g.slots > TC_MAX_SLOTS || g.Cw > TC_MAX_CW || g.total_q + 512 >= (1LL << 31)) return DABNN_ERR_UNSUPPORTED;
   g.ntile = nt; g.n_ntiles = tc_n_ntiles(O, nt);
   g.m_tiles = (g.total_q + 127) / 128;
-  if ((long long)in.N * OH * OW * O > (1LL << 40)) return DABNN_ERR_UNSUPPORTED;
+  if ((long long)in.N * OH * OW >= (1LL << 31) || (long long)in.N * OH * OW * O > (1LL << 40)) return DABNN_ERR_UNSUPPORTED;
   g.pad_neg = cv.pad_value < 0;
   g.out = nullptr; g.out_nchw = 0; g.scale = g.shift = g.residual = nullptr; g.y_out = nullptr;
   g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64);
@@ -421,21 +573,21 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
 using namespace dabnn;
 
 extern "C" size_t dabnn_tc_weights_bytes(int O, int C, int kh, int kw) {
-  if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0 || C % 32 != 0) return 0;
+  if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0 || C % 64 != 0) return 0;
   const int nt = tc_ntile(O, C, kh * kw);
   if (nt == 0) return 0;
-  return (size_t)tc_n_ntiles(O, nt) * nt * kh * kw * C;
+  return (size_t)tc_n_ntiles(O, nt) * nt * kh * kw * (C / 2);
 }
 
 extern "C" dabnn_status dabnn_tc_prepare_weights(const uint64_t* w_packed, int O, int C, int kh, int kw, void* w_tc,
                                                  void* stream) {
   if (!w_packed || !w_tc) return DABNN_ERR_NULL;
   if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0) return DABNN_ERR_SHAPE;
-  if (C % 32 != 0) return DABNN_ERR_UNSUPPORTED;
+  if (C % 64 != 0) return DABNN_ERR_UNSUPPORTED;
   if (!aligned(w_packed, 8) || !aligned(w_tc, 16)) return DABNN_ERR_ALIGNMENT;
   const int nt = tc_ntile(O, C, kh * kw);
   if (nt == 0) return DABNN_ERR_UNSUPPORTED;
-  const int taps = kh * kw, cgroups = C / 16, n_nt = tc_n_ntiles(O, nt);
+  const int taps = kh * kw, cgroups = C / 32, n_nt = tc_n_ntiles(O, nt);
   const long long units = (long long)n_nt * taps * cgroups * nt;
   tc_prepare_weights_kernel<<<ceil_div(units, 256), 256, 0, as_stream(stream)>>>(w_packed, O, taps, (C + 63) / 64, cgroups,
                                                                                  nt, units, static_cast<uint4*>(w_tc));
@@ -491,3 +643,9 @@ extern "C" int dabnn_tc_error_flag(void) {
   }
   return v;
 }
+
+#ifdef TC_TIMING
+extern "C" int dabnn_tc_debug_read(unsigned long long* out24) {
+  return cudaMemcpyFromSymbol(out24, g_tc_prof, 24 * sizeof(unsigned long long)) == cudaSuccess ? 0 : -1;
+}
+#endif

@@ -34,8 +34,8 @@ TC_CASES = [
     (2, 512, 7, 7, 512, 3, 1, -1),      # channel tiles of 32, K = 4608
     (2, 512, 14, 14, 300, 1, 0, -1),    # 1x1, ragged channel tile
     (1, 64, 56, 56, 64, 3, 1, -1),
-    (2, 96, 10, 10, 70, 5, 2, -1),      # C = 96: half-used last word, 5x5
-    (5, 32, 6, 7, 33, 3, 1, -1),        # smallest C, O just over a tile
+    (2, 192, 10, 10, 70, 5, 2, -1),     # three words, 5x5, O just over one sign word
+    (5, 64, 6, 7, 33, 3, 1, -1),        # smallest C, O just over a 32-channel tile
     (9, 128, 28, 28, 128, 3, 1, -1),    # many pixel tiles per CTA? (persistent loop over tiles)
     (300, 64, 8, 8, 64, 3, 0, -1),      # no padding, many images per tile
 ]
@@ -84,8 +84,8 @@ def test_tc_conv_and_epilogues_match_oracle(B, oracle_mod, case):
 
 def test_tc_declines_what_it_does_not_cover(B):
     assert not B.tc_supported(64, 64, 3, 3, stride=(2, 2))
-    assert not B.tc_supported(64, 70, 3, 3)          # C not a multiple of 32
-    assert not B.tc_supported(64, 1024, 7, 7)        # expanded weights larger than the resident budget
+    assert not B.tc_supported(64, 96, 3, 3)          # C not a multiple of 64
+    assert not B.tc_supported(64, 2048, 7, 7)        # expanded weights larger than the resident budget
     a = torch.zeros((1, 8, 8, 1), dtype=torch.int64, device="cuda")
     wt = B.TcWeights(torch.zeros((64, 3, 3, 1), dtype=torch.int64, device="cuda"), 64)
     with pytest.raises(B.DabnnError, match="supported"):
