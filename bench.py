@@ -53,6 +53,17 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
 
 
+def measured_tensor_peak_tops():
+    """Dense 4-bit (e2m1) tensor peak for the roofline: the measured bf16 burst peak x the nominal fp4 : bf16 ratio (4)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"tops": float(d["bf16_tflops"]) * 4.0,
+                "how": "measured bf16 burst peak %.0f TFLOP/s x 4 (nominal dense fp4 : bf16 ratio), of measured" % float(d["bf16_tflops"])}
+    return {"tops": 1590.0 * 4.0, "how": "fallback bf16 peak 1590 TFLOP/s x 4 (nominal dense fp4 : bf16 ratio), of fallback"}
+
+
 def bitop_peak_tbitops(sm_count, sm_mhz):
     """Carry-save bound of sum popcount(a xor w) on the B200 integer pipes: with one POPC (XU pipe, 16 lanes/clk/SM)
     and four logic ops (ALU pipe, 64 lanes/clk/SM) per two 32-bit word pairs both pipes are full at 32 word pairs
@@ -220,9 +231,12 @@ def main():
             "bits": torch.empty((BATCH, HW, HW, (C + 63) // 64), dtype=torch.int64, device=dev),
             "bitops": conv_bitops(BATCH, C, HW, C, 3),
         }
+        L["wt"] = B.TcWeights(L["w"], C)  # the same weights expanded once for the tensor-core engine
         L["call_pack"] = B.prepare_pack(L["x"], L["a"])
-        L["call_conv"] = B.prepare_bconv2d(L["a"], C, L["w"], L["out"], (1, 1), (1, 1), -1, B.NHWC)
-        L["call_fused"] = B.prepare_bconv2d_bn_sign_pack(L["a"], C, L["w"], L["scale"], L["shift"], L["bits"], (1, 1), (1, 1), -1)
+        L["call_conv"] = {"popc": B.prepare_bconv2d(L["a"], C, L["w"], L["out"], (1, 1), (1, 1), -1, B.NHWC),
+                          "tc": B.prepare_tc_bconv2d(L["a"], L["wt"], L["out"], (1, 1), (1, 1), -1, B.NHWC)}
+        L["call_fused"] = {"popc": B.prepare_bconv2d_bn_sign_pack(L["a"], C, L["w"], L["scale"], L["shift"], L["bits"], (1, 1), (1, 1), -1),
+                           "tc": B.prepare_tc_bconv2d_bn_sign_pack(L["a"], L["wt"], L["scale"], L["shift"], L["bits"], (1, 1), (1, 1), -1)}
         L["out_host"] = torch.empty(L["out"].shape, dtype=torch.int32).pin_memory()
         L["bits_host"] = torch.empty(L["bits"].shape, dtype=torch.int64).pin_memory()
         ws_bytes = B.binary_layer_host_workspace_bytes(BATCH, C, HW, HW, C, 3, 3, (1, 1), (1, 1), -1)
@@ -230,22 +244,12 @@ def main():
         layers.append(L)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)  # larger than the 126 MB L2
 
-    conv_events = []  # (start, end, bitops) of every convolution launch in the timed region
-
-    def step(record):
+    def step(engine, convs_only=False):
         for L in layers:
-            L["call_pack"]()
-            for fused in (False, True):
-                if record:
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                if fused:
-                    L["call_fused"]()
-                else:
-                    L["call_conv"]()
-                if record:
-                    e1.record()
-                    conv_events.append((e0, e1, L["bitops"], fused))
+            if not convs_only:
+                L["call_pack"]()
+            L["call_conv"][engine]()
+            L["call_fused"][engine]()
     launches_per_step = 3 * len(layers)
 
     def barrier():
@@ -253,33 +257,52 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    def capture(fn):
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                fn()
+        torch.cuda.current_stream().wait_stream(side)
+        return graph
+
+    def timed_replays(graph, n):
+        """n replays, L2 flushed before each (outside its event pair); returns the per-replay device times in ms."""
+        st = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        en = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for k in range(n):
+            flush.zero_()
+            st[k].record()
+            graph.replay()
+            en[k].record()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in zip(st, en)]
+
     for _ in range(warmup):
-        step(False)
+        step("tc")
+        step("popc")
     barrier()
-    # the step as a CUDA graph: one host call per step, so the timed loop is never host-bound
-    side = torch.cuda.Stream()
-    side.wait_stream(torch.cuda.current_stream())
-    with torch.cuda.stream(side):
-        step(False)
-        side.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            step(False)
-    torch.cuda.current_stream().wait_stream(side)
+    # each step is one CUDA-graph replay (one host call), so the timed loop is never host-bound
+    g_step = {e: capture(lambda e=e: step(e)) for e in ("tc", "popc")}
+    g_conv = {e: capture(lambda e=e: step(e, convs_only=True)) for e in ("tc", "popc")}
     for _ in range(warmup):
-        graph.replay()
+        g_step["tc"].replay()
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.05)
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     barrier()
     host_t0 = time.perf_counter()
+    # ---- the timed region: K steps with the faster (tensor-core) engine ------------------------------------------
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     for k in range(args.steps):
         flush.zero_()  # evict the previous step's data from L2 (outside the step's event pair)
         starts[k].record()
-        graph.replay()
+        g_step["tc"].replay()
         ends[k].record()
     host_issue_ms = (time.perf_counter() - host_t0) * 1e3  # time the host needed to enqueue everything
     barrier()
@@ -290,30 +313,30 @@ def main():
     total_ms = float(total_ms.item())
     value = world * step_bitops(BATCH) * args.steps / (total_ms * 1e-3) / 1e9
 
-    # the same steps again, launch by launch, with an event pair around every convolution.  Each step starts
-    # behind a GPU-side delay so that the host has enqueued the whole step before its first kernel runs: the
-    # event pairs then bracket GPU execution only, never host launch latency.
-    for k in range(args.steps):
-        flush.zero_()
-        torch.cuda._sleep(int(1.5e6))
-        step(True)
-    barrier()
+    # ---- the dominant kernels on their own: the eight convolution launches of a step, per engine ------------------
+    conv_ms = {e: timed_replays(g_conv[e], args.steps) for e in ("tc", "popc")}
+    popc_step_ms = timed_replays(g_step["popc"], args.steps)
     clocks = sampler.stop()
-
-    # dominant kernel: the convolution launches, timed one by one inside the timed region
-    conv_ms = sum(e0.elapsed_time(e1) for e0, e1, _, _ in conv_events)
-    conv_ops = sum(b for _, _, b, _ in conv_events)
-    achieved = conv_ops / (conv_ms * 1e-3) / 1e12
-    peak = bitop_peak_tbitops(sm_count, peaks["sm_max_mhz"])
+    conv_ops = step_bitops(BATCH)
+    tc_ms, popc_ms = sum(conv_ms["tc"]) / args.steps, sum(conv_ms["popc"]) / args.steps
+    tensor_peak = measured_tensor_peak_tops()
+    alu_peak = bitop_peak_tbitops(sm_count, peaks["sm_max_mhz"])
     roofline = {
-        "bound": "alu", "kernel": "bconv_kernel (all 8 launches of a step)", "achieved": achieved, "peak": peak,
-        "unit": "Tbit-ops/s", "frac": achieved / peak,
-        "peak_is": "ALU+XU carry-save bound at %d SMs x %.0f MHz (derived, see DESIGN.md); one-POPC-per-word-pair bound is half of it"
+        "bound": "tensor", "kernel": "bconv_tc_kernel (the 8 convolution launches of a step, one CUDA-graph replay)",
+        "achieved": conv_ops / (tc_ms * 1e-3) / 1e12, "peak": tensor_peak["tops"], "unit": "TFLOP/s",
+        "frac": conv_ops / (tc_ms * 1e-3) / 1e12 / tensor_peak["tops"], "peak_is": tensor_peak["how"],
+        "traffic": None, "avg_launch_ms": tc_ms / 8, "conv_share_of_step": tc_ms / (sum(step_ms) / args.steps),
+        "note": "1 bit-op = 1 op: a +-1 multiply-add counts 2, as in FLOPs",
+    }
+    roofline_bitop = {
+        "bound": "alu", "kernel": "bconv_kernel (integer pipes: xor + carry-save + popc), same 8 launches",
+        "achieved": conv_ops / (popc_ms * 1e-3) / 1e12, "peak": alu_peak, "unit": "Tbit-ops/s",
+        "frac": conv_ops / (popc_ms * 1e-3) / 1e12 / alu_peak,
+        "peak_is": "ALU+XU carry-save bound at %d SMs x %.0f MHz (derived, see DESIGN.md); the one-POPC-per-word-pair bound is half of it"
                    % (sm_count, peaks["sm_max_mhz"]),
-        "traffic": None, "avg_launch_ms": conv_ms / max(1, len(conv_events)),
-        "conv_share_of_step": (conv_ms / args.steps) / (sum(step_ms) / args.steps),
-        "timed": "CUDA events around each of the %d convolution launches of %d eager steps (L2 flushed before each step)"
-                 % (len(conv_events), args.steps),
+        "traffic": 2.69e6, "traffic_is": "dram bytes of one N=64 C=256 28x28 launch (ncu, profiles/bconv_kernel_N64_C256_HW28.md)",
+        "avg_launch_ms": popc_ms / 8,
+        "step_value_with_this_engine": step_bitops(BATCH) / (sum(popc_step_ms) / args.steps * 1e-3) / 1e9,
     }
 
     # ---- end to end through the host-buffer entry point ----------------------------------------------------------
@@ -346,8 +369,10 @@ def main():
         "dtype": "u64 words / int32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "l2": "flushed between timed steps (256 MB write)",
                    "launch": "each step is one CUDA-graph replay of its 12 kernels",
+                   "engine": "tensor-core engine (e2m1 tcgen05) for the timed steps; the integer-pipe engine is timed beside it (roofline_bitop)",
                    "parallelism": "replicas" if world > 1 else "single GPU"},
-        "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        "roofline": roofline, "roofline_bitop": roofline_bitop, "e2e": e2e,
+        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
         "host_issue_ms_per_step": host_issue_ms / args.steps,
     }
 
@@ -416,16 +441,20 @@ def extras(B, torch, dev, peaks, sm_count):
 
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     peak = bitop_peak_tbitops(sm_count, peaks["sm_max_mhz"])
+    tpeak = measured_tensor_peak_tops()["tops"]
     for name, (N, C, HW, O, k, pad) in {"conv_256x256x28x28_3x3": (256, 256, 28, 256, 3, 1),
                                         "conv_256x512x14x14_1x1_to_2048": (256, 512, 14, 2048, 1, 0)}.items():
         g = torch.Generator(device=dev); g.manual_seed(5)
         a = torch.randint(-2**62, 2**62, (N, HW, HW, (C + 63) // 64), dtype=torch.int64, device=dev, generator=g)
         w = torch.randint(-2**62, 2**62, (O, k, k, (C + 63) // 64), dtype=torch.int64, device=dev, generator=g)
         o = torch.empty((N, HW, HW, O), dtype=torch.int32, device=dev)
-        med, best = time_fn(lambda: B.bconv2d(a, C, w, (1, 1), (pad, pad), -1, B.NHWC, out=o), 10, flush)
+        wt = B.TcWeights(w, C)
         ops = conv_bitops(N, C, HW, O, k)
-        out[name] = {"ms": med, "Tbit-ops/s": ops / med / 1e9, "frac_of_bitop_peak": ops / med / 1e9 / peak}
-        del a, w, o
+        med, best = time_fn(lambda: B.bconv2d(a, C, w, (1, 1), (pad, pad), -1, B.NHWC, out=o), 10, flush)
+        out[name] = {"int_pipes": {"ms": med, "Tbit-ops/s": ops / med / 1e9, "frac_of_bitop_peak": ops / med / 1e9 / peak}}
+        med, best = time_fn(lambda: B.tc_bconv2d(a, wt, (1, 1), (pad, pad), -1, B.NHWC, out=o), 10, flush)
+        out[name]["tensor"] = {"ms": med, "Tbit-ops/s": ops / med / 1e9, "frac_of_fp4_peak": ops / med / 1e9 / tpeak}
+        del a, w, o, wt
 
     # batch-1 latency of the four sweep shapes (CUDA-graph replay of 50 launches)
     for C, HW in synth.SWEEP_SHAPES:
@@ -450,7 +479,11 @@ def extras(B, torch, dev, peaks, sm_count):
     img = torch.from_numpy(synth.bireal18_images(128)).to(dev)
     logits = torch.empty((128, 1000), dtype=torch.float32, device=dev)
     med, best = time_fn(lambda: net.forward(img, logits), 5)
-    out["bireal18_batch128"] = {"ms": med, "images/s": 128 / med * 1e3}
+    out["bireal18_batch128"] = {"ms": med, "images/s": 128 / med * 1e3, "engine": "tensor-core engine on the 13 stride-1 blocks"}
+    net_p = B.Bireal18(synth.bireal18_params(), engine="popc")
+    med, best = time_fn(lambda: net_p.forward(img, logits), 5)
+    out["bireal18_batch128_int_pipes"] = {"ms": med, "images/s": 128 / med * 1e3}
+    del net_p
     img1, logits1 = img[:1].contiguous(), torch.empty((1, 1000), dtype=torch.float32, device=dev)
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):

@@ -112,6 +112,9 @@ typedef struct {
   const float* down_shift[3];
   const float* fc_w;             /* fp32 [1000][512] */
   const float* fc_b;             /* fp32 [1000] */
+  const void* block_w_tc[16];    /* optional: weights expanded by dabnn_tc_prepare_weights, or NULL.  Where given and the
+                                    layer is covered by the tensor-core engine (the 13 stride-1 blocks), that engine runs
+                                    the block; results are identical either way */
 } dabnn_bireal18_params;
 
 /* Bytes of device workspace dabnn_bireal18_forward needs for a batch of N images (0 if N <= 0). */

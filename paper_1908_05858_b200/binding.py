@@ -50,6 +50,7 @@ class Bireal18Params(ctypes.Structure):
         ("block_w", ctypes.c_void_p * 16), ("block_scale", ctypes.c_void_p * 16), ("block_shift", ctypes.c_void_p * 16),
         ("down_w", ctypes.c_void_p * 3), ("down_scale", ctypes.c_void_p * 3), ("down_shift", ctypes.c_void_p * 3),
         ("fc_w", ctypes.c_void_p), ("fc_b", ctypes.c_void_p),
+        ("block_w_tc", ctypes.c_void_p * 16),
     ]
 
 
@@ -231,7 +232,8 @@ class Bireal18:
     """Device-resident Bi-Real Net 18 parameters, prepared once with the library's own kernels
     (weights packed by dabnn_pack_weights, BN folded by dabnn_bn_fold)."""
 
-    def __init__(self, params: dict, device="cuda"):
+    def __init__(self, params: dict, device="cuda", engine: str = "auto"):
+        """engine: "auto" / "tc" = tensor-core engine for the blocks it covers, "popc" = integer-pipe kernel only."""
         dev = torch.device(device)
 
         def up(a):
@@ -248,6 +250,12 @@ class Bireal18:
             sc, sh = bn_fold(*[up(t) for t in params["block_bn"][b]], eps=eps)
             self.keep += [wp, sc, sh]
             P.block_w[b], P.block_scale[b], P.block_shift[b] = wp.data_ptr(), sc.data_ptr(), sh.data_ptr()
+            O_b, C_b = int(params["block_w"][b].shape[0]), int(params["block_w"][b].shape[1])
+            stride_b = 2 if (b % 4 == 0 and b > 0) else 1
+            if engine != "popc" and tc_supported(O_b, C_b, 3, 3, (stride_b, stride_b)):
+                wt = TcWeights(wp, C_b)
+                self.keep.append(wt)
+                P.block_w_tc[b] = wt.buf.data_ptr()
         for d in range(3):
             w = up(params["down_w"][d])
             sc, sh = bn_fold(*[up(t) for t in params["down_bn"][d]], eps=eps)
@@ -425,6 +433,21 @@ def prepare_bconv2d_bn_sign_pack(a_packed, C, w_packed, scale, shift, out, strid
     return Prepared(lib().dabnn_bconv2d_bn_sign_pack,
                     (a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O, _conv(kh, kw, stride, pad, pad_value),
                      scale.data_ptr(), shift.data_ptr(), out.data_ptr()), (a, w, scale, shift, out))
+
+
+def prepare_tc_bconv2d(a_packed, wt: TcWeights, out, stride=(1, 1), pad=(0, 0), pad_value=-1, out_layout=NHWC) -> Prepared:
+    a, N, H, W, OH, OW = _tc_geom(a_packed, wt, stride, pad)
+    return Prepared(lib().dabnn_tc_bconv2d, (a.data_ptr(), Shape(N, wt.C, H, W), wt.buf.data_ptr(), wt.O,
+                                             _conv(wt.kh, wt.kw, stride, pad, pad_value), out.data_ptr(), out_layout),
+                    (a, wt, out))
+
+
+def prepare_tc_bconv2d_bn_sign_pack(a_packed, wt: TcWeights, scale, shift, out, stride=(1, 1), pad=(0, 0),
+                                    pad_value=-1) -> Prepared:
+    a, N, H, W, OH, OW = _tc_geom(a_packed, wt, stride, pad)
+    return Prepared(lib().dabnn_tc_bconv2d_bn_sign_pack,
+                    (a.data_ptr(), Shape(N, wt.C, H, W), wt.buf.data_ptr(), wt.O, _conv(wt.kh, wt.kw, stride, pad, pad_value),
+                     scale.data_ptr(), shift.data_ptr(), out.data_ptr()), (a, wt, scale, shift, out))
 
 
 def set_conv_variant(variant: int) -> int:

@@ -568,6 +568,14 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
 
 }  // namespace
 
+bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv) {
+  if (cv.stride_h != 1 || cv.stride_w != 1 || in.C % 64 != 0 || in.C > 64 * TC_MAX_CW) return false;
+  const int nt = tc_ntile(O, in.C, cv.kh * cv.kw);
+  if (nt == 0) return false;
+  const long long slots_total = (long long)in.N * (in.H + 2 * cv.pad_h) * (in.W + 2 * cv.pad_w);
+  return (slots_total / 128) * tc_n_ntiles(O, nt) >= 2LL * sm_count();
+}
+
 }  // namespace dabnn
 
 using namespace dabnn;

@@ -331,8 +331,13 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     const dabnn_shape in = {N, C, HW, HW};
     const int stride = down ? 2 : 1;
     const dabnn_conv cv = {3, 3, stride, stride, 1, 1, -1};
-    s = dabnn_bconv2d_bn_add_sign_pack(bits_in, in, p->block_w[b], O, cv, p->block_scale[b], p->block_shift[b], cur, cur,
-                                       b == 15 ? nullptr : bits_out, st);
+    s = DABNN_ERR_UNSUPPORTED;
+    if (p->block_w_tc[b] != nullptr && tc_worthwhile(in, O, cv))  // tensor-core engine where it covers the layer and pays
+      s = dabnn_tc_bconv2d_bn_add_sign_pack(bits_in, in, p->block_w_tc[b], O, cv, p->block_scale[b], p->block_shift[b], cur,
+                                            cur, b == 15 ? nullptr : bits_out, st);
+    if (s == DABNN_ERR_UNSUPPORTED)
+      s = dabnn_bconv2d_bn_add_sign_pack(bits_in, in, p->block_w[b], O, cv, p->block_scale[b], p->block_shift[b], cur, cur,
+                                         b == 15 ? nullptr : bits_out, st);
     if (s != DABNN_OK) return s;
     uint64_t* tb = bits_in; bits_in = bits_out; bits_out = tb;
     C = O; HW = OHW;

@@ -26,6 +26,7 @@ def main():
     ap.add_argument("--k", type=int, default=3)
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--reps", type=int, default=1, help="launches per timed event pair")
+    ap.add_argument("--graph", action="store_true", help="time a CUDA-graph replay of the `reps` launches")
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--tile", type=int, default=0)
     ap.add_argument("--engine", default="popc", choices=["popc", "tc"])
@@ -71,6 +72,20 @@ def main():
             work = ("Tbit-ops/s", 2.0 * a.N * a.HW * a.HW * O * a.C * a.k * a.k / 1e12)
     fn()
     torch.cuda.synchronize()
+    if a.graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(a.reps):
+                    fn()
+        torch.cuda.current_stream().wait_stream(side)
+        one, reps = fn, a.reps
+        fn = graph.replay
+        a.reps = 1
     ms = []
     for _ in range(a.iters):
         # `reps` launches back to back inside one event pair, so that launch latency is hidden behind the
@@ -81,7 +96,7 @@ def main():
             fn()
         e1.record()
         torch.cuda.synchronize()
-        ms.append(e0.elapsed_time(e1) / a.reps)
+        ms.append(e0.elapsed_time(e1) / (reps if a.graph else a.reps))
     med = statistics.median(ms)
     line = "%s N=%d C=%d HW=%d O=%d k=%d: median %.4f ms" % (a.case, a.N, a.C, a.HW, O, a.k, med)
     if work:
