@@ -32,80 +32,103 @@ __global__ void bn_fold_kernel(const float* gamma, const float* beta, const floa
 constexpr int STEM_K = 147;
 
 template <int TS, int PPT>
-__global__ void __launch_bounds__((TS * TS / PPT) * 4) stem_conv_bn(const float* __restrict__ img,
-                                                                    const float* __restrict__ w,
-                                                                    const float* __restrict__ scale,
-                                                                    const float* __restrict__ shift,
-                                                                    float* __restrict__ out /*[N][112][112][64]*/) {
+__global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const float* __restrict__ img,
+                                                                       const float* __restrict__ w,
+                                                                       const float* __restrict__ scale,
+                                                                       const float* __restrict__ shift, int N,
+                                                                       float* __restrict__ out /*[N][112][112][64]*/) {
   constexpr int IH = 224, IW = 224, OHW = 112;
   constexpr int PS = 2 * TS + 5;         // patch side
   constexpr int HALF = (PS + 1) / 2 + 1; // columns per parity, padded
+  constexpr int PATCH = 3 * PS * 2 * HALF;  // floats per patch buffer
   constexpr int PGROUPS = TS * TS / PPT; // pixel groups = threads per channel group
   constexpr int THREADS = PGROUPS * 4;
   constexpr int RSTEP = TS / PPT;        // a thread's pixels are RSTEP rows apart
+  constexpr int TILES = (OHW + TS - 1) / TS;
   extern __shared__ __align__(16) float sm[];
-  float* w_s = sm;                       // [147][64]
-  float* x_s = sm + STEM_K * 64;         // [3][PS][2][HALF]
+  float* w_s = sm;                       // [147][64], loaded once per CTA
+  float* x_s = sm + STEM_K * 64;         // [2 buffers][3][PS][2][HALF]
   const int tid = threadIdx.x;
-  const int n = blockIdx.z, oh0 = blockIdx.y * TS, ow0 = blockIdx.x * TS;
   for (int t = tid; t < STEM_K * 64; t += THREADS) {
     const int o = t % 64, k = t / 64;    // w is [64][147]
     w_s[k * 64 + o] = w[o * STEM_K + k];
   }
-  const int ih_base = 2 * oh0 - 3, iw_base = 2 * ow0 - 3;
-  for (int t = tid; t < 3 * PS * PS; t += THREADS) {
-    const int lw = t % PS, lh = (t / PS) % PS, c = t / (PS * PS);
-    const int ih = ih_base + lh, iw = iw_base + lw;
-    float v = 0.0f;
-    if (ih >= 0 && ih < IH && iw >= 0 && iw < IW) v = img[(((size_t)n * 3 + c) * IH + ih) * IW + iw];
-    x_s[((c * PS + lh) * 2 + (lw & 1)) * HALF + (lw >> 1)] = v;
-  }
-  __syncthreads();
+  const long long ntiles = (long long)N * TILES * TILES;
+  // asynchronous copy of one tile's zero-padded input patch (even and odd columns apart)
+  auto load_patch = [&](long long tile, float* dst) {
+    const int n = (int)(tile / (TILES * TILES));
+    const int rem = (int)(tile % (TILES * TILES));
+    const int ih_base = 2 * (rem / TILES) * TS - 3, iw_base = 2 * (rem % TILES) * TS - 3;
+    for (int t = tid; t < 3 * PS * PS; t += THREADS) {
+      const int lw = t % PS, lh = (t / PS) % PS, c = t / (PS * PS);
+      const int ih = ih_base + lh, iw = iw_base + lw;
+      const bool in = ih >= 0 && ih < IH && iw >= 0 && iw < IW;
+      const float* src = in ? img + (((size_t)n * 3 + c) * IH + ih) * IW + iw : img;
+      const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst + ((c * PS + lh) * 2 + (lw & 1)) * HALF + (lw >> 1));
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(d), "l"(src), "r"(in ? 4 : 0) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
   const int cg = tid / PGROUPS;          // channel group: 16 channels
   const int pg = tid % PGROUPS;
   const int low = pg % TS, lohb = pg / TS;  // pixels (lohb + RSTEP*i, low)
-  float acc[PPT][16];
-#pragma unroll
-  for (int i = 0; i < PPT; i++)
-#pragma unroll
-    for (int j = 0; j < 16; j++) acc[i][j] = 0.0f;
-  for (int c = 0; c < 3; c++)
-    for (int ki = 0; ki < 7; ki++) {
-#pragma unroll
-      for (int kj = 0; kj < 7; kj++) {
-        const int k = (c * 7 + ki) * 7 + kj;
-        float wv[16];
-#pragma unroll
-        for (int q = 0; q < 4; q++) {
-          const float4 t4 = *reinterpret_cast<const float4*>(w_s + k * 64 + cg * 16 + 4 * q);
-          wv[4 * q] = t4.x; wv[4 * q + 1] = t4.y; wv[4 * q + 2] = t4.z; wv[4 * q + 3] = t4.w;
-        }
-#pragma unroll
-        for (int i = 0; i < PPT; i++) {
-          const int lh = 2 * (lohb + RSTEP * i) + ki;
-          const float xv = x_s[((c * PS + lh) * 2 + (kj & 1)) * HALF + low + (kj >> 1)];
-#pragma unroll
-          for (int j = 0; j < 16; j++) acc[i][j] = __fmaf_rn(xv, wv[j], acc[i][j]);
-        }
-      }
-    }
   float sc[16], sf[16];
 #pragma unroll
   for (int j = 0; j < 16; j++) {
     sc[j] = scale[cg * 16 + j];
     sf[j] = shift[cg * 16 + j];
   }
+  long long tile = blockIdx.x;
+  int buf = 0;
+  if (tile < ntiles) load_patch(tile, x_s);
+  for (; tile < ntiles; tile += gridDim.x, buf ^= 1) {
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();  // this tile's patch (and, the first time, the weights) are in place; the other buffer is free
+    if (tile + gridDim.x < ntiles) load_patch(tile + gridDim.x, x_s + (buf ^ 1) * PATCH);
+    const float* xb = x_s + buf * PATCH;
+    float acc[PPT][16];
 #pragma unroll
-  for (int i = 0; i < PPT; i++) {
-    const int oh = oh0 + lohb + RSTEP * i, ow = ow0 + low;
-    if (oh >= OHW || ow >= OHW) continue;
-    float* dst = out + (((size_t)n * OHW + oh) * OHW + ow) * 64 + cg * 16;
+    for (int i = 0; i < PPT; i++)
 #pragma unroll
-    for (int j = 0; j < 16; j += 4)
-      *reinterpret_cast<float4*>(dst + j) =
-          make_float4(__fmaf_rn(acc[i][j], sc[j], sf[j]), __fmaf_rn(acc[i][j + 1], sc[j + 1], sf[j + 1]),
-                      __fmaf_rn(acc[i][j + 2], sc[j + 2], sf[j + 2]), __fmaf_rn(acc[i][j + 3], sc[j + 3], sf[j + 3]));
+      for (int j = 0; j < 16; j++) acc[i][j] = 0.0f;
+#pragma unroll 1
+    for (int c = 0; c < 3; c++)
+#pragma unroll 1
+      for (int ki = 0; ki < 7; ki++) {  // one row of taps per iteration keeps the loop body inside the instruction cache
+#pragma unroll
+        for (int kj = 0; kj < 7; kj++) {
+          const int k = (c * 7 + ki) * 7 + kj;
+          float wv[16];
+#pragma unroll
+          for (int q = 0; q < 4; q++) {
+            const float4 t4 = *reinterpret_cast<const float4*>(w_s + k * 64 + cg * 16 + 4 * q);
+            wv[4 * q] = t4.x; wv[4 * q + 1] = t4.y; wv[4 * q + 2] = t4.z; wv[4 * q + 3] = t4.w;
+          }
+#pragma unroll
+          for (int i = 0; i < PPT; i++) {
+            const int lh = 2 * (lohb + RSTEP * i) + ki;
+            const float xv = xb[((c * PS + lh) * 2 + (kj & 1)) * HALF + low + (kj >> 1)];
+#pragma unroll
+            for (int j = 0; j < 16; j++) acc[i][j] = __fmaf_rn(xv, wv[j], acc[i][j]);
+          }
+        }
+      }
+    const int n = (int)(tile / (TILES * TILES));
+    const int rem = (int)(tile % (TILES * TILES));
+    const int oh0 = (rem / TILES) * TS, ow0 = (rem % TILES) * TS;
+#pragma unroll
+    for (int i = 0; i < PPT; i++) {
+      const int oh = oh0 + lohb + RSTEP * i, ow = ow0 + low;
+      if (oh >= OHW || ow >= OHW) continue;
+      float* dst = out + (((size_t)n * OHW + oh) * OHW + ow) * 64 + cg * 16;
+#pragma unroll
+      for (int j = 0; j < 16; j += 4)
+        *reinterpret_cast<float4*>(dst + j) =
+            make_float4(__fmaf_rn(acc[i][j], sc[j], sf[j]), __fmaf_rn(acc[i][j + 1], sc[j + 1], sf[j + 1]),
+                        __fmaf_rn(acc[i][j + 2], sc[j + 2], sf[j + 2]), __fmaf_rn(acc[i][j + 3], sc[j + 3], sf[j + 3]));
+    }
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 // ---- maxpool 3x3 / 2, pad 1 (64 channels) -> fp32 residual stream + packed signs -------------------
@@ -142,22 +165,25 @@ __global__ void __launch_bounds__(256) maxpool_pack(const float* __restrict__ x 
 }
 
 // ---- downsample shortcut: avgpool 2x2 / 2 -> fp32 conv 1x1 (C -> O) -> BN ---------------------------
-// CTA tile: 32 output pixels x 64 output channels; a thread owns 8 consecutive pixels x 2 channels (o, o+32).
-// One fmaf chain per output over c ascending.
+// CTA tile: 32 output pixels x 128 output channels; a thread owns 8 consecutive pixels x 4 channels
+// (o, o+32, o+64, o+96).  One fmaf chain per output over c ascending.
+constexpr int SC_TO = 4;
 __global__ void __launch_bounds__(128) shortcut_down(const float* __restrict__ x /*[N][HW][HW][C]*/, int HW, int C,
                                                      const float* __restrict__ w /*[O][C]*/, int O,
                                                      const float* __restrict__ scale, const float* __restrict__ shift,
                                                      long long npix_out, float* __restrict__ y /*[N][HW/2][HW/2][O]*/) {
-  __shared__ __align__(16) float p_s[32][36];   // [c in chunk][pixel], padded
-  __shared__ float w_s[64][33];                 // [o in tile][c in chunk]
+  __shared__ __align__(16) float p_s[32][36];          // [c in chunk][pixel], padded
+  __shared__ float w_s[32 * SC_TO][33];                // [o in tile][c in chunk]
   const int tid = threadIdx.x;
   const long long p0 = (long long)blockIdx.x * 32;
-  const int o0 = blockIdx.y * 64;
+  const int o0 = blockIdx.y * (32 * SC_TO);
   const int OHW = HW / 2;
   const int ol = tid % 32, pgp = tid / 32;      // pixels pgp*8 .. pgp*8+7
-  float acc[8][2];
+  float acc[8][SC_TO];
 #pragma unroll
-  for (int i = 0; i < 8; i++) acc[i][0] = acc[i][1] = 0.0f;
+  for (int i = 0; i < 8; i++)
+#pragma unroll
+    for (int j = 0; j < SC_TO; j++) acc[i][j] = 0.0f;
   for (int c0 = 0; c0 < C; c0 += 32) {
     __syncthreads();
     for (int t = tid; t < 32 * 32; t += 128) {
@@ -175,62 +201,80 @@ __global__ void __launch_bounds__(128) shortcut_down(const float* __restrict__ x
       }
       p_s[cc][pp] = v;
     }
-    for (int t = tid; t < 64 * 32; t += 128) {
+    for (int t = tid; t < 32 * SC_TO * 32; t += 128) {
       const int cc = t % 32, oo = t / 32;
       w_s[oo][cc] = (o0 + oo < O && c0 + cc < C) ? w[(size_t)(o0 + oo) * C + c0 + cc] : 0.0f;
     }
     __syncthreads();
     const int cn = min(32, C - c0);
+#pragma unroll 4
     for (int cc = 0; cc < cn; cc++) {
-      const float w0 = w_s[ol][cc], w1 = w_s[ol + 32][cc];
+      float wv[SC_TO];
+#pragma unroll
+      for (int j = 0; j < SC_TO; j++) wv[j] = w_s[ol + 32 * j][cc];
       const float4 pa = *reinterpret_cast<const float4*>(&p_s[cc][pgp * 8]);
       const float4 pb = *reinterpret_cast<const float4*>(&p_s[cc][pgp * 8 + 4]);
       const float pv[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
 #pragma unroll
-      for (int i = 0; i < 8; i++) {
-        acc[i][0] = __fmaf_rn(pv[i], w0, acc[i][0]);
-        acc[i][1] = __fmaf_rn(pv[i], w1, acc[i][1]);
-      }
+      for (int i = 0; i < 8; i++)
+#pragma unroll
+        for (int j = 0; j < SC_TO; j++) acc[i][j] = __fmaf_rn(pv[i], wv[j], acc[i][j]);
     }
   }
 #pragma unroll
-  for (int h = 0; h < 2; h++) {
-    const int o = o0 + ol + 32 * h;
+  for (int j = 0; j < SC_TO; j++) {
+    const int o = o0 + ol + 32 * j;
     if (o >= O) continue;
     const float sc = scale[o], sf = shift[o];
 #pragma unroll
     for (int i = 0; i < 8; i++) {
       const long long p = p0 + pgp * 8 + i;
-      if (p < npix_out) y[p * O + o] = __fmaf_rn(acc[i][h], sc, sf);
+      if (p < npix_out) y[p * O + o] = __fmaf_rn(acc[i][j], sc, sf);
     }
   }
 }
 
 // ---- head: global average over 7x7 (sequential sum, then /49), fc 512 -> 1000 -----------------------
-__global__ void __launch_bounds__(256) gap_fc(const float* __restrict__ x /*[N][7][7][512]*/,
+// A CTA takes GAP_IMGS images and 256 logits: the pooled vectors sit in shared memory and every fc weight a thread
+// loads is used for all of the CTA's images.  One fmaf chain per logit over k ascending, then + bias.
+constexpr int GAP_IMGS = 8;
+__global__ void __launch_bounds__(256) gap_fc(const float* __restrict__ x /*[N][7][7][512]*/, int N,
                                               const float* __restrict__ fw /*[1000][512]*/,
                                               const float* __restrict__ fb, float* __restrict__ logits) {
-  __shared__ __align__(16) float g[512];
-  const int n = blockIdx.y;
-  for (int c = threadIdx.x; c < 512; c += blockDim.x) {
+  __shared__ __align__(16) float g[GAP_IMGS][512];
+  const int n0 = blockIdx.y * GAP_IMGS;
+  const int nimg = min(GAP_IMGS, N - n0);
+  for (int t = threadIdx.x; t < GAP_IMGS * 512; t += blockDim.x) {
+    const int c = t % 512, im = t / 512;
     float s = 0.0f;
-    for (int q = 0; q < 49; q++) s = __fadd_rn(s, x[((size_t)n * 49 + q) * 512 + c]);
-    g[c] = __fdiv_rn(s, 49.0f);
+    if (im < nimg) {
+      for (int q = 0; q < 49; q++) s = __fadd_rn(s, x[((size_t)(n0 + im) * 49 + q) * 512 + c]);
+      s = __fdiv_rn(s, 49.0f);
+    }
+    g[im][c] = s;
   }
   __syncthreads();
   const int j = blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= 1000) return;
   const float4* wr = reinterpret_cast<const float4*>(fw + (size_t)j * 512);
-  float a = 0.0f;
+  float a[GAP_IMGS];
+#pragma unroll
+  for (int im = 0; im < GAP_IMGS; im++) a[im] = 0.0f;
   for (int k4 = 0; k4 < 128; k4++) {
     const float4 wv = __ldg(wr + k4);
-    const float4 gv = *reinterpret_cast<const float4*>(g + 4 * k4);
-    a = __fmaf_rn(gv.x, wv.x, a);
-    a = __fmaf_rn(gv.y, wv.y, a);
-    a = __fmaf_rn(gv.z, wv.z, a);
-    a = __fmaf_rn(gv.w, wv.w, a);
+#pragma unroll
+    for (int im = 0; im < GAP_IMGS; im++) {
+      const float4 gv = *reinterpret_cast<const float4*>(&g[im][4 * k4]);
+      a[im] = __fmaf_rn(gv.x, wv.x, a[im]);
+      a[im] = __fmaf_rn(gv.y, wv.y, a[im]);
+      a[im] = __fmaf_rn(gv.z, wv.z, a[im]);
+      a[im] = __fmaf_rn(gv.w, wv.w, a[im]);
+    }
   }
-  logits[(size_t)n * 1000 + j] = __fadd_rn(a, fb[j]);
+  const float bias = fb[j];
+#pragma unroll
+  for (int im = 0; im < GAP_IMGS; im++)
+    if (im < nimg) logits[(size_t)(n0 + im) * 1000 + j] = __fadd_rn(a[im], bias);
 }
 
 constexpr int kStageC[4] = {64, 128, 256, 512};
@@ -257,7 +301,7 @@ Workspace plan(int N) {
 template <int TS, int PPT>
 dabnn_status launch_stem(const dabnn_bireal18_params* p, const float* images, int N, float* out, cudaStream_t st) {
   constexpr int PS = 2 * TS + 5, HALF = (PS + 1) / 2 + 1;
-  constexpr size_t SMEM = (size_t)(STEM_K * 64 + 3 * PS * 2 * HALF) * 4;
+  constexpr size_t SMEM = (size_t)(STEM_K * 64 + 2 * 3 * PS * 2 * HALF) * 4;
   auto kern = stem_conv_bn<TS, PPT>;
   static bool configured = false;
   if (!configured) {
@@ -268,7 +312,10 @@ dabnn_status launch_stem(const dabnn_bireal18_params* p, const float* images, in
     configured = true;
   }
   const int tiles = (112 + TS - 1) / TS;
-  kern<<<dim3(tiles, tiles, N), (TS * TS / PPT) * 4, SMEM, st>>>(images, p->stem_w, p->stem_scale, p->stem_shift, out);
+  const long long ntiles = (long long)N * tiles * tiles;
+  const long long cap = 2LL * sm_count();  // persistent: two CTAs per SM, each walking over tiles
+  kern<<<(unsigned)(ntiles < cap ? ntiles : cap), (TS * TS / PPT) * 4, SMEM, st>>>(images, p->stem_w, p->stem_scale,
+                                                                                p->stem_shift, N, out);
   return launch_status();
 }
 
@@ -323,7 +370,7 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     const bool down = stage > 0 && b % 4 == 0;
     if (down) {
       const long long npo = (long long)N * OHW * OHW;
-      shortcut_down<<<dim3(ceil_div(npo, 32), ceil_div(O, 64)), 128, 0, st>>>(
+      shortcut_down<<<dim3(ceil_div(npo, 32), ceil_div(O, 32 * SC_TO)), 128, 0, st>>>(
           cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
       if ((s = launch_status()) != DABNN_OK) return s;
       float* t = cur; cur = other; other = t;
@@ -342,7 +389,7 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     uint64_t* tb = bits_in; bits_in = bits_out; bits_out = tb;
     C = O; HW = OHW;
   }
-  gap_fc<<<dim3(4, N), 256, 0, st>>>(cur, p->fc_w, p->fc_b, logits);
+  gap_fc<<<dim3(4, ceil_div(N, GAP_IMGS)), 256, 0, st>>>(cur, N, p->fc_w, p->fc_b, logits);
   return launch_status();
 }
 
