@@ -143,7 +143,7 @@ dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float*
  *     overlaps on the GPU (different streams, or different threads) race on the area: serialise them.
  * Arguments and results are otherwise exactly those of dabnn_bireal18_forward. */
 #define DABNN_STATIC_MAX_BATCH 2
-#define DABNN_STATIC_SCRATCH_BYTES 8931328
+#define DABNN_STATIC_SCRATCH_BYTES 8935424
 dabnn_status dabnn_bireal18_forward_static(const dabnn_bireal18_params* p, const float* images, int N, float* logits,
                                            void* stream);
 

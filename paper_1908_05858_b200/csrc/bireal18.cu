@@ -234,6 +234,83 @@ __global__ void __launch_bounds__(128) shortcut_down(const float* __restrict__ x
   }
 }
 
+// Small problems (batch 1): one thread per output, so that a 7x7x512 layer still fills the chip.  A CTA takes 4 output
+// pixels x 64 channels; the pooled inputs of its pixels sit in shared memory, each thread walks its weight row.
+// Same order of operations as above.
+__global__ void __launch_bounds__(256) shortcut_down_small(const float* __restrict__ x, int HW, int C,
+                                                           const float* __restrict__ w, int O,
+                                                           const float* __restrict__ scale, const float* __restrict__ shift,
+                                                           long long npix_out, float* __restrict__ y) {
+  __shared__ __align__(16) float pooled[4][512];
+  const int tid = threadIdx.x;
+  const long long p0 = (long long)blockIdx.x * 4;
+  const int OHW = HW / 2;
+  for (int t = tid; t < 4 * C; t += 256) {
+    const int c = t % C, pp = t / C;
+    const long long p = p0 + pp;
+    float v = 0.0f;
+    if (p < npix_out) {
+      const int ow = (int)(p % OHW), oh = (int)((p / OHW) % OHW);
+      const long long n = p / ((long long)OHW * OHW);
+      const float* q = x + ((n * HW + 2 * oh) * HW + 2 * ow) * C + c;
+      float s = __fadd_rn(q[0], q[C]);
+      s = __fadd_rn(s, q[(size_t)HW * C]);
+      s = __fadd_rn(s, q[(size_t)HW * C + C]);
+      v = __fmul_rn(s, 0.25f);
+    }
+    pooled[pp][c] = v;
+  }
+  __syncthreads();
+  const int pp = tid / 64, o = blockIdx.y * 64 + tid % 64;
+  const long long p = p0 + pp;
+  if (o >= O || p >= npix_out) return;
+  const float* wr = w + (size_t)o * C;
+  float a = 0.0f;
+  if ((C & 3) == 0 && (reinterpret_cast<uintptr_t>(w) & 15) == 0) {
+    for (int c = 0; c < C; c += 4) {
+      const float4 wv = __ldg(reinterpret_cast<const float4*>(wr + c));
+      const float4 pv = *reinterpret_cast<const float4*>(&pooled[pp][c]);
+      a = __fmaf_rn(pv.x, wv.x, a);
+      a = __fmaf_rn(pv.y, wv.y, a);
+      a = __fmaf_rn(pv.z, wv.z, a);
+      a = __fmaf_rn(pv.w, wv.w, a);
+    }
+  } else {
+    for (int c = 0; c < C; c++) a = __fmaf_rn(pooled[pp][c], wr[c], a);
+  }
+  y[p * O + o] = __fmaf_rn(a, scale[o], shift[o]);
+}
+
+// Small batches: the pooled vector is written to the workspace by one kernel and 32-thread CTAs compute the logits.
+__global__ void __launch_bounds__(512) gap_small(const float* __restrict__ x /*[N][7][7][512]*/, float* __restrict__ g) {
+  const int n = blockIdx.x, c = threadIdx.x;
+  float s = 0.0f;
+  for (int q = 0; q < 49; q++) s = __fadd_rn(s, x[((size_t)n * 49 + q) * 512 + c]);
+  g[(size_t)n * 512 + c] = __fdiv_rn(s, 49.0f);
+}
+__global__ void __launch_bounds__(32) fc_small(const float* __restrict__ g /*[N][512]*/, const float* __restrict__ fw,
+                                               const float* __restrict__ fb, float* __restrict__ logits) {
+  __shared__ __align__(16) float gs[512];
+  const int n = blockIdx.y;
+  for (int t = threadIdx.x; t < 128; t += 32)
+    reinterpret_cast<float4*>(gs)[t] = reinterpret_cast<const float4*>(g + (size_t)n * 512)[t];
+  __syncwarp();
+  const int j = blockIdx.x * 32 + threadIdx.x;
+  if (j >= 1000) return;
+  const float4* wr = reinterpret_cast<const float4*>(fw + (size_t)j * 512);
+  float a = 0.0f;
+#pragma unroll 8
+  for (int k4 = 0; k4 < 128; k4++) {
+    const float4 wv = __ldg(wr + k4);
+    const float4 gv = reinterpret_cast<const float4*>(gs)[k4];
+    a = __fmaf_rn(gv.x, wv.x, a);
+    a = __fmaf_rn(gv.y, wv.y, a);
+    a = __fmaf_rn(gv.z, wv.z, a);
+    a = __fmaf_rn(gv.w, wv.w, a);
+  }
+  logits[(size_t)n * 1000 + j] = __fadd_rn(a, fb[j]);
+}
+
 // ---- head: global average over 7x7 (sequential sum, then /49), fc 512 -> 1000 -----------------------
 // A CTA takes GAP_IMGS images and 256 logits: the pooled vectors sit in shared memory and every fc weight a thread
 // loads is used for all of the CTA's images.  One fmaf chain per logit over k ascending, then + bias.
@@ -283,7 +360,7 @@ constexpr int kStageHW[4] = {56, 28, 14, 7};
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Workspace {
-  size_t stem_out, res_a, res_b, bits_a, bits_b, total;
+  size_t stem_out, res_a, res_b, bits_a, bits_b, gap, total;
 };
 
 Workspace plan(int N) {
@@ -294,6 +371,7 @@ Workspace plan(int N) {
   ws.res_b = off;    off = align_up(off + (size_t)N * 28 * 28 * 128 * 4, 256);
   ws.bits_a = off;   off = align_up(off + (size_t)N * 56 * 56 * 8, 256);
   ws.bits_b = off;   off = align_up(off + (size_t)N * 56 * 56 * 8, 256);
+  ws.gap = off;      off = align_up(off + (size_t)N * 512 * 4, 256);
   ws.total = off;
   return ws;
 }
@@ -370,8 +448,12 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     const bool down = stage > 0 && b % 4 == 0;
     if (down) {
       const long long npo = (long long)N * OHW * OHW;
-      shortcut_down<<<dim3(ceil_div(npo, 32), ceil_div(O, 32 * SC_TO)), 128, 0, st>>>(
-          cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
+      if ((long long)ceil_div(npo, 32) * ceil_div(O, 32 * SC_TO) < sm_count() && C <= 512)
+        shortcut_down_small<<<dim3(ceil_div(npo, 4), ceil_div(O, 64)), 256, 0, st>>>(
+            cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
+      else
+        shortcut_down<<<dim3(ceil_div(npo, 32), ceil_div(O, 32 * SC_TO)), 128, 0, st>>>(
+            cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
       if ((s = launch_status()) != DABNN_OK) return s;
       float* t = cur; cur = other; other = t;
     }
@@ -389,7 +471,14 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     uint64_t* tb = bits_in; bits_in = bits_out; bits_out = tb;
     C = O; HW = OHW;
   }
-  gap_fc<<<dim3(4, ceil_div(N, GAP_IMGS)), 256, 0, st>>>(cur, N, p->fc_w, p->fc_b, logits);
+  if (N < GAP_IMGS) {
+    float* gbuf = reinterpret_cast<float*>(base + ws.gap);
+    gap_small<<<N, 512, 0, st>>>(cur, gbuf);
+    if ((s = launch_status()) != DABNN_OK) return s;
+    fc_small<<<dim3(ceil_div(1000, 32), N), 32, 0, st>>>(gbuf, p->fc_w, p->fc_b, logits);
+  } else {
+    gap_fc<<<dim3(4, ceil_div(N, GAP_IMGS)), 256, 0, st>>>(cur, N, p->fc_w, p->fc_b, logits);
+  }
   return launch_status();
 }
 
