@@ -77,6 +77,12 @@ dabnn_status dabnn_pack_weights(const float* w_oihw, int O, int C, int kh, int k
 dabnn_status dabnn_bconv2d(const uint64_t* a_packed, dabnn_shape in, const uint64_t* w_packed, int O, dabnn_conv cv,
                            int32_t* out, dabnn_layout out_layout, void* stream);
 
+/* Eq. 1 -- BGEMM on packed vectors, for binary fully-connected layers and im2col'ed inputs.
+ * A: [M][Kw] packed rows; B: [N][Kw] packed rows (row j is column j of the paper's B); Kbits valid bits per row,
+ * Kw = ceil(Kbits/64), tail bits 0.  C: int32 [M][N], the +-1 dot product  Kbits - 2*popcount(xor)  of row i of A and
+ * row j of B.  The paper's count of agreeing positions is (C + Kbits) / 2. */
+dabnn_status dabnn_bgemm(const uint64_t* A, int M, const uint64_t* B, int N, int Kbits, int32_t* C, void* stream);
+
 /* Section 2.1.1 (fused BN-binarization) on top of Eq. 1: the int32 result never leaves the chip.
  * y = fmaf((float)acc, scale[o], shift[o]); bit = (y < 0); out_packed: uint64 [N][OH][OW][ceil(O/64)]. */
 dabnn_status dabnn_bconv2d_bn_sign_pack(const uint64_t* a_packed, dabnn_shape in, const uint64_t* w_packed, int O,

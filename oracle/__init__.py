@@ -160,6 +160,19 @@ def bconv_bits_at(A, C, Wp, coords, stride=(1, 1), pad=(0, 0), pad_value=-1) -> 
     return vals
 
 
+def bgemm_xnor(A: np.ndarray, B: np.ndarray, Kbits: int) -> np.ndarray:
+    """Eq. 1 as printed: C[i][j] = sum_k bitcount(xnor(A[i][k], B[j][k])) over the Kbits valid positions.
+    A: uint64 [M][Kw]; B: uint64 [N][Kw] (row j = column j of the paper's B).  Returns int32 [M][N]."""
+    A = np.ascontiguousarray(A, dtype=np.uint64)
+    B = np.ascontiguousarray(B, dtype=np.uint64)
+    M, Kw = A.shape
+    N, Kw2 = B.shape
+    assert Kw == Kw2 == words_per_pixel(Kbits)
+    C = np.empty((M, N), dtype=np.int32)
+    lib().oracle_bgemm_xnor(_p(A), M, _p(B), N, int(Kbits), _p(C))
+    return C
+
+
 def bn_fold(gamma, beta, mean, var, eps: float = 1e-5):
     """BN parameters -> (scale, shift) in double, rounded once to fp32 each."""
     g, b, m, v = (_f32(t) for t in (gamma, beta, mean, var))

@@ -17,6 +17,7 @@
  *   oracle_bconv_bits                   Eq. 1 (BGEMM: sum_k bitcount(xnor(A_ik, B_kj))) on the
  *                                       packed words, turned into the +-1 dot product
  *                                       2*C_xnor - K  =  K - 2*sum popcount(xor).
+ *   oracle_bgemm_xnor                   Eq. 1 as printed: counts of agreeing bit positions, C in N^{M x N}.
  *   oracle_bn_fold / oracle_bn_sign_pack  Section 2.1.1, last sentence (fused BN + binarize).
  *   oracle_bireal18_forward             Section 2.3 / Table 2: Bi-Real Net 18 (a binary
  *                                       ResNet-18; first conv and last fc in full precision).
@@ -203,6 +204,25 @@ void oracle_bconv_bits_at(const uint64_t* A, int N, int C, int H, int W, const u
   for (int64_t q = 0; q < ncoords; q++)
     vals[q] = bits_one(A, C, H, W, Wp, kh, kw, sh, sw, ph, pw, pad_value, coords[4 * q],
                        coords[4 * q + 1], coords[4 * q + 2], coords[4 * q + 3]);
+}
+
+/* ---- BGEMM exactly as Eq. 1 prints it: C_ij = sum_k bitcount(xnor(A_ik, B_kj)) ------------------------
+ * A is [M][Kw] packed rows, B is given by its columns as [N][Kw] packed rows (column j of the paper's B),
+ * Kbits valid bits per row (tail bits 0 in both).  C is [M][N], a count of agreeing positions in 0..Kbits. */
+void oracle_bgemm_xnor(const uint64_t* A, int M, const uint64_t* B, int N, int Kbits, int32_t* Cout) {
+  int Kw = (int)words_per_pixel(Kbits);
+#pragma omp parallel for num_threads(g_threads) schedule(static)
+  for (int i = 0; i < M; i++)
+    for (int j = 0; j < N; j++) {
+      int count = 0;
+      for (int k = 0; k < Kw; k++) {
+        int valid = Kbits - 64 * k;
+        if (valid > 64) valid = 64;
+        uint64_t mask = (valid == 64) ? ~(uint64_t)0 : ((((uint64_t)1) << valid) - 1);
+        count += popcount64(~(A[(size_t)i * Kw + k] ^ B[(size_t)j * Kw + k]) & mask);
+      }
+      Cout[(size_t)i * N + j] = count;
+    }
 }
 
 /* ---- fused BN + binarize (Section 2.1.1, last sentence) ----------------------------- */

@@ -23,7 +23,7 @@ LIB_PATH = os.path.join(_HERE, "libdabnn_b200.so")
 
 EXPORTS = (
     "dabnn_status_string", "dabnn_words_per_pixel", "dabnn_out_dim", "dabnn_pack", "dabnn_pack_weights",
-    "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack", "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold",
+    "dabnn_bconv2d", "dabnn_bgemm", "dabnn_bconv2d_bn_sign_pack", "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold",
     "dabnn_bireal18_workspace_bytes", "dabnn_bireal18_forward", "dabnn_set_conv_variant",
     "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host", "dabnn_bireal18_forward_static", "dabnn_set_conv_tile",
     "dabnn_tc_weights_bytes", "dabnn_tc_prepare_weights", "dabnn_tc_bconv2d", "dabnn_tc_bconv2d_bn_sign_pack",
@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
         L.dabnn_pack.argtypes = [vp, ci, Shape, vp, vp]
         L.dabnn_pack_weights.argtypes = [vp, ci, ci, ci, ci, vp, vp]
         L.dabnn_bconv2d.argtypes = [vp, Shape, vp, ci, Conv, vp, ci, vp]
+        L.dabnn_bgemm.argtypes = [vp, ci, vp, ci, ci, vp, vp]
+        L.dabnn_bgemm.restype = ci
         L.dabnn_bconv2d_bn_sign_pack.argtypes = [vp, Shape, vp, ci, Conv, vp, vp, vp, vp]
         L.dabnn_bconv2d_bn_add_sign_pack.argtypes = [vp, Shape, vp, ci, Conv, vp, vp, vp, vp, vp, vp]
         L.dabnn_bn_fold.argtypes = [vp, vp, vp, vp, ctypes.c_double, ci, vp, vp, vp]
@@ -178,6 +180,19 @@ def bconv2d(a_packed, C: int, w_packed, stride=(1, 1), pad=(0, 0), pad_value: in
         out = torch.empty(shape, dtype=torch.int32, device=a.device)
     _check(lib().dabnn_bconv2d(a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O, _conv(kh, kw, stride, pad, pad_value),
                                out.data_ptr(), out_layout, _stream()))
+    return out
+
+
+def bgemm(A: torch.Tensor, B: torch.Tensor, Kbits: int) -> torch.Tensor:
+    """dabnn_bgemm: A int64 [M][Kw], B int64 [N][Kw] -> int32 [M][N] of +-1 dot products over Kbits positions."""
+    A = _dev(A, torch.int64, "A")
+    B = _dev(B, torch.int64, "B")
+    M, Kw = A.shape
+    N, Kw2 = B.shape
+    if Kw != Kw2 or Kw != (Kbits + 63) // 64:
+        raise DabnnError("packed word counts do not match Kbits")
+    out = torch.empty((M, N), dtype=torch.int32, device=A.device)
+    _check(lib().dabnn_bgemm(A.data_ptr(), M, B.data_ptr(), N, int(Kbits), out.data_ptr(), _stream()))
     return out
 
 

@@ -517,3 +517,12 @@ extern "C" dabnn_status dabnn_bconv2d_bn_add_sign_pack(const uint64_t* a_packed,
   g.out_packed32 = reinterpret_cast<uint32_t*>(out_packed);
   return launch_epi<EPI_BIREAL>(g, as_stream(stream));
 }
+
+extern "C" dabnn_status dabnn_bgemm(const uint64_t* A, int M, const uint64_t* B, int N, int Kbits, int32_t* C,
+                                    void* stream) {
+  // rows of A are "pixels" of a 1x1 image batch, rows of B the "filters": a 1x1 convolution over Kbits channels
+  if (M <= 0 || N <= 0 || Kbits <= 0) return DABNN_ERR_SHAPE;
+  const dabnn_shape in = {M, Kbits, 1, 1};
+  const dabnn_conv cv = {1, 1, 1, 1, 0, 0, -1};
+  return dabnn_bconv2d(A, in, B, N, cv, C, DABNN_NHWC, stream);
+}

@@ -243,3 +243,16 @@ def test_every_conv_tile_gives_the_same_integers(B, oracle_mod, case, tile):
         B.set_conv_tile(prev)
     assert np.array_equal(got, want)
     assert np.array_equal(got_bits, want_bits)
+
+
+@pytest.mark.parametrize("shape", [(5, 7, 150), (300, 260, 512), (1, 1000, 4608), (129, 65, 64)])
+def test_bgemm_matches_eq1(B, oracle_mod, shape):
+    M, N, K = shape
+    rng = np.random.default_rng(M + N + K)
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    b = rng.standard_normal((N, K)).astype(np.float32)
+    A = B.pack(dev(a.reshape(M, K, 1, 1))).reshape(M, -1)
+    Bm = B.pack(dev(b.reshape(N, K, 1, 1))).reshape(N, -1)
+    got = B.bgemm(A, Bm, K).cpu().numpy()
+    counts = oracle_mod.bgemm_xnor(u64(A), u64(Bm), K)  # Eq. 1 as printed: agreeing positions
+    assert np.array_equal(got, 2 * counts - K)

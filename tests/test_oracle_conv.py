@@ -192,3 +192,24 @@ def test_exhaustive_tiny_with_padding(oracle_mod, pv):
         xs = X[n].astype(int).tolist()
         for f in range(0, 512, 7):
             assert a[n, f].tolist() == brute(xs, Wall[f].astype(int).tolist(), 1, 1, pv)
+
+
+def test_bgemm_xnor_counts_against_brute_force_and_the_dot_product(oracle_mod):
+    """Eq. 1 as printed: counts of agreeing positions, checked bit by bit in Python and against 2*C - K = dot."""
+    o = oracle_mod
+    rng = np.random.default_rng(21)
+    M, N, K = 5, 7, 150  # three words, tail of 22 bits
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    b = rng.standard_normal((N, K)).astype(np.float32)
+    A = o.pack(a.reshape(M, K, 1, 1)).reshape(M, -1)
+    Bm = o.pack(b.reshape(N, K, 1, 1)).reshape(N, -1)
+    C = o.bgemm_xnor(A, Bm, K)
+    sa, sb = np.where(a < 0, -1, 1), np.where(b < 0, -1, 1)
+    for i in range(M):
+        for j in range(N):
+            agree = sum(1 for k in range(K) if sa[i, k] == sb[j, k])
+            assert C[i, j] == agree
+    assert np.array_equal(2 * C - K, sa @ sb.T)
+    # the worked example, by hand: 0x46^0xD3 = 0x95 (4 differ, 4 agree); 0x46^0x87 = 0xC1 (3 differ, 5 agree);
+    # 0x8F^0xD3 = 0x5C (4 differ, 4 agree); 0x8F^0x87 = 0x08 (1 differs, 7 agree)
+    assert o.bgemm_xnor(np.array([[0x46], [0x8F]], dtype=np.uint64), np.array([[0xD3], [0x87]], dtype=np.uint64), 8).tolist() == [[4, 5], [4, 7]]
