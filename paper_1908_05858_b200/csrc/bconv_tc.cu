@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   uint8_t* w_s = smem;                                   // [taps][C/32][NT][16]
   uint8_t* a_s = smem + (size_t)NT * Kb;                 // [abufs][C/32][slots][16]
   uint8_t* misc = a_s + (size_t)g.abufs * a_bytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(misc);    // [0,1] mma_done  [2,3] tmem_free  [4,5] a_full
+  uint64_t* bars = reinterpret_cast<uint64_t*>(misc);    // [0,1] mma_done  [2,3] tmem_free  [4,5] a_full  [6] w_full
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 64);
   volatile int* s_fail = reinterpret_cast<volatile int*>(misc + 72);
   float* s_scale = reinterpret_cast<float*>(misc + 128);     // [NT] this CTA's channels
@@ -167,6 +167,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     mbar_init(smem_u32(&bars[3]), 128);
     mbar_init(smem_u32(&bars[4]), 128);
     mbar_init(smem_u32(&bars[5]), 128);
+    mbar_init(smem_u32(&bars[6]), 160);
     *s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -176,34 +177,35 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // resident weights: one contiguous block per channel tile
-  {
-    const uint8_t* src = g.w_tc + (size_t)nt * NT * Kb;
-    const int units = NT * Kb / 16;
-    for (int u = tid; u < units; u += TC_THREADS) cp_async16(smem_u32(w_s + (size_t)u * 16), src + (size_t)u * 16);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
-  if (warp < 4) {
-    // scale factors: every byte of the scale-factor columns is ue8m0 127 = 1.0, whatever their layout
-    const uint32_t one = 0x7F7F7F7Fu;
-    for (int c = TC_SF_COL; c < TC_TMEM_COLS; c += 16) {
-      const uint32_t taddr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)c;
-      asm volatile(
-          "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr),
-          "r"(one)
-          : "memory");
+  if (warp < 4 || warp == 8) {
+    // One-time set-up by the 160 threads that are not producers, while the producers already expand the first tile:
+    // the resident weights (one contiguous block per channel tile) and the scale factors.
+    const int stid = warp == 8 ? 128 + lane : tid;
+    const uint8_t* src = g.w_tc + (size_t)nt * NT * Kb;
+    const int units = NT * Kb / 16;
+    for (int u = stid; u < units; u += 160) cp_async16(smem_u32(w_s + (size_t)u * 16), src + (size_t)u * 16);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    if (warp < 4) {
+      // every byte of the scale-factor columns is ue8m0 127 = 1.0, whatever their layout
+      const uint32_t one = 0x7F7F7F7Fu;
+      for (int c = TC_SF_COL; c < TC_TMEM_COLS; c += 16) {
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)c;
+        asm volatile(
+            "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};" ::"r"(taddr),
+            "r"(one)
+            : "memory");
+      }
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    mbar_arrive(smem_u32(&bars[6]));  // 160 arrivals: weights and scale factors are in place
   }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
   if (warp == 8) {
     // ================= MMA issue: one thread ======================================================================
@@ -222,7 +224,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       long long tlast = clock64();
 #endif
       int it = 0;
-      for (long long mt = mt_first; mt < g.m_tiles; mt += mt_step, it++) {
+      if (!mbar_wait(smem_u32(&bars[6]), 0)) *s_fail = 1;  // resident weights and scale factors
+      for (long long mt = mt_first; mt < g.m_tiles && *s_fail == 0; mt += mt_step, it++) {
         const int ab = it % g.abufs;
         TC_T(0);
         if (!mbar_wait(smem_u32(&bars[4 + ab]), (uint32_t)(it / g.abufs) & 1)) { *s_fail = 1; break; }      // rows written
@@ -264,13 +267,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     const int ptid = tid - 128;
     const int cgroups = g.C >> 5;
     const uint32_t pad_word4 = g.pad_neg ? 0xAAAAAAAAu : 0x22222222u;
-    uint64_t words[2][TC_MAX_CW];
-    int kind[2];  // 0: inside the image (words valid), 1: padding, 2: beyond the batch, 3: no such slot
-    auto prefetch = [&](long long mt) {
+    struct SlotRegs {
+      uint64_t words[2][TC_MAX_CW];
+      int kind[2];  // 0: inside the image (words valid), 1: padding, 2: beyond the batch, 3: no such slot
+    };
+    auto prefetch = [&](SlotRegs& R, long long mt) {
 #pragma unroll
       for (int h = 0; h < 2; h++) {
         const int s = ptid + 128 * h;
-        kind[h] = 3;
+        R.kind[h] = 3;
         if (s < g.slots) {
           const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)s;  // total_q < 2^31 is checked on the host
           const uint32_t rr = Q / (uint32_t)g.SP;
@@ -278,22 +283,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
           const uint32_t n = rr / (uint32_t)g.HP;
           const int r = (int)(rr - n * (uint32_t)g.HP);
           const int ih = r - g.ph, iw = col - g.pw;
-          if (n >= (uint32_t)g.N) kind[h] = 2;
-          else if (ih < 0 || ih >= g.H || iw < 0 || iw >= g.W) kind[h] = 1;
+          if (n >= (uint32_t)g.N) R.kind[h] = 2;
+          else if (ih < 0 || ih >= g.H || iw < 0 || iw >= g.W) R.kind[h] = 1;
           else {
-            kind[h] = 0;
+            R.kind[h] = 0;
             const uint64_t* src = g.a + (((long long)n * g.H + ih) * g.W + iw) * g.Cw;
 #pragma unroll
             for (int cw = 0; cw < TC_MAX_CW; cw++)
-              if (cw < g.Cw) words[h][cw] = __ldg(src + cw);
+              if (cw < g.Cw) R.words[h][cw] = __ldg(src + cw);
           }
         }
       }
     };
-    auto expand = [&](uint8_t* abuf) {
+    auto expand = [&](const SlotRegs& R, uint8_t* abuf) {
 #pragma unroll
       for (int h = 0; h < 2; h++) {
-        if (kind[h] == 3) continue;
+        if (R.kind[h] == 3) continue;
         const int s = ptid + 128 * h;
 #pragma unroll
         for (int cw = 0; cw < TC_MAX_CW; cw++) {
@@ -303,10 +308,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
             const int grp = cw * 2 + q2;
             if (grp >= cgroups) break;
             uint4 bytes;
-            if (kind[h] == 0) {
-              const uint32_t half = (uint32_t)(words[h][cw] >> (32 * q2));
+            if (R.kind[h] == 0) {
+              const uint32_t half = (uint32_t)(R.words[h][cw] >> (32 * q2));
               bytes = expand32(half);
-            } else if (kind[h] == 2) bytes = make_uint4(0, 0, 0, 0);
+            } else if (R.kind[h] == 2) bytes = make_uint4(0, 0, 0, 0);
             else bytes = make_uint4(pad_word4, pad_word4, pad_word4, pad_word4);
             *reinterpret_cast<uint4*>(abuf + ((size_t)grp * g.slots + s) * 16) = bytes;
           }
@@ -319,19 +324,32 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     long long tlast = clock64();
 #endif
-    if (mt_first < g.m_tiles) prefetch(mt_first);
-    for (long long mt = mt_first; mt < g.m_tiles; mt += mt_step, it++) {
+    // One tile of producer work on register set R; the bits of the tile two steps ahead are requested right after,
+    // so that a whole tile period covers their latency.  Returns false when the loop must stop.
+    auto stage = [&](SlotRegs& R, long long mt) -> bool {
       const int ab = it % g.abufs;
       TC_T(0);
       const int j = it - g.abufs;  // the tile whose MMAs last read this A buffer
-      if (j >= 0 && !mbar_wait(smem_u32(&bars[j & 1]), (uint32_t)(j >> 1) & 1)) { *s_fail = 1; break; }
+      if (j >= 0 && !mbar_wait(smem_u32(&bars[j & 1]), (uint32_t)(j >> 1) & 1)) { *s_fail = 1; return false; }
       TC_T(1);
-      expand(a_s + (size_t)ab * a_bytes);
+      expand(R, a_s + (size_t)ab * a_bytes);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
       mbar_arrive(smem_u32(&bars[4 + ab]));
       TC_T(2);
-      if (mt + mt_step < g.m_tiles) prefetch(mt + mt_step);  // in flight while the tensor core works
-      if (*s_fail != 0) break;
+      if (mt + 2 * mt_step < g.m_tiles) prefetch(R, mt + 2 * mt_step);
+      it++;
+      return *s_fail == 0;
+    };
+    SlotRegs ra, rb;
+    long long mt = mt_first;
+    if (mt < g.m_tiles) prefetch(ra, mt);
+    if (mt + mt_step < g.m_tiles) prefetch(rb, mt + mt_step);
+    while (mt < g.m_tiles) {
+      if (!stage(ra, mt)) break;
+      mt += mt_step;
+      if (mt >= g.m_tiles) break;
+      if (!stage(rb, mt)) break;
+      mt += mt_step;
     }
 #ifdef TC_TIMING
     if (ptid == 0 && blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[i] = prof[i]; g_tc_prof[15] = it; }
