@@ -165,71 +165,149 @@ __global__ void __launch_bounds__(256) maxpool_pack(const float* __restrict__ x 
 }
 
 // ---- downsample shortcut: avgpool 2x2 / 2 -> fp32 conv 1x1 (C -> O) -> BN ---------------------------
-// CTA tile: 32 output pixels x 128 output channels; a thread owns 8 consecutive pixels x 4 channels
-// (o, o+32, o+64, o+96).  One fmaf chain per output over c ascending.
-constexpr int SC_TO = 4;
-__global__ void __launch_bounds__(128) shortcut_down(const float* __restrict__ x /*[N][HW][HW][C]*/, int HW, int C,
+// A register-tiled matrix product with a fixed summation order: CTA tile 128 output pixels x 128 output channels,
+// 256 threads, 8 pixels x 8 channels per thread, K (= C) in chunks of 16 through two shared-memory stages.  The pooled
+// activations are formed on the fly (four loads, three adds, one multiply, in that order) while the previous chunk is
+// being multiplied; weights arrive with cp.async.  Each output is one fmaf chain over c ascending, as pinned.
+constexpr int SC_BM = 128, SC_BN = 128, SC_BK = 16;
+__global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x /*[N][HW][HW][C]*/, int HW, int C,
                                                      const float* __restrict__ w /*[O][C]*/, int O,
                                                      const float* __restrict__ scale, const float* __restrict__ shift,
                                                      long long npix_out, float* __restrict__ y /*[N][HW/2][HW/2][O]*/) {
-  __shared__ __align__(16) float p_s[32][36];          // [c in chunk][pixel], padded
-  __shared__ float w_s[32 * SC_TO][33];                // [o in tile][c in chunk]
+  __shared__ __align__(16) float p_s[2][SC_BK][SC_BM + 4];  // [stage][c][pixel]
+  __shared__ __align__(16) float w_s[2][SC_BK][SC_BN + 4];  // [stage][c][channel]
   const int tid = threadIdx.x;
-  const long long p0 = (long long)blockIdx.x * 32;
-  const int o0 = blockIdx.y * (32 * SC_TO);
+  const long long p0 = (long long)blockIdx.x * SC_BM;
+  const int o0 = blockIdx.y * SC_BN;
   const int OHW = HW / 2;
-  const int ol = tid % 32, pgp = tid / 32;      // pixels pgp*8 .. pgp*8+7
-  float acc[8][SC_TO];
+  // loader roles: a thread pools 8 (pixel, c) pairs per chunk: pixel = tid / 2, c = (tid % 2) * 8 .. +7
+  const int lp = tid >> 1, lc = (tid & 1) * 8;
+  const long long pl = p0 + lp;
+  const float* xq = nullptr;
+  if (pl < npix_out) {
+    const int ow = (int)(pl % OHW), oh = (int)((pl / OHW) % OHW);
+    const long long n = pl / ((long long)OHW * OHW);
+    xq = x + ((n * HW + 2 * oh) * HW + 2 * ow) * C;
+  }
+  // weights: 16 c x 128 channels per chunk = 2048 floats: thread copies 8 floats of one channel row: channel = tid / 2
+  const int wo = tid >> 1, wc = (tid & 1) * 8;
+  const bool c_vec = (C % 8 == 0) && (reinterpret_cast<uintptr_t>(x) % 16 == 0) && (reinterpret_cast<uintptr_t>(w) % 16 == 0);
+  float pooled[8];
+  auto pool_load = [&](int c0) {  // registers <- pooled values of chunk c0
+#pragma unroll
+    for (int k = 0; k < 8; k++) pooled[k] = 0.0f;
+    if (xq == nullptr) return;
+    const int c = c0 + lc;
+    if (c_vec && c + 8 <= C) {
+      const float4* q00 = reinterpret_cast<const float4*>(xq + c);
+      const float4* q01 = reinterpret_cast<const float4*>(xq + C + c);
+      const float4* q10 = reinterpret_cast<const float4*>(xq + (size_t)HW * C + c);
+      const float4* q11 = reinterpret_cast<const float4*>(xq + (size_t)HW * C + C + c);
+#pragma unroll
+      for (int h = 0; h < 2; h++) {
+        const float4 a = q00[h], b = q01[h], cc = q10[h], d = q11[h];
+        pooled[4 * h + 0] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.x, b.x), cc.x), d.x), 0.25f);
+        pooled[4 * h + 1] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.y, b.y), cc.y), d.y), 0.25f);
+        pooled[4 * h + 2] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.z, b.z), cc.z), d.z), 0.25f);
+        pooled[4 * h + 3] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.w, b.w), cc.w), d.w), 0.25f);
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; k++)
+        if (c + k < C) {
+          const float* q = xq + c + k;
+          pooled[k] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(q[0], q[C]), q[(size_t)HW * C]), q[(size_t)HW * C + C]), 0.25f);
+        }
+    }
+  };
+  auto pool_store = [&](int st) {
+#pragma unroll
+    for (int k = 0; k < 8; k++) p_s[st][lc + k][lp] = pooled[k];
+  };
+  float wreg[8];
+  auto w_load = [&](int c0) {
+    const int o = o0 + wo, c = c0 + wc;
+#pragma unroll
+    for (int k = 0; k < 8; k++) wreg[k] = 0.0f;
+    if (o >= O) return;
+    if (c_vec && c + 8 <= C) {
+      const float4 a = *reinterpret_cast<const float4*>(w + (size_t)o * C + c);
+      const float4 b = *reinterpret_cast<const float4*>(w + (size_t)o * C + c + 4);
+      wreg[0] = a.x; wreg[1] = a.y; wreg[2] = a.z; wreg[3] = a.w; wreg[4] = b.x; wreg[5] = b.y; wreg[6] = b.z; wreg[7] = b.w;
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; k++)
+        if (c + k < C) wreg[k] = w[(size_t)o * C + c + k];
+    }
+  };
+  auto w_store = [&](int st) {
+#pragma unroll
+    for (int k = 0; k < 8; k++) w_s[st][wc + k][wo] = wreg[k];
+  };
+  // compute roles: 16 x 16 threads; thread (ty, tx) owns pixels ty*8..+7 and channels tx*4..+3 and 64 + tx*4..+3
+  const int ty = tid >> 4, tx = tid & 15;
+  float acc[8][8];
 #pragma unroll
   for (int i = 0; i < 8; i++)
 #pragma unroll
-    for (int j = 0; j < SC_TO; j++) acc[i][j] = 0.0f;
-  for (int c0 = 0; c0 < C; c0 += 32) {
-    __syncthreads();
-    for (int t = tid; t < 32 * 32; t += 128) {
-      const int cc = t % 32, pp = t / 32;
-      const long long p = p0 + pp;
-      float v = 0.0f;
-      if (p < npix_out && c0 + cc < C) {
-        const int ow = (int)(p % OHW), oh = (int)((p / OHW) % OHW);
-        const long long n = p / ((long long)OHW * OHW);
-        const float* q = x + ((n * HW + 2 * oh) * HW + 2 * ow) * C + c0 + cc;
-        float s = __fadd_rn(q[0], q[C]);
-        s = __fadd_rn(s, q[(size_t)HW * C]);
-        s = __fadd_rn(s, q[(size_t)HW * C + C]);
-        v = __fmul_rn(s, 0.25f);
-      }
-      p_s[cc][pp] = v;
+    for (int j = 0; j < 8; j++) acc[i][j] = 0.0f;
+  const int nchunks = (C + SC_BK - 1) / SC_BK;
+  pool_load(0);
+  w_load(0);
+  pool_store(0);
+  w_store(0);
+  __syncthreads();
+  for (int ch = 0; ch < nchunks; ch++) {
+    const int st = ch & 1;
+    if (ch + 1 < nchunks) {  // next chunk's global loads are in flight during this chunk's multiply-adds
+      pool_load((ch + 1) * SC_BK);
+      w_load((ch + 1) * SC_BK);
     }
-    for (int t = tid; t < 32 * SC_TO * 32; t += 128) {
-      const int cc = t % 32, oo = t / 32;
-      w_s[oo][cc] = (o0 + oo < O && c0 + cc < C) ? w[(size_t)(o0 + oo) * C + c0 + cc] : 0.0f;
-    }
-    __syncthreads();
-    const int cn = min(32, C - c0);
+    const int cn = min(SC_BK, C - ch * SC_BK);
 #pragma unroll 4
     for (int cc = 0; cc < cn; cc++) {
-      float wv[SC_TO];
-#pragma unroll
-      for (int j = 0; j < SC_TO; j++) wv[j] = w_s[ol + 32 * j][cc];
-      const float4 pa = *reinterpret_cast<const float4*>(&p_s[cc][pgp * 8]);
-      const float4 pb = *reinterpret_cast<const float4*>(&p_s[cc][pgp * 8 + 4]);
+      const float4 pa = *reinterpret_cast<const float4*>(&p_s[st][cc][ty * 8]);
+      const float4 pb = *reinterpret_cast<const float4*>(&p_s[st][cc][ty * 8 + 4]);
+      const float4 wa = *reinterpret_cast<const float4*>(&w_s[st][cc][tx * 4]);
+      const float4 wb = *reinterpret_cast<const float4*>(&w_s[st][cc][64 + tx * 4]);
       const float pv[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+      const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
       for (int i = 0; i < 8; i++)
 #pragma unroll
-        for (int j = 0; j < SC_TO; j++) acc[i][j] = __fmaf_rn(pv[i], wv[j], acc[i][j]);
+        for (int j = 0; j < 8; j++) acc[i][j] = __fmaf_rn(pv[i], wv[j], acc[i][j]);
     }
+    if (ch + 1 < nchunks) {
+      pool_store(st ^ 1);
+      w_store(st ^ 1);
+    }
+    __syncthreads();
   }
 #pragma unroll
-  for (int j = 0; j < SC_TO; j++) {
-    const int o = o0 + ol + 32 * j;
+  for (int h = 0; h < 2; h++) {
+    const int o = o0 + 64 * h + tx * 4;
     if (o >= O) continue;
-    const float sc = scale[o], sf = shift[o];
+    float sc[4], sf[4];
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      sc[j] = (o + j < O) ? scale[o + j] : 0.0f;
+      sf[j] = (o + j < O) ? shift[o + j] : 0.0f;
+    }
 #pragma unroll
     for (int i = 0; i < 8; i++) {
-      const long long p = p0 + pgp * 8 + i;
-      if (p < npix_out) y[p * O + o] = __fmaf_rn(acc[i][j], sc, sf);
+      const long long p = p0 + ty * 8 + i;
+      if (p >= npix_out) continue;
+      float* dst = y + p * O + o;
+      const float r0 = __fmaf_rn(acc[i][4 * h], sc[0], sf[0]), r1 = __fmaf_rn(acc[i][4 * h + 1], sc[1], sf[1]);
+      const float r2 = __fmaf_rn(acc[i][4 * h + 2], sc[2], sf[2]), r3 = __fmaf_rn(acc[i][4 * h + 3], sc[3], sf[3]);
+      if (o + 4 <= O && (O & 3) == 0 && (reinterpret_cast<uintptr_t>(y) & 15) == 0) {
+        *reinterpret_cast<float4*>(dst) = make_float4(r0, r1, r2, r3);
+      } else {
+        dst[0] = r0;
+        if (o + 1 < O) dst[1] = r1;
+        if (o + 2 < O) dst[2] = r2;
+        if (o + 3 < O) dst[3] = r3;
+      }
     }
   }
 }
@@ -448,11 +526,11 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     const bool down = stage > 0 && b % 4 == 0;
     if (down) {
       const long long npo = (long long)N * OHW * OHW;
-      if ((long long)ceil_div(npo, 32) * ceil_div(O, 32 * SC_TO) < sm_count() && C <= 512)
+      if ((long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) < sm_count() && C <= 512)
         shortcut_down_small<<<dim3(ceil_div(npo, 4), ceil_div(O, 64)), 256, 0, st>>>(
             cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
       else
-        shortcut_down<<<dim3(ceil_div(npo, 32), ceil_div(O, 32 * SC_TO)), 128, 0, st>>>(
+        shortcut_down<<<dim3(ceil_div(npo, SC_BM), ceil_div(O, SC_BN)), 256, 0, st>>>(
             cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
       if ((s = launch_status()) != DABNN_OK) return s;
       float* t = cur; cur = other; other = t;
