@@ -526,7 +526,7 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     const bool down = stage > 0 && b % 4 == 0;
     if (down) {
       const long long npo = (long long)N * OHW * OHW;
-      if ((long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) < sm_count() && C <= 512)
+      if ((long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) < 8 && C <= 512)  // a handful of tiles: one thread per output
         shortcut_down_small<<<dim3(ceil_div(npo, 4), ceil_div(O, 64)), 256, 0, st>>>(
             cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
       else
@@ -549,7 +549,7 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     uint64_t* tb = bits_in; bits_in = bits_out; bits_out = tb;
     C = O; HW = OHW;
   }
-  if (N < GAP_IMGS) {
+  if (N < 64) {  // few images: more, smaller CTAs
     float* gbuf = reinterpret_cast<float*>(base + ws.gap);
     gap_small<<<N, 512, 0, st>>>(cur, gbuf);
     if ((s = launch_status()) != DABNN_OK) return s;
