@@ -170,8 +170,8 @@ dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const 
  * The same convolutions (Section 2.1.2, Eq. 1 read as a +-1 dot product) computed on the tcgen05 tensor cores with
  * 4-bit {+1,-1} operands (e2m1, block scale 1.0, fp32 accumulation: exact) expanded on chip from the packed bits.
  * Results are identical to dabnn_bconv2d* bit for bit.
- * Covered: stride 1, C a multiple of 64 and at most 512, W + 2*pad_w small enough that a tile's 128 + (kh-1)*(W+2*pad_w)
- * + (kw-1) slots are at most 256, filters whose expanded weights fit the resident budget (dabnn_tc_weights_bytes
+ * Covered: stride 1 or 2 (both axes alike), C a multiple of 64 and at most 512 (256 for stride 2), images narrow enough
+ * that a tile's rows fit the activation buffer (W + 2*pad_w <= 63 for 3x3 stride 1), filters whose expanded weights fit the resident budget (dabnn_tc_weights_bytes
  * returns 0 otherwise); other cases return DABNN_ERR_UNSUPPORTED and are served by dabnn_bconv2d*.
  *   dabnn_tc_weights_bytes    bytes of the expanded weight buffer for a filter bank (0 = not covered)
  *   dabnn_tc_prepare_weights  w_packed [O][kh][kw][Cw] -> w_tc (device, 16-byte aligned, that many bytes); once per model

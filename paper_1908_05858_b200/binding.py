@@ -359,7 +359,7 @@ class TcWeights:
 
 
 def tc_supported(O: int, C: int, kh: int, kw: int, stride=(1, 1)) -> bool:
-    return tuple(stride) == (1, 1) and int(lib().dabnn_tc_weights_bytes(O, C, kh, kw)) > 0
+    return tuple(stride) in ((1, 1), (2, 2)) and int(lib().dabnn_tc_weights_bytes(O, C, kh, kw)) > 0
 
 
 def _tc_geom(a_packed, wt: TcWeights, stride, pad):

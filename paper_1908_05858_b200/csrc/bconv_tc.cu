@@ -35,7 +35,7 @@ constexpr int TC_SMEM_LIMIT = 232448;     // 227 KB opt-in maximum per CTA
 constexpr int TC_SMEM_MISC = 2048;        // barriers, TMEM base, flags, this CTA's scale / shift
 constexpr int TC_WEIGHT_BUDGET = 147456;  // 144 KB of resident weights at most
 constexpr int TC_MAX_CW = 8;              // C <= 512
-constexpr int TC_MAX_SLOTS = 256;         // two slots per producer thread
+constexpr int TC_MAX_SPT = 5;             // slots per producer thread: 2 for stride 1, up to 5 for stride 2
 constexpr int TC_TMEM_COLS = 512;         // 2 accumulators (<= 128 columns each) + the scale-factor columns
 constexpr int TC_SF_COL = 256;            // columns [256, 512) hold scale factors (all 1.0)
 
@@ -52,9 +52,12 @@ struct TcArgs {
   const uint8_t* w_tc;
   int N, H, W, Cw, C;
   int O, kh, kw, ph, pw, OH, OW;
-  int SP, HP;          // slot pitch and slot rows per image
+  int S;               // stride (1 or 2, both axes)
+  int SPin, HPin;      // padded input extent: W + 2*pad_w, H + 2*pad_h
+  int SP, HP;          // slot grid per image: ceil(SPin / S) columns, ceil(HPin / S) rows; output (oh, ow) sits at slot (oh, ow)
   long long total_q;   // N * HP * SP
-  int slots;           // slots per tile, multiple of 8
+  int slots_p;         // slots per parity plane and tile, multiple of 8
+  int slots;           // S*S*slots_p: rows of one 32-channel group in an A buffer
   int abufs;           // A buffers in shared memory (1 or 2)
   int ntile, n_ntiles; // output channels per tile, number of channel tiles
   long long m_tiles;
@@ -136,7 +139,7 @@ __device__ __forceinline__ void ld_global_v8(const void* p, float (&r)[8]) {
                : "l"(p));
 }
 
-template <int NT, int EPI>
+template <int NT, int EPI, int SPT>
 __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -238,9 +241,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         uint32_t accumulate = 0;
         uint64_t bdesc = bdesc0;  // weights are laid out in issue order: [tap][C/32][NT][16]
         for (int ti = 0; ti < g.kh; ti++) {
-          uint64_t arow = adesc0 + (uint64_t)(uint32_t)(ti * g.SP);  // start addresses are in 16-byte units
-          for (int tj = 0; tj < g.kw; tj++, arow += 1) {
-            uint64_t adesc = arow;
+          for (int tj = 0; tj < g.kw; tj++) {
+            // tap (ti, tj) reads parity plane (ti % S, tj % S) from a start shifted by (ti / S) slot rows and (tj / S) slots;
+            // start addresses are in 16-byte units
+            const uint32_t plane = (uint32_t)((ti % g.S) * g.S + (tj % g.S));
+            uint64_t adesc = adesc0 + (uint64_t)(plane * (uint32_t)g.slots_p + (uint32_t)((ti / g.S) * g.SP + (tj / g.S)));
 #pragma unroll 4
             for (int kb = 0; kb < kblocks; kb++, adesc += a_step, bdesc += b_step) {
               asm volatile(
@@ -267,29 +272,32 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     const int ptid = tid - 128;
     const int cgroups = g.C >> 5;
     const uint32_t pad_word4 = g.pad_neg ? 0xAAAAAAAAu : 0x22222222u;
+    constexpr int PCW = SPT > 2 ? 4 : TC_MAX_CW;  // words per slot held in registers (stride 2 is limited to C <= 256)
     struct SlotRegs {
-      uint64_t words[2][TC_MAX_CW];
-      int kind[2];  // 0: inside the image (words valid), 1: padding, 2: beyond the batch, 3: no such slot
+      uint64_t words[SPT][PCW];
+      int kind[SPT];  // 0: inside the image (words valid), 1: padding, 2: beyond the batch, 3: no such slot
     };
     auto prefetch = [&](SlotRegs& R, long long mt) {
 #pragma unroll
-      for (int h = 0; h < 2; h++) {
+      for (int h = 0; h < SPT; h++) {
         const int s = ptid + 128 * h;
         R.kind[h] = 3;
         if (s < g.slots) {
-          const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)s;  // total_q < 2^31 is checked on the host
+          const int plane = s / g.slots_p;              // 0 for stride 1
+          const int sp = s - plane * g.slots_p;
+          const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)sp;  // total_q < 2^31 is checked on the host
           const uint32_t rr = Q / (uint32_t)g.SP;
-          const int col = (int)(Q - rr * (uint32_t)g.SP);
+          const int cp = (int)(Q - rr * (uint32_t)g.SP);
           const uint32_t n = rr / (uint32_t)g.HP;
-          const int r = (int)(rr - n * (uint32_t)g.HP);
-          const int ih = r - g.ph, iw = col - g.pw;
+          const int rp = (int)(rr - n * (uint32_t)g.HP);
+          const int ih = rp * g.S + plane / g.S - g.ph, iw = cp * g.S + plane % g.S - g.pw;  // un-padded input coordinates
           if (n >= (uint32_t)g.N) R.kind[h] = 2;
           else if (ih < 0 || ih >= g.H || iw < 0 || iw >= g.W) R.kind[h] = 1;
           else {
             R.kind[h] = 0;
             const uint64_t* src = g.a + (((long long)n * g.H + ih) * g.W + iw) * g.Cw;
 #pragma unroll
-            for (int cw = 0; cw < TC_MAX_CW; cw++)
+            for (int cw = 0; cw < PCW; cw++)
               if (cw < g.Cw) R.words[h][cw] = __ldg(src + cw);
           }
         }
@@ -297,11 +305,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     };
     auto expand = [&](const SlotRegs& R, uint8_t* abuf) {
 #pragma unroll
-      for (int h = 0; h < 2; h++) {
+      for (int h = 0; h < SPT; h++) {
         if (R.kind[h] == 3) continue;
         const int s = ptid + 128 * h;
 #pragma unroll
-        for (int cw = 0; cw < TC_MAX_CW; cw++) {
+        for (int cw = 0; cw < PCW; cw++) {
           if (cw >= g.Cw) break;
 #pragma unroll
           for (int q2 = 0; q2 < 2; q2++) {  // a 64-bit word = two 32-channel rows
@@ -522,9 +530,9 @@ int tc_ntile(int O, int C, int taps) {
 // Channel tiles cover O rounded up to whole 64-bit sign words (rows beyond O hold zero weights).
 int tc_n_ntiles(int O, int nt) { return ((O + 63) / 64 * 64 + nt - 1) / nt; }
 
-template <int NT, int EPI>
+template <int NT, int EPI, int SPT>
 dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
-  auto kern = bconv_tc_kernel<NT, EPI>;
+  auto kern = bconv_tc_kernel<NT, EPI, SPT>;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT) != cudaSuccess) {
@@ -547,10 +555,18 @@ dabnn_status tc_dispatch(TcArgs& g, cudaStream_t st) {
   g.abufs = (wbytes + 2 * abytes + TC_SMEM_MISC <= (size_t)TC_SMEM_LIMIT) ? 2 : 1;
   const size_t smem = wbytes + g.abufs * abytes + TC_SMEM_MISC;
   if (smem > (size_t)TC_SMEM_LIMIT) return DABNN_ERR_UNSUPPORTED;
-  switch (g.ntile) {
-    case 128: return tc_launch<128, EPI>(g, smem, st);
-    case 64: return tc_launch<64, EPI>(g, smem, st);
-    case 32: return tc_launch<32, EPI>(g, smem, st);
+  if (g.slots <= 256) {
+    switch (g.ntile) {
+      case 128: return tc_launch<128, EPI, 2>(g, smem, st);
+      case 64: return tc_launch<64, EPI, 2>(g, smem, st);
+      case 32: return tc_launch<32, EPI, 2>(g, smem, st);
+    }
+  } else if (g.Cw <= 4) {
+    switch (g.ntile) {
+      case 128: return tc_launch<128, EPI, TC_MAX_SPT>(g, smem, st);
+      case 64: return tc_launch<64, EPI, TC_MAX_SPT>(g, smem, st);
+      case 32: return tc_launch<32, EPI, TC_MAX_SPT>(g, smem, st);
+    }
   }
   return DABNN_ERR_UNSUPPORTED;
 }
@@ -565,16 +581,19 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   const int OH = dabnn_out_dim(in.H, cv.kh, cv.stride_h, cv.pad_h), OW = dabnn_out_dim(in.W, cv.kw, cv.stride_w, cv.pad_w);
   if (OH <= 0 || OW <= 0) return DABNN_ERR_SHAPE;
   // what this engine covers; everything else is served by the xor/popcount kernel
-  if (cv.stride_h != 1 || cv.stride_w != 1 || in.C % 64 != 0) return DABNN_ERR_UNSUPPORTED;
+  if (cv.stride_h != cv.stride_w || cv.stride_h > 2 || in.C % 64 != 0) return DABNN_ERR_UNSUPPORTED;
   const int nt = tc_ntile(O, in.C, cv.kh * cv.kw);
   if (nt == 0) return DABNN_ERR_UNSUPPORTED;
   g.a = a; g.w_tc = static_cast<const uint8_t*>(w_tc);
   g.N = in.N; g.H = in.H; g.W = in.W; g.Cw = (in.C + 63) / 64; g.C = in.C;
   g.O = O; g.kh = cv.kh; g.kw = cv.kw; g.ph = cv.pad_h; g.pw = cv.pad_w; g.OH = OH; g.OW = OW;
-  g.SP = in.W + 2 * cv.pad_w; g.HP = in.H + 2 * cv.pad_h;
+  g.S = cv.stride_h;
+  g.SPin = in.W + 2 * cv.pad_w; g.HPin = in.H + 2 * cv.pad_h;
+  g.SP = (g.SPin + g.S - 1) / g.S; g.HP = (g.HPin + g.S - 1) / g.S;
   g.total_q = (long long)in.N * g.HP * g.SP;
-  g.slots = (128 + (cv.kh - 1) * g.SP + (cv.kw - 1) + 7) / 8 * 8;
-  if (g.slots > TC_MAX_SLOTS || g.Cw > TC_MAX_CW || g.total_q + 512 >= (1LL << 31)) return DABNN_ERR_UNSUPPORTED;
+  g.slots_p = (128 + ((cv.kh - 1) / g.S) * g.SP + (cv.kw - 1) / g.S + 7) / 8 * 8;
+  g.slots = g.S * g.S * g.slots_p;
+  if (g.slots > 128 * TC_MAX_SPT || g.Cw > TC_MAX_CW || g.total_q + 512 >= (1LL << 31)) return DABNN_ERR_UNSUPPORTED;
   g.ntile = nt; g.n_ntiles = tc_n_ntiles(O, nt);
   g.m_tiles = (g.total_q + 127) / 128;
   if ((long long)in.N * OH * OW >= (1LL << 31) || (long long)in.N * OH * OW * O > (1LL << 40)) return DABNN_ERR_UNSUPPORTED;
@@ -587,10 +606,11 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
 }  // namespace
 
 bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv) {
-  if (cv.stride_h != 1 || cv.stride_w != 1 || in.C % 64 != 0 || in.C > 64 * TC_MAX_CW) return false;
+  if (cv.stride_h != cv.stride_w || cv.stride_h > 2 || in.C % 64 != 0 || in.C > 64 * TC_MAX_CW) return false;
   const int nt = tc_ntile(O, in.C, cv.kh * cv.kw);
   if (nt == 0) return false;
-  const long long slots_total = (long long)in.N * (in.H + 2 * cv.pad_h) * (in.W + 2 * cv.pad_w);
+  const int S = cv.stride_h;
+  const long long slots_total = (long long)in.N * ((in.H + 2 * cv.pad_h + S - 1) / S) * ((in.W + 2 * cv.pad_w + S - 1) / S);
   return (slots_total / 128) * tc_n_ntiles(O, nt) >= 2LL * sm_count();
 }
 

@@ -214,7 +214,7 @@ def test_bireal18_forward_matches_oracle(B, oracle_mod):
     got = net.forward(dev(img)).cpu().numpy()
     # the integer-pipe engine alone gives the same bits as the mixed (tensor-core where covered) network
     assert np.array_equal(B.Bireal18(p, engine="popc").forward(dev(img)).cpu().numpy(), got)
-    assert sum(1 for b in range(16) if net.P.block_w_tc[b]) == 13 and B.tc_error_flag() == 0
+    assert sum(1 for b in range(16) if net.P.block_w_tc[b]) == 16 and B.tc_error_flag() == 0
     scale = np.max(np.abs(want))
     assert np.max(np.abs(got - want)) <= 1e-3 * scale
     assert np.array_equal(got.argmax(axis=1), want.argmax(axis=1))

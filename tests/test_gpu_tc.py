@@ -27,7 +27,7 @@ def u64(t):
 
 
 TC_CASES = [
-    # N, C, H, W, O, k, pad, pad_value
+    # N, C, H, W, O, k, pad, pad_value[, stride]
     (1, 64, 14, 14, 64, 3, 1, -1),      # BASELINE config 1
     (2, 128, 9, 11, 100, 3, 1, +1),     # O not a multiple of 16, pad +1
     (3, 256, 14, 14, 256, 3, 1, -1),    # four channel tiles of 64
@@ -38,31 +38,38 @@ TC_CASES = [
     (5, 64, 6, 7, 33, 3, 1, -1),        # smallest C, O just over a 32-channel tile
     (9, 128, 28, 28, 128, 3, 1, -1),    # many pixel tiles per CTA? (persistent loop over tiles)
     (300, 64, 8, 8, 64, 3, 0, -1),      # no padding, many images per tile
+    (3, 64, 56, 56, 128, 3, 1, -1, 2),  # stride 2 (four parity planes): Bi-Real stage 2 entry
+    (5, 128, 28, 28, 256, 3, 1, -1, 2),
+    (7, 256, 14, 14, 512, 3, 1, +1, 2),
+    (2, 64, 13, 11, 70, 3, 1, -1, 2),   # odd sizes, stride 2
+    (2, 128, 12, 12, 64, 1, 0, -1, 2),  # 1x1 stride 2
+    (2, 64, 16, 16, 64, 5, 2, -1, 2),   # 5x5 stride 2
 ]
 
 
 def inputs(case):
-    N, C, H, W, O, k, pad, pv = case
+    N, C, H, W, O, k, pad, pv = case[:8]
     rng = np.random.default_rng(abs(hash(case)) % (2**32))
     return rng.standard_normal((N, C, H, W)).astype(np.float32), rng.standard_normal((O, C, k, k)).astype(np.float32)
 
 
 @pytest.mark.parametrize("case", TC_CASES)
 def test_tc_conv_and_epilogues_match_oracle(B, oracle_mod, case):
-    N, C, H, W, O, k, pad, pv = case
+    N, C, H, W, O, k, pad, pv = case[:8]
+    st = (case[8], case[8]) if len(case) > 8 else (1, 1)
     x, w = inputs(case)
     o = oracle_mod
-    acc = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (1, 1), (pad, pad), pv, o.NHWC)
+    acc = o.bconv_bits(o.pack(x), C, o.pack_weights(w), st, (pad, pad), pv, o.NHWC)
     a = B.pack(dev(x))
     wp = B.pack_weights(dev(w))
-    assert B.tc_supported(O, C, k, k)
+    assert B.tc_supported(O, C, k, k, st)
     wt = B.TcWeights(wp, C)
-    got = B.tc_bconv2d(a, wt, (1, 1), (pad, pad), pv, B.NHWC).cpu().numpy()
+    got = B.tc_bconv2d(a, wt, st, (pad, pad), pv, B.NHWC).cpu().numpy()
     assert np.array_equal(got, acc)
-    got_nchw = B.tc_bconv2d(a, wt, (1, 1), (pad, pad), pv, B.NCHW).cpu().numpy()
+    got_nchw = B.tc_bconv2d(a, wt, st, (pad, pad), pv, B.NCHW).cpu().numpy()
     assert np.array_equal(got_nchw, np.transpose(acc, (0, 3, 1, 2)))
     # the xor/popcount kernel gives the same integers
-    assert np.array_equal(B.bconv2d(a, C, wp, (1, 1), (pad, pad), pv, B.NHWC).cpu().numpy(), acc)
+    assert np.array_equal(B.bconv2d(a, C, wp, st, (pad, pad), pv, B.NHWC).cpu().numpy(), acc)
     # fused BN + sign + pack
     rng = np.random.default_rng(O)
     gamma, beta, mean, var = synth.bn_params(rng, O)
@@ -70,12 +77,12 @@ def test_tc_conv_and_epilogues_match_oracle(B, oracle_mod, case):
     mean *= 30.0
     scale, shift = o.bn_fold(gamma, beta, mean, var)
     want_bits = o.bn_sign_pack(acc, scale, shift)
-    got_bits = u64(B.tc_bconv2d_bn_sign_pack(a, wt, dev(scale), dev(shift), (1, 1), (pad, pad), pv))
+    got_bits = u64(B.tc_bconv2d_bn_sign_pack(a, wt, dev(scale), dev(shift), st, (pad, pad), pv))
     assert np.array_equal(got_bits, want_bits)
     # Bi-Real block epilogue
     res = rng.standard_normal(acc.shape).astype(np.float32) * 20
     y = (acc.astype(np.float64) * scale.astype(np.float64) + shift.astype(np.float64)).astype(np.float32) + res
-    got_y, got_ybits = B.tc_bconv2d_bn_add_sign_pack(a, wt, dev(scale), dev(shift), dev(res), (1, 1), (pad, pad), pv)
+    got_y, got_ybits = B.tc_bconv2d_bn_add_sign_pack(a, wt, dev(scale), dev(shift), dev(res), st, (pad, pad), pv)
     assert np.array_equal(got_y.cpu().numpy().view(np.uint32), y.view(np.uint32))
     assert np.array_equal(u64(got_ybits), o.pack(y, o.NHWC))
     torch.cuda.synchronize()
@@ -83,13 +90,13 @@ def test_tc_conv_and_epilogues_match_oracle(B, oracle_mod, case):
 
 
 def test_tc_declines_what_it_does_not_cover(B):
-    assert not B.tc_supported(64, 64, 3, 3, stride=(2, 2))
+    assert not B.tc_supported(64, 64, 3, 3, stride=(3, 3))
     assert not B.tc_supported(64, 96, 3, 3)          # C not a multiple of 64
     assert not B.tc_supported(64, 2048, 7, 7)        # expanded weights larger than the resident budget
     a = torch.zeros((1, 8, 8, 1), dtype=torch.int64, device="cuda")
     wt = B.TcWeights(torch.zeros((64, 3, 3, 1), dtype=torch.int64, device="cuda"), 64)
     with pytest.raises(B.DabnnError, match="supported"):
-        B.tc_bconv2d(a, wt, (2, 2), (1, 1), -1)
+        B.tc_bconv2d(a, wt, (2, 1), (1, 1), -1)
 
 
 @pytest.mark.parametrize("cfg", [(64, 64, 56, 64, 3, 1), (64, 512, 7, 512, 3, 1), (256, 256, 28, 256, 3, 1), (256, 512, 14, 2048, 1, 0)])
