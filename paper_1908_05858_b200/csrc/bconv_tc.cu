@@ -371,13 +371,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #endif
     for (long long mt = mt_first; mt < g.m_tiles; mt += mt_step, it++) {
       const int buf = it & 1;
-      TC_T(0);
-      if (!mbar_wait(smem_u32(&bars[buf]), (it >> 1) & 1)) {
-        *s_fail = 1;
-        break;
-      }
-      TC_T(1);
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int row = 32 * warp + lane;  // TMEM lane = slot row of the tile
       const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)row;
       const uint32_t rr = Q / (uint32_t)g.SP;
@@ -386,14 +379,41 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       const int r = (int)(rr - n * (uint32_t)g.HP);
       const int my_valid = (n < (uint32_t)g.N && r < g.OH && col < g.OW) ? 1 : 0;
       const int my_m = (int)((n * (uint32_t)g.OH + (uint32_t)r) * (uint32_t)g.OW + (uint32_t)col);  // < 2^31 (host check)
-      const long long m = my_m;
       // wide outputs: 256-bit accesses when rows are 32-byte multiples at 32-byte aligned addresses
       const bool wide_i32 = EPI == EPI_I32 && !g.out_nchw && (g.O & 7) == 0 && (reinterpret_cast<uintptr_t>(g.out) & 31) == 0;
       const bool wide_y = EPI == EPI_BIREAL && (g.O & 7) == 0 &&
                           ((reinterpret_cast<uintptr_t>(g.residual) | reinterpret_cast<uintptr_t>(g.y_out)) & 31) == 0;
+      // The residual does not depend on the MMAs: its first 32 channels are requested before waiting for them, and
+      // every later chunk one chunk ahead of its use.
+      float rpre[32];
+      auto load_res = [&](int c0) {
+        if (EPI == EPI_BIREAL && wide_y && my_valid) {
+          const int o = nt * NT + c0;
+          const int nch = min(32, g.O - o);
+          const float* rs = g.residual + (long long)my_m * g.O + o;
+#pragma unroll
+          for (int q = 0; q < 4; q++)
+            if (8 * q < nch) ld_global_v8(rs + 8 * q, *reinterpret_cast<float(*)[8]>(&rpre[8 * q]));
+        }
+      };
+      load_res(0);
+      TC_T(0);
+      if (!mbar_wait(smem_u32(&bars[buf]), (it >> 1) & 1)) {
+        *s_fail = 1;
+        break;
+      }
+      TC_T(1);
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const long long m = my_m;
 #pragma unroll 1
       for (int c0 = 0; c0 < NT; c0 += 32) {
         __syncwarp();  // the TMEM load is warp-wide: rejoin lanes that took different paths below
+        float rc[32];
+        if (EPI == EPI_BIREAL) {
+#pragma unroll
+          for (int j = 0; j < 32; j++) rc[j] = rpre[j];
+          if (c0 + 32 < NT) load_res(c0 + 32);
+        }
         uint32_t v[32];
         const uint32_t taddr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)(buf * NT + c0);
         asm volatile(
@@ -454,10 +474,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #pragma unroll
               for (int q = 0; q < 4; q++)
                 if (8 * q < nch) {  // nch is a multiple of 8 here
-                  float r8[8];
-                  ld_global_v8(rs + 8 * q, r8);
 #pragma unroll
-                  for (int j = 0; j < 8; j++) y[8 * q + j] = __fadd_rn(y[8 * q + j], r8[j]);
+                  for (int j = 0; j < 8; j++) y[8 * q + j] = __fadd_rn(y[8 * q + j], rc[8 * q + j]);
                   st_global_v8(yd + 8 * q, __float_as_uint(y[8 * q]), __float_as_uint(y[8 * q + 1]), __float_as_uint(y[8 * q + 2]),
                                __float_as_uint(y[8 * q + 3]), __float_as_uint(y[8 * q + 4]), __float_as_uint(y[8 * q + 5]),
                                __float_as_uint(y[8 * q + 6]), __float_as_uint(y[8 * q + 7]));
