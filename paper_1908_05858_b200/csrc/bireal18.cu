@@ -131,6 +131,107 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
   asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
+// Large batches: the same convolution with an 8 pixels (along a row) x 8 channels register tile.  Per (c, kh) a thread
+// loads the 21 input values its 8 pixels need (even and odd columns as 3 + 3 float4) once and reuses them for all 7
+// horizontal taps; per tap it loads 8 weights.  Persistent CTAs as above; the order of every output's fmaf chain is
+// unchanged: c, then kh, then kw.
+__global__ void __launch_bounds__(256, 2) stem_conv_bn_8x8(const float* __restrict__ img, const float* __restrict__ w,
+                                                           const float* __restrict__ scale,
+                                                           const float* __restrict__ shift, int N,
+                                                           float* __restrict__ out /*[N][112][112][64]*/) {
+  constexpr int TS = 16, IH = 224, IW = 224, OHW = 112;
+  constexpr int PS = 2 * TS + 5;         // 37
+  constexpr int HALF = 20;               // columns per parity (19 / 18 used), a multiple of 4
+  constexpr int PATCH = 3 * PS * 2 * HALF;
+  constexpr int THREADS = 256;
+  constexpr int TILES = OHW / TS;        // 7
+  extern __shared__ __align__(16) float sm[];
+  float* w_s = sm;                       // [147][64]
+  float* x_s = sm + STEM_K * 64;         // [2 buffers][3][PS][2][HALF]
+  const int tid = threadIdx.x;
+  for (int t = tid; t < STEM_K * 64; t += THREADS) {
+    const int o = t % 64, k = t / 64;
+    w_s[k * 64 + o] = w[o * STEM_K + k];
+  }
+  const long long ntiles = (long long)N * TILES * TILES;
+  auto load_patch = [&](long long tile, float* dst) {
+    const int n = (int)(tile / (TILES * TILES));
+    const int rem = (int)(tile % (TILES * TILES));
+    const int ih_base = 2 * (rem / TILES) * TS - 3, iw_base = 2 * (rem % TILES) * TS - 3;
+    for (int t = tid; t < 3 * PS * 2 * HALF; t += THREADS) {  // every word of the buffer, padding columns included
+      const int hc = t % HALF, par = (t / HALF) % 2, lh = (t / (2 * HALF)) % PS, c = t / (2 * HALF * PS);
+      const int lw = 2 * hc + par;
+      const int ih = ih_base + lh, iw = iw_base + lw;
+      const bool in = lw < PS && ih >= 0 && ih < IH && iw >= 0 && iw < IW;
+      const float* src = in ? img + (((size_t)n * 3 + c) * IH + ih) * IW + iw : img;
+      const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst + t);
+      asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(d), "l"(src), "r"(in ? 4 : 0) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  const int chg = tid & 7, pg = tid >> 3;        // 8 channel groups x 32 pixel groups
+  const int row = pg >> 1, ow0 = (pg & 1) * 8;   // 8 consecutive pixels of one tile row
+  float sc[8], sf[8];
+#pragma unroll
+  for (int j = 0; j < 8; j++) {
+    sc[j] = scale[chg * 8 + j];
+    sf[j] = shift[chg * 8 + j];
+  }
+  long long tile = blockIdx.x;
+  int buf = 0;
+  if (tile < ntiles) load_patch(tile, x_s);
+  for (; tile < ntiles; tile += gridDim.x, buf ^= 1) {
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    if (tile + gridDim.x < ntiles) load_patch(tile + gridDim.x, x_s + (buf ^ 1) * PATCH);
+    const float* xb = x_s + buf * PATCH;
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; i++)
+#pragma unroll
+      for (int j = 0; j < 8; j++) acc[i][j] = 0.0f;
+#pragma unroll 1
+    for (int c = 0; c < 3; c++)
+#pragma unroll 1
+      for (int ki = 0; ki < 7; ki++) {
+        const float* xr = xb + ((c * PS + 2 * row + ki) * 2) * HALF + ow0;
+        float xe[12], xo[12];  // even / odd input columns 2*(ow0 + t), 2*(ow0 + t) + 1
+#pragma unroll
+        for (int q = 0; q < 3; q++) {
+          const float4 e4 = *reinterpret_cast<const float4*>(xr + 4 * q);
+          const float4 o4 = *reinterpret_cast<const float4*>(xr + HALF + 4 * q);
+          xe[4 * q] = e4.x; xe[4 * q + 1] = e4.y; xe[4 * q + 2] = e4.z; xe[4 * q + 3] = e4.w;
+          xo[4 * q] = o4.x; xo[4 * q + 1] = o4.y; xo[4 * q + 2] = o4.z; xo[4 * q + 3] = o4.w;
+        }
+        const float* wk = w_s + ((c * 7 + ki) * 7) * 64 + chg * 8;
+#pragma unroll
+        for (int kj = 0; kj < 7; kj++) {
+          const float4 wa = *reinterpret_cast<const float4*>(wk + kj * 64);
+          const float4 wb = *reinterpret_cast<const float4*>(wk + kj * 64 + 4);
+          const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+          for (int i = 0; i < 8; i++) {
+            const float xv = (kj & 1) ? xo[i + (kj >> 1)] : xe[i + (kj >> 1)];
+#pragma unroll
+            for (int j = 0; j < 8; j++) acc[i][j] = __fmaf_rn(xv, wv[j], acc[i][j]);
+          }
+        }
+      }
+    const int n = (int)(tile / (TILES * TILES));
+    const int rem = (int)(tile % (TILES * TILES));
+    const int oh = (rem / TILES) * TS + row, owb = (rem % TILES) * TS + ow0;
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+      float* dst = out + (((size_t)n * OHW + oh) * OHW + owb + i) * 64 + chg * 8;
+      *reinterpret_cast<float4*>(dst) = make_float4(__fmaf_rn(acc[i][0], sc[0], sf[0]), __fmaf_rn(acc[i][1], sc[1], sf[1]),
+                                                    __fmaf_rn(acc[i][2], sc[2], sf[2]), __fmaf_rn(acc[i][3], sc[3], sf[3]));
+      *reinterpret_cast<float4*>(dst + 4) = make_float4(__fmaf_rn(acc[i][4], sc[4], sf[4]), __fmaf_rn(acc[i][5], sc[5], sf[5]),
+                                                        __fmaf_rn(acc[i][6], sc[6], sf[6]), __fmaf_rn(acc[i][7], sc[7], sf[7]));
+    }
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
 // ---- maxpool 3x3 / 2, pad 1 (64 channels) -> fp32 residual stream + packed signs -------------------
 // A thread handles 4 channels of one output pixel; 16 lanes make one 64-bit word.
 __global__ void __launch_bounds__(256) maxpool_pack(const float* __restrict__ x /*[N][112][112][64]*/, long long npix,
@@ -454,6 +555,22 @@ Workspace plan(int N) {
   return ws;
 }
 
+dabnn_status launch_stem_8x8(const dabnn_bireal18_params* p, const float* images, int N, float* out, cudaStream_t st) {
+  constexpr size_t SMEM = (size_t)(STEM_K * 64 + 2 * 3 * 37 * 2 * 20) * 4;
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(stem_conv_bn_8x8, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) {
+      cudaGetLastError();
+      return DABNN_ERR_CUDA;
+    }
+    configured = true;
+  }
+  const long long ntiles = (long long)N * 49, cap = 2LL * sm_count();
+  stem_conv_bn_8x8<<<(unsigned)(ntiles < cap ? ntiles : cap), 256, SMEM, st>>>(images, p->stem_w, p->stem_scale,
+                                                                             p->stem_shift, N, out);
+  return launch_status();
+}
+
 template <int TS, int PPT>
 dabnn_status launch_stem(const dabnn_bireal18_params* p, const float* images, int N, float* out, cudaStream_t st) {
   constexpr int PS = 2 * TS + 5, HALF = (PS + 1) / 2 + 1;
@@ -512,7 +629,7 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
   uint64_t* bits_in = reinterpret_cast<uint64_t*>(base + ws.bits_a);
   uint64_t* bits_out = reinterpret_cast<uint64_t*>(base + ws.bits_b);
 
-  dabnn_status s = (N * 49 >= 2 * sm_count()) ? launch_stem<16, 4>(p, images, N, stem_out, st)
+  dabnn_status s = (N * 49 >= 2 * sm_count()) ? launch_stem_8x8(p, images, N, stem_out, st)
                                                : launch_stem<8, 1>(p, images, N, stem_out, st);
   if (s != DABNN_OK) return s;
   {

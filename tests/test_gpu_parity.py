@@ -256,3 +256,16 @@ def test_bgemm_matches_eq1(B, oracle_mod, shape):
     got = B.bgemm(A, Bm, K).cpu().numpy()
     counts = oracle_mod.bgemm_xnor(u64(A), u64(Bm), K)  # Eq. 1 as printed: agreeing positions
     assert np.array_equal(got, 2 * counts - K)
+
+
+def test_bireal18_large_batch_kernels_match_oracle(B, oracle_mod):
+    """Batch 8 is large enough for the persistent 8x8-tile stem, the tiled shortcut kernel and the tensor-core engine
+    on the early stages; the logits must still equal the oracle's bit for bit."""
+    p = synth.bireal18_params()
+    img = synth.bireal18_images(8)
+    want = oracle_mod.bireal18_forward(p, img, conv_form=1)
+    got = B.Bireal18(p).forward(dev(img)).cpu().numpy()
+    assert np.max(np.abs(got - want)) <= 1e-3 * np.max(np.abs(want))
+    assert np.array_equal(got.argmax(axis=1), want.argmax(axis=1))
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert B.tc_error_flag() == 0
