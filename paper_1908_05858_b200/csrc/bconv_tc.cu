@@ -222,6 +222,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       const uint64_t bdesc0 = make_desc(smem_u32(w_s), (uint32_t)NT * 16, 128);
       const uint64_t a_step = (uint64_t)(2u * (uint32_t)g.slots), b_step = (uint64_t)(2u * NT);  // one K = 64 block
       const int kblocks = g.C >> 6;
+      const int sshift = g.S - 1, smask = g.S - 1;  // stride 1 or 2: masks and shifts instead of divisions
 #ifdef TC_TIMING
       long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
       long long tlast = clock64();
@@ -243,9 +244,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         for (int ti = 0; ti < g.kh; ti++) {
           for (int tj = 0; tj < g.kw; tj++) {
             // tap (ti, tj) reads parity plane (ti % S, tj % S) from a start shifted by (ti / S) slot rows and (tj / S) slots;
-            // start addresses are in 16-byte units
-            const uint32_t plane = (uint32_t)((ti % g.S) * g.S + (tj % g.S));
-            uint64_t adesc = adesc0 + (uint64_t)(plane * (uint32_t)g.slots_p + (uint32_t)((ti / g.S) * g.SP + (tj / g.S)));
+            // start addresses are in 16-byte units (S is 1 or 2: masks and shifts, no divisions in this single-thread chain)
+            const uint32_t plane = (uint32_t)(((ti & smask) << sshift) + (tj & smask));
+            uint64_t adesc = adesc0 + (uint64_t)(plane * (uint32_t)g.slots_p + (uint32_t)((ti >> sshift) * g.SP + (tj >> sshift)));
 #pragma unroll 4
             for (int kb = 0; kb < kblocks; kb++, adesc += a_step, bdesc += b_step) {
               asm volatile(
@@ -283,14 +284,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         const int s = ptid + 128 * h;
         R.kind[h] = 3;
         if (s < g.slots) {
-          const int plane = s / g.slots_p;              // 0 for stride 1
-          const int sp = s - plane * g.slots_p;
+          int plane = 0, sp = s;                        // parity plane of this row (always 0 for stride 1)
+          while (sp >= g.slots_p) { sp -= g.slots_p; plane++; }
           const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)sp;  // total_q < 2^31 is checked on the host
           const uint32_t rr = Q / (uint32_t)g.SP;
           const int cp = (int)(Q - rr * (uint32_t)g.SP);
           const uint32_t n = rr / (uint32_t)g.HP;
           const int rp = (int)(rr - n * (uint32_t)g.HP);
-          const int ih = rp * g.S + plane / g.S - g.ph, iw = cp * g.S + plane % g.S - g.pw;  // un-padded input coordinates
+          const int sshift = g.S - 1;                   // stride 1 or 2
+          const int ih = (rp << sshift) + (plane >> sshift) - g.ph, iw = (cp << sshift) + (plane & sshift) - g.pw;  // un-padded input coordinates
           if (n >= (uint32_t)g.N) R.kind[h] = 2;
           else if (ih < 0 || ih >= g.H || iw < 0 || iw >= g.W) R.kind[h] = 1;
           else {
@@ -611,7 +613,8 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   g.total_q = (long long)in.N * g.HP * g.SP;
   g.slots_p = (128 + ((cv.kh - 1) / g.S) * g.SP + (cv.kw - 1) / g.S + 7) / 8 * 8;
   g.slots = g.S * g.S * g.slots_p;
-  if (g.slots > 128 * TC_MAX_SPT || g.Cw > TC_MAX_CW || g.total_q + 512 >= (1LL << 31)) return DABNN_ERR_UNSUPPORTED;
+  if (g.slots > 128 * TC_MAX_SPT || g.Cw > TC_MAX_CW || g.total_q + 512 >= (1LL << 31))
+    return DABNN_ERR_UNSUPPORTED;
   g.ntile = nt; g.n_ntiles = tc_n_ntiles(O, nt);
   g.m_tiles = (g.total_q + 127) / 128;
   if ((long long)in.N * OH * OW >= (1LL << 31) || (long long)in.N * OH * OW * O > (1LL << 40)) return DABNN_ERR_UNSUPPORTED;
@@ -629,7 +632,7 @@ bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv) {
   if (nt == 0) return false;
   const int S = cv.stride_h;
   const long long slots_total = (long long)in.N * ((in.H + 2 * cv.pad_h + S - 1) / S) * ((in.W + 2 * cv.pad_w + S - 1) / S);
-  return (slots_total / 128) * tc_n_ntiles(O, nt) >= 2LL * sm_count();
+  return (slots_total / 128) * tc_n_ntiles(O, nt) >= (long long)sm_count();
 }
 
 }  // namespace dabnn

@@ -460,7 +460,8 @@ __global__ void __launch_bounds__(256) shortcut_down_small(const float* __restri
   y[p * O + o] = __fmaf_rn(a, scale[o], shift[o]);
 }
 
-// Small batches: the pooled vector is written to the workspace by one kernel and 32-thread CTAs compute the logits.
+// ---- head: global average over 7x7 (sequential sum over (h, w), then /49) into the workspace, then fc 512 -> 1000 as
+// one fmaf chain per logit over k ascending, then + bias.  Small batches: 32-thread CTAs, one image each.
 __global__ void __launch_bounds__(512) gap_small(const float* __restrict__ x /*[N][7][7][512]*/, float* __restrict__ g) {
   const int n = blockIdx.x, c = threadIdx.x;
   float s = 0.0f;
@@ -490,37 +491,30 @@ __global__ void __launch_bounds__(32) fc_small(const float* __restrict__ g /*[N]
   logits[(size_t)n * 1000 + j] = __fadd_rn(a, fb[j]);
 }
 
-// ---- head: global average over 7x7 (sequential sum, then /49), fc 512 -> 1000 -----------------------
-// A CTA takes GAP_IMGS images and 256 logits: the pooled vectors sit in shared memory and every fc weight a thread
-// loads is used for all of the CTA's images.  One fmaf chain per logit over k ascending, then + bias.
-constexpr int GAP_IMGS = 8;
-__global__ void __launch_bounds__(256) gap_fc(const float* __restrict__ x /*[N][7][7][512]*/, int N,
-                                              const float* __restrict__ fw /*[1000][512]*/,
-                                              const float* __restrict__ fb, float* __restrict__ logits) {
-  __shared__ __align__(16) float g[GAP_IMGS][512];
-  const int n0 = blockIdx.y * GAP_IMGS;
-  const int nimg = min(GAP_IMGS, N - n0);
-  for (int t = threadIdx.x; t < GAP_IMGS * 512; t += blockDim.x) {
-    const int c = t % 512, im = t / 512;
-    float s = 0.0f;
-    if (im < nimg) {
-      for (int q = 0; q < 49; q++) s = __fadd_rn(s, x[((size_t)(n0 + im) * 49 + q) * 512 + c]);
-      s = __fdiv_rn(s, 49.0f);
-    }
-    g[im][c] = s;
+// Larger batches: pooled vectors come from gap_small; a 64-thread CTA computes 64 logits for 8 images, so every weight
+// it loads is used 8 times and there are 16 x N/8 CTAs.
+__global__ void __launch_bounds__(64) fc_batched(const float* __restrict__ g /*[N][512]*/, int N, const float* __restrict__ fw,
+                                                 const float* __restrict__ fb, float* __restrict__ logits) {
+  __shared__ __align__(16) float gs[8][512];
+  const int n0 = blockIdx.y * 8, nimg = min(8, N - n0);
+  for (int t = threadIdx.x; t < 8 * 128; t += 64) {
+    const int im = t / 128;
+    reinterpret_cast<float4*>(&gs[0][0])[t] =
+        im < nimg ? reinterpret_cast<const float4*>(g + (size_t)n0 * 512)[t] : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   __syncthreads();
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  const int j = blockIdx.x * 64 + threadIdx.x;
   if (j >= 1000) return;
   const float4* wr = reinterpret_cast<const float4*>(fw + (size_t)j * 512);
-  float a[GAP_IMGS];
+  float a[8];
 #pragma unroll
-  for (int im = 0; im < GAP_IMGS; im++) a[im] = 0.0f;
+  for (int im = 0; im < 8; im++) a[im] = 0.0f;
+#pragma unroll 2
   for (int k4 = 0; k4 < 128; k4++) {
     const float4 wv = __ldg(wr + k4);
 #pragma unroll
-    for (int im = 0; im < GAP_IMGS; im++) {
-      const float4 gv = *reinterpret_cast<const float4*>(&g[im][4 * k4]);
+    for (int im = 0; im < 8; im++) {
+      const float4 gv = *reinterpret_cast<const float4*>(&gs[im][4 * k4]);
       a[im] = __fmaf_rn(gv.x, wv.x, a[im]);
       a[im] = __fmaf_rn(gv.y, wv.y, a[im]);
       a[im] = __fmaf_rn(gv.z, wv.z, a[im]);
@@ -529,7 +523,7 @@ __global__ void __launch_bounds__(256) gap_fc(const float* __restrict__ x /*[N][
   }
   const float bias = fb[j];
 #pragma unroll
-  for (int im = 0; im < GAP_IMGS; im++)
+  for (int im = 0; im < 8; im++)
     if (im < nimg) logits[(size_t)(n0 + im) * 1000 + j] = __fadd_rn(a[im], bias);
 }
 
@@ -666,13 +660,12 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     uint64_t* tb = bits_in; bits_in = bits_out; bits_out = tb;
     C = O; HW = OHW;
   }
-  if (N < 64) {  // few images: more, smaller CTAs
+  {
     float* gbuf = reinterpret_cast<float*>(base + ws.gap);
     gap_small<<<N, 512, 0, st>>>(cur, gbuf);
     if ((s = launch_status()) != DABNN_OK) return s;
-    fc_small<<<dim3(ceil_div(1000, 32), N), 32, 0, st>>>(gbuf, p->fc_w, p->fc_b, logits);
-  } else {
-    gap_fc<<<dim3(4, ceil_div(N, GAP_IMGS)), 256, 0, st>>>(cur, N, p->fc_w, p->fc_b, logits);
+    if (N < 64) fc_small<<<dim3(ceil_div(1000, 32), N), 32, 0, st>>>(gbuf, p->fc_w, p->fc_b, logits);  // few images: many small CTAs
+    else fc_batched<<<dim3(ceil_div(1000, 64), ceil_div(N, 8)), 64, 0, st>>>(gbuf, N, p->fc_w, p->fc_b, logits);
   }
   return launch_status();
 }
