@@ -56,6 +56,7 @@ struct TcArgs {
   int SPin, HPin;      // padded input extent: W + 2*pad_w, H + 2*pad_h
   int SP, HP;          // slot grid per image: ceil(SPin / S) columns, ceil(HPin / S) rows; output (oh, ow) sits at slot (oh, ow)
   long long total_q;   // N * HP * SP
+  unsigned long long magic_sp, magic_hp;  // ceil(2^64 / SP), ceil(2^64 / HP) (0 when the divisor is 1)
   int slots_p;         // slots per parity plane and tile, multiple of 8
   int slots;           // S*S*slots_p: rows of one 32-channel group in an A buffer
   int abufs;           // A buffers in shared memory (1 or 2)
@@ -139,6 +140,14 @@ __device__ __forceinline__ void ld_global_v8(const void* p, float (&r)[8]) {
                : "l"(p));
 }
 
+template <int V>
+struct IntC { static constexpr int value = V; };
+
+// floor(q / d) for q < 2^32 and 1 <= d < 2^16 with magic = ceil(2^64 / d): one 64-bit multiply-high instead of a division.
+__device__ __forceinline__ uint32_t fast_div(uint32_t q, unsigned long long magic) {
+  return magic == 0 ? q : (uint32_t)__umul64hi((unsigned long long)q, magic);
+}
+
 template <int NT, int EPI, int SPT>
 __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g) {
   extern __shared__ __align__(1024) uint8_t smem[];
@@ -170,7 +179,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     mbar_init(smem_u32(&bars[3]), 128);
     mbar_init(smem_u32(&bars[4]), 128);
     mbar_init(smem_u32(&bars[5]), 128);
-    mbar_init(smem_u32(&bars[6]), 160);
+    mbar_init(smem_u32(&bars[6]), TC_THREADS);
     *s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -184,14 +193,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
-  if (warp < 4 || warp == 8) {
-    // One-time set-up by the 160 threads that are not producers, while the producers already expand the first tile:
-    // the resident weights (one contiguous block per channel tile) and the scale factors.
-    const int stid = warp == 8 ? 128 + lane : tid;
+  {
+    // Resident weights (one contiguous block per channel tile): every thread requests its share; the producers do not
+    // wait for theirs until their first tile's rows are out, so the copy overlaps the first expansion.
     const uint8_t* src = g.w_tc + (size_t)nt * NT * Kb;
     const int units = NT * Kb / 16;
-    for (int u = stid; u < units; u += 160) cp_async16(smem_u32(w_s + (size_t)u * 16), src + (size_t)u * 16);
+    for (int u = tid; u < units; u += TC_THREADS) cp_async16(smem_u32(w_s + (size_t)u * 16), src + (size_t)u * 16);
     asm volatile("cp.async.commit_group;" ::: "memory");
+  }
+  if (warp < 4 || warp == 8) {
     if (warp < 4) {
       // every byte of the scale-factor columns is ue8m0 127 = 1.0, whatever their layout
       const uint32_t one = 0x7F7F7F7Fu;
@@ -207,7 +217,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    mbar_arrive(smem_u32(&bars[6]));  // 160 arrivals: weights and scale factors are in place
+    mbar_arrive(smem_u32(&bars[6]));  // 288 arrivals in all: weights and scale factors are in place
   }
 
   if (warp == 8) {
@@ -271,60 +281,63 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   } else if (warp >= 4) {
     // ================= producer warps: packed bits -> e2m1 rows ===================================================
     const int ptid = tid - 128;
-    const int cgroups = g.C >> 5;
-    const uint32_t pad_word4 = g.pad_neg ? 0xAAAAAAAAu : 0x22222222u;
     constexpr int PCW = SPT > 2 ? 4 : TC_MAX_CW;  // words per slot held in registers (stride 2 is limited to C <= 256)
+    // Registers of one tile's rows.  A row that is padding carries the pad pattern as its words, a row beyond the batch
+    // carries zero words and live = 0, so that the expansion below is the same straight-line code for every row.
     struct SlotRegs {
       uint64_t words[SPT][PCW];
-      int kind[SPT];  // 0: inside the image (words valid), 1: padding, 2: beyond the batch, 3: no such slot
+      uint32_t live[SPT];  // ~0: expand the words; 0: the row is all zeros (beyond the batch)
     };
-    auto prefetch = [&](SlotRegs& R, long long mt) {
+    const uint64_t pad_bits = g.pad_neg ? ~0ull : 0ull;
+    auto prefetch = [&](SlotRegs& R, long long mt, auto cwc) {
+      constexpr int CW = decltype(cwc)::value;
 #pragma unroll
       for (int h = 0; h < SPT; h++) {
         const int s = ptid + 128 * h;
-        R.kind[h] = 3;
+        R.live[h] = 0;
+#pragma unroll
+        for (int cw = 0; cw < CW; cw++) R.words[h][cw] = 0;
         if (s < g.slots) {
           int plane = 0, sp = s;                        // parity plane of this row (always 0 for stride 1)
           while (sp >= g.slots_p) { sp -= g.slots_p; plane++; }
           const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)sp;  // total_q < 2^31 is checked on the host
-          const uint32_t rr = Q / (uint32_t)g.SP;
+          const uint32_t rr = fast_div(Q, g.magic_sp);
           const int cp = (int)(Q - rr * (uint32_t)g.SP);
-          const uint32_t n = rr / (uint32_t)g.HP;
+          const uint32_t n = fast_div(rr, g.magic_hp);
           const int rp = (int)(rr - n * (uint32_t)g.HP);
           const int sshift = g.S - 1;                   // stride 1 or 2
           const int ih = (rp << sshift) + (plane >> sshift) - g.ph, iw = (cp << sshift) + (plane & sshift) - g.pw;  // un-padded input coordinates
-          if (n >= (uint32_t)g.N) R.kind[h] = 2;
-          else if (ih < 0 || ih >= g.H || iw < 0 || iw >= g.W) R.kind[h] = 1;
-          else {
-            R.kind[h] = 0;
-            const uint64_t* src = g.a + (((long long)n * g.H + ih) * g.W + iw) * g.Cw;
+          if (n < (uint32_t)g.N) {
+            R.live[h] = ~0u;
+            if (ih < 0 || ih >= g.H || iw < 0 || iw >= g.W) {
 #pragma unroll
-            for (int cw = 0; cw < PCW; cw++)
-              if (cw < g.Cw) R.words[h][cw] = __ldg(src + cw);
+              for (int cw = 0; cw < CW; cw++) R.words[h][cw] = pad_bits;
+            } else {
+              const uint64_t* src = g.a + (((long long)n * g.H + ih) * g.W + iw) * g.Cw;
+#pragma unroll
+              for (int cw = 0; cw < CW; cw++)
+                if (cw < g.Cw) R.words[h][cw] = __ldg(src + cw);  // (CW is g.Cw rounded up to 1, 2, 4 or 8)
+            }
           }
         }
       }
     };
-    auto expand = [&](const SlotRegs& R, uint8_t* abuf) {
+    auto expand = [&](const SlotRegs& R, uint8_t* abuf, auto cwc) {
+      constexpr int CW = decltype(cwc)::value;
 #pragma unroll
       for (int h = 0; h < SPT; h++) {
-        if (R.kind[h] == 3) continue;
         const int s = ptid + 128 * h;
+        if (s >= g.slots) break;
+        uint8_t* dst = abuf + (size_t)s * 16;
+        const size_t gstride = (size_t)g.slots * 16;  // bytes between consecutive 32-channel groups
 #pragma unroll
-        for (int cw = 0; cw < PCW; cw++) {
-          if (cw >= g.Cw) break;
-#pragma unroll
-          for (int q2 = 0; q2 < 2; q2++) {  // a 64-bit word = two 32-channel rows
-            const int grp = cw * 2 + q2;
-            if (grp >= cgroups) break;
-            uint4 bytes;
-            if (R.kind[h] == 0) {
-              const uint32_t half = (uint32_t)(R.words[h][cw] >> (32 * q2));
-              bytes = expand32(half);
-            } else if (R.kind[h] == 2) bytes = make_uint4(0, 0, 0, 0);
-            else bytes = make_uint4(pad_word4, pad_word4, pad_word4, pad_word4);
-            *reinterpret_cast<uint4*>(abuf + ((size_t)grp * g.slots + s) * 16) = bytes;
-          }
+        for (int cw = 0; cw < CW; cw++) {
+          if (cw >= g.Cw) break;  // warp-uniform
+          uint4 lo = expand32((uint32_t)R.words[h][cw]), hi = expand32((uint32_t)(R.words[h][cw] >> 32));
+          lo.x &= R.live[h]; lo.y &= R.live[h]; lo.z &= R.live[h]; lo.w &= R.live[h];
+          hi.x &= R.live[h]; hi.y &= R.live[h]; hi.z &= R.live[h]; hi.w &= R.live[h];
+          *reinterpret_cast<uint4*>(dst + (size_t)(2 * cw) * gstride) = lo;
+          *reinterpret_cast<uint4*>(dst + (size_t)(2 * cw + 1) * gstride) = hi;
         }
       }
     };
@@ -334,33 +347,50 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     long long tlast = clock64();
 #endif
-    // One tile of producer work on register set R; the bits of the tile two steps ahead are requested right after,
-    // so that a whole tile period covers their latency.  Returns false when the loop must stop.
-    auto stage = [&](SlotRegs& R, long long mt) -> bool {
-      const int ab = it % g.abufs;
-      TC_T(0);
-      const int j = it - g.abufs;  // the tile whose MMAs last read this A buffer
-      if (j >= 0 && !mbar_wait(smem_u32(&bars[j & 1]), (uint32_t)(j >> 1) & 1)) { *s_fail = 1; return false; }
-      TC_T(1);
-      expand(R, a_s + (size_t)ab * a_bytes);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
-      mbar_arrive(smem_u32(&bars[4 + ab]));
-      TC_T(2);
-      if (mt + 2 * mt_step < g.m_tiles) prefetch(R, mt + 2 * mt_step);
-      it++;
-      return *s_fail == 0;
+    // Per tile: wait until the A buffer is free, expand the rows held in `cur`, hand them over, then request the bits of
+    // the tile two steps ahead into `cur` and swap the two register sets (one copy of the code for both sets).
+    auto run = [&](auto cwc) {  // the words per row (C / 64) as a compile-time constant
+      constexpr int CW = decltype(cwc)::value;
+      SlotRegs cur, nxt;
+      long long mt = mt_first;
+      if (mt < g.m_tiles) prefetch(cur, mt, cwc);
+#pragma unroll 1
+      for (; mt < g.m_tiles; mt += mt_step, it++) {
+        const int ab = it % g.abufs;
+        TC_T(0);
+        const int j = it - g.abufs;  // the tile whose MMAs last read this A buffer
+        if (j >= 0 && !mbar_wait(smem_u32(&bars[j & 1]), (uint32_t)(j >> 1) & 1)) { *s_fail = 1; break; }
+        TC_T(1);
+        expand(cur, a_s + (size_t)ab * a_bytes, cwc);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+        mbar_arrive(smem_u32(&bars[4 + ab]));
+        if (it == 0) {
+          // the first tile's rows went out before anything else: a short launch is all start-up.  Now this thread's
+          // share of the weights, and the second tile's bits.
+          asm volatile("cp.async.wait_group 0;" ::: "memory");
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          mbar_arrive(smem_u32(&bars[6]));
+          if (mt + mt_step < g.m_tiles) prefetch(nxt, mt + mt_step, cwc);
+        }
+        TC_T(2);
+        if (mt + 2 * mt_step < g.m_tiles) prefetch(cur, mt + 2 * mt_step, cwc);
+        // swap the register sets: `cur` now holds the next tile
+#pragma unroll
+        for (int h = 0; h < SPT; h++) {
+          const uint32_t tl = cur.live[h]; cur.live[h] = nxt.live[h]; nxt.live[h] = tl;
+#pragma unroll
+          for (int cw = 0; cw < CW; cw++) {
+            const uint64_t tw = cur.words[h][cw]; cur.words[h][cw] = nxt.words[h][cw]; nxt.words[h][cw] = tw;
+          }
+        }
+        if (*s_fail != 0) break;
+      }
     };
-    SlotRegs ra, rb;
-    long long mt = mt_first;
-    if (mt < g.m_tiles) prefetch(ra, mt);
-    if (mt + mt_step < g.m_tiles) prefetch(rb, mt + mt_step);
-    while (mt < g.m_tiles) {
-      if (!stage(ra, mt)) break;
-      mt += mt_step;
-      if (mt >= g.m_tiles) break;
-      if (!stage(rb, mt)) break;
-      mt += mt_step;
-    }
+    // C is a multiple of 64 up to 512: 1..8 words; the common counts get their own straight-line code
+    if (g.Cw == 1) run(IntC<1>{});
+    else if (g.Cw == 2) run(IntC<2>{});
+    else if (g.Cw <= 4) run(IntC<4>{});
+    else if constexpr (PCW > 4) run(IntC<8>{});
 #ifdef TC_TIMING
     if (ptid == 0 && blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[i] = prof[i]; g_tc_prof[15] = it; }
 #endif
@@ -375,9 +405,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       const int buf = it & 1;
       const int row = 32 * warp + lane;  // TMEM lane = slot row of the tile
       const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)row;
-      const uint32_t rr = Q / (uint32_t)g.SP;
+      const uint32_t rr = fast_div(Q, g.magic_sp);
       const int col = (int)(Q - rr * (uint32_t)g.SP);
-      const uint32_t n = rr / (uint32_t)g.HP;
+      const uint32_t n = fast_div(rr, g.magic_hp);
       const int r = (int)(rr - n * (uint32_t)g.HP);
       const int my_valid = (n < (uint32_t)g.N && r < g.OH && col < g.OW) ? 1 : 0;
       const int my_m = (int)((n * (uint32_t)g.OH + (uint32_t)r) * (uint32_t)g.OW + (uint32_t)col);  // < 2^31 (host check)
@@ -611,6 +641,9 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   g.SPin = in.W + 2 * cv.pad_w; g.HPin = in.H + 2 * cv.pad_h;
   g.SP = (g.SPin + g.S - 1) / g.S; g.HP = (g.HPin + g.S - 1) / g.S;
   g.total_q = (long long)in.N * g.HP * g.SP;
+  if (g.SP >= 65536 || g.HP >= 65536) return DABNN_ERR_UNSUPPORTED;
+  g.magic_sp = g.SP == 1 ? 0ull : ~0ull / (unsigned long long)g.SP + 1ull;
+  g.magic_hp = g.HP == 1 ? 0ull : ~0ull / (unsigned long long)g.HP + 1ull;
   g.slots_p = (128 + ((cv.kh - 1) / g.S) * g.SP + (cv.kw - 1) / g.S + 7) / 8 * 8;
   g.slots = g.S * g.S * g.slots_p;
   if (g.slots > 128 * TC_MAX_SPT || g.Cw > TC_MAX_CW || g.total_q + 512 >= (1LL << 31))
