@@ -171,11 +171,14 @@ __global__ void __launch_bounds__(256, 2) stem_conv_bn_8x8(const float* __restri
   };
   const int chg = tid & 7, pg = tid >> 3;        // 8 channel groups x 32 pixel groups
   const int row = pg >> 1, ow0 = (pg & 1) * 8;   // 8 consecutive pixels of one tile row
+  // a thread's 8 channels are chg*4 .. +3 and 32 + chg*4 .. +3, so that the 8 lanes of a quarter-warp read 128 contiguous
+  // bytes of weights (no bank conflict) and write 128 contiguous bytes of output
   float sc[8], sf[8];
 #pragma unroll
   for (int j = 0; j < 8; j++) {
-    sc[j] = scale[chg * 8 + j];
-    sf[j] = shift[chg * 8 + j];
+    const int ch = (j < 4) ? chg * 4 + j : 32 + chg * 4 + (j - 4);
+    sc[j] = scale[ch];
+    sf[j] = shift[ch];
   }
   long long tile = blockIdx.x;
   int buf = 0;
@@ -203,11 +206,11 @@ __global__ void __launch_bounds__(256, 2) stem_conv_bn_8x8(const float* __restri
           xe[4 * q] = e4.x; xe[4 * q + 1] = e4.y; xe[4 * q + 2] = e4.z; xe[4 * q + 3] = e4.w;
           xo[4 * q] = o4.x; xo[4 * q + 1] = o4.y; xo[4 * q + 2] = o4.z; xo[4 * q + 3] = o4.w;
         }
-        const float* wk = w_s + ((c * 7 + ki) * 7) * 64 + chg * 8;
+        const float* wk = w_s + ((c * 7 + ki) * 7) * 64 + chg * 4;
 #pragma unroll
         for (int kj = 0; kj < 7; kj++) {
           const float4 wa = *reinterpret_cast<const float4*>(wk + kj * 64);
-          const float4 wb = *reinterpret_cast<const float4*>(wk + kj * 64 + 4);
+          const float4 wb = *reinterpret_cast<const float4*>(wk + kj * 64 + 32);
           const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
           for (int i = 0; i < 8; i++) {
@@ -222,10 +225,10 @@ __global__ void __launch_bounds__(256, 2) stem_conv_bn_8x8(const float* __restri
     const int oh = (rem / TILES) * TS + row, owb = (rem % TILES) * TS + ow0;
 #pragma unroll
     for (int i = 0; i < 8; i++) {
-      float* dst = out + (((size_t)n * OHW + oh) * OHW + owb + i) * 64 + chg * 8;
+      float* dst = out + (((size_t)n * OHW + oh) * OHW + owb + i) * 64 + chg * 4;
       *reinterpret_cast<float4*>(dst) = make_float4(__fmaf_rn(acc[i][0], sc[0], sf[0]), __fmaf_rn(acc[i][1], sc[1], sf[1]),
                                                     __fmaf_rn(acc[i][2], sc[2], sf[2]), __fmaf_rn(acc[i][3], sc[3], sf[3]));
-      *reinterpret_cast<float4*>(dst + 4) = make_float4(__fmaf_rn(acc[i][4], sc[4], sf[4]), __fmaf_rn(acc[i][5], sc[5], sf[5]),
+      *reinterpret_cast<float4*>(dst + 32) = make_float4(__fmaf_rn(acc[i][4], sc[4], sf[4]), __fmaf_rn(acc[i][5], sc[5], sf[5]),
                                                         __fmaf_rn(acc[i][6], sc[6], sf[6]), __fmaf_rn(acc[i][7], sc[7], sf[7]));
     }
   }
