@@ -15,8 +15,10 @@
 //     value -- and every filter tap (i, j) is the SAME array read from a start address shifted by (i*SP + j) rows:
 //     with a 16-byte row pitch a shift by one slot is a 16-byte step of the matrix descriptor, so no im2col copy
 //     is ever materialised.  Rows that fall on padding columns / rows compute garbage that is never stored.
-//   * Warp-specialised and mbarrier-driven: four producer warps prefetch the next tile's bits, expand them through a
-//     256-entry table (8 bits -> 8 nibbles) into one of up to two A buffers and arrive on `a_full`; one thread of a
+//   * Stride 2 keeps four parity planes of the padded input; tap (i, j) reads plane (i mod 2, j mod 2) shifted by
+//     (i div 2, j div 2).
+//   * Warp-specialised and mbarrier-driven: four producer warps prefetch the bits two tiles ahead, expand them
+//     (table-free, see expand16) into one of up to two A buffers and arrive on `a_full`; one thread of a
 //     ninth warp waits for it, issues kh*kw*(C/64) tcgen05.mma (M = 128, N = NT, K = 64) into one of two TMEM
 //     accumulators and commits to `mma_done`; four epilogue warps wait for that, read the accumulator with
 //     tcgen05.ld, write the output form, and hand the accumulator back through `tmem_free`.
