@@ -224,57 +224,100 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 
   if (warp == 8) {
     // ================= MMA issue: one thread ======================================================================
+    // The chain below is all there is between two MMAs of this CTA, so it is kept to 32-bit adds: only the start-address
+    // field (low 14 bits of a descriptor's low word) changes from one MMA to the next, and shared-memory addresses in
+    // 16-byte units never carry out of it.
     if (lane == 0) {
       const uint32_t idesc = (1u << 7) | (1u << 10)          // A, B: e2m1
                              | ((uint32_t)(NT >> 3) << 17)   // N
                              | (1u << 23)                    // scale factors: ue8m0
                              | ((uint32_t)(128 >> 4) << 24); // M = 128; both operands K-major; K = 64
       const uint32_t tsfa = tmem_base + TC_SF_COL, tsfb = tmem_base + TC_SF_COL + 128;
-      const int cgroups = g.C >> 5;  // 32-channel groups (16-byte rows)
       const uint64_t bdesc0 = make_desc(smem_u32(w_s), (uint32_t)NT * 16, 128);
-      const uint64_t a_step = (uint64_t)(2u * (uint32_t)g.slots), b_step = (uint64_t)(2u * NT);  // one K = 64 block
-      const int kblocks = g.C >> 6;
-      const int sshift = g.S - 1, smask = g.S - 1;  // stride 1 or 2: masks and shifts instead of divisions
+      const uint32_t desc_hi = (uint32_t)(bdesc0 >> 32);  // same for A and B: core matrices 128 bytes apart along M / N
+      const uint32_t b_lo0 = (uint32_t)bdesc0;
+      uint32_t a_lo_buf[2];
+      a_lo_buf[0] = (uint32_t)make_desc(smem_u32(a_s), (uint32_t)g.slots * 16, 128);
+      a_lo_buf[1] = (uint32_t)make_desc(smem_u32(a_s + a_bytes), (uint32_t)g.slots * 16, 128);
+      const uint32_t a_step = 2u * (uint32_t)g.slots;  // one K = 64 block of A, in 16-byte units
+      constexpr uint32_t b_step = 2u * NT;             // weights are laid out in issue order: [tap][C/32][NT][16]
+      const int sshift = g.S - 1, smask = g.S - 1;     // stride 1 or 2: masks and shifts instead of divisions
+      // tap (ti, tj) reads parity plane (ti % S, tj % S) from a start shifted by (ti / S) slot rows and (tj / S) slots
+      auto tap_offset = [&](int ti, int tj) {
+        const uint32_t plane = (uint32_t)(((ti & smask) << sshift) + (tj & smask));
+        return plane * (uint32_t)g.slots_p + (uint32_t)((ti >> sshift) * g.SP + (tj >> sshift));
+      };
+      auto mma = [&](uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t accumulate) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %4, [%6], [%7], p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+            : "memory");
+      };
+      const bool k3 = g.kh == 3 && g.kw == 3;
+      uint32_t off9[9];
+#pragma unroll
+      for (int t = 0; t < 9; t++) off9[t] = k3 ? tap_offset(t / 3, t % 3) : 0u;
 #ifdef TC_TIMING
       long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
       long long tlast = clock64();
 #endif
+      // all MMAs of one tile; KB = C / 64 as a compile-time constant, the 3x3 filter fully unrolled
+      auto issue_tile = [&](uint32_t d_tmem, uint32_t a_lo0, auto kbc) {
+        constexpr int KB = decltype(kbc)::value;
+        if (k3) {
+#pragma unroll
+          for (int t = 0; t < 9; t++) {
+            const uint32_t a_lo = a_lo0 + off9[t];
+#pragma unroll
+            for (int kb = 0; kb < KB; kb++)
+              mma(d_tmem, a_lo + (uint32_t)kb * a_step, b_lo0 + (uint32_t)(t * KB + kb) * b_step, (t | kb) ? 1u : 0u);
+          }
+        } else {
+          uint32_t b_lo = b_lo0, accumulate = 0;
+          for (int ti = 0; ti < g.kh; ti++)
+            for (int tj = 0; tj < g.kw; tj++) {
+              const uint32_t a_lo = a_lo0 + tap_offset(ti, tj);
+#pragma unroll
+              for (int kb = 0; kb < KB; kb++, b_lo += b_step) {
+                mma(d_tmem, a_lo + (uint32_t)kb * a_step, b_lo, accumulate);
+                accumulate = 1;
+              }
+            }
+        }
+      };
       int it = 0;
+      uint32_t ab = 0, a_phase = 0;  // A buffer of this tile and the parity of its `a_full` phase
       if (!mbar_wait(smem_u32(&bars[6]), 0)) *s_fail = 1;  // resident weights and scale factors
+#pragma unroll 1
       for (long long mt = mt_first; mt < g.m_tiles && *s_fail == 0; mt += mt_step, it++) {
-        const int ab = it % g.abufs;
         TC_T(0);
-        if (!mbar_wait(smem_u32(&bars[4 + ab]), (uint32_t)(it / g.abufs) & 1)) { *s_fail = 1; break; }      // rows written
+        if (!mbar_wait(smem_u32(&bars[4 + ab]), a_phase)) { *s_fail = 1; break; }      // rows written
         TC_T(1);
         if (it >= 2 && !mbar_wait(smem_u32(&bars[2 + (it & 1)]), ((it - 2) >> 1) & 1)) { *s_fail = 1; break; }  // accumulator drained
         TC_T(2);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + (uint32_t)((it & 1) * NT);
-        const uint64_t adesc0 = make_desc(smem_u32(a_s + (size_t)ab * a_bytes), (uint32_t)g.slots * 16, 128);
-        uint32_t accumulate = 0;
-        uint64_t bdesc = bdesc0;  // weights are laid out in issue order: [tap][C/32][NT][16]
-        for (int ti = 0; ti < g.kh; ti++) {
-          for (int tj = 0; tj < g.kw; tj++) {
-            // tap (ti, tj) reads parity plane (ti % S, tj % S) from a start shifted by (ti / S) slot rows and (tj / S) slots;
-            // start addresses are in 16-byte units (S is 1 or 2: masks and shifts, no divisions in this single-thread chain)
-            const uint32_t plane = (uint32_t)(((ti & smask) << sshift) + (tj & smask));
-            uint64_t adesc = adesc0 + (uint64_t)(plane * (uint32_t)g.slots_p + (uint32_t)((ti >> sshift) * g.SP + (tj >> sshift)));
-#pragma unroll 4
-            for (int kb = 0; kb < kblocks; kb++, adesc += a_step, bdesc += b_step) {
-              asm volatile(
-                  "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                  "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
-                  : "memory");
-              accumulate = 1;
+        const uint32_t a_lo0 = ab ? a_lo_buf[1] : a_lo_buf[0];
+        if (g.Cw == 1) issue_tile(d_tmem, a_lo0, IntC<1>{});
+        else if (g.Cw == 2) issue_tile(d_tmem, a_lo0, IntC<2>{});
+        else if (g.Cw == 4) issue_tile(d_tmem, a_lo0, IntC<4>{});
+        else if (g.Cw == 8) issue_tile(d_tmem, a_lo0, IntC<8>{});
+        else {
+          for (int ti = 0; ti < g.kh; ti++)
+            for (int tj = 0; tj < g.kw; tj++) {
+              const uint32_t a_lo = a_lo0 + tap_offset(ti, tj);
+              for (int kb = 0; kb < g.Cw; kb++)
+                mma(d_tmem, a_lo + (uint32_t)kb * a_step, b_lo0 + (uint32_t)((ti * g.kw + tj) * g.Cw + kb) * b_step,
+                    (ti | tj | kb) ? 1u : 0u);
             }
-          }
         }
-        (void)cgroups;
         asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
                          smem_u32(&bars[it & 1]))
                      : "memory");
         TC_T(3);
+        if (g.abufs == 2) { a_phase ^= ab; ab ^= 1u; } else { a_phase ^= 1u; }
       }
 #ifdef TC_TIMING
       if (blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[16 + i] = prof[i]; }
@@ -358,7 +401,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       if (mt < g.m_tiles) prefetch(cur, mt, cwc);
 #pragma unroll 1
       for (; mt < g.m_tiles; mt += mt_step, it++) {
-        const int ab = it % g.abufs;
+        const int ab = g.abufs == 2 ? (it & 1) : 0;
         TC_T(0);
         const int j = it - g.abufs;  // the tile whose MMAs last read this A buffer
         if (j >= 0 && !mbar_wait(smem_u32(&bars[j & 1]), (uint32_t)(j >> 1) & 1)) { *s_fail = 1; break; }
