@@ -142,6 +142,12 @@ __device__ __forceinline__ void ld_global_v8(const void* p, float (&r)[8]) {
                : "l"(p));
 }
 
+// The fp32 accumulator holds an exact integer of magnitude <= K < 2^22: adding 1.5 * 2^23 leaves it in the low mantissa
+// bits (two full-rate instructions instead of a conversion).
+__device__ __forceinline__ uint32_t acc_to_int(uint32_t acc_bits) {
+  return __float_as_uint(__fadd_rn(__uint_as_float(acc_bits), 12582912.0f)) - 0x4B400000u;
+}
+
 template <int V>
 struct IntC { static constexpr int value = V; };
 
@@ -327,43 +333,53 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     // ================= producer warps: packed bits -> e2m1 rows ===================================================
     const int ptid = tid - 128;
     constexpr int PCW = SPT > 2 ? 4 : TC_MAX_CW;  // words per slot held in registers (stride 2 is limited to C <= 256)
-    // Registers of one tile's rows.  A row that is padding carries the pad pattern as its words, a row beyond the batch
-    // carries zero words and live = 0, so that the expansion below is the same straight-line code for every row.
+    // Registers of one tile's rows.  A row that is padding -- or lies beyond the batch, where no stored output reads
+    // it -- carries the pad pattern as its words, so that the expansion is the same straight-line code for every row.
     struct SlotRegs {
       uint64_t words[SPT][PCW];
-      uint32_t live[SPT];  // ~0: expand the words; 0: the row is all zeros (beyond the batch)
     };
     const uint64_t pad_bits = g.pad_neg ? ~0ull : 0ull;
-    auto prefetch = [&](SlotRegs& R, long long mt, auto cwc) {
+    // Slot coordinates (image, slot row, slot column) of this thread's rows in the next tile to request.  Tiles are
+    // requested in order, each `mt_step` tiles = a fixed (dn, dr, dc) after the one before: divisions happen once here.
+    int co_n[SPT], co_r[SPT], co_c[SPT], co_plane[SPT];
+    const uint32_t D = (uint32_t)mt_step * 128u;
+    const uint32_t d_rows = fast_div(D, g.magic_sp);
+    const int dc = (int)(D - d_rows * (uint32_t)g.SP);
+    const int dn = (int)fast_div(d_rows, g.magic_hp);
+    const int dr = (int)(d_rows - (uint32_t)dn * (uint32_t)g.HP);
+#pragma unroll
+    for (int h = 0; h < SPT; h++) {
+      int plane = 0, sp = ptid + 128 * h;  // parity plane of this row (always 0 for stride 1)
+      while (sp >= g.slots_p && plane < 3) { sp -= g.slots_p; plane++; }
+      const uint32_t Q = (uint32_t)mt_first * 128u + (uint32_t)sp;  // total_q < 2^31 is checked on the host
+      const uint32_t rr = fast_div(Q, g.magic_sp);
+      const uint32_t n = fast_div(rr, g.magic_hp);
+      co_c[h] = (int)(Q - rr * (uint32_t)g.SP);
+      co_r[h] = (int)(rr - n * (uint32_t)g.HP);
+      co_n[h] = (int)n;
+      co_plane[h] = plane;
+    }
+    auto prefetch = [&](SlotRegs& R, auto cwc) {
       constexpr int CW = decltype(cwc)::value;
+      const int sshift = g.S - 1;  // stride 1 or 2
 #pragma unroll
       for (int h = 0; h < SPT; h++) {
-        const int s = ptid + 128 * h;
-        R.live[h] = 0;
 #pragma unroll
-        for (int cw = 0; cw < CW; cw++) R.words[h][cw] = 0;
-        if (s < g.slots) {
-          int plane = 0, sp = s;                        // parity plane of this row (always 0 for stride 1)
-          while (sp >= g.slots_p) { sp -= g.slots_p; plane++; }
-          const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)sp;  // total_q < 2^31 is checked on the host
-          const uint32_t rr = fast_div(Q, g.magic_sp);
-          const int cp = (int)(Q - rr * (uint32_t)g.SP);
-          const uint32_t n = fast_div(rr, g.magic_hp);
-          const int rp = (int)(rr - n * (uint32_t)g.HP);
-          const int sshift = g.S - 1;                   // stride 1 or 2
-          const int ih = (rp << sshift) + (plane >> sshift) - g.ph, iw = (cp << sshift) + (plane & sshift) - g.pw;  // un-padded input coordinates
-          if (n < (uint32_t)g.N) {
-            R.live[h] = ~0u;
-            if (ih < 0 || ih >= g.H || iw < 0 || iw >= g.W) {
+        for (int cw = 0; cw < CW; cw++) R.words[h][cw] = pad_bits;
+        if (ptid + 128 * h < g.slots) {
+          const int ih = (co_r[h] << sshift) + (co_plane[h] >> sshift) - g.ph;  // un-padded input coordinates
+          const int iw = (co_c[h] << sshift) + (co_plane[h] & sshift) - g.pw;
+          if (co_n[h] < g.N && ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) {
+            const uint64_t* src = g.a + (((long long)co_n[h] * g.H + ih) * g.W + iw) * g.Cw;
 #pragma unroll
-              for (int cw = 0; cw < CW; cw++) R.words[h][cw] = pad_bits;
-            } else {
-              const uint64_t* src = g.a + (((long long)n * g.H + ih) * g.W + iw) * g.Cw;
-#pragma unroll
-              for (int cw = 0; cw < CW; cw++)
-                if (cw < g.Cw) R.words[h][cw] = __ldg(src + cw);  // (CW is g.Cw rounded up to 1, 2, 4 or 8)
-            }
+            for (int cw = 0; cw < CW; cw++)
+              if (cw < g.Cw) R.words[h][cw] = __ldg(src + cw);  // (CW is g.Cw rounded up to 1, 2, 4 or 8)
           }
+          co_c[h] += dc;
+          if (co_c[h] >= g.SP) { co_c[h] -= g.SP; co_r[h]++; }
+          co_r[h] += dr;
+          if (co_r[h] >= g.HP) { co_r[h] -= g.HP; co_n[h]++; }
+          co_n[h] += dn;
         }
       }
     };
@@ -378,9 +394,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #pragma unroll
         for (int cw = 0; cw < CW; cw++) {
           if (cw >= g.Cw) break;  // warp-uniform
-          uint4 lo = expand32((uint32_t)R.words[h][cw]), hi = expand32((uint32_t)(R.words[h][cw] >> 32));
-          lo.x &= R.live[h]; lo.y &= R.live[h]; lo.z &= R.live[h]; lo.w &= R.live[h];
-          hi.x &= R.live[h]; hi.y &= R.live[h]; hi.z &= R.live[h]; hi.w &= R.live[h];
+          const uint4 lo = expand32((uint32_t)R.words[h][cw]), hi = expand32((uint32_t)(R.words[h][cw] >> 32));
           *reinterpret_cast<uint4*>(dst + (size_t)(2 * cw) * gstride) = lo;
           *reinterpret_cast<uint4*>(dst + (size_t)(2 * cw + 1) * gstride) = hi;
         }
@@ -392,13 +406,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     long long tlast = clock64();
 #endif
-    // Per tile: wait until the A buffer is free, expand the rows held in `cur`, hand them over, then request the bits of
-    // the tile two steps ahead into `cur` and swap the two register sets (one copy of the code for both sets).
+    // Per tile: wait until the A buffer is free, expand the rows held in `cur`, hand them over, move the next tile's
+    // bits (requested one tile ago, so they have landed) from `nxt` into `cur`, and request the tile after that into
+    // `nxt`: registers that a load is still filling are never touched before the next iteration.
     auto run = [&](auto cwc) {  // the words per row (C / 64) as a compile-time constant
       constexpr int CW = decltype(cwc)::value;
       SlotRegs cur, nxt;
       long long mt = mt_first;
-      if (mt < g.m_tiles) prefetch(cur, mt, cwc);
+      prefetch(cur, cwc);  // (rows of a tile beyond the last one are beyond the batch: nothing is read for them)
+      prefetch(nxt, cwc);
 #pragma unroll 1
       for (; mt < g.m_tiles; mt += mt_step, it++) {
         const int ab = g.abufs == 2 ? (it & 1) : 0;
@@ -411,23 +427,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         mbar_arrive(smem_u32(&bars[4 + ab]));
         if (it == 0) {
           // the first tile's rows went out before anything else: a short launch is all start-up.  Now this thread's
-          // share of the weights, and the second tile's bits.
+          // share of the weights.
           asm volatile("cp.async.wait_group 0;" ::: "memory");
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           mbar_arrive(smem_u32(&bars[6]));
-          if (mt + mt_step < g.m_tiles) prefetch(nxt, mt + mt_step, cwc);
         }
         TC_T(2);
-        if (mt + 2 * mt_step < g.m_tiles) prefetch(cur, mt + 2 * mt_step, cwc);
-        // swap the register sets: `cur` now holds the next tile
 #pragma unroll
         for (int h = 0; h < SPT; h++) {
-          const uint32_t tl = cur.live[h]; cur.live[h] = nxt.live[h]; nxt.live[h] = tl;
 #pragma unroll
-          for (int cw = 0; cw < CW; cw++) {
-            const uint64_t tw = cur.words[h][cw]; cur.words[h][cw] = nxt.words[h][cw]; nxt.words[h][cw] = tw;
-          }
+          for (int cw = 0; cw < CW; cw++) cur.words[h][cw] = nxt.words[h][cw];
         }
+        prefetch(nxt, cwc);
         if (*s_fail != 0) break;
       }
     };
@@ -512,25 +523,25 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #pragma unroll
             for (int q = 0; q < 4; q++)
               if (8 * q < nch)  // nch is a multiple of 8 here
-                st_global_v8(dst + 8 * q, (uint32_t)__float2int_rn(__uint_as_float(v[8 * q])),
-                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 1])),
-                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 2])),
-                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 3])),
-                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 4])),
-                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 5])),
-                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 6])),
-                             (uint32_t)__float2int_rn(__uint_as_float(v[8 * q + 7])));
+                st_global_v8(dst + 8 * q, acc_to_int(v[8 * q]),
+                             acc_to_int(v[8 * q + 1]),
+                             acc_to_int(v[8 * q + 2]),
+                             acc_to_int(v[8 * q + 3]),
+                             acc_to_int(v[8 * q + 4]),
+                             acc_to_int(v[8 * q + 5]),
+                             acc_to_int(v[8 * q + 6]),
+                             acc_to_int(v[8 * q + 7]));
           } else if (!g.out_nchw) {
             int32_t* dst = g.out + m * g.O + o;
 #pragma unroll
             for (int j = 0; j < 32; j++)
-              if (j < nch) dst[j] = __float2int_rn(__uint_as_float(v[j]));
+              if (j < nch) dst[j] = acc_to_int(v[j]);
           } else {
             const long long ohw = (long long)g.OH * g.OW;
             const long long nn = m / ohw, q = m - nn * ohw;
 #pragma unroll
             for (int j = 0; j < 32; j++)
-              if (j < nch) g.out[(nn * g.O + o + j) * ohw + q] = __float2int_rn(__uint_as_float(v[j]));
+              if (j < nch) g.out[(nn * g.O + o + j) * ohw + q] = acc_to_int(v[j]);
           }
         } else {
           if (o >= g.Ow32 * 32) continue;  // sign words are written whole (tail bits 0), nothing beyond them
@@ -691,6 +702,7 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   g.magic_hp = g.HP == 1 ? 0ull : ~0ull / (unsigned long long)g.HP + 1ull;
   g.slots_p = (128 + ((cv.kh - 1) / g.S) * g.SP + (cv.kw - 1) / g.S + 7) / 8 * 8;
   g.slots = g.S * g.S * g.slots_p;
+  if ((long long)in.C * cv.kh * cv.kw >= (1LL << 22)) return DABNN_ERR_UNSUPPORTED;  // exact fp32 sums and acc_to_int
   if (g.slots > 128 * TC_MAX_SPT || g.Cw > TC_MAX_CW || g.total_q + 512 >= (1LL << 31))
     return DABNN_ERR_UNSUPPORTED;
   g.ntile = nt; g.n_ntiles = tc_n_ntiles(O, nt);
