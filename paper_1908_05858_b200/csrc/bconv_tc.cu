@@ -6,9 +6,15 @@
 // the block-scaled kind::mxf4 with every scale factor set to 1.0 (ue8m0 127).  Products are +-1 and the fp32
 // accumulator adds at most K < 2^24 of them, so the result is the exact integer.  HBM still holds one bit per value.
 //
-//   * Weights: expanded once (dabnn_tc_prepare_weights) to e2m1 in the UMMA K-major, no-swizzle core-matrix layout
-//     (rows of 16 bytes = 32 channels), one contiguous block per tile of NT output channels; a persistent CTA copies
-//     its block to shared memory once and keeps it for all its pixel tiles.
+//   * Weights: expanded once (dabnn_tc_prepare_weights) to e2m1 rows of 16 bytes = 32 channels, stored in blocks of 32
+//     output channels ([O/32][tap][C/32][32][16 B]); a persistent CTA copies the rows of its output channels into the
+//     UMMA K-major, no-swizzle core-matrix layout in shared memory once and keeps them for all its pixel tiles -- as
+//     many channel tiles as fit, so that a tile of activations is expanded once for all of them.
+//   * CTA pairs: where the launch is large enough, two CTAs of a cluster share every MMA (cta_group::2, M = 256: each
+//     CTA's 128 rows against N columns of which each CTA holds half).  Per MMA a CTA then reads half the weights from
+//     its shared memory -- the tensor pipe's operand reads are what saturates shared memory in the one-CTA form -- and
+//     the pair keeps twice the channels resident.  The leader CTA issues; producers and epilogue warps of the peer
+//     signal the leader's barriers through the cluster's shared-memory window.
 //   * Activations: a tile is 128 consecutive "slots" q of the padded image grid (slot pitch SP = W + 2*pad_w,
 //     H + 2*pad_h slot rows per image).  The CTA reads the packed bits of the 128 + (kh-1)*SP + (kw-1) slots it
 //     needs, expands them to e2m1 rows of 32 channels ([C/32][slots][16 B]) -- padded slots get the declared pad
@@ -20,8 +26,9 @@
 //   * Warp-specialised and mbarrier-driven: four producer warps prefetch the bits two tiles ahead, expand them
 //     (table-free, see expand16) into one of up to two A buffers and arrive on `a_full`; one thread of a
 //     ninth warp waits for it, issues kh*kw*(C/64) tcgen05.mma (M = 128, N = NT, K = 64) into one of two TMEM
-//     accumulators and commits to `mma_done`; four epilogue warps wait for that, read the accumulator with
-//     tcgen05.ld, write the output form, and hand the accumulator back through `tmem_free`.
+//     accumulators per resident channel tile and commits to `mma_done` (and, after the tile's last MMA, to `a_free`);
+//     four epilogue warps wait for that, read the accumulator with tcgen05.ld, write the output form, and hand the
+//     accumulator back through `tmem_free`.
 //
 // Every wait on an mbarrier is bounded: on expiry the kernel records an error flag, stops, frees its TMEM and returns.
 #include "common.cuh"
@@ -34,7 +41,8 @@ enum { EPI_I32 = 0, EPI_BNPACK = 1, EPI_BIREAL = 2 };
 
 constexpr int TC_THREADS = 288;           // 4 epilogue warps, 4 producer warps, 1 MMA-issue warp
 constexpr int TC_SMEM_LIMIT = 232448;     // 227 KB opt-in maximum per CTA
-constexpr int TC_SMEM_MISC = 2048;        // barriers, TMEM base, flags, this CTA's scale / shift
+constexpr int TC_MAX_RES = 4;              // channel tiles resident per CTA (pair) at most
+constexpr int TC_SMEM_MISC = 128 + 2 * TC_MAX_RES * 128 * 4;  // barriers, TMEM base, flags; this CTA's scale / shift
 constexpr int TC_WEIGHT_BUDGET = 147456;  // 144 KB of resident weights at most
 constexpr int TC_MAX_CW = 8;              // C <= 512
 constexpr int TC_MAX_SPT = 5;             // slots per producer thread: 2 for stride 1, up to 5 for stride 2
@@ -62,8 +70,10 @@ struct TcArgs {
   int slots_p;         // slots per parity plane and tile, multiple of 8
   int slots;           // S*S*slots_p: rows of one 32-channel group in an A buffer
   int abufs;           // A buffers in shared memory (1 or 2)
-  int ntile, n_ntiles; // output channels per tile, number of channel tiles
-  long long m_tiles;
+  int ntile, n_ntiles; // output channels per MMA (N), number of such channel tiles
+  int pair;            // 1: CTA pairs (cta_group::2), each CTA holds ntile / 2 weight rows per channel tile
+  int nres, n_groups;  // channel tiles resident per CTA (pair), groups of `nres` channel tiles
+  long long m_tiles;   // tiles of 128 slots (a pair takes two consecutive ones at a time)
   int pad_neg;
   int32_t* out;
   int out_nchw;
@@ -88,8 +98,9 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-// Bounded wait for the given phase parity; false if it ran out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait for the given phase parity; false if it ran out, or if another role of this CTA has given up (`fail`,
+// looked at only now and then: shared-memory reads are slow while the tensor pipe streams its operands).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* fail) {
   for (int tries = 0; tries < (1 << 20); tries++) {  // about a second at most, then give up
     uint32_t done;
     asm volatile(
@@ -100,8 +111,42 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         : "r"(bar), "r"(parity)
         : "memory");
     if (done) return true;
+    if ((tries & 1023) == 1023 && *fail != 0) return false;
   }
   return false;
+}
+// The same with cluster-scope acquire: the arrivals may come from the peer CTA.
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* fail) {
+  for (int tries = 0; tries < (1 << 20); tries++) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, 0x400;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if ((tries & 1023) == 1023 && *fail != 0) return false;
+  }
+  return false;
+}
+// Address of the leader CTA's copy of a shared-memory object, in the cluster's shared window; arrive on it.
+__device__ __forceinline__ uint32_t leader_addr(uint32_t local) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(r) : "r"(local));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 // 64-bit shared-memory matrix descriptor: K-major, no swizzle.  Core matrix = 8 rows x 16 bytes, rows 16 bytes
@@ -156,57 +201,95 @@ __device__ __forceinline__ uint32_t fast_div(uint32_t q, unsigned long long magi
   return magic == 0 ? q : (uint32_t)__umul64hi((unsigned long long)q, magic);
 }
 
-template <int NT, int EPI, int SPT>
+template <int NT, int EPI, int SPT, bool PAIR>
 __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g) {
   extern __shared__ __align__(1024) uint8_t smem[];
+  constexpr int WR = PAIR ? NT / 2 : NT;  // weight rows (output channels) of one channel tile held by this CTA
+  constexpr uint32_t PEERS = PAIR ? 2 : 1;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // 0: the CTA that issues the pair's MMAs
   const int Kb = g.kh * g.kw * (g.C >> 1);               // bytes per weight row
   const int a_bytes = g.slots * (g.C >> 1);              // bytes of one A buffer
-  uint8_t* w_s = smem;                                   // [taps][C/32][NT][16]
-  uint8_t* a_s = smem + (size_t)NT * Kb;                 // [abufs][C/32][slots][16]
+  uint8_t* w_s = smem;                                   // [nres][taps][C/32][WR][16]
+  uint8_t* a_s = smem + (size_t)g.nres * WR * Kb;        // [abufs][C/32][slots][16]
   uint8_t* misc = a_s + (size_t)g.abufs * a_bytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(misc);    // [0,1] mma_done  [2,3] tmem_free  [4,5] a_full  [6] w_full
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 64);
-  volatile int* s_fail = reinterpret_cast<volatile int*>(misc + 72);
-  float* s_scale = reinterpret_cast<float*>(misc + 128);     // [NT] this CTA's channels
-  float* s_shift = s_scale + NT;                             // [NT]
+  // [0,1] mma_done  [2,3] tmem_free  [4,5] a_full  [6] w_full  [7,8] a_free; of a pair, the leader's 2..6 are used
+  uint64_t* bars = reinterpret_cast<uint64_t*>(misc);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 96);
+  volatile int* s_fail = reinterpret_cast<volatile int*>(misc + 104);
+  float* s_scale = reinterpret_cast<float*>(misc + 128);     // [nres][NT] this CTA's channels
+  float* s_shift = s_scale + TC_MAX_RES * NT;                // [nres][NT]
 
-  const int nt = blockIdx.x % g.n_ntiles;
-  const long long mt_first = blockIdx.x / g.n_ntiles;
-  const long long mt_step = gridDim.x / g.n_ntiles;
+  // work: CTA (pair) `unit` takes channel-tile group `ng` and every `unit_step`-th tile (pair of tiles) of 128 slots
+  const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int ng = unit % g.n_groups;
+  const long long mt_first = (long long)(unit / g.n_groups) * PEERS + rank;
+  const long long mt_step = (long long)(units / g.n_groups) * PEERS;
+  const int nres_here = min(g.nres, g.n_ntiles - ng * g.nres);  // channel tiles of this group that exist
+  // a pair runs while its leader has a tile (the peer's last tile may lie beyond the end: pad rows, nothing stored)
+  const long long mt_end = PAIR ? (g.m_tiles + 1) / 2 * 2 : g.m_tiles;
 
-  if (EPI != EPI_I32 && tid < NT) {
-    const int o = nt * NT + tid;
-    s_scale[tid] = (o < g.O) ? g.scale[o] : 0.0f;
-    s_shift[tid] = (o < g.O) ? g.shift[o] : 0.0f;
+  if (EPI != EPI_I32) {
+    for (int i = tid; i < nres_here * NT; i += TC_THREADS) {
+      const int o = (ng * g.nres + i / NT) * NT + (i % NT);
+      s_scale[i] = (o < g.O) ? g.scale[o] : 0.0f;
+      s_shift[i] = (o < g.O) ? g.shift[o] : 0.0f;
+    }
   }
   if (tid == 0) {
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
-    mbar_init(smem_u32(&bars[2]), 128);
-    mbar_init(smem_u32(&bars[3]), 128);
-    mbar_init(smem_u32(&bars[4]), 128);
-    mbar_init(smem_u32(&bars[5]), 128);
-    mbar_init(smem_u32(&bars[6]), TC_THREADS);
+    mbar_init(smem_u32(&bars[2]), 128 * PEERS);
+    mbar_init(smem_u32(&bars[3]), 128 * PEERS);
+    mbar_init(smem_u32(&bars[4]), 128 * PEERS);
+    mbar_init(smem_u32(&bars[5]), 128 * PEERS);
+    mbar_init(smem_u32(&bars[6]), TC_THREADS * PEERS);
+    mbar_init(smem_u32(&bars[7]), 1);
+    mbar_init(smem_u32(&bars[8]), 1);
     *s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"((uint32_t)TC_TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"((uint32_t)TC_TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"((uint32_t)TC_TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  if (PAIR) cluster_sync_all();  // both CTAs' barriers exist before either signals the other's
+  else __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  // barriers that both CTAs of a pair signal live in the leader
+  const uint32_t bar_tmem_free0 = PAIR ? leader_addr(smem_u32(&bars[2])) : smem_u32(&bars[2]);
+  const uint32_t bar_a_full0 = PAIR ? leader_addr(smem_u32(&bars[4])) : smem_u32(&bars[4]);
+  const uint32_t bar_w_full = PAIR ? leader_addr(smem_u32(&bars[6])) : smem_u32(&bars[6]);
+  auto arrive = [&](uint32_t bar) {
+    if (PAIR) mbar_arrive_cluster(bar);
+    else mbar_arrive(bar);
+  };
   {
-    // Resident weights (one contiguous block per channel tile): every thread requests its share; the producers do not
-    // wait for theirs until their first tile's rows are out, so the copy overlaps the first expansion.
-    const uint8_t* src = g.w_tc + (size_t)nt * NT * Kb;
-    const int units = NT * Kb / 16;
-    for (int u = tid; u < units; u += TC_THREADS) cp_async16(smem_u32(w_s + (size_t)u * 16), src + (size_t)u * 16);
+    // Resident weights: rows [rank * WR, +WR) of every channel tile of this group, one (tile, tap, 32-channel group)
+    // block of WR rows per warp and step; the source holds blocks of 32 output channels.  The producers do not wait
+    // for their share until their first tile's rows are out, so the copy overlaps the first expansion.
+    const int TG = g.kh * g.kw * (g.C >> 5);
+    for (int tb = warp; tb < nres_here * TG; tb += TC_THREADS / 32) {
+      const int r = tb / TG, tg = tb - r * TG;
+      const int col0 = (ng * g.nres + r) * NT + (int)rank * WR;
+      uint8_t* dst = w_s + (size_t)tb * WR * 16;
+      for (int n = lane; n < WR; n += 32) {
+        const int col = col0 + n;
+        cp_async16(smem_u32(dst + n * 16), g.w_tc + (((size_t)(col >> 5) * TG + tg) * 32 + (col & 31)) * 16);
+      }
+    }
     asm volatile("cp.async.commit_group;" ::: "memory");
   }
   if (warp < 4 || warp == 8) {
@@ -225,28 +308,29 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    mbar_arrive(smem_u32(&bars[6]));  // 288 arrivals in all: weights and scale factors are in place
+    arrive(bar_w_full);  // 288 arrivals per CTA in all: weights and scale factors are in place
   }
 
   if (warp == 8) {
-    // ================= MMA issue: one thread ======================================================================
+    // ================= MMA issue: one thread (of the leader CTA) ==================================================
     // The chain below is all there is between two MMAs of this CTA, so it is kept to 32-bit adds: only the start-address
     // field (low 14 bits of a descriptor's low word) changes from one MMA to the next, and shared-memory addresses in
     // 16-byte units never carry out of it.
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       const uint32_t idesc = (1u << 7) | (1u << 10)          // A, B: e2m1
                              | ((uint32_t)(NT >> 3) << 17)   // N
                              | (1u << 23)                    // scale factors: ue8m0
-                             | ((uint32_t)(128 >> 4) << 24); // M = 128; both operands K-major; K = 64
+                             | ((uint32_t)((PAIR ? 256 : 128) >> 4) << 24);  // M; both operands K-major; K = 64
       const uint32_t tsfa = tmem_base + TC_SF_COL, tsfb = tmem_base + TC_SF_COL + 128;
-      const uint64_t bdesc0 = make_desc(smem_u32(w_s), (uint32_t)NT * 16, 128);
+      const uint64_t bdesc0 = make_desc(smem_u32(w_s), (uint32_t)WR * 16, 128);
       const uint32_t desc_hi = (uint32_t)(bdesc0 >> 32);  // same for A and B: core matrices 128 bytes apart along M / N
       const uint32_t b_lo0 = (uint32_t)bdesc0;
       uint32_t a_lo_buf[2];
       a_lo_buf[0] = (uint32_t)make_desc(smem_u32(a_s), (uint32_t)g.slots * 16, 128);
       a_lo_buf[1] = (uint32_t)make_desc(smem_u32(a_s + a_bytes), (uint32_t)g.slots * 16, 128);
       const uint32_t a_step = 2u * (uint32_t)g.slots;  // one K = 64 block of A, in 16-byte units
-      constexpr uint32_t b_step = 2u * NT;             // weights are laid out in issue order: [tap][C/32][NT][16]
+      constexpr uint32_t b_step = 2u * WR;             // weights are laid out in issue order: [tile][tap][C/32][WR][16]
+      const uint32_t b_tile = (uint32_t)(g.kh * g.kw * g.Cw) * b_step;  // one resident channel tile
       const int sshift = g.S - 1, smask = g.S - 1;     // stride 1 or 2: masks and shifts instead of divisions
       // tap (ti, tj) reads parity plane (ti % S, tj % S) from a start shifted by (ti / S) slot rows and (tj / S) slots
       auto tap_offset = [&](int ti, int tj) {
@@ -254,12 +338,33 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         return plane * (uint32_t)g.slots_p + (uint32_t)((ti >> sshift) * g.SP + (tj >> sshift));
       };
       auto mma = [&](uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t accumulate) {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %4, [%6], [%7], p;\n\t}"
-            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
-            : "memory");
+        if (PAIR) {
+          asm volatile(
+              "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+              "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+              "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.block32 [%0], da, db, %4, [%6], [%7], p;\n\t}"
+              ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+              : "memory");
+        } else {
+          asm volatile(
+              "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+              "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\tsetp.ne.b32 p, %5, 0;\n\t"
+              "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], da, db, %4, [%6], [%7], p;\n\t}"
+              ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(tsfa), "r"(tsfb)
+              : "memory");
+        }
+      };
+      // completion of everything issued so far -> one arrival on the barrier at this offset (in both CTAs of a pair)
+      auto commit = [&](uint32_t bar) {
+        if (PAIR)
+          asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                       "h"((uint16_t)3)
+                       : "memory");
+        else
+          asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+      };
+      auto wait = [&](uint32_t bar, uint32_t parity) {
+        return PAIR ? mbar_wait_cluster(bar, parity, s_fail) : mbar_wait(bar, parity, s_fail);
       };
       const bool k3 = g.kh == 3 && g.kw == 3;
       uint32_t off9[9];
@@ -269,8 +374,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
       long long tlast = clock64();
 #endif
-      // all MMAs of one tile; KB = C / 64 as a compile-time constant, the 3x3 filter fully unrolled
-      auto issue_tile = [&](uint32_t d_tmem, uint32_t a_lo0, auto kbc) {
+      // all MMAs of one tile and channel tile; KB = C / 64 as a compile-time constant, the 3x3 filter fully unrolled
+      auto issue_tile = [&](uint32_t d_tmem, uint32_t a_lo0, uint32_t b_base, uint32_t a_stp, auto kbc) {
         constexpr int KB = decltype(kbc)::value;
         if (k3) {
 #pragma unroll
@@ -278,50 +383,54 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
             const uint32_t a_lo = a_lo0 + off9[t];
 #pragma unroll
             for (int kb = 0; kb < KB; kb++)
-              mma(d_tmem, a_lo + (uint32_t)kb * a_step, b_lo0 + (uint32_t)(t * KB + kb) * b_step, (t | kb) ? 1u : 0u);
+              mma(d_tmem, a_lo + (uint32_t)kb * a_stp, b_base + (uint32_t)(t * KB + kb) * b_step, (t | kb) ? 1u : 0u);
           }
         } else {
-          uint32_t b_lo = b_lo0, accumulate = 0;
+          uint32_t b_lo = b_base, accumulate = 0;
           for (int ti = 0; ti < g.kh; ti++)
             for (int tj = 0; tj < g.kw; tj++) {
               const uint32_t a_lo = a_lo0 + tap_offset(ti, tj);
 #pragma unroll
               for (int kb = 0; kb < KB; kb++, b_lo += b_step) {
-                mma(d_tmem, a_lo + (uint32_t)kb * a_step, b_lo, accumulate);
+                mma(d_tmem, a_lo + (uint32_t)kb * a_stp, b_lo, accumulate);
                 accumulate = 1;
               }
             }
         }
       };
-      int it = 0;
       uint32_t ab = 0, a_phase = 0;  // A buffer of this tile and the parity of its `a_full` phase
-      if (!mbar_wait(smem_u32(&bars[6]), 0)) *s_fail = 1;  // resident weights and scale factors
+      int ar = 0;                    // accumulator rounds so far: one per (tile, resident channel tile)
+      bool ok = wait(smem_u32(&bars[6]), 0);  // resident weights and scale factors
+      if (!ok) *s_fail = 1;
 #pragma unroll 1
-      for (long long mt = mt_first; mt < g.m_tiles && *s_fail == 0; mt += mt_step, it++) {
+      for (long long mt = mt_first; mt < mt_end && ok; mt += mt_step) {
         TC_T(0);
-        if (!mbar_wait(smem_u32(&bars[4 + ab]), a_phase)) { *s_fail = 1; break; }      // rows written
+        if (!wait(smem_u32(&bars[4 + ab]), a_phase)) { *s_fail = 1; break; }  // rows written
         TC_T(1);
-        if (it >= 2 && !mbar_wait(smem_u32(&bars[2 + (it & 1)]), ((it - 2) >> 1) & 1)) { *s_fail = 1; break; }  // accumulator drained
-        TC_T(2);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t d_tmem = tmem_base + (uint32_t)((it & 1) * NT);
         const uint32_t a_lo0 = ab ? a_lo_buf[1] : a_lo_buf[0];
-        if (g.Cw == 1) issue_tile(d_tmem, a_lo0, IntC<1>{});
-        else if (g.Cw == 2) issue_tile(d_tmem, a_lo0, IntC<2>{});
-        else if (g.Cw == 4) issue_tile(d_tmem, a_lo0, IntC<4>{});
-        else if (g.Cw == 8) issue_tile(d_tmem, a_lo0, IntC<8>{});
-        else {
-          for (int ti = 0; ti < g.kh; ti++)
-            for (int tj = 0; tj < g.kw; tj++) {
-              const uint32_t a_lo = a_lo0 + tap_offset(ti, tj);
-              for (int kb = 0; kb < g.Cw; kb++)
-                mma(d_tmem, a_lo + (uint32_t)kb * a_step, b_lo0 + (uint32_t)((ti * g.kw + tj) * g.Cw + kb) * b_step,
-                    (ti | tj | kb) ? 1u : 0u);
-            }
+        // (opaque to the compiler, so that it does not keep every tap's and K block's offset in a register of its own
+        // across tiles: the sums are recomputed per tile, one add each)
+        uint32_t a_step_t = a_step;
+        asm volatile("" : "+r"(a_step_t));
+#pragma unroll 1
+        for (int r = 0; r < nres_here; r++, ar++) {
+          if (ar >= 2 && !wait(smem_u32(&bars[2 + (ar & 1)]), ((ar - 2) >> 1) & 1)) { *s_fail = 1; ok = false; break; }  // accumulator drained
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t d_tmem = tmem_base + (uint32_t)((ar & 1) * NT);
+          const uint32_t b_base = b_lo0 + (uint32_t)r * b_tile;
+          switch (g.Cw) {  // C / 64 = 1..8
+            case 1: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<1>{}); break;
+            case 2: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<2>{}); break;
+            case 3: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<3>{}); break;
+            case 4: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<4>{}); break;
+            case 5: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<5>{}); break;
+            case 6: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<6>{}); break;
+            case 7: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<7>{}); break;
+            default: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<8>{}); break;
+          }
+          commit(smem_u32(&bars[ar & 1]));
         }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
-                         smem_u32(&bars[it & 1]))
-                     : "memory");
+        commit(smem_u32(&bars[7 + ab]));  // the tile's rows have been read: the A buffer may be refilled
         TC_T(3);
         if (g.abufs == 2) { a_phase ^= ab; ab ^= 1u; } else { a_phase ^= 1u; }
       }
@@ -416,21 +525,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       prefetch(cur, cwc);  // (rows of a tile beyond the last one are beyond the batch: nothing is read for them)
       prefetch(nxt, cwc);
 #pragma unroll 1
-      for (; mt < g.m_tiles; mt += mt_step, it++) {
+      for (; mt < mt_end; mt += mt_step, it++) {
         const int ab = g.abufs == 2 ? (it & 1) : 0;
+        const int use = g.abufs == 2 ? (it >> 1) : it;  // how often this A buffer has been filled before
         TC_T(0);
-        const int j = it - g.abufs;  // the tile whose MMAs last read this A buffer
-        if (j >= 0 && !mbar_wait(smem_u32(&bars[j & 1]), (uint32_t)(j >> 1) & 1)) { *s_fail = 1; break; }
+        // its last reader: all MMAs of the tile that used it, signalled through `a_free` (in both CTAs of a pair)
+        if (use > 0 && !mbar_wait(smem_u32(&bars[7 + ab]), (uint32_t)(use - 1) & 1, s_fail)) { *s_fail = 1; break; }
         TC_T(1);
         expand(cur, a_s + (size_t)ab * a_bytes, cwc);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
-        mbar_arrive(smem_u32(&bars[4 + ab]));
+        arrive(bar_a_full0 + 8u * (uint32_t)ab);
         if (it == 0) {
           // the first tile's rows went out before anything else: a short launch is all start-up.  Now this thread's
           // share of the weights.
           asm volatile("cp.async.wait_group 0;" ::: "memory");
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          mbar_arrive(smem_u32(&bars[6]));
+          arrive(bar_w_full);
         }
         TC_T(2);
 #pragma unroll
@@ -439,7 +549,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
           for (int cw = 0; cw < CW; cw++) cur.words[h][cw] = nxt.words[h][cw];
         }
         prefetch(nxt, cwc);
-        if (*s_fail != 0) break;
       }
     };
     // C is a multiple of 64 up to 512: 1..8 words; the common counts get their own straight-line code
@@ -452,13 +561,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #endif
   } else {
     // ================= epilogue warps: TMEM accumulator -> output ===============================================
-    int it = 0;
+    int ar = 0;  // accumulator rounds so far: one per (tile, resident channel tile)
+    bool failed = false;
 #ifdef TC_TIMING
     long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     long long tlast = clock64();
 #endif
-    for (long long mt = mt_first; mt < g.m_tiles; mt += mt_step, it++) {
-      const int buf = it & 1;
+    for (long long mt = mt_first; mt < mt_end && !failed; mt += mt_step) {
       const int row = 32 * warp + lane;  // TMEM lane = slot row of the tile
       const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)row;
       const uint32_t rr = fast_div(Q, g.magic_sp);
@@ -471,6 +580,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       const bool wide_i32 = EPI == EPI_I32 && !g.out_nchw && (g.O & 7) == 0 && (reinterpret_cast<uintptr_t>(g.out) & 31) == 0;
       const bool wide_y = EPI == EPI_BIREAL && (g.O & 7) == 0 &&
                           ((reinterpret_cast<uintptr_t>(g.residual) | reinterpret_cast<uintptr_t>(g.y_out)) & 31) == 0;
+      for (int r = 0; r < nres_here; r++, ar++) {
+      const int buf = ar & 1;
+      const int nt = ng * g.nres + r;  // this round's channel tile
+      const float* r_scale = s_scale + r * NT;
+      const float* r_shift = s_shift + r * NT;
       // The residual does not depend on the MMAs: its first 32 channels are requested before waiting for them, and
       // every later chunk one chunk ahead of its use.
       float rpre[32];
@@ -486,8 +600,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       };
       load_res(0);
       TC_T(0);
-      if (!mbar_wait(smem_u32(&bars[buf]), (it >> 1) & 1)) {
+      if (!mbar_wait(smem_u32(&bars[buf]), (ar >> 1) & 1, s_fail)) {
         *s_fail = 1;
+        failed = true;
         break;
       }
       TC_T(1);
@@ -496,6 +611,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #pragma unroll 1
       for (int c0 = 0; c0 < NT; c0 += 32) {
         __syncwarp();  // the TMEM load is warp-wide: rejoin lanes that took different paths below
+        TC_T(4);
         float rc[32];
         if (EPI == EPI_BIREAL) {
 #pragma unroll
@@ -513,6 +629,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
               "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
             : "r"(taddr));
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        TC_T(3);
         const int o = nt * NT + c0;  // first of the 32 channels of this chunk; the lane owns them all for its row
         if (!my_valid) continue;
         const int nch = min(32, g.O - o);  // channels of this chunk that exist (<= 0: none)
@@ -548,8 +665,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
           float y[32];
 #pragma unroll
           for (int q = 0; q < 8; q++) {  // channels beyond O have scale = shift = 0: y = +0
-            const float4 sc = *reinterpret_cast<const float4*>(s_scale + c0 + 4 * q);
-            const float4 sh = *reinterpret_cast<const float4*>(s_shift + c0 + 4 * q);
+            const float4 sc = *reinterpret_cast<const float4*>(r_scale + c0 + 4 * q);
+            const float4 sh = *reinterpret_cast<const float4*>(r_shift + c0 + 4 * q);
             y[4 * q] = __fmaf_rn(__uint_as_float(v[4 * q]), sc.x, sh.x);
             y[4 * q + 1] = __fmaf_rn(__uint_as_float(v[4 * q + 1]), sc.y, sh.y);
             y[4 * q + 2] = __fmaf_rn(__uint_as_float(v[4 * q + 2]), sc.z, sh.z);
@@ -587,35 +704,41 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       }
       // this accumulator buffer may be overwritten by the tile after next
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(smem_u32(&bars[2 + buf]));
+      arrive(bar_tmem_free0 + 8u * (uint32_t)buf);
       TC_T(2);
+      }
     }
 #ifdef TC_TIMING
-    if (tid == 0 && blockIdx.x == 0) { for (int i = 0; i < 4; i++) g_tc_prof[8 + i] = prof[i]; }
+    if (tid == 0 && blockIdx.x == 0) { for (int i = 0; i < 6; i++) g_tc_prof[8 + i] = prof[i]; }
 #endif
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
+  if (PAIR) cluster_sync_all();  // neither CTA leaves, or frees tensor memory, while the other may still use it
+  else __syncthreads();
   if (*s_fail != 0 && tid == 0) atomicExch(&g_tc_error, 1);
   if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TC_TMEM_COLS)
-                 : "memory");
+    if (PAIR)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TC_TMEM_COLS)
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TC_TMEM_COLS)
+                   : "memory");
   }
 }
 
-// Weights: packed bits [O][taps][Cw] -> e2m1 [n_ntiles][taps][C/32][NT][16 bytes = 32 channels].
-__global__ void tc_prepare_weights_kernel(const uint64_t* __restrict__ wp, int O, int taps, int Cw, int cgroups, int NT,
+// Weights: packed bits [O][taps][Cw] -> e2m1 [blocks of 32 output channels][taps][C/32][32][16 bytes = 32 channels];
+// the blocks cover O rounded up to 128, rows beyond O are zero (e2m1 0.0: they contribute nothing).
+__global__ void tc_prepare_weights_kernel(const uint64_t* __restrict__ wp, int O, int taps, int Cw, int cgroups,
                                           long long units, uint4* __restrict__ out) {
   const long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (u >= units) return;
-  const int n = (int)(u % NT);
-  long long t = u / NT;
+  const int n = (int)(u & 31);
+  long long t = u >> 5;
   const int grp = (int)(t % cgroups);
   t /= cgroups;
   const int tap = (int)(t % taps);
-  const int nt = (int)(t / taps);
-  const int o = nt * NT + n;
-  uint4 bytes = make_uint4(0, 0, 0, 0);  // channels beyond O contribute nothing (e2m1 zero)
+  const int o = (int)(t / taps) * 32 + n;
+  uint4 bytes = make_uint4(0, 0, 0, 0);
   if (o < O) {
     const uint32_t half = (uint32_t)(wp[((long long)o * taps + tap) * Cw + (grp >> 1)] >> (32 * (grp & 1)));
     bytes = expand32(half);
@@ -623,11 +746,26 @@ __global__ void tc_prepare_weights_kernel(const uint64_t* __restrict__ wp, int O
   out[u] = bytes;
 }
 
-int tc_ntile(int O, int C, int taps) {
+// 0: choose by size; 1: one CTA per tile; 2: CTA pairs wherever they are possible (environment DABNN_TC_MODE, read once).
+int tc_mode() {
+  static const int mode = [] {
+    const char* e = getenv("DABNN_TC_MODE");
+    return e ? atoi(e) : 0;
+  }();
+  return mode;
+}
+
+bool tc_covers(int O, int C, int taps) {
+  return O > 0 && C > 0 && C % 64 == 0 && C <= 64 * TC_MAX_CW && 32LL * (C / 2) * taps <= TC_WEIGHT_BUDGET;
+}
+
+// Channels per MMA for a launch: the widest of 128 / 64 / 32 whose rows (half of them per CTA of a pair) fit the
+// resident budget, without padding a small O to a wide tile.
+int tc_ntile(int O, int C, int taps, bool pair) {
   const long long Kb = (long long)C / 2 * taps;  // bytes per weight row
-  for (int nt = 128; nt >= 32; nt >>= 1) {
-    if (nt * Kb > TC_WEIGHT_BUDGET) continue;
-    if (nt > 32 && nt / 2 >= O) continue;  // do not pad a small O to a wide tile
+  for (int nt = 128; nt >= (pair ? 64 : 32); nt >>= 1) {
+    if ((pair ? nt / 2 : nt) * Kb > TC_WEIGHT_BUDGET) continue;
+    if (nt > 32 && nt / 2 >= O) continue;
     return nt;
   }
   return 0;
@@ -636,45 +774,114 @@ int tc_ntile(int O, int C, int taps) {
 // Channel tiles cover O rounded up to whole 64-bit sign words (rows beyond O hold zero weights).
 int tc_n_ntiles(int O, int nt) { return ((O + 63) / 64 * 64 + nt - 1) / nt; }
 
-template <int NT, int EPI, int SPT>
+template <int NT, int EPI, int SPT, bool PAIR>
 dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
-  auto kern = bconv_tc_kernel<NT, EPI, SPT>;
+  auto kern = bconv_tc_kernel<NT, EPI, SPT, PAIR>;
   static bool configured = false;
+  static int max_units = 0;  // CTAs (pairs) that can be resident at once
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT) != cudaSuccess) {
       cudaGetLastError();
       return DABNN_ERR_CUDA;
     }
+    max_units = sm_count();
+    if (PAIR) {
+      cudaLaunchConfig_t probe = {};
+      probe.gridDim = dim3((unsigned)(sm_count() / 2 * 2));
+      probe.blockDim = dim3(TC_THREADS);
+      probe.dynamicSmemBytes = TC_SMEM_LIMIT;
+      cudaLaunchAttribute at;
+      at.id = cudaLaunchAttributeClusterDimension;
+      at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+      probe.attrs = &at; probe.numAttrs = 1;
+      int clusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&clusters, kern, &probe) != cudaSuccess || clusters <= 0) {
+        cudaGetLastError();
+        return DABNN_ERR_UNSUPPORTED;
+      }
+      max_units = clusters < sm_count() / 2 ? clusters : sm_count() / 2;
+    }
     configured = true;
   }
-  long long ctas = (long long)g.n_ntiles * g.m_tiles;
-  const long long cap = (long long)sm_count() / g.n_ntiles * g.n_ntiles;
+  const long long m_units = PAIR ? (g.m_tiles + 1) / 2 : g.m_tiles;
+  long long units = (long long)g.n_groups * m_units;
+  const long long cap = (long long)max_units / g.n_groups * g.n_groups;
   if (cap <= 0) return DABNN_ERR_UNSUPPORTED;
-  if (ctas > cap) ctas = cap;
-  kern<<<(unsigned)ctas, TC_THREADS, smem, st>>>(g);
+  if (units > cap) units = cap;
+  if (!PAIR) {
+    kern<<<(unsigned)units, TC_THREADS, smem, st>>>(g);
+    return launch_status();
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(2 * units));
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at;
+  at.id = cudaLaunchAttributeClusterDimension;
+  at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+  cfg.attrs = &at; cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, g) != cudaSuccess) {
+    cudaGetLastError();
+    return DABNN_ERR_CUDA;
+  }
   return launch_status();
 }
 
-template <int EPI>
-dabnn_status tc_dispatch(TcArgs& g, cudaStream_t st) {
-  const size_t wbytes = (size_t)g.ntile * g.kh * g.kw * (g.C / 2), abytes = (size_t)g.slots * (g.C / 2);
+template <int EPI, bool PAIR>
+dabnn_status tc_dispatch_mode(TcArgs& g, cudaStream_t st) {
+  const size_t wr = (size_t)g.ntile / (PAIR ? 2 : 1);
+  const size_t wbytes = (size_t)g.nres * wr * g.kh * g.kw * (g.C / 2), abytes = (size_t)g.slots * (g.C / 2);
   g.abufs = (wbytes + 2 * abytes + TC_SMEM_MISC <= (size_t)TC_SMEM_LIMIT) ? 2 : 1;
   const size_t smem = wbytes + g.abufs * abytes + TC_SMEM_MISC;
   if (smem > (size_t)TC_SMEM_LIMIT) return DABNN_ERR_UNSUPPORTED;
   if (g.slots <= 256) {
     switch (g.ntile) {
-      case 128: return tc_launch<128, EPI, 2>(g, smem, st);
-      case 64: return tc_launch<64, EPI, 2>(g, smem, st);
-      case 32: return tc_launch<32, EPI, 2>(g, smem, st);
+      case 128: return tc_launch<128, EPI, 2, PAIR>(g, smem, st);
+      case 64: return tc_launch<64, EPI, 2, PAIR>(g, smem, st);
+      case 32: if constexpr (!PAIR) return tc_launch<32, EPI, 2, false>(g, smem, st);
     }
   } else if (g.Cw <= 4) {
     switch (g.ntile) {
-      case 128: return tc_launch<128, EPI, TC_MAX_SPT>(g, smem, st);
-      case 64: return tc_launch<64, EPI, TC_MAX_SPT>(g, smem, st);
-      case 32: return tc_launch<32, EPI, TC_MAX_SPT>(g, smem, st);
+      case 128: return tc_launch<128, EPI, TC_MAX_SPT, PAIR>(g, smem, st);
+      case 64: return tc_launch<64, EPI, TC_MAX_SPT, PAIR>(g, smem, st);
+      case 32: if constexpr (!PAIR) return tc_launch<32, EPI, TC_MAX_SPT, false>(g, smem, st);
     }
   }
   return DABNN_ERR_UNSUPPORTED;
+}
+
+template <int EPI>
+dabnn_status tc_dispatch(TcArgs& g, cudaStream_t st) {
+  return g.pair ? tc_dispatch_mode<EPI, true>(g, st) : tc_dispatch_mode<EPI, false>(g, st);
+}
+
+// Launch form for a problem: CTA pairs when there are enough tiles to fill the chip with pairs, and as many channel
+// tiles resident per CTA (pair) as fit while every CTA (pair) still gets work.
+void tc_plan(TcArgs& g, int O, int C, int taps) {
+  const long long Kb = (long long)C / 2 * taps;
+  const int mode = tc_mode();
+  const int units1 = sm_count(), units2 = sm_count() / 2;
+  const int nt2 = tc_ntile(O, C, taps, true);
+  bool pair = nt2 != 0 && mode != 1;
+  if (pair && mode == 0) {
+    // Measured: pairs win where one CTA cannot keep a 128-channel tile resident (C = 512 at 3x3) and there are
+    // enough double tiles to go round; elsewhere the one-CTA form is as fast or faster.
+    const long long work = (g.m_tiles + 1) / 2 * tc_n_ntiles(O, nt2);
+    pair = nt2 > tc_ntile(O, C, taps, false) && work >= units2;
+  }
+  g.pair = pair ? 1 : 0;
+  g.ntile = pair ? nt2 : tc_ntile(O, C, taps, false);
+  if (g.ntile == 0) return;
+  g.n_ntiles = tc_n_ntiles(O, g.ntile);
+  const long long wr = pair ? g.ntile / 2 : g.ntile;
+  long long nres = TC_WEIGHT_BUDGET / (wr * Kb);
+  if (nres > TC_MAX_RES) nres = TC_MAX_RES;
+  if (nres > g.n_ntiles) nres = g.n_ntiles;
+  const long long m_units = pair ? (g.m_tiles + 1) / 2 : g.m_tiles;
+  while (nres > 1 && (g.n_ntiles + nres - 1) / nres * m_units < (pair ? units2 : units1)) nres--;
+  g.nres = (int)nres;
+  g.n_groups = (g.n_ntiles + g.nres - 1) / g.nres;
 }
 
 dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w_tc, int O, dabnn_conv cv) {
@@ -688,8 +895,7 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   if (OH <= 0 || OW <= 0) return DABNN_ERR_SHAPE;
   // what this engine covers; everything else is served by the xor/popcount kernel
   if (cv.stride_h != cv.stride_w || cv.stride_h > 2 || in.C % 64 != 0) return DABNN_ERR_UNSUPPORTED;
-  const int nt = tc_ntile(O, in.C, cv.kh * cv.kw);
-  if (nt == 0) return DABNN_ERR_UNSUPPORTED;
+  if (!tc_covers(O, in.C, cv.kh * cv.kw)) return DABNN_ERR_UNSUPPORTED;
   g.a = a; g.w_tc = static_cast<const uint8_t*>(w_tc);
   g.N = in.N; g.H = in.H; g.W = in.W; g.Cw = (in.C + 63) / 64; g.C = in.C;
   g.O = O; g.kh = cv.kh; g.kw = cv.kw; g.ph = cv.pad_h; g.pw = cv.pad_w; g.OH = OH; g.OW = OW;
@@ -705,8 +911,9 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   if ((long long)in.C * cv.kh * cv.kw >= (1LL << 22)) return DABNN_ERR_UNSUPPORTED;  // exact fp32 sums and acc_to_int
   if (g.slots > 128 * TC_MAX_SPT || g.Cw > TC_MAX_CW || g.total_q + 512 >= (1LL << 31))
     return DABNN_ERR_UNSUPPORTED;
-  g.ntile = nt; g.n_ntiles = tc_n_ntiles(O, nt);
   g.m_tiles = (g.total_q + 127) / 128;
+  tc_plan(g, O, in.C, cv.kh * cv.kw);
+  if (g.ntile == 0) return DABNN_ERR_UNSUPPORTED;
   if ((long long)in.N * OH * OW >= (1LL << 31) || (long long)in.N * OH * OW * O > (1LL << 40)) return DABNN_ERR_UNSUPPORTED;
   g.pad_neg = cv.pad_value < 0;
   g.out = nullptr; g.out_nchw = 0; g.scale = g.shift = g.residual = nullptr; g.y_out = nullptr;
@@ -717,8 +924,8 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
 }  // namespace
 
 bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv) {
-  if (cv.stride_h != cv.stride_w || cv.stride_h > 2 || in.C % 64 != 0 || in.C > 64 * TC_MAX_CW) return false;
-  const int nt = tc_ntile(O, in.C, cv.kh * cv.kw);
+  if (cv.stride_h != cv.stride_w || cv.stride_h > 2 || !tc_covers(O, in.C, cv.kh * cv.kw)) return false;
+  const int nt = tc_ntile(O, in.C, cv.kh * cv.kw, false);
   if (nt == 0) return false;
   const int S = cv.stride_h;
   const long long slots_total = (long long)in.N * ((in.H + 2 * cv.pad_h + S - 1) / S) * ((in.W + 2 * cv.pad_w + S - 1) / S);
@@ -730,24 +937,20 @@ bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv) {
 using namespace dabnn;
 
 extern "C" size_t dabnn_tc_weights_bytes(int O, int C, int kh, int kw) {
-  if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0 || C % 64 != 0) return 0;
-  const int nt = tc_ntile(O, C, kh * kw);
-  if (nt == 0) return 0;
-  return (size_t)tc_n_ntiles(O, nt) * nt * kh * kw * (C / 2);
+  if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0 || !tc_covers(O, C, kh * kw)) return 0;
+  return (size_t)((O + 127) / 128 * 128) * kh * kw * (C / 2);
 }
 
 extern "C" dabnn_status dabnn_tc_prepare_weights(const uint64_t* w_packed, int O, int C, int kh, int kw, void* w_tc,
                                                  void* stream) {
   if (!w_packed || !w_tc) return DABNN_ERR_NULL;
   if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0) return DABNN_ERR_SHAPE;
-  if (C % 64 != 0) return DABNN_ERR_UNSUPPORTED;
+  if (!tc_covers(O, C, kh * kw)) return DABNN_ERR_UNSUPPORTED;
   if (!aligned(w_packed, 8) || !aligned(w_tc, 16)) return DABNN_ERR_ALIGNMENT;
-  const int nt = tc_ntile(O, C, kh * kw);
-  if (nt == 0) return DABNN_ERR_UNSUPPORTED;
-  const int taps = kh * kw, cgroups = C / 32, n_nt = tc_n_ntiles(O, nt);
-  const long long units = (long long)n_nt * taps * cgroups * nt;
+  const int taps = kh * kw, cgroups = C / 32;
+  const long long units = (long long)((O + 127) / 128 * 128) * taps * cgroups;
   tc_prepare_weights_kernel<<<ceil_div(units, 256), 256, 0, as_stream(stream)>>>(w_packed, O, taps, (C + 63) / 64, cgroups,
-                                                                                 nt, units, static_cast<uint4*>(w_tc));
+                                                                                 units, static_cast<uint4*>(w_tc));
   return launch_status();
 }
 

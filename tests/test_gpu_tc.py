@@ -44,6 +44,12 @@ TC_CASES = [
     (2, 64, 13, 11, 70, 3, 1, -1, 2),   # odd sizes, stride 2
     (2, 128, 12, 12, 64, 1, 0, -1, 2),  # 1x1 stride 2
     (2, 64, 16, 16, 64, 5, 2, -1, 2),   # 5x5 stride 2
+    (2, 448, 10, 10, 70, 3, 1, -1),     # seven words
+    (2, 192, 10, 10, 70, 4, 2, -1),     # even filter size
+    (2, 320, 10, 10, 32, 5, 2, -1),     # five words, 5x5, one 32-channel tile
+    (40, 256, 14, 14, 256, 3, 1, -1),   # enough tiles for CTA pairs with two resident channel tiles
+    (33, 512, 7, 7, 512, 3, 1, +1),     # pairs, odd number of tiles, four channel-tile groups
+    (70, 128, 28, 28, 128, 3, 1, -1, 2),  # pairs, stride 2
 ]
 
 
