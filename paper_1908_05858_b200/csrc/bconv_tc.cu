@@ -25,9 +25,9 @@
 //     (i div 2, j div 2).
 //   * Warp-specialised and mbarrier-driven: four producer warps prefetch the bits two tiles ahead, expand them
 //     (table-free, see expand16) into one of up to two A buffers and arrive on `a_full`; one thread of a
-//     ninth warp waits for it, issues kh*kw*(C/64) tcgen05.mma (M = 128, N = NT, K = 64) into one of two TMEM
+//     separate warp waits for it, issues kh*kw*(C/64) tcgen05.mma (M = 128, N = NT, K = 64) into one of two TMEM
 //     accumulators per resident channel tile and commits to `mma_done` (and, after the tile's last MMA, to `a_free`);
-//     four epilogue warps wait for that, read the accumulator with tcgen05.ld, write the output form, and hand the
+//     four (or eight) epilogue warps wait for that, read the accumulator with tcgen05.ld, write the output form, and hand the
 //     accumulator back through `tmem_free`.
 //
 // Every wait on an mbarrier is bounded: on expiry the kernel records an error flag, stops, frees its TMEM and returns.
@@ -39,7 +39,7 @@ namespace {
 
 enum { EPI_I32 = 0, EPI_BNPACK = 1, EPI_BIREAL = 2 };
 
-constexpr int TC_THREADS = 288;           // 4 epilogue warps, 4 producer warps, 1 MMA-issue warp
+constexpr int TC_THREADS = 416;           // warps 0-3 and (optionally) 8-11: epilogue, 4-7: producers, 12: MMA issue
 constexpr int TC_SMEM_LIMIT = 232448;     // 227 KB opt-in maximum per CTA
 constexpr int TC_MAX_RES = 4;              // channel tiles resident per CTA (pair) at most
 constexpr int TC_SMEM_MISC = 128 + 2 * TC_MAX_RES * 128 * 4;  // barriers, TMEM base, flags; this CTA's scale / shift
@@ -73,6 +73,7 @@ struct TcArgs {
   int ntile, n_ntiles; // output channels per MMA (N), number of such channel tiles
   int pair;            // 1: CTA pairs (cta_group::2), each CTA holds ntile / 2 weight rows per channel tile
   int nres, n_groups;  // channel tiles resident per CTA (pair), groups of `nres` channel tiles
+  int epi2;            // 1: warps 8-11 share the epilogue with warps 0-3
   long long m_tiles;   // tiles of 128 slots (a pair takes two consecutive ones at a time)
   int pad_neg;
   int32_t* out;
@@ -240,8 +241,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   if (tid == 0) {
     mbar_init(smem_u32(&bars[0]), 1);
     mbar_init(smem_u32(&bars[1]), 1);
-    mbar_init(smem_u32(&bars[2]), 128 * PEERS);
-    mbar_init(smem_u32(&bars[3]), 128 * PEERS);
+    mbar_init(smem_u32(&bars[2]), (g.epi2 ? 256 : 128) * PEERS);
+    mbar_init(smem_u32(&bars[3]), (g.epi2 ? 256 : 128) * PEERS);
     mbar_init(smem_u32(&bars[4]), 128 * PEERS);
     mbar_init(smem_u32(&bars[5]), 128 * PEERS);
     mbar_init(smem_u32(&bars[6]), TC_THREADS * PEERS);
@@ -292,7 +293,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   }
-  if (warp < 4 || warp == 8) {
+  if (warp < 4 || warp >= 8) {
     if (warp < 4) {
       // every byte of the scale-factor columns is ue8m0 127 = 1.0, whatever their layout
       const uint32_t one = 0x7F7F7F7Fu;
@@ -308,10 +309,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    arrive(bar_w_full);  // 288 arrivals per CTA in all: weights and scale factors are in place
+    arrive(bar_w_full);  // one arrival per thread of the CTA (pair) in all: weights and scale factors are in place
   }
 
-  if (warp == 8) {
+  if (warp == 12) {
     // ================= MMA issue: one thread (of the leader CTA) ==================================================
     // The chain below is all there is between two MMAs of this CTA, so it is kept to 32-bit adds: only the start-address
     // field (low 14 bits of a descriptor's low word) changes from one MMA to the next, and shared-memory addresses in
@@ -438,7 +439,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       if (blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[16 + i] = prof[i]; }
 #endif
     }
-  } else if (warp >= 4) {
+  } else if (warp >= 4 && warp < 8) {
     // ================= producer warps: packed bits -> e2m1 rows ===================================================
     const int ptid = tid - 128;
     constexpr int PCW = SPT > 2 ? 4 : TC_MAX_CW;  // words per slot held in registers (stride 2 is limited to C <= 256)
@@ -520,10 +521,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     // `nxt`: registers that a load is still filling are never touched before the next iteration.
     auto run = [&](auto cwc) {  // the words per row (C / 64) as a compile-time constant
       constexpr int CW = decltype(cwc)::value;
+      // (stride 2 holds up to five rows per thread: one register set, requested one tile ahead only)
+      constexpr bool TWO_SETS = SPT <= 2;
       SlotRegs cur, nxt;
       long long mt = mt_first;
       prefetch(cur, cwc);  // (rows of a tile beyond the last one are beyond the batch: nothing is read for them)
-      prefetch(nxt, cwc);
+      if (TWO_SETS) prefetch(nxt, cwc);
 #pragma unroll 1
       for (; mt < mt_end; mt += mt_step, it++) {
         const int ab = g.abufs == 2 ? (it & 1) : 0;
@@ -543,12 +546,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
           arrive(bar_w_full);
         }
         TC_T(2);
+        if (TWO_SETS) {
 #pragma unroll
-        for (int h = 0; h < SPT; h++) {
+          for (int h = 0; h < SPT; h++) {
 #pragma unroll
-          for (int cw = 0; cw < CW; cw++) cur.words[h][cw] = nxt.words[h][cw];
+            for (int cw = 0; cw < CW; cw++) cur.words[h][cw] = nxt.words[h][cw];
+          }
+          prefetch(nxt, cwc);
+        } else {
+          prefetch(cur, cwc);
         }
-        prefetch(nxt, cwc);
       }
     };
     // C is a multiple of 64 up to 512: 1..8 words; the common counts get their own straight-line code
@@ -559,16 +566,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #ifdef TC_TIMING
     if (ptid == 0 && blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[i] = prof[i]; g_tc_prof[15] = it; }
 #endif
-  } else {
+  } else if (warp < 4 || g.epi2) {
     // ================= epilogue warps: TMEM accumulator -> output ===============================================
     int ar = 0;  // accumulator rounds so far: one per (tile, resident channel tile)
     bool failed = false;
+    // with the second group, two warps share each quarter of the accumulator's rows: warps 0-3 take the even
+    // 32-column chunks, warps 8-11 the odd ones
+    const int c_first = warp >= 8 ? 32 : 0;
+    const int c_step = g.epi2 ? 64 : 32;
 #ifdef TC_TIMING
     long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     long long tlast = clock64();
 #endif
     for (long long mt = mt_first; mt < mt_end && !failed; mt += mt_step) {
-      const int row = 32 * warp + lane;  // TMEM lane = slot row of the tile
+      const int row = 32 * (warp & 3) + lane;  // TMEM lane = slot row of the tile
       const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)row;
       const uint32_t rr = fast_div(Q, g.magic_sp);
       const int col = (int)(Q - rr * (uint32_t)g.SP);
@@ -598,7 +609,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
             if (8 * q < nch) ld_global_v8(rs + 8 * q, *reinterpret_cast<float(*)[8]>(&rpre[8 * q]));
         }
       };
-      load_res(0);
+      load_res(c_first);
       TC_T(0);
       if (!mbar_wait(smem_u32(&bars[buf]), (ar >> 1) & 1, s_fail)) {
         *s_fail = 1;
@@ -609,17 +620,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const long long m = my_m;
 #pragma unroll 1
-      for (int c0 = 0; c0 < NT; c0 += 32) {
+      for (int c0 = c_first; c0 < NT; c0 += c_step) {
         __syncwarp();  // the TMEM load is warp-wide: rejoin lanes that took different paths below
         TC_T(4);
         float rc[32];
         if (EPI == EPI_BIREAL) {
 #pragma unroll
           for (int j = 0; j < 32; j++) rc[j] = rpre[j];
-          if (c0 + 32 < NT) load_res(c0 + 32);
+          if (c0 + c_step < NT) load_res(c0 + c_step);
         }
         uint32_t v[32];
-        const uint32_t taddr = tmem_base + ((uint32_t)(32 * warp) << 16) + (uint32_t)(buf * NT + c0);
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(buf * NT + c0);
         asm volatile(
             "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
             "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
@@ -853,6 +864,11 @@ dabnn_status tc_dispatch_mode(TcArgs& g, cudaStream_t st) {
 
 template <int EPI>
 dabnn_status tc_dispatch(TcArgs& g, cudaStream_t st) {
+  // A second group of epilogue warps (measured): it pays for the residual epilogue, which moves two fp32 rows per
+  // output row, and for the sign-bit epilogue at C = 128; elsewhere the extra warps only add contention.
+  // (environment DABNN_TC_EPI2 = 0 / 1 overrides, for measurements)
+  static const int epi_env = [] { const char* e = getenv("DABNN_TC_EPI2"); return e ? atoi(e) : -1; }();
+  g.epi2 = epi_env >= 0 ? (epi_env != 0) : (EPI == EPI_BIREAL || (EPI == EPI_BNPACK && g.Cw == 2));
   return g.pair ? tc_dispatch_mode<EPI, true>(g, st) : tc_dispatch_mode<EPI, false>(g, st);
 }
 
