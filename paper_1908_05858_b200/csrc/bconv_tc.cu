@@ -214,7 +214,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   uint8_t* w_s = smem;                                   // [nres][taps][C/32][WR][16]
   uint8_t* a_s = smem + (size_t)g.nres * WR * Kb;        // [abufs][C/32][slots][16]
   uint8_t* misc = a_s + (size_t)g.abufs * a_bytes;
-  // [0,1] mma_done  [2,3] tmem_free  [4,5] a_full  [6] w_full  [7,8] a_free; of a pair, the leader's 2..6 are used
+  // [0,1] mma_done  [2,3] tmem_free  [4,5] a_full  [6] w_full (first third of the filter taps)  [7,8] a_free
+  // [9,10] w_full (second and last third); of a pair, the leader's tmem_free, a_full and w_full are used
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 96);
   volatile int* s_fail = reinterpret_cast<volatile int*>(misc + 104);
@@ -248,6 +249,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     mbar_init(smem_u32(&bars[6]), TC_THREADS * PEERS);
     mbar_init(smem_u32(&bars[7]), 1);
     mbar_init(smem_u32(&bars[8]), 1);
+    mbar_init(smem_u32(&bars[9]), TC_THREADS * PEERS);
+    mbar_init(smem_u32(&bars[10]), TC_THREADS * PEERS);
     *s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -272,7 +275,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   // barriers that both CTAs of a pair signal live in the leader
   const uint32_t bar_tmem_free0 = PAIR ? leader_addr(smem_u32(&bars[2])) : smem_u32(&bars[2]);
   const uint32_t bar_a_full0 = PAIR ? leader_addr(smem_u32(&bars[4])) : smem_u32(&bars[4]);
-  const uint32_t bar_w_full = PAIR ? leader_addr(smem_u32(&bars[6])) : smem_u32(&bars[6]);
+  const uint32_t bar_w_full = PAIR ? leader_addr(smem_u32(&bars[6])) : smem_u32(&bars[6]);  // + 24, + 32: the later thirds
   auto arrive = [&](uint32_t bar) {
     if (PAIR) mbar_arrive_cluster(bar);
     else mbar_arrive(bar);
@@ -281,18 +284,36 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     // Resident weights: rows [rank * WR, +WR) of every channel tile of this group, one (tile, tap, 32-channel group)
     // block of WR rows per warp and step; the source holds blocks of 32 output channels.  The producers do not wait
     // for their share until their first tile's rows are out, so the copy overlaps the first expansion.
+    // The copy goes in three groups, thirds of the (tap, 32-channel group) blocks in issue order -- for a 3x3 filter
+    // one row of taps each -- with a barrier per group: the first MMAs start when the first third has landed.
     const int TG = g.kh * g.kw * (g.C >> 5);
-    for (int tb = warp; tb < nres_here * TG; tb += TC_THREADS / 32) {
-      const int r = tb / TG, tg = tb - r * TG;
-      const int col0 = (ng * g.nres + r) * NT + (int)rank * WR;
-      uint8_t* dst = w_s + (size_t)tb * WR * 16;
-      for (int n = lane; n < WR; n += 32) {
-        const int col = col0 + n;
-        cp_async16(smem_u32(dst + n * 16), g.w_tc + (((size_t)(col >> 5) * TG + tg) * 32 + (col & 31)) * 16);
+#pragma unroll 1
+    for (int j = 0; j < 3; j++) {
+      const int lo = TG * j / 3, cnt = TG * (j + 1) / 3 - lo;
+      for (int idx = warp; idx < nres_here * cnt; idx += TC_THREADS / 32) {
+        const int r = idx / cnt, tg = lo + idx - r * cnt;
+        const int col0 = (ng * g.nres + r) * NT + (int)rank * WR;
+        uint8_t* dst = w_s + (size_t)(r * TG + tg) * WR * 16;
+        for (int n = lane; n < WR; n += 32) {
+          const int col = col0 + n;
+          cp_async16(smem_u32(dst + n * 16), g.w_tc + (((size_t)(col >> 5) * TG + tg) * 32 + (col & 31)) * 16);
+        }
       }
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    asm volatile("cp.async.commit_group;" ::: "memory");
   }
+  // this thread's share of each third has landed -> one arrival on that third's barrier
+  auto weights_arrive = [&]() {
+    asm volatile("cp.async.wait_group 2;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    arrive(bar_w_full);
+    asm volatile("cp.async.wait_group 1;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    arrive(bar_w_full + 24u);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    arrive(bar_w_full + 32u);
+  };
   if (warp < 4 || warp >= 8) {
     if (warp < 4) {
       // every byte of the scale-factor columns is ue8m0 127 = 1.0, whatever their layout
@@ -306,10 +327,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       }
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
     }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    arrive(bar_w_full);  // one arrival per thread of the CTA (pair) in all: weights and scale factors are in place
+    weights_arrive();  // one arrival per thread of the CTA (pair) in all: weights (by thirds) and scale factors are in place
   }
 
   if (warp == 12) {
@@ -376,17 +395,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       long long tlast = clock64();
 #endif
       // all MMAs of one tile and channel tile; KB = C / 64 as a compile-time constant, the 3x3 filter fully unrolled
-      auto issue_tile = [&](uint32_t d_tmem, uint32_t a_lo0, uint32_t b_base, uint32_t a_stp, auto kbc) {
+      auto issue_tile = [&](uint32_t d_tmem, uint32_t a_lo0, uint32_t b_base, uint32_t a_stp, bool first, auto kbc) {
         constexpr int KB = decltype(kbc)::value;
         if (k3) {
 #pragma unroll
           for (int t = 0; t < 9; t++) {
+            if (first && (t == 3 || t == 6) && !wait(smem_u32(&bars[t == 3 ? 9 : 10]), 0)) *s_fail = 1;  // that row of taps
             const uint32_t a_lo = a_lo0 + off9[t];
 #pragma unroll
             for (int kb = 0; kb < KB; kb++)
               mma(d_tmem, a_lo + (uint32_t)kb * a_stp, b_base + (uint32_t)(t * KB + kb) * b_step, (t | kb) ? 1u : 0u);
           }
         } else {
+          if (first && !(wait(smem_u32(&bars[9]), 0) && wait(smem_u32(&bars[10]), 0))) *s_fail = 1;
           uint32_t b_lo = b_base, accumulate = 0;
           for (int ti = 0; ti < g.kh; ti++)
             for (int tj = 0; tj < g.kw; tj++) {
@@ -420,14 +441,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
           const uint32_t d_tmem = tmem_base + (uint32_t)((ar & 1) * NT);
           const uint32_t b_base = b_lo0 + (uint32_t)r * b_tile;
           switch (g.Cw) {  // C / 64 = 1..8
-            case 1: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<1>{}); break;
-            case 2: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<2>{}); break;
-            case 3: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<3>{}); break;
-            case 4: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<4>{}); break;
-            case 5: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<5>{}); break;
-            case 6: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<6>{}); break;
-            case 7: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<7>{}); break;
-            default: issue_tile(d_tmem, a_lo0, b_base, a_step_t, IntC<8>{}); break;
+            case 1: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<1>{}); break;
+            case 2: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<2>{}); break;
+            case 3: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<3>{}); break;
+            case 4: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<4>{}); break;
+            case 5: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<5>{}); break;
+            case 6: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<6>{}); break;
+            case 7: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<7>{}); break;
+            default: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<8>{}); break;
           }
           commit(smem_u32(&bars[ar & 1]));
         }
@@ -541,9 +562,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         if (it == 0) {
           // the first tile's rows went out before anything else: a short launch is all start-up.  Now this thread's
           // share of the weights.
-          asm volatile("cp.async.wait_group 0;" ::: "memory");
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          arrive(bar_w_full);
+          weights_arrive();
         }
         TC_T(2);
         if (TWO_SETS) {
@@ -791,7 +810,10 @@ dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
   static bool configured = false;
   static int max_units = 0;  // CTAs (pairs) that can be resident at once
   if (!configured) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT) != cudaSuccess) {
+    // the largest shared-memory carve-out for every instance, whatever it needs: consecutive launches of different
+    // instances then never make the SMs re-partition their L1 / shared memory
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT) != cudaSuccess ||
+        cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
       cudaGetLastError();
       return DABNN_ERR_CUDA;
     }
