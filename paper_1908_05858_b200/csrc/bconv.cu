@@ -253,22 +253,24 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(cons
         v[j] = g.Kbits - 2 * cnt;
       }
       const int o = o0 + wrow0;
+      // (streaming stores: the int32 sums are read by nothing in this library, and kept out of the way in L2 they do
+      // not displace the weights and activations that the following launches read)
       if (!g.out_nchw) {
         int32_t* dst = g.out + m * g.O + o;
         if (TO % 4 == 0 && o + TO <= g.O && (g.O & 3) == 0 && (reinterpret_cast<uintptr_t>(g.out) & 15) == 0) {
 #pragma unroll
-          for (int j = 0; j < TO; j += 4) *reinterpret_cast<int4*>(dst + j) = make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+          for (int j = 0; j < TO; j += 4) __stcs(reinterpret_cast<int4*>(dst + j), make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]));
         } else {
 #pragma unroll
           for (int j = 0; j < TO; j++)
-            if (o + j < g.O) dst[j] = v[j];
+            if (o + j < g.O) __stcs(dst + j, v[j]);
         }
       } else {
         const long long ohw = (long long)g.OH * g.OW;
         const long long n = m / ohw, q = m % ohw;
 #pragma unroll
         for (int j = 0; j < TO; j++)
-          if (o + j < g.O) g.out[(n * g.O + o + j) * ohw + q] = v[j];
+          if (o + j < g.O) __stcs(g.out + (n * g.O + o + j) * ohw + q, v[j]);
       }
     }
   } else {

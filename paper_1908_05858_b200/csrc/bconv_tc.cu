@@ -182,6 +182,16 @@ __device__ __forceinline__ void st_global_v8(void* p, uint32_t a, uint32_t b, ui
                "r"(f), "r"(g2), "r"(h)
                : "memory");
 }
+// The same with an evict-first policy in L2: for output that nothing in this library reads back (the int32 sums), so that
+// it drains to DRAM as it is produced instead of displacing the weights and activations that the next launches read.
+__device__ __forceinline__ void st_global_v8_stream(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e,
+                                                    uint32_t f, uint32_t g2, uint32_t h) {
+  asm volatile(
+      "{\n\t.reg .b64 pol;\n\tcreatepolicy.fractional.L2::evict_first.b64 pol, 1.0;\n\t"
+      "st.global.L2::cache_hint.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8}, pol;\n\t}" ::"l"(p),
+      "r"(a), "r"(b), "r"(c), "r"(d), "r"(e), "r"(f), "r"(g2), "r"(h)
+      : "memory");
+}
 __device__ __forceinline__ void ld_global_v8(const void* p, float (&r)[8]) {
   asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                : "=f"(r[0]), "=f"(r[1]), "=f"(r[2]), "=f"(r[3]), "=f"(r[4]), "=f"(r[5]), "=f"(r[6]), "=f"(r[7])
@@ -267,11 +277,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
   }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  if (PAIR) cluster_sync_all();  // both CTAs' barriers exist before either signals the other's
-  else __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = *tmem_slot;
+  // The start-up barrier: barriers initialised (in both CTAs of a pair, before either signals the other's) and the
+  // tensor-memory address published.  Each warp passes it once, as late as its role allows: the weight copy and the
+  // producers' first requests for activation bits are already in flight by then.
+  auto prologue_sync = [&]() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    if (PAIR) cluster_sync_all();
+    else __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  };
+  const bool is_producer = warp >= 4 && warp < 8;
+  uint32_t tmem_base = 0;
   // barriers that both CTAs of a pair signal live in the leader
   const uint32_t bar_tmem_free0 = PAIR ? leader_addr(smem_u32(&bars[2])) : smem_u32(&bars[2]);
   const uint32_t bar_a_full0 = PAIR ? leader_addr(smem_u32(&bars[4])) : smem_u32(&bars[4]);
@@ -314,6 +330,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     arrive(bar_w_full + 32u);
   };
+  if (!is_producer) {
+    prologue_sync();
+    tmem_base = *tmem_slot;
+  }
   if (warp < 4 || warp >= 8) {
     if (warp < 4) {
       // every byte of the scale-factor columns is ue8m0 127 = 1.0, whatever their layout
@@ -548,6 +568,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       long long mt = mt_first;
       prefetch(cur, cwc);  // (rows of a tile beyond the last one are beyond the batch: nothing is read for them)
       if (TWO_SETS) prefetch(nxt, cwc);
+      prologue_sync();
 #pragma unroll 1
       for (; mt < mt_end; mt += mt_step, it++) {
         const int ab = g.abufs == 2 ? (it & 1) : 0;
@@ -582,6 +603,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     else if (g.Cw == 2) run(IntC<2>{});
     else if (g.Cw <= 4) run(IntC<4>{});
     else if constexpr (PCW > 4) run(IntC<8>{});
+    else prologue_sync();  // (not reached: the host launches this instance for C <= 256 only)
 #ifdef TC_TIMING
     if (ptid == 0 && blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[i] = prof[i]; g_tc_prof[15] = it; }
 #endif
@@ -670,7 +692,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #pragma unroll
             for (int q = 0; q < 4; q++)
               if (8 * q < nch)  // nch is a multiple of 8 here
-                st_global_v8(dst + 8 * q, acc_to_int(v[8 * q]),
+                st_global_v8_stream(dst + 8 * q, acc_to_int(v[8 * q]),
                              acc_to_int(v[8 * q + 1]),
                              acc_to_int(v[8 * q + 2]),
                              acc_to_int(v[8 * q + 3]),
@@ -682,13 +704,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
             int32_t* dst = g.out + m * g.O + o;
 #pragma unroll
             for (int j = 0; j < 32; j++)
-              if (j < nch) dst[j] = acc_to_int(v[j]);
+              if (j < nch) __stcs(reinterpret_cast<uint32_t*>(dst) + j, acc_to_int(v[j]));
           } else {
             const long long ohw = (long long)g.OH * g.OW;
             const long long nn = m / ohw, q = m - nn * ohw;
 #pragma unroll
             for (int j = 0; j < 32; j++)
-              if (j < nch) g.out[(nn * g.O + o + j) * ohw + q] = acc_to_int(v[j]);
+              if (j < nch) __stcs(reinterpret_cast<uint32_t*>(g.out) + (nn * g.O + o + j) * ohw + q, acc_to_int(v[j]));
           }
         } else {
           if (o >= g.Ow32 * 32) continue;  // sign words are written whole (tail bits 0), nothing beyond them
