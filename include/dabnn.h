@@ -173,7 +173,14 @@ dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const 
  * Covered: stride 1 or 2 (both axes alike), C a multiple of 64 and at most 512 (256 for stride 2), images narrow enough
  * that a tile's rows fit the activation buffer (W + 2*pad_w <= 63 for 3x3 stride 1), filters whose expanded weights fit the resident budget (dabnn_tc_weights_bytes
  * returns 0 otherwise); other cases return DABNN_ERR_UNSUPPORTED and are served by dabnn_bconv2d*.
- *   dabnn_tc_weights_bytes    bytes of the expanded weight buffer for a filter bank (0 = not covered)
+ * A launch takes one of two forms, chosen by the library from the problem size: one CTA per tile of 128 output
+ * positions, or pairs of CTAs of a thread-block cluster that share every tensor-core instruction (used where one CTA
+ * cannot keep 128 output channels of weights resident: C = 512 with a 3x3 filter).  Both give the same bits.
+ * The int32 output is written with a streaming (evict-first) cache policy.
+ * Environment, read once, for measurements only: DABNN_TC_MODE = 1 (never pairs) or 2 (pairs wherever possible);
+ * DABNN_TC_EPI2 = 0 / 1 (second group of epilogue warps off / on).
+ *   dabnn_tc_weights_bytes    bytes of the expanded weight buffer for a filter bank (0 = not covered): O rounded up to
+ *                             128 rows of C*kh*kw/2 bytes, the same buffer for every launch form
  *   dabnn_tc_prepare_weights  w_packed [O][kh][kw][Cw] -> w_tc (device, 16-byte aligned, that many bytes); once per model
  *   dabnn_tc_bconv2d*         as dabnn_bconv2d*, with w_tc in place of w_packed
  *   dabnn_tc_error_flag       synchronises nothing itself; copies the device-side error flag (1 if a bounded wait inside
