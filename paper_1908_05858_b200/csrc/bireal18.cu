@@ -131,6 +131,20 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
   asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
+// Two fp32 fused multiply-adds in one instruction (fma.rn.f32x2): each lane of the pair is the same correctly rounded
+// fmaf as the scalar instruction, so results do not change; it halves the issue slots of an FMA-bound loop.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma_f32x2(unsigned long long& acc, unsigned long long a, unsigned long long b) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+
 // Large batches: the same convolution with an 8 pixels (along a row) x 8 channels register tile.  Per (c, kh) a thread
 // loads the 21 input values its 8 pixels need (even and odd columns as 3 + 3 float4) once and reuses them for all 7
 // horizontal taps; per tap it loads 8 weights.  Persistent CTAs as above; the order of every output's fmaf chain is
@@ -188,11 +202,11 @@ __global__ void __launch_bounds__(256, 2) stem_conv_bn_8x8(const float* __restri
     __syncthreads();
     if (tile + gridDim.x < ntiles) load_patch(tile + gridDim.x, x_s + (buf ^ 1) * PATCH);
     const float* xb = x_s + buf * PATCH;
-    float acc[8][8];
+    unsigned long long acc2[8][4];  // channel pairs (0,1) (2,3) (4,5) (6,7) of each pixel
 #pragma unroll
     for (int i = 0; i < 8; i++)
 #pragma unroll
-      for (int j = 0; j < 8; j++) acc[i][j] = 0.0f;
+      for (int j = 0; j < 4; j++) acc2[i][j] = 0ull;  // (+0.0, +0.0)
 #pragma unroll 1
     for (int c = 0; c < 3; c++)
 #pragma unroll 1
@@ -211,15 +225,22 @@ __global__ void __launch_bounds__(256, 2) stem_conv_bn_8x8(const float* __restri
         for (int kj = 0; kj < 7; kj++) {
           const float4 wa = *reinterpret_cast<const float4*>(wk + kj * 64);
           const float4 wb = *reinterpret_cast<const float4*>(wk + kj * 64 + 32);
-          const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+          const unsigned long long w2[4] = {pack_f32x2(wa.x, wa.y), pack_f32x2(wa.z, wa.w), pack_f32x2(wb.x, wb.y),
+                                            pack_f32x2(wb.z, wb.w)};
 #pragma unroll
           for (int i = 0; i < 8; i++) {
             const float xv = (kj & 1) ? xo[i + (kj >> 1)] : xe[i + (kj >> 1)];
+            const unsigned long long x2 = pack_f32x2(xv, xv);
 #pragma unroll
-            for (int j = 0; j < 8; j++) acc[i][j] = __fmaf_rn(xv, wv[j], acc[i][j]);
+            for (int j = 0; j < 4; j++) fma_f32x2(acc2[i][j], x2, w2[j]);
           }
         }
       }
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; i++)
+#pragma unroll
+      for (int j = 0; j < 4; j++) unpack_f32x2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
     const int n = (int)(tile / (TILES * TILES));
     const int rem = (int)(tile % (TILES * TILES));
     const int oh = (rem / TILES) * TS + row, owb = (rem % TILES) * TS + ow0;
@@ -350,11 +371,11 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
   };
   // compute roles: 16 x 16 threads; thread (ty, tx) owns pixels ty*8..+7 and channels tx*4..+3 and 64 + tx*4..+3
   const int ty = tid >> 4, tx = tid & 15;
-  float acc[8][8];
+  unsigned long long acc2[8][4];  // channel pairs of each pixel (packed fp32 FMAs, same rounding as scalar fmaf)
 #pragma unroll
   for (int i = 0; i < 8; i++)
 #pragma unroll
-    for (int j = 0; j < 8; j++) acc[i][j] = 0.0f;
+    for (int j = 0; j < 4; j++) acc2[i][j] = 0ull;
   const int nchunks = (C + SC_BK - 1) / SC_BK;
   pool_load(0);
   w_load(0);
@@ -375,11 +396,14 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
       const float4 wa = *reinterpret_cast<const float4*>(&w_s[st][cc][tx * 4]);
       const float4 wb = *reinterpret_cast<const float4*>(&w_s[st][cc][64 + tx * 4]);
       const float pv[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
-      const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+      const unsigned long long w2[4] = {pack_f32x2(wa.x, wa.y), pack_f32x2(wa.z, wa.w), pack_f32x2(wb.x, wb.y),
+                                        pack_f32x2(wb.z, wb.w)};
 #pragma unroll
-      for (int i = 0; i < 8; i++)
+      for (int i = 0; i < 8; i++) {
+        const unsigned long long p2 = pack_f32x2(pv[i], pv[i]);
 #pragma unroll
-        for (int j = 0; j < 8; j++) acc[i][j] = __fmaf_rn(pv[i], wv[j], acc[i][j]);
+        for (int j = 0; j < 4; j++) fma_f32x2(acc2[i][j], p2, w2[j]);
+      }
     }
     if (ch + 1 < nchunks) {
       pool_store(st ^ 1);
@@ -387,6 +411,11 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
     }
     __syncthreads();
   }
+  float acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; i++)
+#pragma unroll
+    for (int j = 0; j < 4; j++) unpack_f32x2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
 #pragma unroll
   for (int h = 0; h < 2; h++) {
     const int o = o0 + 64 * h + tx * 4;
