@@ -66,6 +66,10 @@ int dabnn_out_dim(int in, int k, int stride, int pad);
 /* Section 2.1.1 -- binarize + pack activations.
  * x: fp32, N*C*H*W elements in `in_layout`.  packed: uint64 [N][H][W][Cw], fully overwritten. */
 dabnn_status dabnn_pack(const float* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed, void* stream);
+/* The same for 32-bit integers (Section 2.1.1: the packer takes the sign bit of int32 values as it does of floats), e.g. a
+ * convolution's raw sums binarized without a BN in between.  bit = (x < 0): 0 packs as +1.  Same layouts, output and
+ * errors as dabnn_pack; x must be 4-byte aligned (16-byte aligned input takes the vector path). */
+dabnn_status dabnn_pack_i32(const int32_t* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed, void* stream);
 
 /* Section 3 (weights are binarized and packed once, 32x smaller).
  * w_oihw: fp32 [O][C][kh][kw].  wpacked: uint64 [O][kh][kw][Cw], fully overwritten. */

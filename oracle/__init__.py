@@ -94,6 +94,18 @@ def pack(x: np.ndarray, layout: int = NCHW) -> np.ndarray:
     return P
 
 
+def pack_i32(x: np.ndarray, layout: int = NCHW) -> np.ndarray:
+    """Pack the sign bits of int32 values (Section 2.1.1).  x: int32 NCHW or NHWC."""
+    x = np.ascontiguousarray(x, dtype=np.int32)
+    if layout == NCHW:
+        N, C, H, W = x.shape
+    else:
+        N, H, W, C = x.shape
+    P = np.empty((N, H, W, words_per_pixel(C)), dtype=np.uint64)
+    lib().oracle_pack_i32(_p(x), ctypes.c_int(layout), N, C, H, W, _p(P))
+    return P
+
+
 def pack_weights(w_oihw: np.ndarray) -> np.ndarray:
     w = _f32(w_oihw)
     O, C, kh, kw = w.shape

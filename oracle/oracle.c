@@ -8,7 +8,8 @@
  * the benchmark's CPU-baseline leg may load it.
  *
  * What each function follows:
- *   oracle_pack / oracle_pack_weights   Section 2.1.1 (bit-packing), the "naive" sequential
+ *   oracle_pack / oracle_pack_i32 / oracle_pack_weights
+ *                                       Section 2.1.1 (bit-packing), the "naive" sequential
  *                                       packer the paper describes as the prior method:
  *                                       test every element, set its bit.
  *   oracle_bconv_pm1                    Section 2.1.2, last paragraph: A = weights (M = C_out),
@@ -86,6 +87,21 @@ void oracle_pack(const float* x, int layout, int N, int C, int H, int W, uint64_
           size_t xi = (layout == LAYOUT_NCHW) ? (((size_t)n * C + c) * H + h) * W + w
                                               : (((size_t)n * H + h) * W + w) * C + c;
           uint64_t bit = (binarize(x[xi]) == -1) ? 1u : 0u;
+          P[(((size_t)n * H + h) * W + w) * Cw + (size_t)(c >> 6)] |= bit << (c & 63);
+        }
+}
+
+/* Section 2.1.1, int32 input: the bit is the sign bit of the integer, i.e. 1 for x < 0 (0 packs as +1). */
+void oracle_pack_i32(const int32_t* x, int layout, int N, int C, int H, int W, uint64_t* P) {
+  size_t Cw = words_per_pixel(C);
+  memset(P, 0, (size_t)N * H * W * Cw * sizeof(uint64_t));
+  for (int n = 0; n < N; n++)
+    for (int h = 0; h < H; h++)
+      for (int w = 0; w < W; w++)
+        for (int c = 0; c < C; c++) {
+          size_t xi = (layout == LAYOUT_NCHW) ? (((size_t)n * C + c) * H + h) * W + w
+                                              : (((size_t)n * H + h) * W + w) * C + c;
+          uint64_t bit = (x[xi] < 0) ? 1u : 0u;
           P[(((size_t)n * H + h) * W + w) * Cw + (size_t)(c >> 6)] |= bit << (c & 63);
         }
 }

@@ -22,7 +22,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdabnn_b200.so")
 
 EXPORTS = (
-    "dabnn_status_string", "dabnn_words_per_pixel", "dabnn_out_dim", "dabnn_pack", "dabnn_pack_weights",
+    "dabnn_status_string", "dabnn_words_per_pixel", "dabnn_out_dim", "dabnn_pack", "dabnn_pack_i32", "dabnn_pack_weights",
     "dabnn_bconv2d", "dabnn_bgemm", "dabnn_bconv2d_bn_sign_pack", "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold",
     "dabnn_bireal18_workspace_bytes", "dabnn_bireal18_forward", "dabnn_set_conv_variant",
     "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host", "dabnn_bireal18_forward_static", "dabnn_set_conv_tile",
@@ -73,6 +73,8 @@ def lib() -> ctypes.CDLL:
         L.dabnn_out_dim.restype = ci
         L.dabnn_out_dim.argtypes = [ci, ci, ci, ci]
         L.dabnn_pack.argtypes = [vp, ci, Shape, vp, vp]
+        L.dabnn_pack_i32.argtypes = [vp, ci, Shape, vp, vp]
+        L.dabnn_pack_i32.restype = ci
         L.dabnn_pack_weights.argtypes = [vp, ci, ci, ci, ci, vp, vp]
         L.dabnn_bconv2d.argtypes = [vp, Shape, vp, ci, Conv, vp, ci, vp]
         L.dabnn_bgemm.argtypes = [vp, ci, vp, ci, ci, vp, vp]
@@ -148,6 +150,19 @@ def pack(x: torch.Tensor, layout: int = NCHW, out: Optional[torch.Tensor] = None
     if out is None:
         out = torch.empty((N, H, W, words_per_pixel(C)), dtype=torch.int64, device=x.device)
     _check(lib().dabnn_pack(x.data_ptr(), layout, Shape(N, C, H, W), out.data_ptr(), _stream()))
+    return out
+
+
+def pack_i32(x: torch.Tensor, layout: int = NCHW, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_pack_i32: int32 NCHW or NHWC -> packed int64 [N][H][W][Cw] (bit = x < 0)."""
+    x = _dev(x, torch.int32, "x")
+    if layout == NCHW:
+        N, C, H, W = x.shape
+    else:
+        N, H, W, C = x.shape
+    if out is None:
+        out = torch.empty((N, H, W, words_per_pixel(C)), dtype=torch.int64, device=x.device)
+    _check(lib().dabnn_pack_i32(x.data_ptr(), layout, Shape(N, C, H, W), out.data_ptr(), _stream()))
     return out
 
 

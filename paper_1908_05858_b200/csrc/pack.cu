@@ -1,11 +1,12 @@
-// Binarize + bit-pack kernels (Section 2.1.1 of the paper): fp32 -> one bit per element, 64 channels
+// Binarize + bit-pack kernels (Section 2.1.1 of the paper): fp32 (or int32) -> one bit per element, 64 channels
 // per word, words of a pixel contiguous (channel-packed NHWC).  Pure HBM streaming: 4 bytes read and
 // 1/8 byte written per element.
 //
 // The paper gathers IEEE sign bits with NEON shift-and-insert instructions spread over several
 // registers.  Here the sign test is a compare (so -0.0 and NaN pack as +1), 128-bit loads keep the
 // memory system busy, bits are gathered in registers by shift-or, and the words leave through shared
-// memory so that global stores are whole, contiguous 16-byte pieces.
+// memory so that global stores are whole, contiguous 16-byte pieces.  The int32 form (the paper packs the sign bit
+// of 32-bit integers the same way, e.g. a convolution's raw sums) runs the same kernels with an integer compare.
 #include "common.cuh"
 
 namespace dabnn {
@@ -16,17 +17,29 @@ constexpr int kPackThreads = 128;
 
 // Streaming 16-byte load.  Written as volatile asm so that a batch of them is issued back to back, in program
 // order, before the first result is consumed (memory-level parallelism is what an HBM-bound kernel lives on).
-__device__ __forceinline__ float4 ld_stream_f4(const float4* p) {
+__device__ __forceinline__ float4 ld_stream_v4(const float4* p) {
   float4 v;
   asm volatile("ld.global.cs.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
   return v;
 }
+__device__ __forceinline__ int4 ld_stream_v4(const int4* p) {
+  int4 v;
+  asm volatile("ld.global.cs.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+template <typename T> struct Vec4;
+template <> struct Vec4<float> { using type = float4; };
+template <> struct Vec4<int32_t> { using type = int4; };
+// the bit: 1 where the value is negative (a compare: -0.0 and NaN give 0, i.e. +1)
+__device__ __forceinline__ unsigned neg(float v) { return (unsigned)(v < 0.0f); }
+__device__ __forceinline__ unsigned neg(int32_t v) { return (unsigned)(v < 0); }
 
 // NCHW, H*W a multiple of 4, 16-byte aligned input.  A CTA covers 128 consecutive pixels of one image and all
 // channels.  Each lane owns 4 consecutive pixels (one float4 per channel); the four warps split every word's 64
 // channels into quarters of 16, so a thread has 16 independent 16-byte loads in flight per word, and the 16-bit
 // quarters are placed side by side in shared memory, which assembles the 64-bit words without any exchange.
-__global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const float* __restrict__ x, int C, int HW, int Cw,
+template <typename T>
+__global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const T* __restrict__ x, int C, int HW, int Cw,
                                                                uint64_t* __restrict__ packed) {
   extern __shared__ __align__(16) uint64_t s_words[];  // [128][Cw]
   uint16_t* s_q = reinterpret_cast<uint16_t*>(s_words);
@@ -35,31 +48,32 @@ __global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const float* __re
   const int pix0 = blockIdx.x * 128;
   const int p = pix0 + lane * 4;  // first of this lane's 4 pixels
   const bool live = p < HW;       // HW % 4 == 0, so all 4 pixels are live together
-  const float* xn = x + (size_t)n * C * HW;
+  using V4 = typename Vec4<T>::type;
+  const T* xn = x + (size_t)n * C * HW;
   const size_t cstride = (size_t)HW / 4;
   for (int cw = 0; cw < Cw; cw++) {
     const int c0 = cw * 64 + warp * 16;
     unsigned b0 = 0, b1 = 0, b2 = 0, b3 = 0;  // 16 channels of each of the 4 pixels
     if (live && c0 < C) {
-      const float4* src = reinterpret_cast<const float4*>(xn + (size_t)c0 * HW + p);
+      const V4* src = reinterpret_cast<const V4*>(xn + (size_t)c0 * HW + p);
       if (c0 + 16 <= C) {
-        float4 v[16];
+        V4 v[16];
 #pragma unroll
-        for (int u = 0; u < 16; u++) v[u] = ld_stream_f4(src + (size_t)u * cstride);
+        for (int u = 0; u < 16; u++) v[u] = ld_stream_v4(src + (size_t)u * cstride);
 #pragma unroll
         for (int u = 0; u < 16; u++) {
-          b0 |= (unsigned)(v[u].x < 0.0f) << u;
-          b1 |= (unsigned)(v[u].y < 0.0f) << u;
-          b2 |= (unsigned)(v[u].z < 0.0f) << u;
-          b3 |= (unsigned)(v[u].w < 0.0f) << u;
+          b0 |= neg(v[u].x) << u;
+          b1 |= neg(v[u].y) << u;
+          b2 |= neg(v[u].z) << u;
+          b3 |= neg(v[u].w) << u;
         }
       } else {
         for (int u = 0; u < C - c0; u++) {
-          const float4 v = __ldcs(src + (size_t)u * cstride);
-          b0 |= (unsigned)(v.x < 0.0f) << u;
-          b1 |= (unsigned)(v.y < 0.0f) << u;
-          b2 |= (unsigned)(v.z < 0.0f) << u;
-          b3 |= (unsigned)(v.w < 0.0f) << u;
+          const V4 v = __ldcs(src + (size_t)u * cstride);
+          b0 |= neg(v.x) << u;
+          b1 |= neg(v.y) << u;
+          b2 |= neg(v.z) << u;
+          b3 |= neg(v.w) << u;
         }
       }
     }
@@ -89,21 +103,22 @@ __global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const float* __re
 // NCHW, any H*W and alignment: a CTA takes 128 consecutive pixels of one image and one 64-channel word.  The
 // 64 x 128 sign flags are gathered with coalesced scalar loads (lanes along pixels) into shared memory; each
 // thread then assembles 32 channel bits of one pixel and stores that half word.
-__global__ void __launch_bounds__(256) pack_nchw_tile(const float* __restrict__ x, int C, int HW, int Cw,
+template <typename T>
+__global__ void __launch_bounds__(256) pack_nchw_tile(const T* __restrict__ x, int C, int HW, int Cw,
                                                       uint64_t* __restrict__ packed) {
   __shared__ unsigned char s_sign[64 * 128];
   const int tid = threadIdx.x, lane = tid & 31, ty = tid >> 5;
   const int n = blockIdx.y, p0 = blockIdx.x * 128, cw = blockIdx.z;
   const int npix = min(128, HW - p0);
-  const float* xn = x + (size_t)n * C * HW + p0;
+  const T* xn = x + (size_t)n * C * HW + p0;
   const int c0 = cw * 64, cn = min(64, C - c0);
 #pragma unroll
   for (int c = ty; c < 64; c += 8) {
-    const float* row = xn + (size_t)(c0 + c) * HW;
+    const T* row = xn + (size_t)(c0 + c) * HW;
 #pragma unroll
     for (int q = 0; q < 4; q++) {
       const int p = lane + 32 * q;
-      s_sign[c * 128 + p] = (c < cn && p < npix) ? (unsigned char)(__ldcs(row + p) < 0.0f) : (unsigned char)0;
+      s_sign[c * 128 + p] = (c < cn && p < npix) ? (unsigned char)neg(__ldcs(row + p)) : (unsigned char)0;
     }
   }
   __syncthreads();
@@ -117,7 +132,8 @@ __global__ void __launch_bounds__(256) pack_nchw_tile(const float* __restrict__ 
 }
 
 // Any layout, any shape: one thread per output word.
-__global__ void pack_generic(const float* __restrict__ x, int nhwc, int C, int HW, int Cw, long long total_words,
+template <typename T>
+__global__ void pack_generic(const T* __restrict__ x, int nhwc, int C, int HW, int Cw, long long total_words,
                              uint64_t* __restrict__ packed) {
   long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= total_words) return;
@@ -126,37 +142,38 @@ __global__ void pack_generic(const float* __restrict__ x, int nhwc, int C, int H
   const int c0 = cw * 64, cn = min(64, C - c0);
   uint64_t w = 0;
   if (nhwc) {
-    const float* src = x + (size_t)pix * C + c0;
-    for (int c = 0; c < cn; c++) w |= (uint64_t)(src[c] < 0.0f) << c;
+    const T* src = x + (size_t)pix * C + c0;
+    for (int c = 0; c < cn; c++) w |= (uint64_t)neg(src[c]) << c;
   } else {
     const long long n = pix / HW, hw = pix % HW;
-    const float* src = x + ((size_t)n * C + c0) * HW + hw;
-    for (int c = 0; c < cn; c++) w |= (uint64_t)(src[(size_t)c * HW] < 0.0f) << c;
+    const T* src = x + ((size_t)n * C + c0) * HW + hw;
+    for (int c = 0; c < cn; c++) w |= (uint64_t)neg(src[(size_t)c * HW]) << c;
   }
   packed[t] = w;
 }
 
 // NHWC with C a multiple of 64 and 16-byte aligned input: 16 lanes share one word; each lane tests 4
 // channels (one float4), places its nibble, and an OR-reduction over 8-lane groups builds each half.
-__global__ void __launch_bounds__(256) pack_nhwc_c64(const float* __restrict__ x, long long total_words,
+template <typename T>
+__global__ void __launch_bounds__(256) pack_nhwc_c64(const T* __restrict__ x, long long total_words,
                                                      uint64_t* __restrict__ packed) {
   const int lane = threadIdx.x & 31;
   const long long warp_global = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
   const unsigned gmask = 0xFFu << (lane & 24);  // this lane's 8-lane group
+  using V4 = typename Vec4<T>::type;
   // a warp handles 2 words (128 floats) per step; 4 steps in flight per iteration
   for (long long w0 = warp_global * 8; w0 < total_words; w0 += nwarps * 8) {
-    float4 v[4];
+    V4 v[4];
 #pragma unroll
     for (int u = 0; u < 4; u++) {
       const long long word = w0 + 2 * u + (lane >> 4);
-      v[u] = (word < total_words) ? __ldcs(reinterpret_cast<const float4*>(x) + word * 16 + (lane & 15))
-                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+      v[u] = V4{0, 0, 0, 0};
+      if (word < total_words) v[u] = __ldcs(reinterpret_cast<const V4*>(x) + word * 16 + (lane & 15));
     }
 #pragma unroll
     for (int u = 0; u < 4; u++) {
-      unsigned nib = (unsigned)(v[u].x < 0.0f) | ((unsigned)(v[u].y < 0.0f) << 1) |
-                     ((unsigned)(v[u].z < 0.0f) << 2) | ((unsigned)(v[u].w < 0.0f) << 3);
+      unsigned nib = neg(v[u].x) | (neg(v[u].y) << 1) | (neg(v[u].z) << 2) | (neg(v[u].w) << 3);
       unsigned half = __reduce_or_sync(gmask, nib << (4 * (lane & 7)));  // 32 channels of this 8-lane group
       unsigned other = __shfl_xor_sync(0xFFFFFFFFu, half, 8);            // the other half of the word
       const long long word = w0 + 2 * u + (lane >> 4);
@@ -186,8 +203,8 @@ __global__ void pack_weights_kernel(const float* __restrict__ w, int O, int C, i
 
 using namespace dabnn;
 
-extern "C" dabnn_status dabnn_pack(const float* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed,
-                                   void* stream) {
+template <typename T>
+dabnn_status pack_any(const T* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed, void* stream) {
   if (!x || !packed) return DABNN_ERR_NULL;
   if (s.N <= 0 || s.C <= 0 || s.H <= 0 || s.W <= 0) return DABNN_ERR_SHAPE;
   if (in_layout != DABNN_NCHW && in_layout != DABNN_NHWC) return DABNN_ERR_SHAPE;
@@ -199,23 +216,33 @@ extern "C" dabnn_status dabnn_pack(const float* x, dabnn_layout in_layout, dabnn
   cudaStream_t st = as_stream(stream);
   if (in_layout == DABNN_NCHW && HW % 4 == 0 && aligned(x, 16) && s.N <= 65535 && Cw * 128 * 8 <= 48 * 1024) {
     dim3 grid(ceil_div(HW, 128), s.N);
-    pack_nchw_vec4<<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, packed);
+    pack_nchw_vec4<T><<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, packed);
   } else if (in_layout == DABNN_NCHW && s.N <= 65535 && Cw <= 65535) {
     dim3 grid(ceil_div(HW, 128), s.N, (unsigned)Cw);
-    pack_nchw_tile<<<grid, 256, 0, st>>>(x, s.C, (int)HW, (int)Cw, packed);
+    pack_nchw_tile<T><<<grid, 256, 0, st>>>(x, s.C, (int)HW, (int)Cw, packed);
   } else if (in_layout == DABNN_NHWC && s.C % 64 == 0 && aligned(x, 16)) {
     const long long warps_needed = (total_words + 7) / 8;
     long long blocks = (warps_needed + 7) / 8;
     const long long cap = (long long)sm_count() * 16;
     if (blocks > cap) blocks = cap;
-    pack_nhwc_c64<<<(unsigned)blocks, 256, 0, st>>>(x, total_words, packed);
+    pack_nhwc_c64<T><<<(unsigned)blocks, 256, 0, st>>>(x, total_words, packed);
   } else {
     const long long blocks = (total_words + 255) / 256;
     if (blocks > 0x7FFFFFFF) return DABNN_ERR_UNSUPPORTED;
-    pack_generic<<<(unsigned)blocks, 256, 0, st>>>(x, in_layout == DABNN_NHWC, s.C, (int)HW, (int)Cw, total_words,
+    pack_generic<T><<<(unsigned)blocks, 256, 0, st>>>(x, in_layout == DABNN_NHWC, s.C, (int)HW, (int)Cw, total_words,
                                                    packed);
   }
   return launch_status();
+}
+
+extern "C" dabnn_status dabnn_pack(const float* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed,
+                                   void* stream) {
+  return pack_any<float>(x, in_layout, s, packed, stream);
+}
+
+extern "C" dabnn_status dabnn_pack_i32(const int32_t* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed,
+                                       void* stream) {
+  return pack_any<int32_t>(x, in_layout, s, packed, stream);
 }
 
 extern "C" dabnn_status dabnn_pack_weights(const float* w_oihw, int O, int C, int kh, int kw, uint64_t* wpacked,

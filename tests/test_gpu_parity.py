@@ -64,6 +64,34 @@ def test_pack_nhwc(B, oracle_mod, shape):
     assert np.array_equal(got, oracle_mod.pack(x, oracle_mod.NHWC))
 
 
+@pytest.mark.parametrize("shape", PACK_SHAPES)
+def test_pack_i32_nchw(B, oracle_mod, shape):
+    rng = np.random.default_rng(sum(shape) + 2)
+    x = rng.integers(-2**31, 2**31, size=shape, dtype=np.int64).astype(np.int32)
+    x[rng.random(shape) < 0.05] = 0
+    got = u64(B.pack_i32(dev(x), B.NCHW))
+    assert np.array_equal(got, oracle_mod.pack_i32(x, oracle_mod.NCHW))
+
+
+@pytest.mark.parametrize("shape", [(2, 14, 14, 64), (3, 9, 7, 256), (2, 5, 5, 70), (4, 31, 17, 128)])
+def test_pack_i32_nhwc(B, oracle_mod, shape):
+    rng = np.random.default_rng(sum(shape) + 3)
+    x = rng.integers(-50, 50, size=shape).astype(np.int32)
+    got = u64(B.pack_i32(dev(x), B.NHWC))
+    assert np.array_equal(got, oracle_mod.pack_i32(x, oracle_mod.NHWC))
+
+
+def test_pack_i32_of_conv_sums_equals_fused_sign(B, oracle_mod):
+    """Binarizing a convolution's int32 sums with the int32 packer = the fused epilogue with scale 1, shift 0."""
+    x, w = synth.conv_case(1, 2, 128, 9, 11, 128, 3, 3)
+    a = B.pack(dev(x))
+    wp = B.pack_weights(dev(w))
+    sums = B.bconv2d(a, 128, wp, (1, 1), (1, 1), -1, B.NHWC)
+    ones = torch.ones(128, device=a.device)
+    fused = B.bconv2d_bn_sign_pack(a, 128, wp, ones, torch.zeros_like(ones), (1, 1), (1, 1), -1)
+    assert np.array_equal(u64(B.pack_i32(sums, B.NHWC)), u64(fused))
+
+
 def test_pack_unaligned_input_takes_the_generic_path(B, oracle_mod):
     rng = np.random.default_rng(8)
     buf = rng.standard_normal(1 + 2 * 64 * 8 * 8).astype(np.float32)

@@ -57,6 +57,27 @@ def test_unpack_matches_comparison(oracle_mod, shape):
     assert np.array_equal(P, P2)
 
 
+def test_int32_sign_bits(oracle_mod):
+    """int32 input: the packed bit is the integer's sign bit (two's complement top bit), independently extracted here."""
+    o = oracle_mod
+    vals = [0, 1, -1, 2**31 - 1, -2**31, 5, -5, 7]
+    x = np.asarray(vals, dtype=np.int32).reshape(1, len(vals), 1, 1)
+    word = int(o.pack_i32(x, o.NCHW).reshape(-1)[0])
+    assert [(word >> i) & 1 for i in range(len(vals))] == [0, 0, 1, 0, 1, 0, 1, 0]
+    rng = np.random.default_rng(5)
+    shape = (2, 130, 3, 5)
+    x = rng.integers(-2**31, 2**31, size=shape, dtype=np.int64).astype(np.int32)
+    x[rng.random(shape) < 0.1] = 0
+    P = o.pack_i32(x, o.NCHW)
+    bits, tail = unpack_words(P, shape[1])
+    top_bit = (np.transpose(x, (0, 2, 3, 1)).view(np.uint32) >> np.uint32(31)).astype(np.uint8)
+    assert np.array_equal(bits, top_bit) and not tail.any()
+    assert np.array_equal(P, o.pack_i32(np.ascontiguousarray(np.transpose(x, (0, 2, 3, 1))), o.NHWC))
+    # where floats represent the integers exactly (|x| < 2^24) both packers agree
+    small = rng.integers(-1000, 1000, size=shape).astype(np.int32)
+    assert np.array_equal(o.pack_i32(small, o.NCHW), o.pack(small.astype(np.float32), o.NCHW))
+
+
 def test_size_is_32x_smaller(oracle_mod):
     # one bit per fp32 element (Section 3: packed weights are 32x smaller)
     o = oracle_mod
