@@ -121,3 +121,37 @@ def test_tc_full_size_configs_on_sampled_outputs(B, oracle_mod, cfg):
     want = oracle_mod.bconv_pm1_at(x, w, coords, (1, 1), (pad, pad), -1)
     assert np.array_equal(g[coords[:, 0], coords[:, 2], coords[:, 3], coords[:, 1]], want)
     assert B.tc_error_flag() == 0
+
+
+_FORCED_FORM_SCRIPT = r"""
+import sys, numpy as np, torch
+from paper_1908_05858_b200 import binding as B
+import oracle as o
+o.set_threads(o.max_threads())
+rng = np.random.default_rng(77)
+cases = [(3, 64, 14, 14, 64, 3, 1, -1, 1), (40, 256, 14, 14, 256, 3, 1, -1, 1), (9, 512, 7, 7, 512, 3, 1, +1, 1),
+         (2, 192, 10, 10, 70, 5, 2, -1, 1), (6, 128, 28, 28, 256, 3, 1, -1, 2), (2, 448, 10, 10, 70, 3, 1, -1, 1)]
+for N, C, H, W, O, k, pad, pv, st in cases:
+    x = rng.standard_normal((N, C, H, W)).astype(np.float32); w = rng.standard_normal((O, C, k, k)).astype(np.float32)
+    want = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (st, st), (pad, pad), pv, o.NHWC)
+    a = B.pack(torch.from_numpy(x).cuda()); wt = B.TcWeights(B.pack_weights(torch.from_numpy(w).cuda()), C)
+    got = B.tc_bconv2d(a, wt, (st, st), (pad, pad), pv, B.NHWC).cpu().numpy()
+    assert np.array_equal(got, want), (N, C, H, W, O, k)
+    sc = torch.from_numpy(rng.uniform(0.5, 1.5, O).astype(np.float32)).cuda(); sh = torch.from_numpy(rng.normal(0, 3, O).astype(np.float32)).cuda()
+    bits = B.tc_bconv2d_bn_sign_pack(a, wt, sc, sh, (st, st), (pad, pad), pv).cpu().numpy().view(np.uint64)
+    assert np.array_equal(bits, o.bn_sign_pack(want, sc.cpu().numpy(), sh.cpu().numpy())), (N, C, H, W, O, k)
+torch.cuda.synchronize()
+assert B.tc_error_flag() == 0
+print("forced form ok")
+"""
+
+
+@pytest.mark.parametrize("mode", ["1", "2"])
+def test_both_launch_forms_in_a_child_process(mode):
+    """The launch form is chosen by size; DABNN_TC_MODE (read once per process) forces one CTA per tile (1) or CTA
+    pairs (2), so each form is run on the same cases in a child process and compared with the oracle."""
+    import os, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, DABNN_TC_MODE=mode, PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
+    r = subprocess.run([sys.executable, "-c", _FORCED_FORM_SCRIPT], env=env, cwd=root, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "forced form ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
