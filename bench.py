@@ -338,7 +338,7 @@ def main():
         "bound": "tensor", "kernel": "bconv_tc_kernel (the 8 convolution launches of a step, one CUDA-graph replay)",
         "achieved": conv_ops / (tc_ms * 1e-3) / 1e12, "peak": tensor_peak["tops"], "unit": "TFLOP/s",
         "frac": conv_ops / (tc_ms * 1e-3) / 1e12 / tensor_peak["tops"], "peak_is": tensor_peak["how"],
-        "traffic": 4.15e6, "traffic_is": "dram bytes of one N=64 C=256 28x28 launch (ncu, profiles/bconv_tc_kernel_N64_C256_HW28.md); its int32 output (51 MB) is still in L2 when the kernel ends",
+        "traffic": 4.52e6, "traffic_is": "dram bytes of one N=64 C=256 28x28 launch (ncu, profiles/bconv_tc_kernel_N64_C256_HW28.md); most of its int32 output (51 MB, evict-first) is still in L2 when the kernel ends",
         "avg_launch_ms": tc_ms / 8, "conv_share_of_step": tc_ms / (total_ms / args.steps),
         "note": "1 bit-op = 1 op: a +-1 multiply-add counts 2, as in FLOPs",
     }
@@ -469,6 +469,31 @@ def extras(B, torch, dev, peaks, sm_count):
         med, best = time_fn(lambda: B.tc_bconv2d(a, wt, (1, 1), (pad, pad), -1, B.NHWC, out=o), 10, flush)
         out[name]["tensor"] = {"ms": med, "Tbit-ops/s": ops / med / 1e9, "frac_of_fp4_peak": ops / med / 1e9 / tpeak}
         del a, w, o, wt
+
+    # BGEMM against direct convolution, the comparison of the paper's Fig. 4, on config 5a: the im2col matrix of the packed
+    # activations (padding taps hold the pad word) is materialised with torch slicing (plumbing, 58 MB of packed rows) and
+    # multiplied by dabnn_bgemm; dabnn_bconv2d gathers the same rows on the fly (implicit BGEMM)
+    N, C, HW, O = 256, 256, 28, 256
+    g = torch.Generator(device=dev); g.manual_seed(9)
+    a = torch.randint(-2**62, 2**62, (N, HW, HW, C // 64), dtype=torch.int64, device=dev, generator=g)
+    w = torch.randint(-2**62, 2**62, (O, 3, 3, C // 64), dtype=torch.int64, device=dev, generator=g)
+
+    def im2col():
+        ap = torch.nn.functional.pad(a, (0, 0, 1, 1, 1, 1), value=-1)  # pad word: all bits set = -1 everywhere
+        return torch.stack([ap[:, i:i + HW, j:j + HW, :] for i in range(3) for j in range(3)], dim=3).reshape(N * HW * HW, 9 * (C // 64))
+    A = im2col()
+    Bm = w.reshape(O, 9 * (C // 64))
+    direct = B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC)
+    same = bool((B.bgemm(A, Bm, 9 * C).reshape(N, HW, HW, O) == direct).all())
+    ops = conv_bitops(N, C, HW, O, 3)
+    t_gemm, _ = time_fn(lambda: B.bgemm(A, Bm, 9 * C), 5, flush)
+    t_both, _ = time_fn(lambda: B.bgemm(im2col(), Bm, 9 * C), 5, flush)
+    t_direct, _ = time_fn(lambda: B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC, out=direct), 5, flush)
+    out["bgemm_vs_direct_256x256x28x28"] = {"identical": same, "bgemm_ms": t_gemm, "im2col_plus_bgemm_ms": t_both,
+                                            "direct_ms": t_direct, "direct_Tbit-ops/s": ops / t_direct / 1e9,
+                                            "bgemm_Tbit-ops/s": ops / t_gemm / 1e9,
+                                            "note": "integer-pipe engine for both; im2col is torch slicing, not a tuned kernel"}
+    del a, w, A, Bm, direct
 
     # batch-1 latency of the four sweep shapes (CUDA-graph replay of 50 launches)
     for C, HW in synth.SWEEP_SHAPES:
