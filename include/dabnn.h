@@ -164,7 +164,11 @@ dabnn_status dabnn_bireal18_forward_static(const dabnn_bireal18_params* p, const
  *     packed result [N][OH][OW][ceil(O/64)] to bits_host.
  * w_packed, scale, shift and workspace are DEVICE pointers; workspace must be 256-byte aligned and hold at least
  * dabnn_binary_layer_host_workspace_bytes(in, O, cv) bytes (0 is returned for an invalid geometry).
- * Everything is enqueued on `stream`; the host results are complete once the stream has been synchronised. */
+ * The batch is processed in up to four chunks whose copies run on two internal copy streams (created per device on first
+ * use, kept until exit), so that the copy in, the kernels and the copy out of different chunks overlap; `stream` waits for
+ * all of it: the host results are complete once `stream` has been synchronised.  x_host must hold its data when the
+ * function is called (its copy may start before earlier work on `stream` has finished).  Not thread-safe against
+ * concurrent calls on the same device; calls that share a workspace belong on one stream. */
 size_t dabnn_binary_layer_host_workspace_bytes(dabnn_shape in, int O, dabnn_conv cv);
 dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const uint64_t* w_packed, int O, dabnn_conv cv,
                                      const float* scale, const float* shift, int32_t* out_host, uint64_t* bits_host,

@@ -297,3 +297,32 @@ def test_bireal18_large_batch_kernels_match_oracle(B, oracle_mod):
     assert np.array_equal(got.argmax(axis=1), want.argmax(axis=1))
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
     assert B.tc_error_flag() == 0
+
+
+@pytest.mark.parametrize("N,pinned", [(1, True), (3, True), (5, False), (9, True)])
+def test_binary_layer_host_matches_oracle(B, oracle_mod, N, pinned):
+    """The host-buffer entry point (chunked, copies on side streams): int32 sums and fused sign words against the oracle,
+    called twice in a row on the same workspace with different inputs, results read after one stream synchronisation."""
+    o = oracle_mod
+    C, H, W, O = 128, 9, 11, 70
+    rng = np.random.default_rng(N)
+    w = rng.standard_normal((O, C, 3, 3)).astype(np.float32)
+    scale_np, shift_np = rng.uniform(0.5, 1.5, O).astype(np.float32), rng.normal(0, 5, O).astype(np.float32)
+    wp = B.pack_weights(dev(w))
+    scale, shift = dev(scale_np), dev(shift_np)
+    ws = torch.empty(B.binary_layer_host_workspace_bytes(N, C, H, W, O, 3, 3, (1, 1), (1, 1), -1), dtype=torch.uint8, device="cuda")
+    runs = []
+    for rep in range(2):
+        x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+        xh = torch.from_numpy(x)
+        out_h = torch.empty((N, H, W, O), dtype=torch.int32)
+        bits_h = torch.empty((N, H, W, 2), dtype=torch.int64)
+        if pinned:
+            xh, out_h, bits_h = xh.pin_memory(), out_h.pin_memory(), bits_h.pin_memory()
+        B.binary_layer_host(xh, wp, ws, (1, 1), (1, 1), -1, scale, shift, out_host=out_h, bits_host=bits_h)
+        runs.append((x, out_h, bits_h, xh))
+    torch.cuda.synchronize()
+    for x, out_h, bits_h, _ in runs:
+        want = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (1, 1), (1, 1), -1, o.NHWC)
+        assert np.array_equal(out_h.numpy(), want)
+        assert np.array_equal(bits_h.numpy().view(np.uint64), o.bn_sign_pack(want, scale_np, shift_np))
