@@ -31,6 +31,20 @@ __global__ void bn_fold_kernel(const float* gamma, const float* beta, const floa
 // fmaf(0, w, acc) returns acc.
 constexpr int STEM_K = 147;
 
+// Two fp32 fused multiply-adds in one instruction (fma.rn.f32x2): each lane of the pair is the same correctly rounded
+// fmaf as the scalar instruction, so results do not change; it halves the issue slots of an FMA-bound loop.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma_f32x2(unsigned long long& acc, unsigned long long a, unsigned long long b) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+
 template <int TS, int PPT>
 __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const float* __restrict__ img,
                                                                        const float* __restrict__ w,
@@ -86,11 +100,11 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
     __syncthreads();  // this tile's patch (and, the first time, the weights) are in place; the other buffer is free
     if (tile + gridDim.x < ntiles) load_patch(tile + gridDim.x, x_s + (buf ^ 1) * PATCH);
     const float* xb = x_s + buf * PATCH;
-    float acc[PPT][16];
+    unsigned long long acc2[PPT][8];  // channel pairs (packed fp32 FMAs, same rounding as scalar fmaf)
 #pragma unroll
     for (int i = 0; i < PPT; i++)
 #pragma unroll
-      for (int j = 0; j < 16; j++) acc[i][j] = 0.0f;
+      for (int j = 0; j < 8; j++) acc2[i][j] = 0ull;
 #pragma unroll 1
     for (int c = 0; c < 3; c++)
 #pragma unroll 1
@@ -98,21 +112,28 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
 #pragma unroll
         for (int kj = 0; kj < 7; kj++) {
           const int k = (c * 7 + ki) * 7 + kj;
-          float wv[16];
+          unsigned long long w2[8];
 #pragma unroll
           for (int q = 0; q < 4; q++) {
             const float4 t4 = *reinterpret_cast<const float4*>(w_s + k * 64 + cg * 16 + 4 * q);
-            wv[4 * q] = t4.x; wv[4 * q + 1] = t4.y; wv[4 * q + 2] = t4.z; wv[4 * q + 3] = t4.w;
+            w2[2 * q] = pack_f32x2(t4.x, t4.y);
+            w2[2 * q + 1] = pack_f32x2(t4.z, t4.w);
           }
 #pragma unroll
           for (int i = 0; i < PPT; i++) {
             const int lh = 2 * (lohb + RSTEP * i) + ki;
             const float xv = xb[((c * PS + lh) * 2 + (kj & 1)) * HALF + low + (kj >> 1)];
+            const unsigned long long x2 = pack_f32x2(xv, xv);
 #pragma unroll
-            for (int j = 0; j < 16; j++) acc[i][j] = __fmaf_rn(xv, wv[j], acc[i][j]);
+            for (int j = 0; j < 8; j++) fma_f32x2(acc2[i][j], x2, w2[j]);
           }
         }
       }
+    float acc[PPT][16];
+#pragma unroll
+    for (int i = 0; i < PPT; i++)
+#pragma unroll
+      for (int j = 0; j < 8; j++) unpack_f32x2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
     const int n = (int)(tile / (TILES * TILES));
     const int rem = (int)(tile % (TILES * TILES));
     const int oh0 = (rem / TILES) * TS, ow0 = (rem % TILES) * TS;
@@ -129,20 +150,6 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
     }
   }
   asm volatile("cp.async.wait_group 0;" ::: "memory");
-}
-
-// Two fp32 fused multiply-adds in one instruction (fma.rn.f32x2): each lane of the pair is the same correctly rounded
-// fmaf as the scalar instruction, so results do not change; it halves the issue slots of an FMA-bound loop.
-__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
-  unsigned long long r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ void fma_f32x2(unsigned long long& acc, unsigned long long a, unsigned long long b) {
-  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
 }
 
 // Large batches: the same convolution with an 8 pixels (along a row) x 8 channels register tile.  Per (c, kh) a thread
