@@ -42,12 +42,14 @@ enum { EPI_I32 = 0, EPI_BNPACK = 1, EPI_BIREAL = 2 };
 constexpr int TC_THREADS = 416;           // warps 0-3 and (optionally) 8-11: epilogue, 4-7: producers, 12: MMA issue
 constexpr int TC_SMEM_LIMIT = 232448;     // 227 KB opt-in maximum per CTA
 constexpr int TC_MAX_RES = 4;              // channel tiles resident per CTA (pair) at most
-constexpr int TC_SMEM_MISC = 128 + 2 * TC_MAX_RES * 128 * 4;  // barriers, TMEM base, flags; this CTA's scale / shift
+constexpr int TC_SMEM_MISC = 256 + 2 * TC_MAX_RES * 128 * 4;  // barriers, TMEM base, flags; this CTA's scale / shift
 constexpr int TC_WEIGHT_BUDGET = 147456;  // 144 KB of resident weights at most
 constexpr int TC_MAX_CW = 8;              // C <= 512
 constexpr int TC_MAX_SPT = 5;             // slots per producer thread: 2 for stride 1, up to 5 for stride 2
 constexpr int TC_TMEM_COLS = 512;         // 2 accumulators (<= 128 columns each) + the scale-factor columns
-constexpr int TC_SF_COL = 256;            // columns [256, 512) hold scale factors (all 1.0)
+constexpr int TC_ACC_COLS = 384;          // columns [0, 384): up to four accumulators (three of 128 columns)
+constexpr int TC_SF_COL = 384;            // columns [384, 512) hold scale factors (all 1.0)
+constexpr int TC_MAX_BUFS = 4;            // accumulators / activation buffers in flight at most
 
 __device__ int g_tc_error = 0;  // 1: an mbarrier wait ran out
 #ifdef TC_TIMING
@@ -69,7 +71,8 @@ struct TcArgs {
   unsigned long long magic_sp, magic_hp;  // ceil(2^64 / SP), ceil(2^64 / HP) (0 when the divisor is 1)
   int slots_p;         // slots per parity plane and tile, multiple of 8
   int slots;           // S*S*slots_p: rows of one 32-channel group in an A buffer
-  int abufs;           // A buffers in shared memory (1 or 2)
+  int abufs;           // A buffers in shared memory (1 to 4)
+  int nacc;            // accumulators in tensor memory (2 to 4: as many as fit 384 columns)
   int ntile, n_ntiles; // output channels per MMA (N), number of such channel tiles
   int pair;            // 1: CTA pairs (cta_group::2), each CTA holds ntile / 2 weight rows per channel tile
   int nres, n_groups;  // channel tiles resident per CTA (pair), groups of `nres` channel tiles
@@ -224,12 +227,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   uint8_t* w_s = smem;                                   // [nres][taps][C/32][WR][16]
   uint8_t* a_s = smem + (size_t)g.nres * WR * Kb;        // [abufs][C/32][slots][16]
   uint8_t* misc = a_s + (size_t)g.abufs * a_bytes;
-  // [0,1] mma_done  [2,3] tmem_free  [4,5] a_full  [6] w_full (first third of the filter taps)  [7,8] a_free
-  // [9,10] w_full (second and last third); of a pair, the leader's tmem_free, a_full and w_full are used
+  // [0..3] mma_done  [4..7] tmem_free  [8..11] a_full  [12..15] a_free  [16..18] w_full (thirds of the filter taps);
+  // of a pair, the leader's tmem_free, a_full and w_full are used
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 96);
-  volatile int* s_fail = reinterpret_cast<volatile int*>(misc + 104);
-  float* s_scale = reinterpret_cast<float*>(misc + 128);     // [nres][NT] this CTA's channels
+  constexpr int B_MMA_DONE = 0, B_TMEM_FREE = 4, B_A_FULL = 8, B_A_FREE = 12, B_W_FULL = 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 160);
+  volatile int* s_fail = reinterpret_cast<volatile int*>(misc + 168);
+  float* s_scale = reinterpret_cast<float*>(misc + 256);     // [nres][NT] this CTA's channels
   float* s_shift = s_scale + TC_MAX_RES * NT;                // [nres][NT]
 
   // work: CTA (pair) `unit` takes channel-tile group `ng` and every `unit_step`-th tile (pair of tiles) of 128 slots
@@ -250,17 +254,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     }
   }
   if (tid == 0) {
-    mbar_init(smem_u32(&bars[0]), 1);
-    mbar_init(smem_u32(&bars[1]), 1);
-    mbar_init(smem_u32(&bars[2]), (g.epi2 ? 256 : 128) * PEERS);
-    mbar_init(smem_u32(&bars[3]), (g.epi2 ? 256 : 128) * PEERS);
-    mbar_init(smem_u32(&bars[4]), 128 * PEERS);
-    mbar_init(smem_u32(&bars[5]), 128 * PEERS);
-    mbar_init(smem_u32(&bars[6]), TC_THREADS * PEERS);
-    mbar_init(smem_u32(&bars[7]), 1);
-    mbar_init(smem_u32(&bars[8]), 1);
-    mbar_init(smem_u32(&bars[9]), TC_THREADS * PEERS);
-    mbar_init(smem_u32(&bars[10]), TC_THREADS * PEERS);
+    for (int i = 0; i < TC_MAX_BUFS; i++) {
+      mbar_init(smem_u32(&bars[B_MMA_DONE + i]), 1);
+      mbar_init(smem_u32(&bars[B_TMEM_FREE + i]), (g.epi2 ? 256 : 128) * PEERS);
+      mbar_init(smem_u32(&bars[B_A_FULL + i]), 128 * PEERS);
+      mbar_init(smem_u32(&bars[B_A_FREE + i]), 1);
+    }
+    for (int i = 0; i < 3; i++) mbar_init(smem_u32(&bars[B_W_FULL + i]), TC_THREADS * PEERS);
     *s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -289,9 +289,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   const bool is_producer = warp >= 4 && warp < 8;
   uint32_t tmem_base = 0;
   // barriers that both CTAs of a pair signal live in the leader
-  const uint32_t bar_tmem_free0 = PAIR ? leader_addr(smem_u32(&bars[2])) : smem_u32(&bars[2]);
-  const uint32_t bar_a_full0 = PAIR ? leader_addr(smem_u32(&bars[4])) : smem_u32(&bars[4]);
-  const uint32_t bar_w_full = PAIR ? leader_addr(smem_u32(&bars[6])) : smem_u32(&bars[6]);  // + 24, + 32: the later thirds
+  const uint32_t bar_tmem_free0 = PAIR ? leader_addr(smem_u32(&bars[B_TMEM_FREE])) : smem_u32(&bars[B_TMEM_FREE]);
+  const uint32_t bar_a_full0 = PAIR ? leader_addr(smem_u32(&bars[B_A_FULL])) : smem_u32(&bars[B_A_FULL]);
+  const uint32_t bar_w_full = PAIR ? leader_addr(smem_u32(&bars[B_W_FULL])) : smem_u32(&bars[B_W_FULL]);  // + 8, + 16: the later thirds
   auto arrive = [&](uint32_t bar) {
     if (PAIR) mbar_arrive_cluster(bar);
     else mbar_arrive(bar);
@@ -325,10 +325,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     arrive(bar_w_full);
     asm volatile("cp.async.wait_group 1;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    arrive(bar_w_full + 24u);
+    arrive(bar_w_full + 8u);
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    arrive(bar_w_full + 32u);
+    arrive(bar_w_full + 16u);
   };
   if (!is_producer) {
     prologue_sync();
@@ -361,13 +361,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
                              | ((uint32_t)(NT >> 3) << 17)   // N
                              | (1u << 23)                    // scale factors: ue8m0
                              | ((uint32_t)((PAIR ? 256 : 128) >> 4) << 24);  // M; both operands K-major; K = 64
-      const uint32_t tsfa = tmem_base + TC_SF_COL, tsfb = tmem_base + TC_SF_COL + 128;
+      const uint32_t tsfa = tmem_base + TC_SF_COL, tsfb = tmem_base + TC_SF_COL + 64;
       const uint64_t bdesc0 = make_desc(smem_u32(w_s), (uint32_t)WR * 16, 128);
       const uint32_t desc_hi = (uint32_t)(bdesc0 >> 32);  // same for A and B: core matrices 128 bytes apart along M / N
       const uint32_t b_lo0 = (uint32_t)bdesc0;
-      uint32_t a_lo_buf[2];
-      a_lo_buf[0] = (uint32_t)make_desc(smem_u32(a_s), (uint32_t)g.slots * 16, 128);
-      a_lo_buf[1] = (uint32_t)make_desc(smem_u32(a_s + a_bytes), (uint32_t)g.slots * 16, 128);
+      const uint32_t a_lo_first = (uint32_t)make_desc(smem_u32(a_s), (uint32_t)g.slots * 16, 128);
+      const uint32_t a_buf_units = (uint32_t)a_bytes >> 4;  // one A buffer, in 16-byte units
       const uint32_t a_step = 2u * (uint32_t)g.slots;  // one K = 64 block of A, in 16-byte units
       constexpr uint32_t b_step = 2u * WR;             // weights are laid out in issue order: [tile][tap][C/32][WR][16]
       const uint32_t b_tile = (uint32_t)(g.kh * g.kw * g.Cw) * b_step;  // one resident channel tile
@@ -420,14 +419,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         if (k3) {
 #pragma unroll
           for (int t = 0; t < 9; t++) {
-            if (first && (t == 3 || t == 6) && !wait(smem_u32(&bars[t == 3 ? 9 : 10]), 0)) *s_fail = 1;  // that row of taps
+            if (first && (t == 3 || t == 6) && !wait(smem_u32(&bars[B_W_FULL + t / 3]), 0)) *s_fail = 1;  // that row of taps
             const uint32_t a_lo = a_lo0 + off9[t];
 #pragma unroll
             for (int kb = 0; kb < KB; kb++)
               mma(d_tmem, a_lo + (uint32_t)kb * a_stp, b_base + (uint32_t)(t * KB + kb) * b_step, (t | kb) ? 1u : 0u);
           }
         } else {
-          if (first && !(wait(smem_u32(&bars[9]), 0) && wait(smem_u32(&bars[10]), 0))) *s_fail = 1;
+          if (first && !(wait(smem_u32(&bars[B_W_FULL + 1]), 0) && wait(smem_u32(&bars[B_W_FULL + 2]), 0))) *s_fail = 1;
           uint32_t b_lo = b_base, accumulate = 0;
           for (int ti = 0; ti < g.kh; ti++)
             for (int tj = 0; tj < g.kw; tj++) {
@@ -441,24 +440,25 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         }
       };
       uint32_t ab = 0, a_phase = 0;  // A buffer of this tile and the parity of its `a_full` phase
+      uint32_t accb = 0, acc_phase = 0;  // accumulator of this round and the parity of its uses so far
       int ar = 0;                    // accumulator rounds so far: one per (tile, resident channel tile)
-      bool ok = wait(smem_u32(&bars[6]), 0);  // resident weights and scale factors
+      bool ok = wait(smem_u32(&bars[B_W_FULL]), 0);  // first third of the resident weights, and the scale factors
       if (!ok) *s_fail = 1;
 #pragma unroll 1
       for (long long mt = mt_first; mt < mt_end && ok; mt += mt_step) {
         TC_T(0);
-        if (!wait(smem_u32(&bars[4 + ab]), a_phase)) { *s_fail = 1; break; }  // rows written
+        if (!wait(smem_u32(&bars[B_A_FULL + ab]), a_phase)) { *s_fail = 1; break; }  // rows written
         TC_T(1);
-        const uint32_t a_lo0 = ab ? a_lo_buf[1] : a_lo_buf[0];
+        const uint32_t a_lo0 = a_lo_first + ab * a_buf_units;
         // (opaque to the compiler, so that it does not keep every tap's and K block's offset in a register of its own
         // across tiles: the sums are recomputed per tile, one add each)
         uint32_t a_step_t = a_step;
         asm volatile("" : "+r"(a_step_t));
 #pragma unroll 1
         for (int r = 0; r < nres_here; r++, ar++) {
-          if (ar >= 2 && !wait(smem_u32(&bars[2 + (ar & 1)]), ((ar - 2) >> 1) & 1)) { *s_fail = 1; ok = false; break; }  // accumulator drained
+          if (ar >= g.nacc && !wait(smem_u32(&bars[B_TMEM_FREE + accb]), acc_phase ^ 1u)) { *s_fail = 1; ok = false; break; }  // accumulator drained
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t d_tmem = tmem_base + (uint32_t)((ar & 1) * NT);
+          const uint32_t d_tmem = tmem_base + accb * (uint32_t)NT;
           const uint32_t b_base = b_lo0 + (uint32_t)r * b_tile;
           switch (g.Cw) {  // C / 64 = 1..8
             case 1: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<1>{}); break;
@@ -470,11 +470,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
             case 7: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<7>{}); break;
             default: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<8>{}); break;
           }
-          commit(smem_u32(&bars[ar & 1]));
+          commit(smem_u32(&bars[B_MMA_DONE + accb]));
+          if (++accb == (uint32_t)g.nacc) { accb = 0; acc_phase ^= 1u; }
         }
-        commit(smem_u32(&bars[7 + ab]));  // the tile's rows have been read: the A buffer may be refilled
+        commit(smem_u32(&bars[B_A_FREE + ab]));  // the tile's rows have been read: the A buffer may be refilled
         TC_T(3);
-        if (g.abufs == 2) { a_phase ^= ab; ab ^= 1u; } else { a_phase ^= 1u; }
+        if (++ab == (uint32_t)g.abufs) { ab = 0; a_phase ^= 1u; }
       }
 #ifdef TC_TIMING
       if (blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[16 + i] = prof[i]; }
@@ -569,13 +570,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       prefetch(cur, cwc);  // (rows of a tile beyond the last one are beyond the batch: nothing is read for them)
       if (TWO_SETS) prefetch(nxt, cwc);
       prologue_sync();
+      uint32_t ab = 0, use_phase = 0;  // A buffer of this tile and the parity of the number of times it has been filled
 #pragma unroll 1
       for (; mt < mt_end; mt += mt_step, it++) {
-        const int ab = g.abufs == 2 ? (it & 1) : 0;
-        const int use = g.abufs == 2 ? (it >> 1) : it;  // how often this A buffer has been filled before
         TC_T(0);
         // its last reader: all MMAs of the tile that used it, signalled through `a_free` (in both CTAs of a pair)
-        if (use > 0 && !mbar_wait(smem_u32(&bars[7 + ab]), (uint32_t)(use - 1) & 1, s_fail)) { *s_fail = 1; break; }
+        if (it >= g.abufs && !mbar_wait(smem_u32(&bars[B_A_FREE + ab]), use_phase ^ 1u, s_fail)) { *s_fail = 1; break; }
         TC_T(1);
         expand(cur, a_s + (size_t)ab * a_bytes, cwc);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
@@ -596,6 +596,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         } else {
           prefetch(cur, cwc);
         }
+        if (++ab == (uint32_t)g.abufs) { ab = 0; use_phase ^= 1u; }
       }
     };
     // C is a multiple of 64 up to 512: 1..8 words; the common counts get their own straight-line code
@@ -609,7 +610,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #endif
   } else if (warp < 4 || g.epi2) {
     // ================= epilogue warps: TMEM accumulator -> output ===============================================
-    int ar = 0;  // accumulator rounds so far: one per (tile, resident channel tile)
+    uint32_t accb = 0, acc_phase = 0;  // accumulator of this round (one per tile and resident channel tile), parity of its uses
     bool failed = false;
     // with the second group, two warps share each quarter of the accumulator's rows: warps 0-3 take the even
     // 32-column chunks, warps 8-11 the odd ones
@@ -632,8 +633,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       const bool wide_i32 = EPI == EPI_I32 && !g.out_nchw && (g.O & 7) == 0 && (reinterpret_cast<uintptr_t>(g.out) & 31) == 0;
       const bool wide_y = EPI == EPI_BIREAL && (g.O & 7) == 0 &&
                           ((reinterpret_cast<uintptr_t>(g.residual) | reinterpret_cast<uintptr_t>(g.y_out)) & 31) == 0;
-      for (int r = 0; r < nres_here; r++, ar++) {
-      const int buf = ar & 1;
+      for (int r = 0; r < nres_here; r++) {
+      const uint32_t buf = accb;
       const int nt = ng * g.nres + r;  // this round's channel tile
       const float* r_scale = s_scale + r * NT;
       const float* r_shift = s_shift + r * NT;
@@ -652,7 +653,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       };
       load_res(c_first);
       TC_T(0);
-      if (!mbar_wait(smem_u32(&bars[buf]), (ar >> 1) & 1, s_fail)) {
+      if (!mbar_wait(smem_u32(&bars[B_MMA_DONE + buf]), acc_phase, s_fail)) {
         *s_fail = 1;
         failed = true;
         break;
@@ -756,7 +757,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       }
       // this accumulator buffer may be overwritten by the tile after next
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      arrive(bar_tmem_free0 + 8u * (uint32_t)buf);
+      arrive(bar_tmem_free0 + 8u * buf);
+      if (++accb == (uint32_t)g.nacc) { accb = 0; acc_phase ^= 1u; }
       TC_T(2);
       }
     }
@@ -887,7 +889,9 @@ template <int EPI, bool PAIR>
 dabnn_status tc_dispatch_mode(TcArgs& g, cudaStream_t st) {
   const size_t wr = (size_t)g.ntile / (PAIR ? 2 : 1);
   const size_t wbytes = (size_t)g.nres * wr * g.kh * g.kw * (g.C / 2), abytes = (size_t)g.slots * (g.C / 2);
-  g.abufs = (wbytes + 2 * abytes + TC_SMEM_MISC <= (size_t)TC_SMEM_LIMIT) ? 2 : 1;
+  g.abufs = 1;
+  while (g.abufs < TC_MAX_BUFS && wbytes + (size_t)(g.abufs + 1) * abytes + TC_SMEM_MISC <= (size_t)TC_SMEM_LIMIT) g.abufs++;
+  g.nacc = TC_ACC_COLS / g.ntile < TC_MAX_BUFS ? TC_ACC_COLS / g.ntile : TC_MAX_BUFS;
   const size_t smem = wbytes + g.abufs * abytes + TC_SMEM_MISC;
   if (smem > (size_t)TC_SMEM_LIMIT) return DABNN_ERR_UNSUPPORTED;
   if (g.slots <= 256) {
