@@ -24,9 +24,9 @@
 //   * Stride 2 keeps four parity planes of the padded input; tap (i, j) reads plane (i mod 2, j mod 2) shifted by
 //     (i div 2, j div 2).
 //   * Warp-specialised and mbarrier-driven: four producer warps prefetch the bits two tiles ahead, expand them
-//     (table-free, see expand16) into one of up to two A buffers and arrive on `a_full`; one thread of a
-//     separate warp waits for it, issues kh*kw*(C/64) tcgen05.mma (M = 128, N = NT, K = 64) into one of two TMEM
-//     accumulators per resident channel tile and commits to `mma_done` (and, after the tile's last MMA, to `a_free`);
+//     (table-free, see expand16) into one of up to four A buffers and arrive on `a_full`; one thread of a
+//     separate warp waits for it, issues kh*kw*(C/64) tcgen05.mma (M = 128, N = NT, K = 64) into one of up to four
+//     TMEM accumulators per resident channel tile and commits to `mma_done` (and, after the tile's last MMA, to `a_free`);
 //     four (or eight) epilogue warps wait for that, read the accumulator with tcgen05.ld, write the output form, and hand the
 //     accumulator back through `tmem_free`.
 //
