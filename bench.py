@@ -450,7 +450,22 @@ def extras(B, torch, dev, peaks, sm_count):
     med, best = time_fn(lambda: B.pack(x, B.NCHW, out=packed), 10)
     nbytes = x.numel() * 4 + packed.numel() * 8
     out["pack_128x256x56x56"] = {"ms": med, "GB/s": nbytes / med / 1e6, "frac_of_hbm_peak": nbytes / med / 1e6 / peaks["hbm_gbs"],
-                                 "peak_GB/s": peaks["hbm_gbs"], "peak_source": peaks["source"], "bytes": nbytes}
+                                 "peak_GB/s": peaks["hbm_gbs"], "peak_source": peaks["source"], "bytes": nbytes,
+                                 "how": "one launch per CUDA-event pair (includes the launch gap of a lone kernel)"}
+    # the same launch ten times in one CUDA graph: the 411 MB input is larger than L2, so every launch reads DRAM, and
+    # the gaps between a lone kernel and its events drop out
+    s_pack = torch.cuda.Stream()
+    with torch.cuda.stream(s_pack):
+        B.pack(x, B.NCHW, out=packed)
+        s_pack.synchronize()
+        g_pack = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_pack, stream=s_pack):
+            for _ in range(10):
+                B.pack(x, B.NCHW, out=packed)
+        med10, _ = time_fn(g_pack.replay, 5)
+    out["pack_128x256x56x56_back_to_back"] = {"ms": med10 / 10, "GB/s": nbytes / (med10 / 10) / 1e6,
+                                              "frac_of_hbm_peak": nbytes / (med10 / 10) / 1e6 / peaks["hbm_gbs"]}
+    del g_pack
     del x, packed
 
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
