@@ -337,7 +337,7 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
       const float4* q11 = reinterpret_cast<const float4*>(xq + (size_t)HW * C + C + c);
 #pragma unroll
       for (int h = 0; h < 2; h++) {
-        const float4 a = q00[h], b = q01[h], cc = q10[h], d = q11[h];
+        const float4 a = __ldcs(q00 + h), b = __ldcs(q01 + h), cc = __ldcs(q10 + h), d = __ldcs(q11 + h);  // read once
         pooled[4 * h + 0] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.x, b.x), cc.x), d.x), 0.25f);
         pooled[4 * h + 1] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.y, b.y), cc.y), d.y), 0.25f);
         pooled[4 * h + 2] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.z, b.z), cc.z), d.z), 0.25f);
