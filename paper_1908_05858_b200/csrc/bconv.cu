@@ -306,7 +306,7 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(cons
             ((reinterpret_cast<uintptr_t>(g.residual) | reinterpret_cast<uintptr_t>(g.y_out)) & 15) == 0) {
 #pragma unroll
           for (int j = 0; j < TO; j += 4) {
-            const float4 r4 = *reinterpret_cast<const float4*>(rs + j);
+            const float4 r4 = __ldcs(reinterpret_cast<const float4*>(rs + j));  // the residual is read once
             y[j] = __fadd_rn(y[j], r4.x);
             y[j + 1] = __fadd_rn(y[j + 1], r4.y);
             y[j + 2] = __fadd_rn(y[j + 2], r4.z);
