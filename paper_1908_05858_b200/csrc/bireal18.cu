@@ -531,35 +531,54 @@ __global__ void __launch_bounds__(32) fc_small(const float* __restrict__ g /*[N]
 }
 
 // Larger batches: pooled vectors come from gap_small; a 64-thread CTA computes 64 logits for 8 images, so every weight
-// it loads is used 8 times and there are 16 x N/8 CTAs.
+// it loads is used 8 times and there are 16 x N/8 CTAs.  The weight rows of the 64 logits pass through shared memory in
+// chunks of 32 inputs (coalesced 128-byte pieces of each row in, conflict-free columns out), the next chunk in flight
+// while the current one is multiplied.  Each logit is still one fmaf chain over the inputs in ascending order.
 __global__ void __launch_bounds__(64) fc_batched(const float* __restrict__ g /*[N][512]*/, int N, const float* __restrict__ fw,
                                                  const float* __restrict__ fb, float* __restrict__ logits) {
   __shared__ __align__(16) float gs[8][512];
+  __shared__ float ws[64][33];
+  const int tid = threadIdx.x;
   const int n0 = blockIdx.y * 8, nimg = min(8, N - n0);
-  for (int t = threadIdx.x; t < 8 * 128; t += 64) {
+  for (int t = tid; t < 8 * 128; t += 64) {
     const int im = t / 128;
     reinterpret_cast<float4*>(&gs[0][0])[t] =
         im < nimg ? reinterpret_cast<const float4*>(g + (size_t)n0 * 512)[t] : make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  __syncthreads();
-  const int j = blockIdx.x * 64 + threadIdx.x;
-  if (j >= 1000) return;
-  const float4* wr = reinterpret_cast<const float4*>(fw + (size_t)j * 512);
+  const int j0 = blockIdx.x * 64, j = j0 + tid;
+  float4 wreg[8];
+  auto w_load = [&](int k0) {  // 64 rows x 32 inputs: piece u of this thread is row (tid + 64u) / 8, float4 (tid + 64u) % 8
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+      const int idx = tid + 64 * u, row = idx >> 3, q = idx & 7;
+      wreg[u] = (j0 + row < 1000) ? __ldg(reinterpret_cast<const float4*>(fw + (size_t)(j0 + row) * 512 + k0) + q)
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  auto w_store = [&]() {
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+      const int idx = tid + 64 * u, row = idx >> 3, q = idx & 7;
+      ws[row][4 * q] = wreg[u].x; ws[row][4 * q + 1] = wreg[u].y; ws[row][4 * q + 2] = wreg[u].z; ws[row][4 * q + 3] = wreg[u].w;
+    }
+  };
   float a[8];
 #pragma unroll
   for (int im = 0; im < 8; im++) a[im] = 0.0f;
-#pragma unroll 2
-  for (int k4 = 0; k4 < 128; k4++) {
-    const float4 wv = __ldg(wr + k4);
+  w_load(0);
+  for (int k0 = 0; k0 < 512; k0 += 32) {
+    __syncthreads();  // the previous chunk has been read (and, the first time, gs is complete)
+    w_store();
+    __syncthreads();
+    if (k0 + 32 < 512) w_load(k0 + 32);
+#pragma unroll 8
+    for (int kk = 0; kk < 32; kk++) {
+      const float wv = ws[tid][kk];
 #pragma unroll
-    for (int im = 0; im < 8; im++) {
-      const float4 gv = *reinterpret_cast<const float4*>(&gs[im][4 * k4]);
-      a[im] = __fmaf_rn(gv.x, wv.x, a[im]);
-      a[im] = __fmaf_rn(gv.y, wv.y, a[im]);
-      a[im] = __fmaf_rn(gv.z, wv.z, a[im]);
-      a[im] = __fmaf_rn(gv.w, wv.w, a[im]);
+      for (int im = 0; im < 8; im++) a[im] = __fmaf_rn(gs[im][k0 + kk], wv, a[im]);
     }
   }
+  if (j >= 1000) return;
   const float bias = fb[j];
 #pragma unroll
   for (int im = 0; im < 8; im++)
