@@ -503,7 +503,23 @@ def extras(B, torch, dev, peaks, sm_count):
         out[name] = {"int_pipes": {"ms": med, "Tbit-ops/s": ops / med / 1e9, "frac_of_bitop_peak": ops / med / 1e9 / peak}}
         med, best = time_fn(lambda: B.tc_bconv2d(a, wt, (1, 1), (pad, pad), -1, B.NHWC, out=o), 10, flush)
         out[name]["tensor"] = {"ms": med, "Tbit-ops/s": ops / med / 1e9, "frac_of_fp4_peak": ops / med / 1e9 / tpeak}
-        del a, w, o, wt
+        # the same launch with the fused BN + sign + pack epilogue (what a stack of binary layers runs), back to back
+        sc = torch.rand(O, device=dev) + 0.5
+        sh = torch.randn(O, device=dev)
+        bits = torch.empty((N, HW, HW, (O + 63) // 64), dtype=torch.int64, device=dev)
+        fused_call = B.prepare_tc_bconv2d_bn_sign_pack(a, wt, sc, sh, bits, (1, 1), (pad, pad), -1)
+        s_f = torch.cuda.Stream()
+        with torch.cuda.stream(s_f):
+            fused_call()
+            s_f.synchronize()
+            g_f = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_f, stream=s_f):
+                for _ in range(10):
+                    fused_call()
+            med10, _ = time_fn(g_f.replay, 5)
+        out[name]["tensor_fused_back_to_back"] = {"ms": med10 / 10, "Tbit-ops/s": ops / (med10 / 10) / 1e9,
+                                                  "frac_of_fp4_peak": ops / (med10 / 10) / 1e9 / tpeak}
+        del a, w, o, wt, g_f, fused_call, bits
 
     # BGEMM against direct convolution, the comparison of the paper's Fig. 4, on config 5a: the im2col matrix of the packed
     # activations (padding taps hold the pad word) is materialised with torch slicing (plumbing, 58 MB of packed rows) and

@@ -247,11 +247,43 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   // a pair runs while its leader has a tile (the peer's last tile may lie beyond the end: pad rows, nothing stored)
   const long long mt_end = PAIR ? (g.m_tiles + 1) / 2 * 2 : g.m_tiles;
 
-  if (EPI != EPI_I32) {
+  if (EPI == EPI_BIREAL) {
     for (int i = tid; i < nres_here * NT; i += TC_THREADS) {
       const int o = (ng * g.nres + i / NT) * NT + (i % NT);
       s_scale[i] = (o < g.O) ? g.scale[o] : 0.0f;
       s_shift[i] = (o < g.O) ? g.shift[o] : 0.0f;
+    }
+  }
+  if (EPI == EPI_BNPACK) {
+    // The sign of fmaf(acc, scale, shift) as a threshold on the integer acc: fmaf is monotone in acc (the exact value is,
+    // and rounding keeps order), so { acc in [-K, K] : fmaf(acc, scale, shift) < 0 } is empty, everything, a prefix
+    // (scale > 0) or a suffix (scale < 0) of the range -- also for infinite or NaN scale / shift, where the comparison is
+    // false wherever the value is NaN.  A bisection with the very fmaf finds the boundary; the epilogue then needs one
+    // compare per value: bit = (acc <= T) xor flip, with T in s_scale and one flip bit per channel in s_shift's place.
+    uint32_t* s_flip = reinterpret_cast<uint32_t*>(s_shift);
+    const int K = g.kh * g.kw * g.C;
+    for (int i = tid; i < nres_here * NT; i += TC_THREADS) {  // (whole warps: NT is a multiple of 32)
+      const int o = (ng * g.nres + i / NT) * NT + (i % NT);
+      const float sc = (o < g.O) ? g.scale[o] : 0.0f, sh = (o < g.O) ? g.shift[o] : 0.0f;
+      auto neg = [&](int a) { return __fmaf_rn((float)a, sc, sh) < 0.0f; };
+      const bool first = neg(-K), last = neg(K);
+      float T;
+      uint32_t flip = 0;
+      if (first == last) {
+        T = first ? (float)(K + 1) : (float)(-K - 1);  // everything / nothing
+      } else {
+        int lo = -K, hi = K;  // neg(lo) == first, neg(hi) == last
+        while (hi - lo > 1) {
+          const int mid = lo + ((hi - lo) >> 1);
+          if (neg(mid) == first) lo = mid;
+          else hi = mid;
+        }
+        T = (float)lo;        // prefix: negative for acc <= lo; suffix: negative for acc >= hi, i.e. not (acc <= lo)
+        flip = first ? 0u : 1u;
+      }
+      s_scale[i] = T;
+      const uint32_t mask = __ballot_sync(0xFFFFFFFFu, flip != 0);
+      if (lane == 0) s_flip[i >> 5] = mask;
     }
   }
   if (tid == 0) {
@@ -714,6 +746,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
             for (int j = 0; j < 32; j++)
               if (j < nch) __stcs(reinterpret_cast<uint32_t*>(g.out) + (nn * g.O + o + j) * ohw + q, acc_to_int(v[j]));
           }
+        } else if (EPI == EPI_BNPACK) {
+          if (o >= g.Ow32 * 32) continue;  // sign words are written whole (tail bits 0), nothing beyond them
+          uint32_t word = 0;
+#pragma unroll
+          for (int q = 0; q < 8; q++) {
+            const float4 t4 = *reinterpret_cast<const float4*>(r_scale + c0 + 4 * q);  // thresholds (see the prologue)
+            word |= (uint32_t)(__uint_as_float(v[4 * q]) <= t4.x) << (4 * q);
+            word |= (uint32_t)(__uint_as_float(v[4 * q + 1]) <= t4.y) << (4 * q + 1);
+            word |= (uint32_t)(__uint_as_float(v[4 * q + 2]) <= t4.z) << (4 * q + 2);
+            word |= (uint32_t)(__uint_as_float(v[4 * q + 3]) <= t4.w) << (4 * q + 3);
+          }
+          word ^= reinterpret_cast<const uint32_t*>(s_shift)[(r * NT + c0) >> 5];
+          word &= nch >= 32 ? 0xFFFFFFFFu : (nch > 0 ? (1u << nch) - 1u : 0u);  // channels beyond O: bit 0
+          g.out_packed32[m * g.Ow32 + (o >> 5)] = word;
         } else {
           if (o >= g.Ow32 * 32) continue;  // sign words are written whole (tail bits 0), nothing beyond them
           float y[32];

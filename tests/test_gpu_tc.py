@@ -123,6 +123,38 @@ def test_tc_full_size_configs_on_sampled_outputs(B, oracle_mod, cfg):
     assert B.tc_error_flag() == 0
 
 
+@pytest.mark.parametrize("C,k,pad", [(64, 3, 1), (128, 3, 1), (256, 1, 0)])
+def test_tc_sign_epilogue_is_exact_for_awkward_bn_vectors(B, oracle_mod, C, k, pad):
+    """The fused epilogue decides sign(fmaf(acc, scale, shift)) through an integer threshold per channel: negative, zero,
+    huge, tiny, infinite and NaN scales and shifts, and shifts that put y exactly on zero, against the oracle's fmaf."""
+    o = oracle_mod
+    N, H, W, O = 3, 9, 10, 128
+    rng = np.random.default_rng(C + k)
+    x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+    w = rng.standard_normal((O, C, k, k)).astype(np.float32)
+    acc = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (1, 1), (pad, pad), -1, o.NHWC)
+    scale = rng.uniform(0.5, 1.5, O).astype(np.float32)
+    shift = rng.normal(0, 4, O).astype(np.float32)
+    scale[0:8] *= -1                                     # decreasing in acc
+    scale[8:12] = [0.0, -0.0, 0.0, -0.0]; shift[8:12] = [1.0, -1.0, -0.0, 0.0]
+    scale[12:16] = [np.inf, -np.inf, np.inf, -np.inf]; shift[12:16] = [3.0, 3.0, -np.inf, np.inf]
+    scale[16:18] = np.nan; shift[18:20] = np.nan
+    scale[20:24] = [1e-30, -1e-30, 1e30, -1e30]; shift[20:24] = [1e-31, 1e-31, -1e29, 5e30]
+    scale[24:32] = [1, 1, -1, -1, 2, 0.5, -2, -0.5]      # y exactly zero at an attainable acc, and just beside it
+    shift[24:32] = [-4, 4, 6, -6, -8, 1, 12, -3]
+    scale[32:36] = [1.0000001, 0.99999994, -1.0000001, -0.99999994]; shift[32:36] = [-10, -10, 10, 10]
+    shift[36:40] = [np.inf, -np.inf, 1e38, -1e38]
+    want = o.bn_sign_pack(acc, scale, shift)
+    a = B.pack(dev(x))
+    wt = B.TcWeights(B.pack_weights(dev(w)), C)
+    got = u64(B.tc_bconv2d_bn_sign_pack(a, wt, dev(scale), dev(shift), (1, 1), (pad, pad), -1))
+    assert np.array_equal(got, want)
+    # and the integer-pipe engine, which evaluates the fmaf itself
+    got2 = u64(B.bconv2d_bn_sign_pack(a, C, B.pack_weights(dev(w)), dev(scale), dev(shift), (1, 1), (pad, pad), -1))
+    assert np.array_equal(got2, want)
+    assert B.tc_error_flag() == 0
+
+
 _FORCED_FORM_SCRIPT = r"""
 import sys, numpy as np, torch
 from paper_1908_05858_b200 import binding as B
