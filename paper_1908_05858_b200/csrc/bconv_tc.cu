@@ -960,10 +960,10 @@ dabnn_status tc_dispatch_mode(TcArgs& g, cudaStream_t st) {
 template <int EPI>
 dabnn_status tc_dispatch(TcArgs& g, cudaStream_t st) {
   // A second group of epilogue warps (measured): it pays for the residual epilogue, which moves two fp32 rows per
-  // output row, and for the sign-bit epilogue at C = 128; elsewhere the extra warps only add contention.
+  // output row; elsewhere the extra warps only add contention.
   // (environment DABNN_TC_EPI2 = 0 / 1 overrides, for measurements)
   static const int epi_env = [] { const char* e = getenv("DABNN_TC_EPI2"); return e ? atoi(e) : -1; }();
-  g.epi2 = epi_env >= 0 ? (epi_env != 0) : (EPI == EPI_BIREAL || (EPI == EPI_BNPACK && g.Cw == 2));
+  g.epi2 = epi_env >= 0 ? (epi_env != 0) : (EPI == EPI_BIREAL);
   return g.pair ? tc_dispatch_mode<EPI, true>(g, st) : tc_dispatch_mode<EPI, false>(g, st);
 }
 
