@@ -20,7 +20,8 @@
 //     needs, expands them to e2m1 rows of 32 channels ([C/32][slots][16 B]) -- padded slots get the declared pad
 //     value -- and every filter tap (i, j) is the SAME array read from a start address shifted by (i*SP + j) rows:
 //     with a 16-byte row pitch a shift by one slot is a 16-byte step of the matrix descriptor, so no im2col copy
-//     is ever materialised.  Rows that fall on padding columns / rows compute garbage that is never stored.
+//     is ever materialised.  Rows that fall on padding columns / rows compute garbage that is never stored; at stride 1
+//     only the left / top padding has slots of its own (the right / bottom taps read the next row's / image's).
 //   * Stride 2 keeps four parity planes of the padded input; tap (i, j) reads plane (i mod 2, j mod 2) shifted by
 //     (i div 2, j div 2).
 //   * Warp-specialised and mbarrier-driven: four producer warps prefetch the bits two tiles ahead, expand them
@@ -65,7 +66,7 @@ struct TcArgs {
   int N, H, W, Cw, C;
   int O, kh, kw, ph, pw, OH, OW;
   int S;               // stride (1 or 2, both axes)
-  int SPin, HPin;      // padded input extent: W + 2*pad_w, H + 2*pad_h
+  int SPin, HPin;      // padded input extent covered by the slot grid: W + 2*pad_w, H + 2*pad_h (one pad each at stride 1)
   int SP, HP;          // slot grid per image: ceil(SPin / S) columns, ceil(HPin / S) rows; output (oh, ow) sits at slot (oh, ow)
   long long total_q;   // N * HP * SP
   unsigned long long magic_sp, magic_hp;  // ceil(2^64 / SP), ceil(2^64 / HP) (0 when the divisor is 1)
@@ -1011,7 +1012,12 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   g.N = in.N; g.H = in.H; g.W = in.W; g.Cw = (in.C + 63) / 64; g.C = in.C;
   g.O = O; g.kh = cv.kh; g.kw = cv.kw; g.ph = cv.pad_h; g.pw = cv.pad_w; g.OH = OH; g.OW = OW;
   g.S = cv.stride_h;
-  g.SPin = in.W + 2 * cv.pad_w; g.HPin = in.H + 2 * cv.pad_h;
+  // Stride 1 with pad <= k - 1: the slot grid keeps only the left and top padding of each image.  A tap that reaches the
+  // right padding of a slot row reads the first slots of the next row -- that row's left padding -- and one that reaches
+  // the bottom padding reads the top padding of the next image (or rows beyond the batch), which hold the same pad value:
+  // (W + pad_w) x (H + pad_h) slots per image instead of (W + 2 pad_w) x (H + 2 pad_h), 64 instead of 81 at 7 x 7.
+  const bool shared_pad = g.S == 1 && cv.pad_h <= cv.kh - 1 && cv.pad_w <= cv.kw - 1;
+  g.SPin = in.W + (shared_pad ? 1 : 2) * cv.pad_w; g.HPin = in.H + (shared_pad ? 1 : 2) * cv.pad_h;
   g.SP = (g.SPin + g.S - 1) / g.S; g.HP = (g.HPin + g.S - 1) / g.S;
   g.total_q = (long long)in.N * g.HP * g.SP;
   if (g.SP >= 65536 || g.HP >= 65536) return DABNN_ERR_UNSUPPORTED;
