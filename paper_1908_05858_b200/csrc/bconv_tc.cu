@@ -980,7 +980,7 @@ void tc_plan(TcArgs& g, int O, int C, int taps) {
     // Measured: pairs win where one CTA cannot keep a 128-channel tile resident (C = 512 at 3x3) and there are
     // enough double tiles to go round; elsewhere the one-CTA form is as fast or faster.
     const long long work = (g.m_tiles + 1) / 2 * tc_n_ntiles(O, nt2);
-    pair = nt2 > tc_ntile(O, C, taps, false) && work >= units2;
+    pair = nt2 > tc_ntile(O, C, taps, false) && 4 * work >= 3LL * units2;
   }
   g.pair = pair ? 1 : 0;
   g.ntile = pair ? nt2 : tc_ntile(O, C, taps, false);
@@ -1045,7 +1045,8 @@ bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv) {
   const int nt = tc_ntile(O, in.C, cv.kh * cv.kw, false);
   if (nt == 0) return false;
   const int S = cv.stride_h;
-  const long long slots_total = (long long)in.N * ((in.H + 2 * cv.pad_h + S - 1) / S) * ((in.W + 2 * cv.pad_w + S - 1) / S);
+  const int pads = (S == 1 && cv.pad_h <= cv.kh - 1 && cv.pad_w <= cv.kw - 1) ? 1 : 2;  // as in tc_fill
+  const long long slots_total = (long long)in.N * ((in.H + pads * cv.pad_h + S - 1) / S) * ((in.W + pads * cv.pad_w + S - 1) / S);
   return (slots_total / 128) * tc_n_ntiles(O, nt) >= (long long)sm_count();
 }
 
