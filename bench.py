@@ -356,7 +356,7 @@ def main():
         "bound": "tensor", "kernel": "bconv_tc_kernel (the 8 convolution launches of a step, one CUDA-graph replay)",
         "achieved": conv_ops / (tc_ms * 1e-3) / 1e12, "peak": tensor_peak["tops"], "unit": "TFLOP/s",
         "frac": conv_ops / (tc_ms * 1e-3) / 1e12 / tensor_peak["tops"], "peak_is": tensor_peak["how"],
-        "traffic": 4.52e6, "traffic_is": "dram bytes of one N=64 C=256 28x28 launch (ncu, profiles/bconv_tc_kernel_N64_C256_HW28.md); most of its int32 output (51 MB, evict-first) is still in L2 when the kernel ends",
+        "traffic": 5.34e6, "traffic_is": "dram bytes of one N=64 C=256 28x28 launch (ncu, profiles/bconv_tc_kernel_N64_C256_HW28.md); most of its int32 output (51 MB, evict-first) is still in L2 when the kernel ends",
         "avg_launch_ms": tc_ms / 8, "conv_share_of_step": tc_ms / serial_step_ms,
         "conv_share_is": "the eight convolutions one after another / the 12 kernels one after another (%.4f ms)" % serial_step_ms,
         "note": "1 bit-op = 1 op: a +-1 multiply-add counts 2, as in FLOPs",
