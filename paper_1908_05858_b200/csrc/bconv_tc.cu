@@ -15,8 +15,8 @@
 //     its shared memory -- the tensor pipe's operand reads are what saturates shared memory in the one-CTA form -- and
 //     the pair keeps twice the channels resident.  The leader CTA issues; producers and epilogue warps of the peer
 //     signal the leader's barriers through the cluster's shared-memory window.
-//   * Activations: a tile is 128 consecutive "slots" q of the padded image grid (slot pitch SP = W + 2*pad_w,
-//     H + 2*pad_h slot rows per image).  The CTA reads the packed bits of the 128 + (kh-1)*SP + (kw-1) slots it
+//   * Activations: a tile is 128 consecutive "slots" q of the padded image grid (slot pitch SP and HP slot rows per
+//     image: W + pad_w and H + pad_h at stride 1, see below).  The CTA reads the packed bits of the 128 + (kh-1)*SP + (kw-1) slots it
 //     needs, expands them to e2m1 rows of 32 channels ([C/32][slots][16 B]) -- padded slots get the declared pad
 //     value -- and every filter tap (i, j) is the SAME array read from a start address shifted by (i*SP + j) rows:
 //     with a 16-byte row pitch a shift by one slot is a 16-byte step of the matrix descriptor, so no im2col copy
@@ -29,7 +29,8 @@
 //     separate warp waits for it, issues kh*kw*(C/64) tcgen05.mma (M = 128, N = NT, K = 64) into one of up to four
 //     TMEM accumulators per resident channel tile and commits to `mma_done` (and, after the tile's last MMA, to `a_free`);
 //     four (or eight) epilogue warps wait for that, read the accumulator with tcgen05.ld, write the output form, and hand the
-//     accumulator back through `tmem_free`.
+//     accumulator back through `tmem_free`.  The fused BN + sign form is one compare per value against a per-channel
+//     integer threshold that each CTA derives from (scale, shift) at start-up.
 //
 // Every wait on an mbarrier is bounded: on expiry the kernel records an error flag, stops, frees its TMEM and returns.
 #include "common.cuh"
