@@ -299,6 +299,23 @@ def test_bireal18_large_batch_kernels_match_oracle(B, oracle_mod):
     assert B.tc_error_flag() == 0
 
 
+def test_bireal18_batch72_all_blocks_on_the_tensor_engine(B, oracle_mod):
+    """At batch 72 every binary block runs on the tensor-core engine (CTA pairs in the last stage, stride-2 planes in the
+    three downsampling blocks, the second epilogue group) and the head uses the batched fc kernel with a ragged last
+    group of images; logits bit for bit against the oracle."""
+    p = synth.bireal18_params()
+    img = synth.bireal18_images(72)
+    want = oracle_mod.bireal18_forward(p, img, conv_form=1)
+    net = B.Bireal18(p)
+    got = net.forward(dev(img)).cpu().numpy()
+    assert np.array_equal(got.argmax(axis=1), want.argmax(axis=1))
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    # the same images through the integer-pipe engine only
+    got_p = B.Bireal18(p, engine="popc").forward(dev(img)).cpu().numpy()
+    assert np.array_equal(got_p.view(np.uint32), want.view(np.uint32))
+    assert B.tc_error_flag() == 0
+
+
 @pytest.mark.parametrize("N,pinned", [(1, True), (3, True), (5, False), (9, True)])
 def test_binary_layer_host_matches_oracle(B, oracle_mod, N, pinned):
     """The host-buffer entry point (chunked, copies on side streams): int32 sums and fused sign words against the oracle,

@@ -120,6 +120,19 @@ def test_tc_full_size_configs_on_sampled_outputs(B, oracle_mod, cfg):
     coords = np.stack([rng.integers(0, N, 20000), rng.integers(0, O, 20000), rng.integers(0, HW, 20000), rng.integers(0, HW, 20000)], axis=1).astype(np.int32)
     want = oracle_mod.bconv_pm1_at(x, w, coords, (1, 1), (pad, pad), -1)
     assert np.array_equal(g[coords[:, 0], coords[:, 2], coords[:, 3], coords[:, 1]], want)
+    # the fused sign epilogue at full size: the whole tensor against the integer-pipe engine's fused kernel, and the
+    # oracle's fmaf + sign on the sampled pixels
+    rng2 = np.random.default_rng(C + N + 1)
+    scale = rng2.uniform(0.5, 1.5, O).astype(np.float32)
+    shift = rng2.normal(0, 0.3 * np.sqrt(K), O).astype(np.float32)
+    bits = B.tc_bconv2d_bn_sign_pack(a, B.TcWeights(wp, C), dev(scale), dev(shift), (1, 1), (pad, pad), -1)
+    assert bool((bits == B.bconv2d_bn_sign_pack(a, C, wp, dev(scale), dev(shift), (1, 1), (pad, pad), -1)).all())
+    px = coords[:2000]
+    acc_px = oracle_mod.bconv_pm1_at(x, w, np.stack([np.repeat(px[:, 0], O), np.tile(np.arange(O), len(px)), np.repeat(px[:, 2], O),
+                                                     np.repeat(px[:, 3], O)], axis=1).astype(np.int32), (1, 1), (pad, pad), -1)
+    want_bits = oracle_mod.bn_sign_pack(acc_px.reshape(len(px), 1, 1, O), scale, shift).reshape(len(px), -1)
+    got_bits = bits.cpu().numpy().view(np.uint64)[px[:, 0], px[:, 2], px[:, 3]]
+    assert np.array_equal(got_bits, want_bits)
     assert B.tc_error_flag() == 0
 
 

@@ -56,3 +56,30 @@ def test_sign_decision_is_the_sign_of_the_exact_value(oracle_mod):
         assert int(np.count_nonzero(np.diff(bits.astype(int)))) <= 1
     # tail bits of the last word are zero
     assert not np.any(P[:, 1] >> np.uint64(O - 64))
+
+
+def test_sign_of_bn_output_is_a_threshold_on_the_integer_sum(oracle_mod):
+    """sign(fmaf(acc, scale, shift)) is monotone in the integer acc (the exact value is, and rounding keeps order), so for
+    every channel the sums that give bit 1 form a prefix (scale > 0), a suffix (scale < 0), everything or nothing --
+    also for zero, infinite and NaN parameters.  The GPU's fused epilogue relies on it; here it is checked on the oracle
+    for every integer in [-K, K]."""
+    o = oracle_mod
+    K = 600
+    rng = np.random.default_rng(3)
+    scale = np.concatenate([rng.uniform(-2, 2, 40), [0.0, -0.0, np.inf, -np.inf, np.nan, 1e-30, -1e30, 1.0, -1.0, 0.5]]).astype(np.float32)
+    shift = np.concatenate([rng.normal(0, 200, 40), [1.0, -1.0, 5.0, 5.0, 0.0, -1e-31, 1e29, -7.0, -7.0, np.nan]]).astype(np.float32)
+    O = scale.size
+    acc = np.repeat(np.arange(-K, K + 1, dtype=np.int32)[:, None], O, axis=1).reshape(2 * K + 1, 1, 1, O)
+    words = o.bn_sign_pack(acc, scale, shift).reshape(2 * K + 1, -1)
+    bits = np.stack([(words[:, c >> 6] >> np.uint64(c & 63)) & np.uint64(1) for c in range(O)], axis=1).astype(np.int8)
+    for c in range(O):
+        col = bits[:, c]
+        changes = np.count_nonzero(np.diff(col))
+        assert changes <= 1, (c, scale[c], shift[c])
+        if changes == 1:  # a prefix of ones for an increasing y, a suffix for a decreasing one
+            assert (col[0] == 1) == (scale[c] > 0), (c, scale[c], shift[c])
+    # and the bit is what a direct evaluation in fp64 says wherever that is unambiguous (|y| well away from zero)
+    with np.errstate(invalid="ignore"):  # 0 * inf and inf - inf are NaN on purpose
+        y = acc.reshape(2 * K + 1, O).astype(np.float64) * scale.astype(np.float64) + shift.astype(np.float64)
+    clear = np.isfinite(y) & (np.abs(y) > 1e-3 * (np.abs(shift.astype(np.float64)) + 1))
+    assert np.array_equal(bits[clear], (y[clear] < 0).astype(np.int8))
