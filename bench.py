@@ -318,7 +318,10 @@ def main():
     barrier()
     # each step is one CUDA-graph replay (one host call), so the timed loop is never host-bound
     g_step = {e: [capture(lambda e=e, w=w: step(e, which=w)) for w in (0, 1)] for e in ("tc", "popc")}
+    # side by side, launches capped at half the chip each fill it better than launches that each take all of it
+    B.tc_set_max_ctas(sm_count // 2)
     g_branched = [capture(lambda w=w: step_branched("tc", which=w)) for w in (0, 1)]
+    B.tc_set_max_ctas(0)
     g_conv = {e: [capture(lambda e=e, w=w: step(e, convs_only=True, which=w)) for w in (0, 1)] for e in ("tc", "popc")}
     for _ in range(warmup):
         g_branched[0].replay()
@@ -401,7 +404,7 @@ def main():
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u64 words / int32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "l2": "no flush: steps alternate between two buffer sets (about 390 MB touched between two uses of a buffer; L2 is 126 MB)",
-                   "launch": "each step is one CUDA-graph replay of its 12 kernels: four branches, one per shape (pack -> conv int32 -> conv fused), that the GPU overlaps",
+                   "launch": "each step is one CUDA-graph replay of its 12 kernels: four branches, one per shape (pack -> conv int32 -> conv fused), that the GPU overlaps, tensor-engine launches capped at half the SMs each (dabnn_tc_set_max_ctas)",
                    "serial_ms_per_step": serial_step_ms,
                    "engine": "tensor-core engine (e2m1 tcgen05) for the timed steps; the integer-pipe engine is timed beside it (roofline_bitop)",
                    "parallelism": "replicas" if world > 1 else "single GPU"},

@@ -203,6 +203,11 @@ dabnn_status dabnn_tc_bconv2d_bn_add_sign_pack(const uint64_t* a_packed, dabnn_s
                                                dabnn_conv cv, const float* scale, const float* shift, const float* residual,
                                                float* y_out, uint64_t* out_packed, void* stream);
 int dabnn_tc_error_flag(void);
+/* CTAs per tensor-engine launch at most (0 = the default: one persistent CTA, or CTA of a pair, per SM).  A launch takes
+ * every SM it is given; a caller that runs independent layers side by side (several streams, or branches of a CUDA graph)
+ * gets more out of the chip with launches capped at about half of it (74 on a B200).  Results do not depend on it.
+ * Returns the previous setting.  Not thread-safe against concurrent calls into the library. */
+int dabnn_tc_set_max_ctas(int max_ctas);
 
 /* Selects the convolution inner loop for measurement runs: 0 = automatic (default),
  * 1 = one POPC per 32-bit word pair, 2 = carry-save (one POPC per two word pairs).  All give identical results.

@@ -26,7 +26,7 @@ EXPORTS = (
     "dabnn_bconv2d", "dabnn_bgemm", "dabnn_bconv2d_bn_sign_pack", "dabnn_bconv2d_bn_add_sign_pack", "dabnn_bn_fold",
     "dabnn_bireal18_workspace_bytes", "dabnn_bireal18_forward", "dabnn_set_conv_variant",
     "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host", "dabnn_bireal18_forward_static", "dabnn_set_conv_tile",
-    "dabnn_tc_weights_bytes", "dabnn_tc_prepare_weights", "dabnn_tc_bconv2d", "dabnn_tc_bconv2d_bn_sign_pack",
+    "dabnn_tc_set_max_ctas", "dabnn_tc_weights_bytes", "dabnn_tc_prepare_weights", "dabnn_tc_bconv2d", "dabnn_tc_bconv2d_bn_sign_pack",
     "dabnn_tc_bconv2d_bn_add_sign_pack", "dabnn_tc_error_flag",
 )
 
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
         L.dabnn_binary_layer_host.restype = ci
         L.dabnn_set_conv_variant.restype = ci
         L.dabnn_set_conv_variant.argtypes = [ci]
+        L.dabnn_tc_set_max_ctas.restype = ci
+        L.dabnn_tc_set_max_ctas.argtypes = [ci]
         L.dabnn_tc_weights_bytes.restype = ctypes.c_size_t
         L.dabnn_tc_weights_bytes.argtypes = [ci, ci, ci, ci]
         L.dabnn_tc_prepare_weights.argtypes = [vp, ci, ci, ci, ci, vp, vp]
@@ -424,6 +426,11 @@ def tc_bconv2d_bn_add_sign_pack(a_packed, wt: TcWeights, scale, shift, residual,
                                                    shift.data_ptr(), residual.data_ptr(), y.data_ptr(),
                                                    bits.data_ptr() if want_bits else None, _stream()))
     return y, bits
+
+
+def tc_set_max_ctas(max_ctas: int) -> int:
+    """dabnn_tc_set_max_ctas: cap the CTAs of a tensor-engine launch (0 = all SMs); returns the previous setting."""
+    return int(lib().dabnn_tc_set_max_ctas(int(max_ctas)))
 
 
 def tc_error_flag() -> int:

@@ -54,6 +54,7 @@ constexpr int TC_SF_COL = 384;            // columns [384, 512) hold scale facto
 constexpr int TC_MAX_BUFS = 4;            // accumulators / activation buffers in flight at most
 
 __device__ int g_tc_error = 0;  // 1: an mbarrier wait ran out
+int g_tc_max_ctas = 0;          // host: CTAs per launch at most (0: one per SM)
 #ifdef TC_TIMING
 __device__ unsigned long long g_tc_prof[24];
 #define TC_T(i) do { long long t_ = clock64(); prof[i] += t_ - tlast; tlast = t_; } while (0)
@@ -911,7 +912,13 @@ dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
   }
   const long long m_units = PAIR ? (g.m_tiles + 1) / 2 : g.m_tiles;
   long long units = (long long)g.n_groups * m_units;
-  const long long cap = (long long)max_units / g.n_groups * g.n_groups;
+  // (a caller that runs several layers side by side may cap the CTAs of a launch: dabnn_tc_set_max_ctas)
+  int avail = max_units;
+  if (g_tc_max_ctas > 0) {
+    const int capped = PAIR ? g_tc_max_ctas / 2 : g_tc_max_ctas;
+    if (capped < avail) avail = capped > g.n_groups ? capped : g.n_groups;
+  }
+  const long long cap = (long long)avail / g.n_groups * g.n_groups;
   if (cap <= 0) return DABNN_ERR_UNSUPPORTED;
   if (units > cap) units = cap;
   if (!PAIR) {
@@ -1112,6 +1119,12 @@ extern "C" dabnn_status dabnn_tc_bconv2d_bn_add_sign_pack(const uint64_t* a_pack
   g.scale = scale; g.shift = shift; g.residual = residual; g.y_out = y_out;
   g.out_packed32 = reinterpret_cast<uint32_t*>(out_packed);
   return tc_dispatch<EPI_BIREAL>(g, as_stream(stream));
+}
+
+extern "C" int dabnn_tc_set_max_ctas(int max_ctas) {
+  const int prev = g_tc_max_ctas;
+  g_tc_max_ctas = max_ctas > 0 ? max_ctas : 0;
+  return prev;
 }
 
 extern "C" int dabnn_tc_error_flag(void) {

@@ -168,6 +168,24 @@ def test_tc_sign_epilogue_is_exact_for_awkward_bn_vectors(B, oracle_mod, C, k, p
     assert B.tc_error_flag() == 0
 
 
+@pytest.mark.parametrize("cap", [1, 10, 74])
+def test_tc_results_do_not_depend_on_the_cta_cap(B, oracle_mod, cap):
+    o = oracle_mod
+    rng = np.random.default_rng(cap)
+    try:
+        for N, C, H, W, O in ((5, 128, 14, 14, 128), (20, 512, 7, 7, 512), (3, 64, 20, 20, 192)):
+            x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+            w = rng.standard_normal((O, C, 3, 3)).astype(np.float32)
+            want = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (1, 1), (1, 1), -1, o.NHWC)
+            a, wt = B.pack(dev(x)), B.TcWeights(B.pack_weights(dev(w)), C)
+            assert B.tc_set_max_ctas(cap) in (0, cap)
+            got = B.tc_bconv2d(a, wt, (1, 1), (1, 1), -1, B.NHWC).cpu().numpy()
+            assert np.array_equal(got, want)
+    finally:
+        B.tc_set_max_ctas(0)
+    assert B.tc_error_flag() == 0
+
+
 _FORCED_FORM_SCRIPT = r"""
 import sys, numpy as np, torch
 from paper_1908_05858_b200 import binding as B
