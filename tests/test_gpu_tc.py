@@ -186,6 +186,23 @@ def test_tc_results_do_not_depend_on_the_cta_cap(B, oracle_mod, cap):
     assert B.tc_error_flag() == 0
 
 
+@pytest.mark.parametrize("kh,kw,ph,pw", [(1, 3, 0, 1), (3, 1, 1, 0), (3, 5, 1, 2), (3, 3, 0, 1), (3, 3, 2, 2), (2, 2, 1, 1), (3, 3, 3, 3)])
+def test_asymmetric_filters_and_paddings_on_both_engines(B, oracle_mod, kh, kw, ph, pw):
+    """Filters and paddings that differ between the axes, padding smaller and larger than (k - 1) / 2, and padding beyond
+    k - 1 (where the tensor engine keeps both padding columns in its slot grid)."""
+    o = oracle_mod
+    N, C, H, W, O = 3, 64, 9, 11, 64
+    rng = np.random.default_rng(kh * 100 + kw * 10 + ph + pw)
+    x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+    w = rng.standard_normal((O, C, kh, kw)).astype(np.float32)
+    for pv in (-1, 1):
+        want = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (1, 1), (ph, pw), pv, o.NHWC)
+        a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
+        assert np.array_equal(B.bconv2d(a, C, wp, (1, 1), (ph, pw), pv, B.NHWC).cpu().numpy(), want)
+        assert np.array_equal(B.tc_bconv2d(a, B.TcWeights(wp, C), (1, 1), (ph, pw), pv, B.NHWC).cpu().numpy(), want)
+    assert B.tc_error_flag() == 0
+
+
 _FORCED_FORM_SCRIPT = r"""
 import sys, numpy as np, torch
 from paper_1908_05858_b200 import binding as B
