@@ -214,7 +214,8 @@ int dabnn_tc_set_max_ctas(int max_ctas);
  * Returns the previous setting.  Not thread-safe against concurrent calls into the library. */
 int dabnn_set_conv_variant(int variant);
 /* Forces the convolution's CTA tile for measurement runs: 0 = automatic (default), 1 = 128 pixels x 128 channels,
- * 2 = 128 x 64, 3 = 64 x 64, 4 = 32 x 32.  All give identical results.  Returns the previous setting. */
+ * 2 = 128 x 64, 3 = 64 x 64, 4 = 32 x 32, 5 = 16 x 32 with all of K in flight (the choice for launches of less than
+ * one wave).  All give identical results.  Returns the previous setting. */
 int dabnn_set_conv_tile(int tile);
 
 #ifdef __cplusplus

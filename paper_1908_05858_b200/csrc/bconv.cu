@@ -25,7 +25,7 @@ enum { EPI_I32 = 0, EPI_BNPACK = 1, EPI_BIREAL = 2 };
 
 constexpr int KC64 = 16;             // 64-bit words per K chunk and smem row
 constexpr int PITCH = 2 * KC64 + 4;  // 32-bit words per smem row: 144 B, keeps 8 consecutive rows on distinct banks
-constexpr int STAGES = 3;
+constexpr int STAGES_DEFAULT = 3;  // ring depth of the throughput tiles; the small-problem tile holds all of K at once
 
 struct BConvArgs {
   const uint64_t* a;
@@ -84,7 +84,7 @@ __device__ __forceinline__ void bit_mac(uint32_t a0, uint32_t a1, uint32_t w0, u
   }
 }
 
-template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16>
+template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16, int STAGES>
 __global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(const BConvArgs g) {
   constexpr int THREADS = (BP / TP) * (BO / TO);
   constexpr int UW = VEC16 ? 2 : 1;         // 64-bit words per copy unit
@@ -346,11 +346,11 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(cons
 int g_conv_variant = 0;
 int g_conv_tile = 0;
 
-template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16>
+template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16, int STAGES>
 dabnn_status launch_one(const BConvArgs& g, cudaStream_t st) {
   constexpr int THREADS = (BP / TP) * (BO / TO);
   constexpr size_t SMEM = (size_t)STAGES * (BP + BO) * PITCH * 4 + (size_t)BP * sizeof(RowInfo);
-  auto kern = bconv_kernel<BP, BO, TP, TO, MINB, EPI, CSA, VEC16>;
+  auto kern = bconv_kernel<BP, BO, TP, TO, MINB, EPI, CSA, VEC16, STAGES>;
   static bool configured = false;  // one attribute call per instantiation (idempotent if raced)
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) {
@@ -367,14 +367,14 @@ dabnn_status launch_one(const BConvArgs& g, cudaStream_t st) {
   return launch_status();
 }
 
-template <int BP, int BO, int TP, int TO, int MINB, int EPI>
+template <int BP, int BO, int TP, int TO, int MINB, int EPI, int STAGES = STAGES_DEFAULT>
 dabnn_status launch_tile(const BConvArgs& g, bool csa, cudaStream_t st) {
   const bool vec16 = (g.Cw % 2 == 0) && aligned(g.a, 16) && aligned(g.w, 16);
   if (csa)
-    return vec16 ? launch_one<BP, BO, TP, TO, MINB, EPI, true, true>(g, st)
-                 : launch_one<BP, BO, TP, TO, MINB, EPI, true, false>(g, st);
-  return vec16 ? launch_one<BP, BO, TP, TO, MINB, EPI, false, true>(g, st)
-               : launch_one<BP, BO, TP, TO, MINB, EPI, false, false>(g, st);
+    return vec16 ? launch_one<BP, BO, TP, TO, MINB, EPI, true, true, STAGES>(g, st)
+                 : launch_one<BP, BO, TP, TO, MINB, EPI, true, false, STAGES>(g, st);
+  return vec16 ? launch_one<BP, BO, TP, TO, MINB, EPI, false, true, STAGES>(g, st)
+               : launch_one<BP, BO, TP, TO, MINB, EPI, false, false, STAGES>(g, st);
 }
 
 template <int EPI>
@@ -388,13 +388,17 @@ dabnn_status launch_epi(const BConvArgs& g, cudaStream_t st) {
     if (ochan > 64 && ctas(128, 128) >= 2LL * sms) tile = 1;
     else if (ctas(128, 64) >= 4LL * sms) tile = 2;
     else if (ctas(64, 64) >= 2LL * sms) tile = 3;
-    else tile = 4;
+    else if (ctas(32, 32) >= sms || g.K64 > 5 * KC64) tile = 4;
+    else tile = 5;  // less than one wave of the smallest tile: latency is all that counts
   }
   switch (tile) {
     case 1: return launch_tile<128, 128, 8, 8, 1, EPI>(g, csa, st);
     case 2: return launch_tile<128, 64, 8, 4, 2, EPI>(g, csa, st);
     case 3: return launch_tile<64, 64, 4, 4, 2, EPI>(g, csa, st);
-    default: return launch_tile<32, 32, 2, 4, 4, EPI>(g, csa, st);
+    case 4: return launch_tile<32, 32, 2, 4, 4, EPI>(g, csa, st);
+    // 16 x 32 outputs per CTA and a ring of 6 stages: every chunk of K up to 80 words (a 3x3 filter over 512 channels is
+    // 72) is requested before the first one is used, so the CTA waits for memory once
+    default: return launch_tile<16, 32, 1, 4, 4, EPI, 6>(g, csa, st);
   }
 }
 
@@ -451,7 +455,7 @@ extern "C" int dabnn_set_conv_variant(int variant) {
 
 extern "C" int dabnn_set_conv_tile(int tile) {
   const int prev = g_conv_tile;
-  if (tile >= 0 && tile <= 4) g_conv_tile = tile;
+  if (tile >= 0 && tile <= 5) g_conv_tile = tile;
   return prev;
 }
 

@@ -499,6 +499,64 @@ __global__ void __launch_bounds__(256) shortcut_down_small(const float* __restri
   y[p * O + o] = __fmaf_rn(a, scale[o], shift[o]);
 }
 
+// The same for a few images, with every global load issued before the first fmaf: a CTA takes 16 output pixels x 16
+// channels; its 16 weight rows and the pooled inputs of its 16 pixels go through shared memory (coalesced float4 loads,
+// all in flight at once), then each thread runs the one fmaf chain of its output over c ascending.  C <= 256, C % 4 == 0.
+__global__ void __launch_bounds__(256) shortcut_down_tile16(const float* __restrict__ x, int HW, int C,
+                                                            const float* __restrict__ w, int O,
+                                                            const float* __restrict__ scale, const float* __restrict__ shift,
+                                                            long long npix_out, float* __restrict__ y) {
+  constexpr int PITCH = 260;  // floats per row: 16 rows, read as float4, fall on distinct banks
+  __shared__ __align__(16) float pooled[16][PITCH];
+  __shared__ __align__(16) float ws[16][PITCH];
+  const int tid = threadIdx.x;
+  const long long p0 = (long long)blockIdx.x * 16;
+  const int o0 = blockIdx.y * 16;
+  const int OHW = HW / 2, C4 = C / 4;
+#pragma unroll 4
+  for (int t = tid; t < 16 * C4; t += 256) {
+    const int row = t / C4, q = t - row * C4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (o0 + row < O) v = __ldg(reinterpret_cast<const float4*>(w + (size_t)(o0 + row) * C) + q);
+    *reinterpret_cast<float4*>(&ws[row][4 * q]) = v;
+  }
+#pragma unroll 4
+  for (int t = tid; t < 16 * C4; t += 256) {
+    const int pp = t / C4, q = t - pp * C4;
+    const long long p = p0 + pp;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (p < npix_out) {
+      const int ow = (int)(p % OHW), oh = (int)((p / OHW) % OHW);
+      const long long n = p / ((long long)OHW * OHW);
+      const float* src = x + ((n * HW + 2 * oh) * HW + 2 * ow) * C + 4 * q;
+      const float4 a = __ldg(reinterpret_cast<const float4*>(src));
+      const float4 b = __ldg(reinterpret_cast<const float4*>(src + C));
+      const float4 c = __ldg(reinterpret_cast<const float4*>(src + (size_t)HW * C));
+      const float4 d = __ldg(reinterpret_cast<const float4*>(src + (size_t)HW * C + C));
+      v.x = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.x, b.x), c.x), d.x), 0.25f);
+      v.y = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.y, b.y), c.y), d.y), 0.25f);
+      v.z = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.z, b.z), c.z), d.z), 0.25f);
+      v.w = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.w, b.w), c.w), d.w), 0.25f);
+    }
+    *reinterpret_cast<float4*>(&pooled[pp][4 * q]) = v;
+  }
+  __syncthreads();
+  const int pp = tid >> 4, oo = tid & 15, o = o0 + oo;
+  const long long p = p0 + pp;
+  if (o >= O || p >= npix_out) return;
+  float a = 0.0f;
+#pragma unroll 4
+  for (int c = 0; c < C; c += 4) {
+    const float4 wv = *reinterpret_cast<const float4*>(&ws[oo][c]);
+    const float4 pv = *reinterpret_cast<const float4*>(&pooled[pp][c]);
+    a = __fmaf_rn(pv.x, wv.x, a);
+    a = __fmaf_rn(pv.y, wv.y, a);
+    a = __fmaf_rn(pv.z, wv.z, a);
+    a = __fmaf_rn(pv.w, wv.w, a);
+  }
+  y[p * O + o] = __fmaf_rn(a, scale[o], shift[o]);
+}
+
 // ---- head: global average over 7x7 (sequential sum over (h, w), then /49) into the workspace, then fc 512 -> 1000 as
 // one fmaf chain per logit over k ascending, then + bias.  Small batches: 32-thread CTAs, one image each.
 __global__ void __launch_bounds__(512) gap_small(const float* __restrict__ x /*[N][7][7][512]*/, float* __restrict__ g) {
@@ -526,6 +584,48 @@ __global__ void __launch_bounds__(32) fc_small(const float* __restrict__ g /*[N]
     a = __fmaf_rn(gv.y, wv.y, a);
     a = __fmaf_rn(gv.z, wv.z, a);
     a = __fmaf_rn(gv.w, wv.w, a);
+  }
+  logits[(size_t)n * 1000 + j] = __fadd_rn(a, fb[j]);
+}
+
+// One to four images: pooling and fc in one launch.  A 512-thread CTA takes 8 logits of one image: it pools the image's
+// 7x7x512 map itself (thread c owns channel c; same sum order and division as gap_small) while its 8 weight rows are in
+// flight, then 8 threads run the 8 fmaf chains out of shared memory.
+__global__ void __launch_bounds__(512) head_small(const float* __restrict__ x /*[N][7][7][512]*/,
+                                                  const float* __restrict__ fw, const float* __restrict__ fb,
+                                                  float* __restrict__ logits) {
+  constexpr int PITCH = 516;
+  __shared__ __align__(16) float gs[512];
+  __shared__ __align__(16) float ws[8][PITCH];
+  const int n = blockIdx.y, tid = threadIdx.x, j0 = blockIdx.x * 8;
+  float4 wv[2];
+#pragma unroll
+  for (int u = 0; u < 2; u++) {
+    const int idx = tid + 512 * u, row = idx >> 7, q = idx & 127;
+    wv[u] = (j0 + row < 1000) ? __ldg(reinterpret_cast<const float4*>(fw + (size_t)(j0 + row) * 512) + q)
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float s = 0.0f;
+#pragma unroll 7
+  for (int q = 0; q < 49; q++) s = __fadd_rn(s, __ldg(x + ((size_t)n * 49 + q) * 512 + tid));
+  gs[tid] = __fdiv_rn(s, 49.0f);
+#pragma unroll
+  for (int u = 0; u < 2; u++) {
+    const int idx = tid + 512 * u, row = idx >> 7, q = idx & 127;
+    *reinterpret_cast<float4*>(&ws[row][4 * q]) = wv[u];
+  }
+  __syncthreads();
+  const int j = j0 + tid;
+  if (tid >= 8 || j >= 1000) return;
+  float a = 0.0f;
+#pragma unroll 8
+  for (int k = 0; k < 512; k += 4) {
+    const float4 w4 = *reinterpret_cast<const float4*>(&ws[tid][k]);
+    const float4 g4 = *reinterpret_cast<const float4*>(&gs[k]);
+    a = __fmaf_rn(g4.x, w4.x, a);
+    a = __fmaf_rn(g4.y, w4.y, a);
+    a = __fmaf_rn(g4.z, w4.z, a);
+    a = __fmaf_rn(g4.w, w4.w, a);
   }
   logits[(size_t)n * 1000 + j] = __fadd_rn(a, fb[j]);
 }
@@ -695,7 +795,11 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     const bool down = stage > 0 && b % 4 == 0;
     if (down) {
       const long long npo = (long long)N * OHW * OHW;
-      if ((long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) < 8 && C <= 512)  // a handful of tiles: one thread per output
+      const bool few = (long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) < 8;  // a handful of tiles: one thread per output
+      if (few && C <= 256 && C % 4 == 0 && aligned(p->down_w[stage - 1], 16))
+        shortcut_down_tile16<<<dim3(ceil_div(npo, 16), ceil_div(O, 16)), 256, 0, st>>>(
+            cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
+      else if (few && C <= 512)
         shortcut_down_small<<<dim3(ceil_div(npo, 4), ceil_div(O, 64)), 256, 0, st>>>(
             cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
       else
@@ -719,6 +823,10 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     C = O; HW = OHW;
   }
   {
+    if (N <= 4) {
+      head_small<<<dim3(125, N), 512, 0, st>>>(cur, p->fc_w, p->fc_b, logits);
+      return launch_status();
+    }
     float* gbuf = reinterpret_cast<float*>(base + ws.gap);
     gap_small<<<N, 512, 0, st>>>(cur, gbuf);
     if ((s = launch_status()) != DABNN_OK) return s;

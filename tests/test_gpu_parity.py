@@ -253,8 +253,9 @@ def test_bireal18_forward_matches_oracle(B, oracle_mod):
     assert np.array_equal(got1, got[:1])
 
 
-@pytest.mark.parametrize("tile", [1, 2, 3, 4])
-@pytest.mark.parametrize("case", [CONV_CASES[1], CONV_CASES[4], CONV_CASES[9]])
+@pytest.mark.parametrize("tile", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("case", [CONV_CASES[1], CONV_CASES[4], CONV_CASES[9],
+                                  (1, 640, 6, 5, 40, 3, 3, (1, 1), (1, 1), -1)])  # 90 words of K: every ring wraps
 def test_every_conv_tile_gives_the_same_integers(B, oracle_mod, case, tile):
     N, C, H, W, O, kh, kw, stride, pad, pv = case
     x, w = conv_inputs(case)
