@@ -60,12 +60,17 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
   constexpr int RSTEP = TS / PPT;        // a thread's pixels are RSTEP rows apart
   constexpr int TILES = (OHW + TS - 1) / TS;
   extern __shared__ __align__(16) float sm[];
-  float* w_s = sm;                       // [147][64], loaded once per CTA
+  float* w_s = sm;                       // [147][64], filled once per CTA
   float* x_s = sm + STEM_K * 64;         // [2 buffers][3][PS][2][HALF]
+  float* w_raw = x_s + 2 * PATCH;        // [64][147] as in global memory, until it has been transposed into w_s
   const int tid = threadIdx.x;
-  for (int t = tid; t < STEM_K * 64; t += THREADS) {
-    const int o = t % 64, k = t / 64;    // w is [64][147]
-    w_s[k * 64 + o] = w[o * STEM_K + k];
+  if ((reinterpret_cast<uintptr_t>(w) & 15) == 0) {  // one coalesced asynchronous copy, in flight together with the first patch
+    for (int t = tid; t < STEM_K * 16; t += THREADS) {
+      const uint32_t d = (uint32_t)__cvta_generic_to_shared(w_raw + 4 * t);
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(w + 4 * t) : "memory");
+    }
+  } else {
+    for (int t = tid; t < STEM_K * 64; t += THREADS) w_raw[t] = w[t];
   }
   const long long ntiles = (long long)N * TILES * TILES;
   // asynchronous copy of one tile's zero-padded input patch (even and odd columns apart)
@@ -95,6 +100,10 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
   long long tile = blockIdx.x;
   int buf = 0;
   if (tile < ntiles) load_patch(tile, x_s);
+  asm volatile("cp.async.wait_all;" ::: "memory");
+  __syncthreads();
+  // [64][147] -> [147][64]: lanes walk over o, 147 words apart in w_raw (an odd stride: distinct banks) and consecutive in w_s
+  for (int t = tid; t < STEM_K * 64; t += THREADS) w_s[t] = w_raw[(t & 63) * STEM_K + (t >> 6)];
   for (; tile < ntiles; tile += gridDim.x, buf ^= 1) {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();  // this tile's patch (and, the first time, the weights) are in place; the other buffer is free
@@ -726,7 +735,7 @@ dabnn_status launch_stem_8x8(const dabnn_bireal18_params* p, const float* images
 template <int TS, int PPT>
 dabnn_status launch_stem(const dabnn_bireal18_params* p, const float* images, int N, float* out, cudaStream_t st) {
   constexpr int PS = 2 * TS + 5, HALF = (PS + 1) / 2 + 1;
-  constexpr size_t SMEM = (size_t)(STEM_K * 64 + 2 * 3 * PS * 2 * HALF) * 4;
+  constexpr size_t SMEM = (size_t)(2 * STEM_K * 64 + 2 * 3 * PS * 2 * HALF) * 4;
   auto kern = stem_conv_bn<TS, PPT>;
   static bool configured = false;
   if (!configured) {
@@ -795,7 +804,8 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     const bool down = stage > 0 && b % 4 == 0;
     if (down) {
       const long long npo = (long long)N * OHW * OHW;
-      const bool few = (long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) < 8;  // a handful of tiles: one thread per output
+      // less than half a wave of 128 x 128 tiles: one thread per output
+      const bool few = 2 * (long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) < sm_count();
       if (few && C <= 256 && C % 4 == 0 && aligned(p->down_w[stage - 1], 16))
         shortcut_down_tile16<<<dim3(ceil_div(npo, 16), ceil_div(O, 16)), 256, 0, st>>>(
             cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
