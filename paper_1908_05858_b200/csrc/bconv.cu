@@ -123,6 +123,7 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(cons
     rows[r] = ri;
   }
   __syncthreads();
+  chain_wait();  // (chained launches: everything above is index arithmetic)
 
   const int unit = tid % UNITS;
   const int row_first = tid / UNITS;
@@ -239,6 +240,7 @@ __global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(cons
     }
   }
   cp_async_wait<0>();
+  chain_trigger();
 
   // ---- epilogue: counts -> K - 2*count, then the selected output form -------------------------
   if (EPI == EPI_I32) {
@@ -363,7 +365,7 @@ dabnn_status launch_one(const BConvArgs& g, cudaStream_t st) {
   const int ochan = (EPI == EPI_I32) ? g.O : g.Ow32 * 32;
   const int gy = (ochan + BO - 1) / BO;
   if (gx > 0x7FFFFFFF || gy > 65535) return DABNN_ERR_UNSUPPORTED;
-  kern<<<dim3((unsigned)gx, (unsigned)gy), THREADS, SMEM, st>>>(g);
+  launch_chain(kern, dim3((unsigned)gx, (unsigned)gy), dim3(THREADS), (size_t)SMEM, st, g);
   return launch_status();
 }
 

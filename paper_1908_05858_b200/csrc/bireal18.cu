@@ -11,6 +11,8 @@
 
 namespace dabnn {
 
+bool g_chain_launch = false;  // see launch_chain() in common.cuh
+
 namespace {
 
 // ---- BN fold, in double ---------------------------------------------------------------------------
@@ -143,6 +145,7 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
     for (int i = 0; i < PPT; i++)
 #pragma unroll
       for (int j = 0; j < 8; j++) unpack_f32x2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
+    if (tile + gridDim.x >= ntiles) chain_trigger();  // the CTA's last tile: the next kernel may start its set-up
     const int n = (int)(tile / (TILES * TILES));
     const int rem = (int)(tile % (TILES * TILES));
     const int oh0 = (rem / TILES) * TS, ow0 = (rem % TILES) * TS;
@@ -283,6 +286,8 @@ __global__ void __launch_bounds__(256) maxpool_pack(const float* __restrict__ x 
   const int c4 = (int)(t & 15);
   const bool live = pix < npix;
   float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+  chain_wait();
+  chain_trigger();
   if (live) {
     const int ow = (int)(pix % 56), oh = (int)((pix / 56) % 56);
     const long long n = pix / (56 * 56);
@@ -529,6 +534,7 @@ __global__ void __launch_bounds__(256) shortcut_down_tile16(const float* __restr
     if (o0 + row < O) v = __ldg(reinterpret_cast<const float4*>(w + (size_t)(o0 + row) * C) + q);
     *reinterpret_cast<float4*>(&ws[row][4 * q]) = v;
   }
+  chain_wait();  // (chained launches: the weights above do not depend on the previous kernel)
 #pragma unroll 4
   for (int t = tid; t < 16 * C4; t += 256) {
     const int pp = t / C4, q = t - pp * C4;
@@ -550,6 +556,7 @@ __global__ void __launch_bounds__(256) shortcut_down_tile16(const float* __restr
     *reinterpret_cast<float4*>(&pooled[pp][4 * q]) = v;
   }
   __syncthreads();
+  chain_trigger();
   const int pp = tid >> 4, oo = tid & 15, o = o0 + oo;
   const long long p = p0 + pp;
   if (o >= O || p >= npix_out) return;
@@ -614,9 +621,10 @@ __global__ void __launch_bounds__(512) head_small(const float* __restrict__ x /*
     wv[u] = (j0 + row < 1000) ? __ldg(reinterpret_cast<const float4*>(fw + (size_t)(j0 + row) * 512) + q)
                               : make_float4(0.f, 0.f, 0.f, 0.f);
   }
+  chain_wait();  // (chained launches: the weight rows above do not depend on the previous kernel)
   float s = 0.0f;
 #pragma unroll 7
-  for (int q = 0; q < 49; q++) s = __fadd_rn(s, __ldg(x + ((size_t)n * 49 + q) * 512 + tid));
+  for (int q = 0; q < 49; q++) s = __fadd_rn(s, x[((size_t)n * 49 + q) * 512 + tid]);
   gs[tid] = __fdiv_rn(s, 49.0f);
 #pragma unroll
   for (int u = 0; u < 2; u++) {
@@ -749,7 +757,7 @@ dabnn_status launch_stem(const dabnn_bireal18_params* p, const float* images, in
   const long long ntiles = (long long)N * tiles * tiles;
   const long long cap = 2LL * sm_count();  // persistent: two CTAs per SM, each walking over tiles
   kern<<<(unsigned)(ntiles < cap ? ntiles : cap), (TS * TS / PPT) * 4, SMEM, st>>>(images, p->stem_w, p->stem_scale,
-                                                                                p->stem_shift, N, out);
+                                                                                p->stem_shift, N, out);  // head of a chain
   return launch_status();
 }
 
@@ -783,6 +791,13 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
   const Workspace ws = plan(N);
   if (workspace_bytes < ws.total) return DABNN_ERR_WORKSPACE;
   cudaStream_t st = as_stream(stream);
+  // One to four images: a chain of 22 short launches, each allowed to start its set-up while its predecessor finishes
+  // (see launch_chain; DABNN_NO_CHAIN=1 in the environment keeps the ordinary stream order, for measurements).
+  static const bool chain_off = getenv("DABNN_NO_CHAIN") != nullptr;
+  struct ChainScope {
+    explicit ChainScope(bool on) { g_chain_launch = on; }
+    ~ChainScope() { g_chain_launch = false; }
+  } chain_scope(N <= 4 && !chain_off);
   char* base = static_cast<char*>(workspace);
   float* stem_out = reinterpret_cast<float*>(base + ws.stem_out);
   float* cur = reinterpret_cast<float*>(base + ws.res_a);
@@ -795,7 +810,7 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
   if (s != DABNN_OK) return s;
   {
     const long long npix = (long long)N * 56 * 56;
-    maxpool_pack<<<ceil_div(npix * 16, 256), 256, 0, st>>>(stem_out, npix, cur, bits_in);
+    launch_chain(maxpool_pack, dim3(ceil_div(npix * 16, 256)), dim3(256), (size_t)0, st, stem_out, npix, cur, bits_in);
     if ((s = launch_status()) != DABNN_OK) return s;
   }
   int C = 64, HW = 56;
@@ -807,8 +822,8 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
       // less than half a wave of 128 x 128 tiles: one thread per output
       const bool few = 2 * (long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) < sm_count();
       if (few && C <= 256 && C % 4 == 0 && aligned(p->down_w[stage - 1], 16))
-        shortcut_down_tile16<<<dim3(ceil_div(npo, 16), ceil_div(O, 16)), 256, 0, st>>>(
-            cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
+        launch_chain(shortcut_down_tile16, dim3(ceil_div(npo, 16), ceil_div(O, 16)), dim3(256), (size_t)0, st, cur, HW, C,
+                     p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
       else if (few && C <= 512)
         shortcut_down_small<<<dim3(ceil_div(npo, 4), ceil_div(O, 64)), 256, 0, st>>>(
             cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
@@ -834,7 +849,7 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
   }
   {
     if (N <= 4) {
-      head_small<<<dim3(125, N), 512, 0, st>>>(cur, p->fc_w, p->fc_b, logits);
+      launch_chain(head_small, dim3(125, N), dim3(512), (size_t)0, st, cur, p->fc_w, p->fc_b, logits);
       return launch_status();
     }
     float* gbuf = reinterpret_cast<float*>(base + ws.gap);

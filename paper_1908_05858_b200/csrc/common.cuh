@@ -21,6 +21,37 @@ inline int ceil_div(long long a, long long b) { return static_cast<int>((a + b -
 // weights busy (below that the integer-pipe kernel, which spreads small problems over many small CTAs, is faster).
 bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv);
 
+// Chained launches for forwards of a few images, where every kernel is shorter than the time it takes to start one.  A
+// kernel started by launch_chain() while g_chain_launch is set may begin before its predecessor in the stream has
+// finished: it may do what does not depend on the predecessor (index set-up, fetching weights) and must call
+// chain_wait() -- which returns once the predecessor has completed and its writes are visible -- before it touches
+// anything else.  chain_trigger(), called by every CTA once its main work is done, lets the successor start.  In a
+// kernel launched the ordinary way both are no-ops.
+extern bool g_chain_launch;
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline void launch_chain(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  if (!g_chain_launch) {
+    kern<<<grid, block, smem, st>>>(args...);
+    return;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Number of SMs of the current device (cached per process; the library runs on one device at a time).
 int sm_count();
 
