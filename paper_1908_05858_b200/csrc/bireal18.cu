@@ -513,30 +513,32 @@ __global__ void __launch_bounds__(256) shortcut_down_small(const float* __restri
   y[p * O + o] = __fmaf_rn(a, scale[o], shift[o]);
 }
 
-// The same for a few images, with every global load issued before the first fmaf: a CTA takes 16 output pixels x 16
+// The same for a few images, with every global load issued before the first fmaf: a tile is 16 output pixels x 16
 // channels; its 16 weight rows and the pooled inputs of its 16 pixels go through shared memory (coalesced float4 loads,
-// all in flight at once), then each thread runs the one fmaf chain of its output over c ascending.  C <= 256, C % 4 == 0.
-__global__ void __launch_bounds__(256) shortcut_down_tile16(const float* __restrict__ x, int HW, int C,
-                                                            const float* __restrict__ w, int O,
-                                                            const float* __restrict__ scale, const float* __restrict__ shift,
-                                                            long long npix_out, float* __restrict__ y) {
-  constexpr int PITCH = 260;  // floats per row: 16 rows, read as float4, fall on distinct banks
-  __shared__ __align__(16) float pooled[16][PITCH];
-  __shared__ __align__(16) float ws[16][PITCH];
+// all in flight at once), then each thread runs the fmaf chain(s) of its output(s) over c ascending.  C <= 256, C % 4 == 0.
+// `sm` holds 2 x 16 x SC16_PITCH floats.  CHAINED: hooks of a kernel launched by launch_chain (see common.cuh).
+constexpr int SC16_PITCH = 260;  // floats per row: 16 rows, read as float4, fall on distinct banks
+template <int THREADS, bool CHAINED>
+__device__ __forceinline__ void shortcut_tile16(const float* x, int HW, int C, const float* __restrict__ w, int O,
+                                                const float* __restrict__ scale, const float* __restrict__ shift,
+                                                long long npix_out, float* y, const long long bx, const int by, float* sm) {
+  constexpr int NOUT = 256 / THREADS;  // outputs per thread, 128 apart in the tile
+  float(*pooled)[SC16_PITCH] = reinterpret_cast<float(*)[SC16_PITCH]>(sm);
+  float(*ws)[SC16_PITCH] = reinterpret_cast<float(*)[SC16_PITCH]>(sm + 16 * SC16_PITCH);
   const int tid = threadIdx.x;
-  const long long p0 = (long long)blockIdx.x * 16;
-  const int o0 = blockIdx.y * 16;
+  const long long p0 = bx * 16;
+  const int o0 = by * 16;
   const int OHW = HW / 2, C4 = C / 4;
 #pragma unroll 4
-  for (int t = tid; t < 16 * C4; t += 256) {
+  for (int t = tid; t < 16 * C4; t += THREADS) {
     const int row = t / C4, q = t - row * C4;
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (o0 + row < O) v = __ldg(reinterpret_cast<const float4*>(w + (size_t)(o0 + row) * C) + q);
     *reinterpret_cast<float4*>(&ws[row][4 * q]) = v;
   }
-  chain_wait();  // (chained launches: the weights above do not depend on the previous kernel)
+  if (CHAINED) chain_wait();  // (the weights above do not depend on the previous kernel)
 #pragma unroll 4
-  for (int t = tid; t < 16 * C4; t += 256) {
+  for (int t = tid; t < 16 * C4; t += THREADS) {
     const int pp = t / C4, q = t - pp * C4;
     const long long p = p0 + pp;
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -544,10 +546,10 @@ __global__ void __launch_bounds__(256) shortcut_down_tile16(const float* __restr
       const int ow = (int)(p % OHW), oh = (int)((p / OHW) % OHW);
       const long long n = p / ((long long)OHW * OHW);
       const float* src = x + ((n * HW + 2 * oh) * HW + 2 * ow) * C + 4 * q;
-      const float4 a = __ldg(reinterpret_cast<const float4*>(src));
-      const float4 b = __ldg(reinterpret_cast<const float4*>(src + C));
-      const float4 c = __ldg(reinterpret_cast<const float4*>(src + (size_t)HW * C));
-      const float4 d = __ldg(reinterpret_cast<const float4*>(src + (size_t)HW * C + C));
+      const float4 a = *reinterpret_cast<const float4*>(src);
+      const float4 b = *reinterpret_cast<const float4*>(src + C);
+      const float4 c = *reinterpret_cast<const float4*>(src + (size_t)HW * C);
+      const float4 d = *reinterpret_cast<const float4*>(src + (size_t)HW * C + C);
       v.x = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.x, b.x), c.x), d.x), 0.25f);
       v.y = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.y, b.y), c.y), d.y), 0.25f);
       v.z = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.z, b.z), c.z), d.z), 0.25f);
@@ -556,21 +558,37 @@ __global__ void __launch_bounds__(256) shortcut_down_tile16(const float* __restr
     *reinterpret_cast<float4*>(&pooled[pp][4 * q]) = v;
   }
   __syncthreads();
-  chain_trigger();
-  const int pp = tid >> 4, oo = tid & 15, o = o0 + oo;
-  const long long p = p0 + pp;
-  if (o >= O || p >= npix_out) return;
-  float a = 0.0f;
+  if (CHAINED) chain_trigger();
+  const int oo = tid & 15, o = o0 + oo;
+  float a[NOUT];
+#pragma unroll
+  for (int u = 0; u < NOUT; u++) a[u] = 0.0f;
 #pragma unroll 4
   for (int c = 0; c < C; c += 4) {
     const float4 wv = *reinterpret_cast<const float4*>(&ws[oo][c]);
-    const float4 pv = *reinterpret_cast<const float4*>(&pooled[pp][c]);
-    a = __fmaf_rn(pv.x, wv.x, a);
-    a = __fmaf_rn(pv.y, wv.y, a);
-    a = __fmaf_rn(pv.z, wv.z, a);
-    a = __fmaf_rn(pv.w, wv.w, a);
+#pragma unroll
+    for (int u = 0; u < NOUT; u++) {
+      const float4 pv = *reinterpret_cast<const float4*>(&pooled[(tid >> 4) + u * (THREADS / 16)][c]);
+      a[u] = __fmaf_rn(pv.x, wv.x, a[u]);
+      a[u] = __fmaf_rn(pv.y, wv.y, a[u]);
+      a[u] = __fmaf_rn(pv.z, wv.z, a[u]);
+      a[u] = __fmaf_rn(pv.w, wv.w, a[u]);
+    }
   }
-  y[p * O + o] = __fmaf_rn(a, scale[o], shift[o]);
+  if (o < O) {
+    const float sc = scale[o], sf = shift[o];
+#pragma unroll
+    for (int u = 0; u < NOUT; u++) {
+      const long long p = p0 + (tid >> 4) + u * (THREADS / 16);
+      if (p < npix_out) y[p * O + o] = __fmaf_rn(a[u], sc, sf);
+    }
+  }
+}
+__global__ void __launch_bounds__(256) shortcut_down_tile16(const float* x, int HW, int C, const float* __restrict__ w, int O,
+                                                            const float* __restrict__ scale, const float* __restrict__ shift,
+                                                            long long npix_out, float* y) {
+  __shared__ __align__(16) float sm[2 * 16 * SC16_PITCH];
+  shortcut_tile16<256, true>(x, HW, C, w, O, scale, shift, npix_out, y, blockIdx.x, blockIdx.y, sm);
 }
 
 // ---- head: global average over 7x7 (sequential sum over (h, w), then /49) into the workspace, then fc 512 -> 1000 as
