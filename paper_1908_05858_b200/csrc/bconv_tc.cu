@@ -1055,7 +1055,7 @@ bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv) {
   const int S = cv.stride_h;
   const int pads = (S == 1 && cv.pad_h <= cv.kh - 1 && cv.pad_w <= cv.kw - 1) ? 1 : 2;  // as in tc_fill
   const long long slots_total = (long long)in.N * ((in.H + pads * cv.pad_h + S - 1) / S) * ((in.W + pads * cv.pad_w + S - 1) / S);
-  return (slots_total / 128) * tc_n_ntiles(O, nt) >= (long long)sm_count();
+  return 2 * (slots_total / 128) * tc_n_ntiles(O, nt) >= (long long)sm_count();  // measured: from half a wave of tiles on
 }
 
 }  // namespace dabnn

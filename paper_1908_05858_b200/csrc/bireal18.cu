@@ -837,8 +837,10 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     const bool down = stage > 0 && b % 4 == 0;
     if (down) {
       const long long npo = (long long)N * OHW * OHW;
-      // less than half a wave of 128 x 128 tiles: one thread per output
-      const bool few = 2 * (long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) < sm_count();
+      // At most one wave of 128 x 128 tiles (whose time is then set by the length of the chain over c alone) and at most
+      // three resident rounds of 16 x 16 tiles (about 6 CTAs per SM): one thread per output.  Measured crossover.
+      const bool few = (long long)ceil_div(npo, SC_BM) * ceil_div(O, SC_BN) <= sm_count() &&
+                       (long long)ceil_div(npo, 16) * ceil_div(O, 16) <= 18LL * sm_count();
       if (few && C <= 256 && C % 4 == 0 && aligned(p->down_w[stage - 1], 16))
         launch_chain(shortcut_down_tile16, dim3(ceil_div(npo, 16), ceil_div(O, 16)), dim3(256), (size_t)0, st, cur, HW, C,
                      p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);

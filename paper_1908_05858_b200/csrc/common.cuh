@@ -17,8 +17,8 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 inline int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
 
-// True when the tensor-core engine covers this layer AND the layer has enough pixel tiles to keep every SM's resident
-// weights busy (below that the integer-pipe kernel, which spreads small problems over many small CTAs, is faster).
+// True when the tensor-core engine covers this layer AND the layer has enough pixel tiles for at least half of the SMs
+// (below that the integer-pipe kernel, which spreads small problems over many small CTAs, is faster).
 bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv);
 
 // Chained launches for forwards of a few images, where every kernel is shorter than the time it takes to start one.  A
