@@ -11,7 +11,7 @@
 
 namespace dabnn {
 
-bool g_chain_launch = false;  // see launch_chain() in common.cuh
+thread_local bool g_chain_launch = false;  // see launch_chain() in common.cuh
 
 namespace {
 
@@ -311,23 +311,27 @@ __global__ void __launch_bounds__(256) maxpool_pack(const float* __restrict__ x 
 }
 
 // ---- downsample shortcut: avgpool 2x2 / 2 -> fp32 conv 1x1 (C -> O) -> BN ---------------------------
-// A register-tiled matrix product with a fixed summation order: CTA tile 128 output pixels x 128 output channels,
-// 256 threads, 8 pixels x 8 channels per thread, K (= C) in chunks of 16 through two shared-memory stages.  The pooled
-// activations are formed on the fly (four loads, three adds, one multiply, in that order) while the previous chunk is
-// being multiplied; weights arrive with cp.async.  Each output is one fmaf chain over c ascending, as pinned.
-constexpr int SC_BM = 128, SC_BN = 128, SC_BK = 16;
-__global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x /*[N][HW][HW][C]*/, int HW, int C,
+// A register-tiled matrix product with a fixed summation order: CTA tile BM (64 or 128) output pixels x 128 output
+// channels, 256 threads, BM/16 pixels x 8 channels per thread, K (= C) in chunks of 16 through two shared-memory stages.
+// The pooled activations are formed on the fly (four loads, three adds, one multiply, in that order) and the weights loaded
+// while the previous chunk is being multiplied.  Each output is one fmaf chain over c ascending, as pinned.
+constexpr int SC_BM = 128, SC_BN = 128, SC_BK = 16;  // SC_BM: the pixel tile the small-batch crossover below was measured with
+template <int BM>
+__global__ void __launch_bounds__(256, BM == 128 ? 2 : 3) shortcut_down(const float* __restrict__ x /*[N][HW][HW][C]*/, int HW, int C,
                                                      const float* __restrict__ w /*[O][C]*/, int O,
                                                      const float* __restrict__ scale, const float* __restrict__ shift,
                                                      long long npix_out, float* __restrict__ y /*[N][HW/2][HW/2][O]*/) {
-  __shared__ __align__(16) float p_s[2][SC_BK][SC_BM + 4];  // [stage][c][pixel]
+  constexpr int PV = BM * SC_BK / 256;   // pooled values a thread forms per chunk: 8 or 4 consecutive c of one pixel
+  constexpr int TYP = BM / 16;           // pixels per thread in the register tile
+  static_assert(BM == 128 || BM == 64, "pixel tile");
+  __shared__ __align__(16) float p_s[2][SC_BK][BM + 4];  // [stage][c][pixel]
   __shared__ __align__(16) float w_s[2][SC_BK][SC_BN + 4];  // [stage][c][channel]
   const int tid = threadIdx.x;
-  const long long p0 = (long long)blockIdx.x * SC_BM;
+  const long long p0 = (long long)blockIdx.x * BM;
   const int o0 = blockIdx.y * SC_BN;
   const int OHW = HW / 2;
-  // loader roles: a thread pools 8 (pixel, c) pairs per chunk: pixel = tid / 2, c = (tid % 2) * 8 .. +7
-  const int lp = tid >> 1, lc = (tid & 1) * 8;
+  // loader roles: a thread pools PV (pixel, c) pairs per chunk: pixel = tid / (16 / PV), c = (tid % (16 / PV)) * PV .. + PV - 1
+  const int lp = tid / (SC_BK / PV), lc = (tid % (SC_BK / PV)) * PV;
   const long long pl = p0 + lp;
   const float* xq = nullptr;
   if (pl < npix_out) {
@@ -338,19 +342,19 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
   // weights: 16 c x 128 channels per chunk = 2048 floats: thread copies 8 floats of one channel row: channel = tid / 2
   const int wo = tid >> 1, wc = (tid & 1) * 8;
   const bool c_vec = (C % 8 == 0) && (reinterpret_cast<uintptr_t>(x) % 16 == 0) && (reinterpret_cast<uintptr_t>(w) % 16 == 0);
-  float pooled[8];
+  float pooled[PV];
   auto pool_load = [&](int c0) {  // registers <- pooled values of chunk c0
 #pragma unroll
-    for (int k = 0; k < 8; k++) pooled[k] = 0.0f;
+    for (int k = 0; k < PV; k++) pooled[k] = 0.0f;
     if (xq == nullptr) return;
     const int c = c0 + lc;
-    if (c_vec && c + 8 <= C) {
+    if (c_vec && c + PV <= C) {
       const float4* q00 = reinterpret_cast<const float4*>(xq + c);
       const float4* q01 = reinterpret_cast<const float4*>(xq + C + c);
       const float4* q10 = reinterpret_cast<const float4*>(xq + (size_t)HW * C + c);
       const float4* q11 = reinterpret_cast<const float4*>(xq + (size_t)HW * C + C + c);
 #pragma unroll
-      for (int h = 0; h < 2; h++) {
+      for (int h = 0; h < PV / 4; h++) {
         const float4 a = __ldcs(q00 + h), b = __ldcs(q01 + h), cc = __ldcs(q10 + h), d = __ldcs(q11 + h);  // read once
         pooled[4 * h + 0] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.x, b.x), cc.x), d.x), 0.25f);
         pooled[4 * h + 1] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(a.y, b.y), cc.y), d.y), 0.25f);
@@ -359,7 +363,7 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
       }
     } else {
 #pragma unroll
-      for (int k = 0; k < 8; k++)
+      for (int k = 0; k < PV; k++)
         if (c + k < C) {
           const float* q = xq + c + k;
           pooled[k] = __fmul_rn(__fadd_rn(__fadd_rn(__fadd_rn(q[0], q[C]), q[(size_t)HW * C]), q[(size_t)HW * C + C]), 0.25f);
@@ -368,7 +372,7 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
   };
   auto pool_store = [&](int st) {
 #pragma unroll
-    for (int k = 0; k < 8; k++) p_s[st][lc + k][lp] = pooled[k];
+    for (int k = 0; k < PV; k++) p_s[st][lc + k][lp] = pooled[k];
   };
   float wreg[8];
   auto w_load = [&](int c0) {
@@ -390,11 +394,11 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
 #pragma unroll
     for (int k = 0; k < 8; k++) w_s[st][wc + k][wo] = wreg[k];
   };
-  // compute roles: 16 x 16 threads; thread (ty, tx) owns pixels ty*8..+7 and channels tx*4..+3 and 64 + tx*4..+3
+  // compute roles: 16 x 16 threads; thread (ty, tx) owns pixels ty*TYP..+TYP-1 and channels tx*4..+3 and 64 + tx*4..+3
   const int ty = tid >> 4, tx = tid & 15;
-  unsigned long long acc2[8][4];  // channel pairs of each pixel (packed fp32 FMAs, same rounding as scalar fmaf)
+  unsigned long long acc2[TYP][4];  // channel pairs of each pixel (packed fp32 FMAs, same rounding as scalar fmaf)
 #pragma unroll
-  for (int i = 0; i < 8; i++)
+  for (int i = 0; i < TYP; i++)
 #pragma unroll
     for (int j = 0; j < 4; j++) acc2[i][j] = 0ull;
   const int nchunks = (C + SC_BK - 1) / SC_BK;
@@ -412,15 +416,18 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
     const int cn = min(SC_BK, C - ch * SC_BK);
 #pragma unroll 4
     for (int cc = 0; cc < cn; cc++) {
-      const float4 pa = *reinterpret_cast<const float4*>(&p_s[st][cc][ty * 8]);
-      const float4 pb = *reinterpret_cast<const float4*>(&p_s[st][cc][ty * 8 + 4]);
+      float pv[TYP];
+#pragma unroll
+      for (int i = 0; i < TYP; i += 4) {
+        const float4 pa = *reinterpret_cast<const float4*>(&p_s[st][cc][ty * TYP + i]);
+        pv[i] = pa.x; pv[i + 1] = pa.y; pv[i + 2] = pa.z; pv[i + 3] = pa.w;
+      }
       const float4 wa = *reinterpret_cast<const float4*>(&w_s[st][cc][tx * 4]);
       const float4 wb = *reinterpret_cast<const float4*>(&w_s[st][cc][64 + tx * 4]);
-      const float pv[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
       const unsigned long long w2[4] = {pack_f32x2(wa.x, wa.y), pack_f32x2(wa.z, wa.w), pack_f32x2(wb.x, wb.y),
                                         pack_f32x2(wb.z, wb.w)};
 #pragma unroll
-      for (int i = 0; i < 8; i++) {
+      for (int i = 0; i < TYP; i++) {
         const unsigned long long p2 = pack_f32x2(pv[i], pv[i]);
 #pragma unroll
         for (int j = 0; j < 4; j++) fma_f32x2(acc2[i][j], p2, w2[j]);
@@ -432,9 +439,9 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
     }
     __syncthreads();
   }
-  float acc[8][8];
+  float acc[TYP][8];
 #pragma unroll
-  for (int i = 0; i < 8; i++)
+  for (int i = 0; i < TYP; i++)
 #pragma unroll
     for (int j = 0; j < 4; j++) unpack_f32x2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
 #pragma unroll
@@ -448,8 +455,8 @@ __global__ void __launch_bounds__(256) shortcut_down(const float* __restrict__ x
       sf[j] = (o + j < O) ? shift[o + j] : 0.0f;
     }
 #pragma unroll
-    for (int i = 0; i < 8; i++) {
-      const long long p = p0 + ty * 8 + i;
+    for (int i = 0; i < TYP; i++) {
+      const long long p = p0 + ty * TYP + i;
       if (p >= npix_out) continue;
       float* dst = y + p * O + o;
       const float r0 = __fmaf_rn(acc[i][4 * h], sc[0], sf[0]), r1 = __fmaf_rn(acc[i][4 * h + 1], sc[1], sf[1]);
@@ -592,36 +599,13 @@ __global__ void __launch_bounds__(256) shortcut_down_tile16(const float* x, int 
 }
 
 // ---- head: global average over 7x7 (sequential sum over (h, w), then /49) into the workspace, then fc 512 -> 1000 as
-// one fmaf chain per logit over k ascending, then + bias.  Small batches: 32-thread CTAs, one image each.
+// one fmaf chain per logit over k ascending, then + bias.  Three forms of the fc, by batch size, below.
 __global__ void __launch_bounds__(512) gap_small(const float* __restrict__ x /*[N][7][7][512]*/, float* __restrict__ g) {
   const int n = blockIdx.x, c = threadIdx.x;
   float s = 0.0f;
   for (int q = 0; q < 49; q++) s = __fadd_rn(s, x[((size_t)n * 49 + q) * 512 + c]);
   g[(size_t)n * 512 + c] = __fdiv_rn(s, 49.0f);
 }
-__global__ void __launch_bounds__(32) fc_small(const float* __restrict__ g /*[N][512]*/, const float* __restrict__ fw,
-                                               const float* __restrict__ fb, float* __restrict__ logits) {
-  __shared__ __align__(16) float gs[512];
-  const int n = blockIdx.y;
-  for (int t = threadIdx.x; t < 128; t += 32)
-    reinterpret_cast<float4*>(gs)[t] = reinterpret_cast<const float4*>(g + (size_t)n * 512)[t];
-  __syncwarp();
-  const int j = blockIdx.x * 32 + threadIdx.x;
-  if (j >= 1000) return;
-  const float4* wr = reinterpret_cast<const float4*>(fw + (size_t)j * 512);
-  float a = 0.0f;
-#pragma unroll 8
-  for (int k4 = 0; k4 < 128; k4++) {
-    const float4 wv = __ldg(wr + k4);
-    const float4 gv = reinterpret_cast<const float4*>(gs)[k4];
-    a = __fmaf_rn(gv.x, wv.x, a);
-    a = __fmaf_rn(gv.y, wv.y, a);
-    a = __fmaf_rn(gv.z, wv.z, a);
-    a = __fmaf_rn(gv.w, wv.w, a);
-  }
-  logits[(size_t)n * 1000 + j] = __fadd_rn(a, fb[j]);
-}
-
 // One to four images: pooling and fc in one launch.  A 512-thread CTA takes 8 logits of one image: it pools the image's
 // 7x7x512 map itself (thread c owns channel c; same sum order and division as gap_small) while its 8 weight rows are in
 // flight, then 8 threads run the 8 fmaf chains out of shared memory.
@@ -663,6 +647,45 @@ __global__ void __launch_bounds__(512) head_small(const float* __restrict__ x /*
     a = __fmaf_rn(g4.w, w4.w, a);
   }
   logits[(size_t)n * 1000 + j] = __fadd_rn(a, fb[j]);
+}
+
+// Five to 63 images: pooled vectors come from gap_small; a 64-thread CTA takes 8 logits of up to 8 images.  Its 8 weight
+// rows and the images' pooled vectors are staged in shared memory by coalesced loads, all in flight at once; thread
+// (image, logit) then runs its fmaf chain over k ascending.
+__global__ void __launch_bounds__(64) fc_mid(const float* __restrict__ g /*[N][512]*/, int N, const float* __restrict__ fw,
+                                             const float* __restrict__ fb, float* __restrict__ logits) {
+  constexpr int PITCH = 516;
+  __shared__ __align__(16) float gs[8][PITCH];
+  __shared__ __align__(16) float ws[8][PITCH];
+  const int tid = threadIdx.x, j0 = blockIdx.x * 8, n0 = blockIdx.y * 8;
+  float4 wv[16], gv[16];
+#pragma unroll
+  for (int u = 0; u < 16; u++) {  // 8 rows x 128 float4 each
+    const int idx = tid + 64 * u, row = idx >> 7, q = idx & 127;
+    wv[u] = (j0 + row < 1000) ? __ldg(reinterpret_cast<const float4*>(fw + (size_t)(j0 + row) * 512) + q)
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
+    gv[u] = (n0 + row < N) ? *(reinterpret_cast<const float4*>(g + (size_t)(n0 + row) * 512) + q)
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll
+  for (int u = 0; u < 16; u++) {
+    const int idx = tid + 64 * u, row = idx >> 7, q = idx & 127;
+    *reinterpret_cast<float4*>(&ws[row][4 * q]) = wv[u];
+    *reinterpret_cast<float4*>(&gs[row][4 * q]) = gv[u];
+  }
+  __syncthreads();
+  const int jj = tid & 7, im = tid >> 3, j = j0 + jj, n = n0 + im;
+  float a = 0.0f;
+#pragma unroll 8
+  for (int k = 0; k < 512; k += 4) {
+    const float4 w4 = *reinterpret_cast<const float4*>(&ws[jj][k]);
+    const float4 g4 = *reinterpret_cast<const float4*>(&gs[im][k]);
+    a = __fmaf_rn(g4.x, w4.x, a);
+    a = __fmaf_rn(g4.y, w4.y, a);
+    a = __fmaf_rn(g4.z, w4.z, a);
+    a = __fmaf_rn(g4.w, w4.w, a);
+  }
+  if (j < 1000 && n < N) logits[(size_t)n * 1000 + j] = __fadd_rn(a, fb[j]);
 }
 
 // Larger batches: pooled vectors come from gap_small; a 64-thread CTA computes 64 logits for 8 images, so every weight
@@ -847,8 +870,8 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
       else if (few && C <= 512)
         shortcut_down_small<<<dim3(ceil_div(npo, 4), ceil_div(O, 64)), 256, 0, st>>>(
             cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
-      else
-        shortcut_down<<<dim3(ceil_div(npo, SC_BM), ceil_div(O, SC_BN)), 256, 0, st>>>(
+      else  // 64-pixel tiles: 80 registers, three CTAs per SM, and less lost to the last, partly filled round than with 128
+        shortcut_down<64><<<dim3(ceil_div(npo, 64), ceil_div(O, SC_BN)), 256, 0, st>>>(
             cur, HW, C, p->down_w[stage - 1], O, p->down_scale[stage - 1], p->down_shift[stage - 1], npo, other);
       if ((s = launch_status()) != DABNN_OK) return s;
       float* t = cur; cur = other; other = t;
@@ -875,7 +898,7 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     float* gbuf = reinterpret_cast<float*>(base + ws.gap);
     gap_small<<<N, 512, 0, st>>>(cur, gbuf);
     if ((s = launch_status()) != DABNN_OK) return s;
-    if (N < 64) fc_small<<<dim3(ceil_div(1000, 32), N), 32, 0, st>>>(gbuf, p->fc_w, p->fc_b, logits);  // few images: many small CTAs
+    if (N < 64) fc_mid<<<dim3(125, ceil_div(N, 8)), 64, 0, st>>>(gbuf, N, p->fc_w, p->fc_b, logits);
     else fc_batched<<<dim3(ceil_div(1000, 64), ceil_div(N, 8)), 64, 0, st>>>(gbuf, N, p->fc_w, p->fc_b, logits);
   }
   return launch_status();

@@ -27,7 +27,7 @@ bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv);
 // chain_wait() -- which returns once the predecessor has completed and its writes are visible -- before it touches
 // anything else.  chain_trigger(), called by every CTA once its main work is done, lets the successor start.  In a
 // kernel launched the ordinary way both are no-ops.
-extern bool g_chain_launch;
+extern thread_local bool g_chain_launch;  // per host thread: set by a forward call for the launches it makes itself
 #ifdef __CUDACC__
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void chain_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
