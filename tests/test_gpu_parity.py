@@ -287,6 +287,32 @@ def test_bgemm_matches_eq1(B, oracle_mod, shape):
     assert np.array_equal(got, 2 * counts - K)
 
 
+def test_bireal18_four_and_five_images_match_oracle(B, oracle_mod):
+    """Four images take the chained launches, the 16x32 convolution tile and the pooling + fc kernel; five take the
+    ordinary stream order and the staged fc kernel.  Both must equal the oracle bit for bit, eagerly and as a CUDA graph."""
+    p = synth.bireal18_params()
+    img = synth.bireal18_images(5)
+    want = oracle_mod.bireal18_forward(p, img, conv_form=1)
+    net = B.Bireal18(p)
+    x5, x4 = dev(img), dev(img[:4])
+    got5 = net.forward(x5).cpu().numpy()
+    got4 = net.forward(x4).cpu().numpy()
+    assert np.array_equal(got5.view(np.uint32), want.view(np.uint32))
+    assert np.array_equal(got4.view(np.uint32), want[:4].view(np.uint32))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        net.forward(x4)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            out = net.forward(x4)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().view(np.uint32), want[:4].view(np.uint32))
+
+
 def test_bireal18_large_batch_kernels_match_oracle(B, oracle_mod):
     """Batch 8 is large enough for the persistent 8x8-tile stem, the tiled shortcut kernel and the tensor-core engine
     on the early stages; the logits must still equal the oracle's bit for bit."""
