@@ -26,12 +26,20 @@ __global__ void bn_fold_kernel(const float* gamma, const float* beta, const floa
 }
 
 // ---- stem: conv 7x7 / 2, 3 -> 64, zero pad 3, then BN ----------------------------------------------
-// A CTA computes a TS x TS tile of output pixels for all 64 channels.  The input patch sits in shared
+// A CTA computes a TS x TS tile of output pixels for 4 * CPT channels (all 64 with CPT = 16; with CPT = 8 two CTAs
+// share a tile, which spreads a single image over twice as many CTAs).  The input patch sits in shared
 // memory with even and odd columns apart, so that lanes walking along ow (input stride 2) read
-// consecutive words.  A thread owns PPT pixels (rows TS/PPT apart... see below) x 16 channels and runs one fmaf
+// consecutive words.  A thread owns PPT pixels (rows TS/PPT apart... see below) x CPT channels and runs one fmaf
 // chain per output over (c, kh, kw) in that order.  Zero padding is held as zeros in the patch:
 // fmaf(0, w, acc) returns acc.
 constexpr int STEM_K = 147;
+// Columns per parity of the input patch, padded: the lanes of a warp read 8 consecutive columns of 4 patch rows that
+// are two rows (4 * half words) apart, which fall on distinct banks when 4 * half is 8 or 24 modulo 32.
+__host__ __device__ constexpr int stem_half(int ps) {
+  int h = (ps + 1) / 2 + 1;
+  while ((4 * h) % 32 != 8 && (4 * h) % 32 != 24) h++;
+  return h;
+}
 
 // Two fp32 fused multiply-adds in one instruction (fma.rn.f32x2): each lane of the pair is the same correctly rounded
 // fmaf as the scalar instruction, so results do not change; it halves the issue slots of an FMA-bound loop.
@@ -47,7 +55,7 @@ __device__ __forceinline__ void fma_f32x2(unsigned long long& acc, unsigned long
   asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
 }
 
-template <int TS, int PPT>
+template <int TS, int PPT, int CPT>
 __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const float* __restrict__ img,
                                                                        const float* __restrict__ w,
                                                                        const float* __restrict__ scale,
@@ -55,24 +63,28 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
                                                                        float* __restrict__ out /*[N][112][112][64]*/) {
   constexpr int IH = 224, IW = 224, OHW = 112;
   constexpr int PS = 2 * TS + 5;         // patch side
-  constexpr int HALF = (PS + 1) / 2 + 1; // columns per parity, padded
+  constexpr int HALF = stem_half(PS);
   constexpr int PATCH = 3 * PS * 2 * HALF;  // floats per patch buffer
   constexpr int PGROUPS = TS * TS / PPT; // pixel groups = threads per channel group
   constexpr int THREADS = PGROUPS * 4;
   constexpr int RSTEP = TS / PPT;        // a thread's pixels are RSTEP rows apart
   constexpr int TILES = (OHW + TS - 1) / TS;
+  constexpr int CB = 4 * CPT;            // channels per CTA (blockIdx.y picks which): four thread groups of CPT channels
+  static_assert(CPT == 16 || CPT == 8, "channels per thread");
   extern __shared__ __align__(16) float sm[];
-  float* w_s = sm;                       // [147][64], filled once per CTA
-  float* x_s = sm + STEM_K * 64;         // [2 buffers][3][PS][2][HALF]
-  float* w_raw = x_s + 2 * PATCH;        // [64][147] as in global memory, until it has been transposed into w_s
+  float* w_s = sm;                       // [147][CB], filled once per CTA
+  float* x_s = sm + STEM_K * CB;         // [2 buffers][3][PS][2][HALF]
+  float* w_raw = x_s + 2 * PATCH;        // [CB][147] as in global memory, until it has been transposed into w_s
+  const int ch0 = blockIdx.y * CB;
+  w += (size_t)ch0 * STEM_K;             // this CTA's rows of the [64][147] weight matrix
   const int tid = threadIdx.x;
   if ((reinterpret_cast<uintptr_t>(w) & 15) == 0) {  // one coalesced asynchronous copy, in flight together with the first patch
-    for (int t = tid; t < STEM_K * 16; t += THREADS) {
+    for (int t = tid; t < STEM_K * CB / 4; t += THREADS) {
       const uint32_t d = (uint32_t)__cvta_generic_to_shared(w_raw + 4 * t);
       asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(w + 4 * t) : "memory");
     }
   } else {
-    for (int t = tid; t < STEM_K * 64; t += THREADS) w_raw[t] = w[t];
+    for (int t = tid; t < STEM_K * CB; t += THREADS) w_raw[t] = w[t];
   }
   const long long ntiles = (long long)N * TILES * TILES;
   // asynchronous copy of one tile's zero-padded input patch (even and odd columns apart)
@@ -93,29 +105,29 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
   const int cg = tid / PGROUPS;          // channel group: 16 channels
   const int pg = tid % PGROUPS;
   const int low = pg % TS, lohb = pg / TS;  // pixels (lohb + RSTEP*i, low)
-  float sc[16], sf[16];
+  float sc[CPT], sf[CPT];
 #pragma unroll
-  for (int j = 0; j < 16; j++) {
-    sc[j] = scale[cg * 16 + j];
-    sf[j] = shift[cg * 16 + j];
+  for (int j = 0; j < CPT; j++) {
+    sc[j] = scale[ch0 + cg * CPT + j];
+    sf[j] = shift[ch0 + cg * CPT + j];
   }
   long long tile = blockIdx.x;
   int buf = 0;
   if (tile < ntiles) load_patch(tile, x_s);
   asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
-  // [64][147] -> [147][64]: lanes walk over o, 147 words apart in w_raw (an odd stride: distinct banks) and consecutive in w_s
-  for (int t = tid; t < STEM_K * 64; t += THREADS) w_s[t] = w_raw[(t & 63) * STEM_K + (t >> 6)];
+  // [CB][147] -> [147][CB]: lanes walk over o, 147 words apart in w_raw (an odd stride: distinct banks) and consecutive in w_s
+  for (int t = tid; t < STEM_K * CB; t += THREADS) w_s[t] = w_raw[(t % CB) * STEM_K + t / CB];
   for (; tile < ntiles; tile += gridDim.x, buf ^= 1) {
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();  // this tile's patch (and, the first time, the weights) are in place; the other buffer is free
     if (tile + gridDim.x < ntiles) load_patch(tile + gridDim.x, x_s + (buf ^ 1) * PATCH);
     const float* xb = x_s + buf * PATCH;
-    unsigned long long acc2[PPT][8];  // channel pairs (packed fp32 FMAs, same rounding as scalar fmaf)
+    unsigned long long acc2[PPT][CPT / 2];  // channel pairs (packed fp32 FMAs, same rounding as scalar fmaf)
 #pragma unroll
     for (int i = 0; i < PPT; i++)
 #pragma unroll
-      for (int j = 0; j < 8; j++) acc2[i][j] = 0ull;
+      for (int j = 0; j < CPT / 2; j++) acc2[i][j] = 0ull;
 #pragma unroll 1
     for (int c = 0; c < 3; c++)
 #pragma unroll 1
@@ -123,10 +135,10 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
 #pragma unroll
         for (int kj = 0; kj < 7; kj++) {
           const int k = (c * 7 + ki) * 7 + kj;
-          unsigned long long w2[8];
+          unsigned long long w2[CPT / 2];
 #pragma unroll
-          for (int q = 0; q < 4; q++) {
-            const float4 t4 = *reinterpret_cast<const float4*>(w_s + k * 64 + cg * 16 + 4 * q);
+          for (int q = 0; q < CPT / 4; q++) {
+            const float4 t4 = *reinterpret_cast<const float4*>(w_s + k * CB + cg * CPT + 4 * q);
             w2[2 * q] = pack_f32x2(t4.x, t4.y);
             w2[2 * q + 1] = pack_f32x2(t4.z, t4.w);
           }
@@ -136,15 +148,15 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
             const float xv = xb[((c * PS + lh) * 2 + (kj & 1)) * HALF + low + (kj >> 1)];
             const unsigned long long x2 = pack_f32x2(xv, xv);
 #pragma unroll
-            for (int j = 0; j < 8; j++) fma_f32x2(acc2[i][j], x2, w2[j]);
+            for (int j = 0; j < CPT / 2; j++) fma_f32x2(acc2[i][j], x2, w2[j]);
           }
         }
       }
-    float acc[PPT][16];
+    float acc[PPT][CPT];
 #pragma unroll
     for (int i = 0; i < PPT; i++)
 #pragma unroll
-      for (int j = 0; j < 8; j++) unpack_f32x2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
+      for (int j = 0; j < CPT / 2; j++) unpack_f32x2(acc2[i][j], acc[i][2 * j], acc[i][2 * j + 1]);
     if (tile + gridDim.x >= ntiles) chain_trigger();  // the CTA's last tile: the next kernel may start its set-up
     const int n = (int)(tile / (TILES * TILES));
     const int rem = (int)(tile % (TILES * TILES));
@@ -153,9 +165,9 @@ __global__ void __launch_bounds__((TS * TS / PPT) * 4, 2) stem_conv_bn(const flo
     for (int i = 0; i < PPT; i++) {
       const int oh = oh0 + lohb + RSTEP * i, ow = ow0 + low;
       if (oh >= OHW || ow >= OHW) continue;
-      float* dst = out + (((size_t)n * OHW + oh) * OHW + ow) * 64 + cg * 16;
+      float* dst = out + (((size_t)n * OHW + oh) * OHW + ow) * 64 + ch0 + cg * CPT;
 #pragma unroll
-      for (int j = 0; j < 16; j += 4)
+      for (int j = 0; j < CPT; j += 4)
         *reinterpret_cast<float4*>(dst + j) =
             make_float4(__fmaf_rn(acc[i][j], sc[j], sf[j]), __fmaf_rn(acc[i][j + 1], sc[j + 1], sf[j + 1]),
                         __fmaf_rn(acc[i][j + 2], sc[j + 2], sf[j + 2]), __fmaf_rn(acc[i][j + 3], sc[j + 3], sf[j + 3]));
@@ -781,11 +793,11 @@ dabnn_status launch_stem_8x8(const dabnn_bireal18_params* p, const float* images
   return launch_status();
 }
 
-template <int TS, int PPT>
+template <int TS, int PPT, int CPT>
 dabnn_status launch_stem(const dabnn_bireal18_params* p, const float* images, int N, float* out, cudaStream_t st) {
-  constexpr int PS = 2 * TS + 5, HALF = (PS + 1) / 2 + 1;
-  constexpr size_t SMEM = (size_t)(2 * STEM_K * 64 + 2 * 3 * PS * 2 * HALF) * 4;
-  auto kern = stem_conv_bn<TS, PPT>;
+  constexpr int PS = 2 * TS + 5, HALF = stem_half(PS);
+  constexpr size_t SMEM = (size_t)(2 * STEM_K * 4 * CPT + 2 * 3 * PS * 2 * HALF) * 4;
+  auto kern = stem_conv_bn<TS, PPT, CPT>;
   static bool configured = false;
   if (!configured) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) {
@@ -797,8 +809,8 @@ dabnn_status launch_stem(const dabnn_bireal18_params* p, const float* images, in
   const int tiles = (112 + TS - 1) / TS;
   const long long ntiles = (long long)N * tiles * tiles;
   const long long cap = 2LL * sm_count();  // persistent: two CTAs per SM, each walking over tiles
-  kern<<<(unsigned)(ntiles < cap ? ntiles : cap), (TS * TS / PPT) * 4, SMEM, st>>>(images, p->stem_w, p->stem_scale,
-                                                                                p->stem_shift, N, out);  // head of a chain
+  kern<<<dim3((unsigned)(ntiles < cap ? ntiles : cap), 16 / CPT), (TS * TS / PPT) * 4, SMEM, st>>>(
+      images, p->stem_w, p->stem_scale, p->stem_shift, N, out);  // head of a chain
   return launch_status();
 }
 
@@ -847,7 +859,8 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
   uint64_t* bits_out = reinterpret_cast<uint64_t*>(base + ws.bits_b);
 
   dabnn_status s = (N * 49 >= 2 * sm_count()) ? launch_stem_8x8(p, images, N, stem_out, st)
-                                               : launch_stem<8, 1>(p, images, N, stem_out, st);
+                                               : (N == 1 ? launch_stem<8, 2, 8>(p, images, N, stem_out, st)  // one image: 392 half-tile CTAs
+                                                          : launch_stem<8, 2, 16>(p, images, N, stem_out, st));
   if (s != DABNN_OK) return s;
   {
     const long long npix = (long long)N * 56 * 56;
