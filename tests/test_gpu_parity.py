@@ -313,6 +313,25 @@ def test_bireal18_four_and_five_images_match_oracle(B, oracle_mod):
     assert np.array_equal(out.cpu().numpy().view(np.uint32), want[:4].view(np.uint32))
 
 
+def test_bireal18_stem_weights_at_an_unaligned_address(B):
+    """The small stem copies its weights with 16-byte asynchronous copies when it can and element by element when the
+    caller's array is only 4-byte aligned; both give the same logits."""
+    p = synth.bireal18_params()
+    img = synth.bireal18_images(2)
+    net = B.Bireal18(p)
+    want2 = net.forward(dev(img)).cpu().numpy()
+    want1 = net.forward(dev(img[:1])).cpu().numpy()
+    flat = net.stem_w.flatten()
+    shifted = torch.empty(flat.numel() + 1, dtype=torch.float32, device=flat.device)
+    shifted[1:].copy_(flat)
+    assert shifted[1:].data_ptr() % 16 == 4
+    net.P.stem_w = shifted[1:].data_ptr()
+    got2 = net.forward(dev(img)).cpu().numpy()
+    got1 = net.forward(dev(img[:1])).cpu().numpy()
+    assert np.array_equal(got2.view(np.uint32), want2.view(np.uint32))
+    assert np.array_equal(got1.view(np.uint32), want1.view(np.uint32))
+
+
 def test_bireal18_large_batch_kernels_match_oracle(B, oracle_mod):
     """Batch 8 is large enough for the persistent 8x8-tile stem, the tiled shortcut kernel and the tensor-core engine
     on the early stages; the logits must still equal the oracle's bit for bit."""
