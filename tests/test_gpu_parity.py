@@ -332,6 +332,33 @@ def test_bireal18_stem_weights_at_an_unaligned_address(B):
     assert np.array_equal(got1.view(np.uint32), want1.view(np.uint32))
 
 
+def test_bireal18_shortcut_and_block_weights_at_unaligned_addresses(B):
+    """The small-batch shortcut kernel with staged weight rows wants 16-byte aligned 1x1 weights, and the convolution's
+    16-byte copies 16-byte aligned packed weights; arrays that are only 4- / 8-byte aligned take the other kernels and
+    copy units and must give the same logits."""
+    p = synth.bireal18_params()
+    img = dev(synth.bireal18_images(2))
+    net = B.Bireal18(p, engine="popc")
+    want = net.forward(img).cpu().numpy()
+    keep = []
+    for d in range(3):
+        n = int(np.prod(p["down_w"][d].shape))
+        src = torch.from_numpy(np.ascontiguousarray(p["down_w"][d], dtype=np.float32)).flatten().to(img.device)
+        buf = torch.empty(n + 1, dtype=torch.float32, device=img.device)
+        buf[1:].copy_(src)
+        keep.append(buf)
+        net.P.down_w[d] = buf[1:].data_ptr()
+    for b in range(16):
+        wp = B.pack_weights(dev(p["block_w"][b])).flatten()
+        buf = torch.empty(wp.numel() + 1, dtype=torch.int64, device=img.device)
+        buf[1:].copy_(wp)
+        assert buf[1:].data_ptr() % 16 == 8
+        keep.append(buf)
+        net.P.block_w[b] = buf[1:].data_ptr()
+    got = net.forward(img).cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
 def test_bireal18_large_batch_kernels_match_oracle(B, oracle_mod):
     """Batch 8 is large enough for the persistent 8x8-tile stem, the tiled shortcut kernel and the tensor-core engine
     on the early stages; the logits must still equal the oracle's bit for bit."""
