@@ -359,6 +359,54 @@ def test_bireal18_shortcut_and_block_weights_at_unaligned_addresses(B):
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
 
 
+def test_forward_and_convolution_from_two_host_threads(B):
+    """A batch-1 forward (chained launches, a per-thread setting inside the library) on one host thread and stream while
+    another thread launches plain convolutions on its own stream: both keep giving their single-threaded results."""
+    import threading
+    p = synth.bireal18_params()
+    net = B.Bireal18(p, engine="popc")
+    img = dev(synth.bireal18_images(1))
+    want_logits = net.forward(img).cpu().numpy()
+    case = CONV_CASES[8]
+    N, C, H, W, O, kh, kw, stride, pad, pv = case
+    x, w = conv_inputs(case)
+    a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
+    want_conv = B.bconv2d(a, C, wp, stride, pad, pv, B.NHWC).cpu().numpy()
+    torch.cuda.synchronize()
+    errors = []
+
+    def forwards():
+        try:
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                for _ in range(40):
+                    got = net.forward(img)
+                s.synchronize()
+                if not np.array_equal(got.cpu().numpy().view(np.uint32), want_logits.view(np.uint32)):
+                    errors.append("logits differ")
+        except Exception as e:  # noqa: BLE001
+            errors.append(repr(e))
+
+    def convs():
+        try:
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                for _ in range(200):
+                    got = B.bconv2d(a, C, wp, stride, pad, pv, B.NHWC)
+                s.synchronize()
+                if not np.array_equal(got.cpu().numpy(), want_conv):
+                    errors.append("convolution differs")
+        except Exception as e:  # noqa: BLE001
+            errors.append(repr(e))
+
+    threads = [threading.Thread(target=forwards), threading.Thread(target=convs)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert errors == []
+
+
 def test_bireal18_large_batch_kernels_match_oracle(B, oracle_mod):
     """Batch 8 is large enough for the persistent 8x8-tile stem, the tiled shortcut kernel and the tensor-core engine
     on the early stages; the logits must still equal the oracle's bit for bit."""
