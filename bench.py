@@ -368,7 +368,7 @@ def main():
         "bound": "alu", "kernel": "bconv_kernel (integer pipes: xor + carry-save + popc), same 8 launches",
         "achieved": conv_ops / (popc_ms * 1e-3) / 1e12, "peak": alu_peak, "unit": "Tbit-ops/s",
         "frac": conv_ops / (popc_ms * 1e-3) / 1e12 / alu_peak,
-        "peak_is": "ALU+XU carry-save bound at %d SMs x %.0f MHz (derived, see DESIGN.md); the one-POPC-per-word-pair bound is half of it"
+        "peak_is": "ALU+XU carry-save bound at %d SMs x %.0f MHz (derived: 64 LOP3 lanes and 16 POPC lanes per clock and SM, carry-save halves the POPCs); the one-POPC-per-word-pair bound is half of it"
                    % (sm_count, peaks["sm_max_mhz"]),
         "traffic": 2.69e6, "traffic_is": "dram bytes of one N=64 C=256 28x28 launch (ncu, profiles/bconv_kernel_N64_C256_HW28.md)",
         "avg_launch_ms": popc_ms / 8,
