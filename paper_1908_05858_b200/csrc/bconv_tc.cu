@@ -292,8 +292,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   if (tid == 0) {
     for (int i = 0; i < TC_MAX_BUFS; i++) {
       mbar_init(smem_u32(&bars[B_MMA_DONE + i]), 1);
-      mbar_init(smem_u32(&bars[B_TMEM_FREE + i]), (g.epi2 ? 256 : 128) * PEERS);
-      mbar_init(smem_u32(&bars[B_A_FULL + i]), 128 * PEERS);
+      mbar_init(smem_u32(&bars[B_TMEM_FREE + i]), (g.epi2 ? 8 : 4) * PEERS);  // one arrival per epilogue warp
+      mbar_init(smem_u32(&bars[B_A_FULL + i]), 4 * PEERS);                     // one arrival per producer warp
       mbar_init(smem_u32(&bars[B_A_FREE + i]), 1);
     }
     for (int i = 0; i < 3; i++) mbar_init(smem_u32(&bars[B_W_FULL + i]), TC_THREADS * PEERS);
@@ -611,11 +611,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       for (; mt < mt_end; mt += mt_step, it++) {
         TC_T(0);
         // its last reader: all MMAs of the tile that used it, signalled through `a_free` (in both CTAs of a pair)
-        if (it >= g.abufs && !mbar_wait(smem_u32(&bars[B_A_FREE + ab]), use_phase ^ 1u, s_fail)) { *s_fail = 1; break; }
+        // (the verdict is taken by the warp as a whole, so that its lanes stay together for the warp-wide steps below)
+        if (it >= g.abufs && !__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&bars[B_A_FREE + ab]), use_phase ^ 1u, s_fail))) { *s_fail = 1; break; }
         TC_T(1);
         expand(cur, a_s + (size_t)ab * a_bytes, cwc);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
-        arrive(bar_a_full0 + 8u * (uint32_t)ab);
+        __syncwarp();  // every lane's rows are written and fenced: one arrival stands for the warp
+        if (lane == 0) arrive(bar_a_full0 + 8u * (uint32_t)ab);
         if (it == 0) {
           // the first tile's rows went out before anything else: a short launch is all start-up.  Now this thread's
           // share of the weights.
@@ -689,7 +691,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       };
       load_res(c_first);
       TC_T(0);
-      if (!mbar_wait(smem_u32(&bars[B_MMA_DONE + buf]), acc_phase, s_fail)) {
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&bars[B_MMA_DONE + buf]), acc_phase, s_fail))) {
         *s_fail = 1;
         failed = true;
         break;
@@ -807,7 +809,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       }
       // this accumulator buffer may be overwritten by the tile after next
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      arrive(bar_tmem_free0 + 8u * buf);
+      __syncwarp();  // (the tensor-memory loads were warp-wide; lanes may have parted since: rejoin, then one arrival per warp)
+      if (lane == 0) arrive(bar_tmem_free0 + 8u * buf);
       if (++accb == (uint32_t)g.nacc) { accb = 0; acc_phase ^= 1u; }
       TC_T(2);
       }
