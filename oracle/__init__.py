@@ -205,6 +205,26 @@ def bn_sign_pack(acc_nhwc: np.ndarray, scale, shift) -> np.ndarray:
     return out
 
 
+def bn_add_sign_pack(acc_nhwc: np.ndarray, scale, shift, residual: np.ndarray):
+    """The Bi-Real block epilogue (Sections 2.1.1 and 2.3): y = fmaf(acc, scale, shift) + residual (one rounded add);
+    returns (y fp32, same shape as acc; packed sign bits of y along the channel axis)."""
+    acc = np.ascontiguousarray(acc_nhwc, dtype=np.int32)
+    r = _f32(residual)
+    assert r.shape == acc.shape
+    O = acc.shape[-1]
+    npix = acc.size // O
+    y = np.empty(acc.shape, dtype=np.float32)
+    bits = np.empty(acc.shape[:-1] + (words_per_pixel(O),), dtype=np.uint64)
+    lib().oracle_bn_add_sign_pack(_p(acc), ctypes.c_int64(npix), O, _p(_f32(scale)), _p(_f32(shift)), _p(r), _p(y), _p(bits))
+    return y, bits
+
+
+def bitcount(v: int) -> int:
+    """The bitcount the C code uses for Eq. 1, on one 64-bit word."""
+    lib().oracle_bitcount.restype = ctypes.c_int
+    return int(lib().oracle_bitcount(ctypes.c_uint64(int(v) & (2**64 - 1))))
+
+
 class _Bireal18Params(ctypes.Structure):
     _fields_ = [
         ("stem_w", ctypes.c_void_p),

@@ -20,6 +20,7 @@
  *                                       2*C_xnor - K  =  K - 2*sum popcount(xor).
  *   oracle_bgemm_xnor                   Eq. 1 as printed: counts of agreeing bit positions, C in N^{M x N}.
  *   oracle_bn_fold / oracle_bn_sign_pack  Section 2.1.1, last sentence (fused BN + binarize).
+ *   oracle_bn_add_sign_pack             the same with the real-valued shortcut of Section 2.3 added before the sign.
  *   oracle_bireal18_forward             Section 2.3 / Table 2: Bi-Real Net 18 (a binary
  *                                       ResNet-18; first conv and last fc in full precision).
  *
@@ -70,11 +71,18 @@ static int binarize(float x) { return (x < 0.0f) ? -1 : +1; }
 
 static size_t words_per_pixel(int C) { return (size_t)((C + 63) / 64); }
 
+/* bitcount of Eq. 1: the number of set bits of a word.  The compiler's builtin (one POPCNT instruction with -mpopcnt) is
+   the default; -DORACLE_BITCOUNT_LOOP selects a bit-by-bit loop instead.  oracle_bitcount exposes it to the pins. */
 static int popcount64(uint64_t v) {
+#ifdef ORACLE_BITCOUNT_LOOP
   int n = 0;
   while (v) { n += (int)(v & 1u); v >>= 1; }
   return n;
+#else
+  return __builtin_popcountll(v);
+#endif
 }
+int oracle_bitcount(uint64_t v) { return popcount64(v); }
 
 /* ---- pack (Section 2.1.1, the sequential packer) ----------------------------------- */
 void oracle_pack(const float* x, int layout, int N, int C, int H, int W, uint64_t* P) {
@@ -262,6 +270,24 @@ void oracle_bn_sign_pack(const int32_t* acc, int64_t npix, int O, const float* s
       float y = fmaf((float)acc[(size_t)p * O + o], scale[o], shift[o]);
       uint64_t bit = (binarize(y) == -1) ? 1u : 0u;
       out[(size_t)p * Ow + (size_t)(o >> 6)] |= bit << (o & 63);
+    }
+}
+
+/* ---- the Bi-Real block epilogue (Section 2.1.1, last sentence, with the real-valued shortcut of Section 2.3) ----
+ * y = fmaf((float)acc, scale[o], shift[o]) + r: the BN as one fused multiply-add, then ONE rounded fp32 add of the
+ * shortcut value; the packed bit is the sign of y.  acc, r and y are [npix][O]; bits is [npix][ceil(O/64)]. */
+void oracle_bn_add_sign_pack(const int32_t* acc, int64_t npix, int O, const float* scale, const float* shift,
+                             const float* r, float* y, uint64_t* bits) {
+  size_t Ow = words_per_pixel(O);
+  memset(bits, 0, (size_t)npix * Ow * sizeof(uint64_t));
+  for (int64_t p = 0; p < npix; p++)
+    for (int o = 0; o < O; o++) {
+      size_t i = (size_t)p * O + o;
+      float bn = fmaf((float)acc[i], scale[o], shift[o]);
+      float v = bn + r[i];
+      y[i] = v;
+      uint64_t bit = (binarize(v) == -1) ? 1u : 0u;
+      bits[(size_t)p * Ow + (size_t)(o >> 6)] |= bit << (o & 63);
     }
 }
 

@@ -83,3 +83,70 @@ def test_sign_of_bn_output_is_a_threshold_on_the_integer_sum(oracle_mod):
         y = acc.reshape(2 * K + 1, O).astype(np.float64) * scale.astype(np.float64) + shift.astype(np.float64)
     clear = np.isfinite(y) & (np.abs(y) > 1e-3 * (np.abs(shift.astype(np.float64)) + 1))
     assert np.array_equal(bits[clear], (y[clear] < 0).astype(np.int8))
+
+
+def round_to_fp32(v: Fraction) -> float:
+    """Round-to-nearest-even of an exact rational to IEEE binary32 (normal and subnormal range), by integer arithmetic."""
+    if v == 0:
+        return 0.0
+    s, a = (-1 if v < 0 else 1), abs(v)
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1
+    assert Fraction(2) ** e <= a < Fraction(2) ** (e + 1)
+    ulp = Fraction(2) ** (max(e, -126) - 23)
+    q = a / ulp
+    n = q.numerator // q.denominator
+    rem = q - n
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and n % 2 == 1):
+        n += 1
+    out = n * ulp
+    assert out < Fraction(2) ** 128
+    return s * float(out)  # exactly representable as a double
+
+
+def test_round_to_fp32_helper_on_known_values():
+    assert round_to_fp32(Fraction(1, 3)) == float(np.float32(1.0) / np.float32(3.0))
+    assert round_to_fp32(Fraction(16777217)) == 16777216.0           # tie -> even
+    assert round_to_fp32(Fraction(16777219)) == 16777220.0           # tie -> even, upwards
+    assert round_to_fp32(Fraction(-5, 2) ** 31) == float(np.float32(float(Fraction(-5, 2) ** 31)))
+    assert round_to_fp32(Fraction(1, 2 ** 149)) == float(np.float32(1.4e-45))
+
+
+def test_block_epilogue_is_one_fma_then_one_rounded_add(oracle_mod):
+    """y = RN(RN(acc*scale + shift) + r) with RN = round-to-nearest-even to fp32, from exact fractions: a contracted or
+    double-precision evaluation, a missing shortcut term or a swapped operand gives different bits somewhere in 9000 values."""
+    o = oracle_mod
+    rng = np.random.default_rng(11)
+    npix, O, K = 120, 75, 1152
+    acc = (rng.integers(0, K + 1, (npix, 1, 1, O)) * 2 - K).astype(np.int32)
+    scale = rng.uniform(-1.5, 1.5, O).astype(np.float32)
+    shift = rng.normal(0, 3.0, O).astype(np.float32)
+    r = (rng.standard_normal((npix, 1, 1, O)) * 20).astype(np.float32)
+    # make some sums cancel (y exactly zero or a tiny difference of large terms)
+    scale[0], shift[0] = 1.0, 0.0
+    r[:, 0, 0, 0] = -acc[:, 0, 0, 0].astype(np.float32)
+    r[::7, 0, 0, 1] = 0.0
+    y, bits = o.bn_add_sign_pack(acc, scale, shift, r)
+    assert y.shape == acc.shape and y.dtype == np.float32 and bits.shape == (npix, 1, 1, 2)
+    for p in range(npix):
+        for c in range(O):
+            bn = round_to_fp32(Fraction(int(acc[p, 0, 0, c])) * Fraction(float(scale[c])) + Fraction(float(shift[c])))
+            want = round_to_fp32(Fraction(bn) + Fraction(float(r[p, 0, 0, c])))
+            assert float(y[p, 0, 0, c]) == want, (p, c)
+            bit = int((bits[p, 0, 0, c >> 6] >> np.uint64(c & 63)) & np.uint64(1))
+            assert bit == (1 if want < 0 else 0)
+    assert np.all(y[:, 0, 0, 0] == 0.0) and not np.any(bits[:, 0, 0, 0] & np.uint64(1))  # exact zero packs as +1
+    assert not np.any(bits[..., 1] >> np.uint64(O - 64))                                  # tail bits zero
+    # without a shortcut it is the plain fused BN + sign
+    y0, bits0 = o.bn_add_sign_pack(acc, scale, shift, np.zeros_like(r))
+    assert np.array_equal(bits0, o.bn_sign_pack(acc, scale, shift))
+
+
+def test_bitcount_of_eq1_counts_set_bits(oracle_mod):
+    o = oracle_mod
+    rng = np.random.default_rng(12)
+    words = [0, 1, 2 ** 63, 2 ** 64 - 1, 0xAAAAAAAAAAAAAAAA, 0x5555555555555555, 0x8000000000000001, 0xFFFFFFFF00000000]
+    words += [int(v) for v in rng.integers(0, 2 ** 63, 200)] + [int(v) | 2 ** 63 for v in rng.integers(0, 2 ** 63, 50)]
+    for v in words:
+        assert o.bitcount(v) == bin(v).count("1"), hex(v)
