@@ -23,7 +23,11 @@
  *     out = K - 2*popcount(xor) lies in [-K, K] with the parity of K.
  *   - Errors: argument problems are reported synchronously, before anything is launched
  *     (DABNN_ERR_NULL / _SHAPE / _ALIGNMENT / _WORKSPACE); a failed launch gives DABNN_ERR_CUDA.
- *     Nothing throws; kernels never trap.
+ *     Nothing throws; kernels never trap.  Waits inside the tensor-core kernels are bounded: a kernel whose wait runs
+ *     out sets a per-device flag, releases what it holds and returns, and its outputs are undefined.  Calls only enqueue
+ *     work, so they still return DABNN_OK then; read the flag with dabnn_stream_status / dabnn_last_device_flag.
+ *   - Devices: a process may use the library on several devices (cudaSetDevice before the call); caches of function
+ *     attributes and SM counts are kept per device ordinal (up to 64).
  *   - Alignment: packed buffers 8 bytes; fp32 buffers 4 bytes (16 bytes enables vector paths,
  *     chosen automatically).
  */
@@ -45,7 +49,8 @@ typedef enum {
   DABNN_ERR_ALIGNMENT = 4,
   DABNN_ERR_WORKSPACE = 5,   /* workspace too small */
   DABNN_ERR_CUDA = 6,        /* the CUDA runtime reported an error at launch */
-  DABNN_ERR_STATIC_LIMIT = 7 /* the request is larger than the library's built-in scratch area */
+  DABNN_ERR_TIMEOUT = 7,     /* a bounded wait inside a kernel ran out (reported by dabnn_stream_status) */
+  DABNN_ERR_STATIC_LIMIT = 8 /* the request is larger than the library's built-in scratch area */
 } dabnn_status;
 
 typedef enum { DABNN_NCHW = 0, DABNN_NHWC = 1 } dabnn_layout;
@@ -123,8 +128,9 @@ typedef struct {
   const float* fc_w;             /* fp32 [1000][512] */
   const float* fc_b;             /* fp32 [1000] */
   const void* block_w_tc[16];    /* optional: weights expanded by dabnn_tc_prepare_weights, or NULL.  Where given and the
-                                    layer is covered by the tensor-core engine (the 13 stride-1 blocks), that engine runs
-                                    the block; results are identical either way */
+                                    batch is large enough for the tensor-core engine to pay (all 16 blocks, stride 1 and
+                                    stride 2, from about 70 images on; the early stages from 8), that engine runs the
+                                    block; results are identical either way */
 } dabnn_bireal18_params;
 
 /* Bytes of device workspace dabnn_bireal18_forward needs for a batch of N images (0 if N <= 0). */
@@ -136,7 +142,9 @@ size_t dabnn_bireal18_workspace_bytes(int N);
  * Kernels are chosen by batch size (results are the same bits whichever runs).  For one to four images the launches are
  * chained with programmatic stream serialization: a kernel may begin its set-up while its predecessor finishes and waits
  * for it before it reads any activation; on the stream the call as a whole is ordered like any other work, and it can
- * be captured into a CUDA graph.  DABNN_NO_CHAIN=1 in the environment (read once) gives ordinary launches. */
+ * be captured into a CUDA graph.  DABNN_NO_CHAIN=1 in the environment (read once) gives ordinary launches.
+ * Where blocks run on the tensor-core engine, a wait that ran out inside one of its kernels leaves the logits undefined
+ * while this call has long returned DABNN_OK: after synchronising, check dabnn_stream_status(stream). */
 dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float* images, int N, float* logits,
                                     void* workspace, size_t workspace_bytes, void* stream);
 
@@ -149,8 +157,9 @@ dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float*
  *   - Limit: N <= DABNN_STATIC_MAX_BATCH images per call; a larger N returns DABNN_ERR_STATIC_LIMIT and nothing runs.
  *   - Cost: the scratch area (DABNN_STATIC_SCRATCH_BYTES, about 8.5 MiB) is reserved on every GPU on which the
  *     library is loaded, from load until the process exits, whether or not this entry point is ever called.
- *   - The first call on each device looks up the area's device address (no allocation, but a runtime query);
- *     make that first call outside any stream capture.  Later calls on that device reuse the address.
+ *   - The first call on each device looks up the area's device address (a runtime query; it may also be the moment at
+ *     which the CUDA runtime loads this library's device code and reserves the area).  Make that first call once at
+ *     start-up, outside any stream capture.  Later calls on that device reuse the address.
  *   - The call itself performs no cudaMalloc / cudaFree and calls no allocating library routine.
  *   - All calls share the one area and it keeps whatever the previous call left in it.  Nothing in it has to start
  *     at zero (every region is fully written before it is read), so no clearing is done.  Two calls whose work
@@ -171,8 +180,12 @@ dabnn_status dabnn_bireal18_forward_static(const dabnn_bireal18_params* p, const
  * The batch is processed in up to four chunks whose copies run on two internal copy streams (created per device on first
  * use, kept until exit), so that the copy in, the kernels and the copy out of different chunks overlap; `stream` waits for
  * all of it: the host results are complete once `stream` has been synchronised.  x_host must hold its data when the
- * function is called (its copy may start before earlier work on `stream` has finished).  Not thread-safe against
- * concurrent calls on the same device; calls that share a workspace belong on one stream. */
+ * function is called (its copy may start before earlier work on `stream` has finished).  The first copy into the
+ * workspace waits for whatever `stream` held when the function was called whenever the workspace is not the one of the
+ * previous call on this device; with the same workspace it waits only for that previous call's kernels, so a caller
+ * that lets other work use the workspace in between must synchronise that work itself.  Not thread-safe against
+ * concurrent calls on the same device; calls that share a workspace belong on one stream.  This entry point uses the
+ * integer-pipe kernels only (no bounded waits), so there is no device flag to read after it. */
 size_t dabnn_binary_layer_host_workspace_bytes(dabnn_shape in, int O, dabnn_conv cv);
 dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const uint64_t* w_packed, int O, dabnn_conv cv,
                                      const float* scale, const float* shift, int32_t* out_host, uint64_t* bits_host,
@@ -183,8 +196,10 @@ dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const 
  * 4-bit {+1,-1} operands (e2m1, block scale 1.0, fp32 accumulation: exact) expanded on chip from the packed bits.
  * Results are identical to dabnn_bconv2d* bit for bit.
  * Covered: stride 1 or 2 (both axes alike), C a multiple of 64 and at most 512 (256 for stride 2), images narrow enough
- * that a tile's rows fit the activation buffer (W + 2*pad_w <= 63 for 3x3 stride 1), filters whose expanded weights fit the resident budget (dabnn_tc_weights_bytes
- * returns 0 otherwise); other cases return DABNN_ERR_UNSUPPORTED and are served by dabnn_bconv2d*.
+ * that the 128 + (kh-1)*SP + kw-1 slots a tile reads fit its activation buffer of 640 rows (SP = W + pad_w slots per
+ * image row at stride 1, so W + pad_w <= 255 for a 3x3 filter; wider still at C <= 256, where a thread holds five rows),
+ * filters whose expanded weights fit the resident budget (dabnn_tc_weights_bytes returns 0 otherwise); other cases
+ * return DABNN_ERR_UNSUPPORTED and are served by dabnn_bconv2d*.
  * A launch takes one of two forms, chosen by the library from the problem size: one CTA per tile of 128 output
  * positions, or pairs of CTAs of a thread-block cluster that share every tensor-core instruction (used where one CTA
  * cannot keep 128 output channels of weights resident: C = 512 with a 3x3 filter).  Both give the same bits.
@@ -195,8 +210,20 @@ dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const 
  *                             128 rows of C*kh*kw/2 bytes, the same buffer for every launch form
  *   dabnn_tc_prepare_weights  w_packed [O][kh][kw][Cw] -> w_tc (device, 16-byte aligned, that many bytes); once per model
  *   dabnn_tc_bconv2d*         as dabnn_bconv2d*, with w_tc in place of w_packed
- *   dabnn_tc_error_flag       synchronises nothing itself; copies the device-side error flag (1 if a bounded wait inside
- *                             a kernel ran out, else 0; -1 if it cannot be read).  Call after synchronising the stream. */
+ *   dabnn_tc_error_flag       synchronises nothing itself; copies the current device's error flag (1 if a bounded wait
+ *                             inside a kernel ran out since the flag was last cleared, else 0; -1 if it cannot be read)
+ *                             and leaves it set.  Call after synchronising the stream.
+ *   dabnn_last_device_flag    synchronises `stream`, returns that flag and clears it (one flag per device, shared by all
+ *                             streams: a value of 1 says that some tensor-engine launch on this device since the last
+ *                             read gave up, and the outputs written since then are undefined).  Not for use during
+ *                             stream capture.
+ *   dabnn_stream_status       the same as a status: DABNN_OK, DABNN_ERR_TIMEOUT (flag was set; now cleared) or
+ *                             DABNN_ERR_CUDA (the stream or the flag could not be read).
+ *   dabnn_tc_wait_expiry_selftest   exercises that failure path without any fault: launches dabnn_tc_bconv2d's kernel (NHWC)
+ *                             with its "activation rows ready" barrier expecting one arrival more than it will ever get
+ *                             and every wait limited to wait_polls polls (1..4096, about a microsecond each).  Each role
+ *                             of each CTA gives up in turn, the flag is set, tensor memory is freed and the kernel
+ *                             returns by itself; `out` is undefined.  The next ordinary launch is unaffected. */
 size_t dabnn_tc_weights_bytes(int O, int C, int kh, int kw);
 dabnn_status dabnn_tc_prepare_weights(const uint64_t* w_packed, int O, int C, int kh, int kw, void* w_tc, void* stream);
 dabnn_status dabnn_tc_bconv2d(const uint64_t* a_packed, dabnn_shape in, const void* w_tc, int O, dabnn_conv cv,
@@ -207,6 +234,10 @@ dabnn_status dabnn_tc_bconv2d_bn_add_sign_pack(const uint64_t* a_packed, dabnn_s
                                                dabnn_conv cv, const float* scale, const float* shift, const float* residual,
                                                float* y_out, uint64_t* out_packed, void* stream);
 int dabnn_tc_error_flag(void);
+int dabnn_last_device_flag(void* stream);
+dabnn_status dabnn_stream_status(void* stream);
+dabnn_status dabnn_tc_wait_expiry_selftest(const uint64_t* a_packed, dabnn_shape in, const void* w_tc, int O, dabnn_conv cv,
+                                           int32_t* out, int wait_polls, void* stream);
 /* CTAs per tensor-engine launch at most (0 = the default: one persistent CTA, or CTA of a pair, per SM).  A launch takes
  * every SM it is given; a caller that runs independent layers side by side (several streams, or branches of a CUDA graph)
  * gets more out of the chip with launches capped at about half of it (74 on a B200).  Results do not depend on it.

@@ -27,8 +27,12 @@ EXPORTS = (
     "dabnn_bireal18_workspace_bytes", "dabnn_bireal18_forward", "dabnn_set_conv_variant",
     "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host", "dabnn_bireal18_forward_static", "dabnn_set_conv_tile",
     "dabnn_tc_set_max_ctas", "dabnn_tc_weights_bytes", "dabnn_tc_prepare_weights", "dabnn_tc_bconv2d", "dabnn_tc_bconv2d_bn_sign_pack",
-    "dabnn_tc_bconv2d_bn_add_sign_pack", "dabnn_tc_error_flag",
+    "dabnn_tc_bconv2d_bn_add_sign_pack", "dabnn_tc_error_flag", "dabnn_last_device_flag", "dabnn_stream_status",
+    "dabnn_tc_wait_expiry_selftest",
 )
+
+ERR_TIMEOUT = 7
+ERR_STATIC_LIMIT = 8
 
 
 class DabnnError(RuntimeError):
@@ -104,6 +108,12 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).restype = ci
         L.dabnn_set_conv_tile.restype = ci
         L.dabnn_set_conv_tile.argtypes = [ci]
+        L.dabnn_last_device_flag.restype = ci
+        L.dabnn_last_device_flag.argtypes = [vp]
+        L.dabnn_stream_status.restype = ci
+        L.dabnn_stream_status.argtypes = [vp]
+        L.dabnn_tc_wait_expiry_selftest.restype = ci
+        L.dabnn_tc_wait_expiry_selftest.argtypes = [vp, Shape, vp, ci, Conv, vp, ci, vp]
         L.dabnn_bireal18_forward_static.restype = ci
         L.dabnn_bireal18_forward_static.argtypes = [ctypes.POINTER(Bireal18Params), vp, ci, vp, vp]
         for name in ("dabnn_pack", "dabnn_pack_weights", "dabnn_bconv2d", "dabnn_bconv2d_bn_sign_pack",
@@ -111,6 +121,23 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).restype = ci
         _lib = L
     return _lib
+
+
+def _default_alloc(shape, dtype, device) -> torch.Tensor:
+    return torch.empty(tuple(shape), dtype=dtype, device=device)
+
+
+_alloc = _default_alloc
+
+
+def set_output_allocator(fn=None):
+    """Every output tensor and workspace that this module creates comes from ``fn(shape, dtype, device)`` (default:
+    ``torch.empty``).  A caller with its own memory pool passes its allocator; the tests pass one that puts guard
+    bytes around each output.  Returns the previous allocator."""
+    global _alloc
+    prev = _alloc
+    _alloc = fn if fn is not None else _default_alloc
+    return prev
 
 
 def _check(status: int) -> None:
@@ -150,7 +177,7 @@ def pack(x: torch.Tensor, layout: int = NCHW, out: Optional[torch.Tensor] = None
     else:
         N, H, W, C = x.shape
     if out is None:
-        out = torch.empty((N, H, W, words_per_pixel(C)), dtype=torch.int64, device=x.device)
+        out = _alloc((N, H, W, words_per_pixel(C)), torch.int64, x.device)
     _check(lib().dabnn_pack(x.data_ptr(), layout, Shape(N, C, H, W), out.data_ptr(), _stream()))
     return out
 
@@ -163,7 +190,7 @@ def pack_i32(x: torch.Tensor, layout: int = NCHW, out: Optional[torch.Tensor] = 
     else:
         N, H, W, C = x.shape
     if out is None:
-        out = torch.empty((N, H, W, words_per_pixel(C)), dtype=torch.int64, device=x.device)
+        out = _alloc((N, H, W, words_per_pixel(C)), torch.int64, x.device)
     _check(lib().dabnn_pack_i32(x.data_ptr(), layout, Shape(N, C, H, W), out.data_ptr(), _stream()))
     return out
 
@@ -172,7 +199,7 @@ def pack_weights(w_oihw: torch.Tensor) -> torch.Tensor:
     """dabnn_pack_weights: fp32 OIHW -> packed int64 [O][kh][kw][Cw]."""
     w = _dev(w_oihw, torch.float32, "w")
     O, C, kh, kw = w.shape
-    out = torch.empty((O, kh, kw, words_per_pixel(C)), dtype=torch.int64, device=w.device)
+    out = _alloc((O, kh, kw, words_per_pixel(C)), torch.int64, w.device)
     _check(lib().dabnn_pack_weights(w.data_ptr(), O, C, kh, kw, out.data_ptr(), _stream()))
     return out
 
@@ -194,7 +221,7 @@ def bconv2d(a_packed, C: int, w_packed, stride=(1, 1), pad=(0, 0), pad_value: in
     a, w, N, H, W, O, kh, kw, OH, OW = _geom(a_packed, C, w_packed, stride, pad)
     if out is None:
         shape = (N, max(OH, 0), max(OW, 0), O) if out_layout == NHWC else (N, O, max(OH, 0), max(OW, 0))
-        out = torch.empty(shape, dtype=torch.int32, device=a.device)
+        out = _alloc(shape, torch.int32, a.device)
     _check(lib().dabnn_bconv2d(a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O, _conv(kh, kw, stride, pad, pad_value),
                                out.data_ptr(), out_layout, _stream()))
     return out
@@ -208,7 +235,7 @@ def bgemm(A: torch.Tensor, B: torch.Tensor, Kbits: int) -> torch.Tensor:
     N, Kw2 = B.shape
     if Kw != Kw2 or Kw != (Kbits + 63) // 64:
         raise DabnnError("packed word counts do not match Kbits")
-    out = torch.empty((M, N), dtype=torch.int32, device=A.device)
+    out = _alloc((M, N), torch.int32, A.device)
     _check(lib().dabnn_bgemm(A.data_ptr(), M, B.data_ptr(), N, int(Kbits), out.data_ptr(), _stream()))
     return out
 
@@ -220,7 +247,7 @@ def bconv2d_bn_sign_pack(a_packed, C: int, w_packed, scale, shift, stride=(1, 1)
     scale = _dev(scale, torch.float32, "scale")
     shift = _dev(shift, torch.float32, "shift")
     if out is None:
-        out = torch.empty((N, max(OH, 0), max(OW, 0), words_per_pixel(O)), dtype=torch.int64, device=a.device)
+        out = _alloc((N, max(OH, 0), max(OW, 0), words_per_pixel(O)), torch.int64, a.device)
     _check(lib().dabnn_bconv2d_bn_sign_pack(a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O,
                                             _conv(kh, kw, stride, pad, pad_value), scale.data_ptr(), shift.data_ptr(),
                                             out.data_ptr(), _stream()))
@@ -236,8 +263,8 @@ def bconv2d_bn_add_sign_pack(a_packed, C: int, w_packed, scale, shift, residual,
     residual = _dev(residual, torch.float32, "residual")
     if tuple(residual.shape) != (N, OH, OW, O):
         raise DabnnError("residual must be NHWC [N][OH][OW][O]")
-    y = torch.empty_like(residual)
-    bits = torch.empty((N, OH, OW, words_per_pixel(O)), dtype=torch.int64, device=a.device) if want_bits else None
+    y = _alloc(residual.shape, torch.float32, a.device)
+    bits = _alloc((N, OH, OW, words_per_pixel(O)), torch.int64, a.device) if want_bits else None
     _check(lib().dabnn_bconv2d_bn_add_sign_pack(a.data_ptr(), Shape(N, C, H, W), w.data_ptr(), O,
                                                 _conv(kh, kw, stride, pad, pad_value), scale.data_ptr(),
                                                 shift.data_ptr(), residual.data_ptr(), y.data_ptr(),
@@ -249,8 +276,8 @@ def bn_fold(gamma, beta, mean, var, eps: float = 1e-5):
     """dabnn_bn_fold: (scale, shift) fp32 device tensors."""
     g, b, m, v = (_dev(t, torch.float32, "bn") for t in (gamma, beta, mean, var))
     O = g.numel()
-    scale = torch.empty(O, dtype=torch.float32, device=g.device)
-    shift = torch.empty(O, dtype=torch.float32, device=g.device)
+    scale = _alloc((O,), torch.float32, g.device)
+    shift = _alloc((O,), torch.float32, g.device)
     _check(lib().dabnn_bn_fold(g.data_ptr(), b.data_ptr(), m.data_ptr(), v.data_ptr(), float(eps), O,
                                scale.data_ptr(), shift.data_ptr(), _stream()))
     return scale, shift
@@ -302,7 +329,7 @@ class Bireal18:
     def workspace(self, N: int) -> torch.Tensor:
         need = bireal18_workspace_bytes(N)
         if self._ws is None or self._ws.numel() < need:
-            self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+            self._ws = _alloc((need,), torch.uint8, self.device)
         return self._ws
 
     def forward(self, images: torch.Tensor, logits: Optional[torch.Tensor] = None) -> torch.Tensor:
@@ -313,7 +340,7 @@ class Bireal18:
             raise DabnnError("images must be [N][3][224][224]")
         ws = self.workspace(N)
         if logits is None:
-            logits = torch.empty((N, 1000), dtype=torch.float32, device=images.device)
+            logits = _alloc((N, 1000), torch.float32, images.device)
         _check(lib().dabnn_bireal18_forward(ctypes.byref(self.P), images.data_ptr(), N, logits.data_ptr(),
                                             ws.data_ptr(), ws.numel(), _stream()))
         return logits
@@ -355,14 +382,14 @@ def bireal18_forward_static(net: "Bireal18", images: torch.Tensor, logits: Optio
     if tuple(images.shape[1:]) != (3, 224, 224):
         raise DabnnError("images must be [N][3][224][224]")
     if logits is None:
-        logits = torch.empty((N, 1000), dtype=torch.float32, device=images.device)
+        logits = _alloc((N, 1000), torch.float32, images.device)
     _check(lib().dabnn_bireal18_forward_static(ctypes.byref(net.P), images.data_ptr(), N, logits.data_ptr(), _stream()))
     return logits
 
 
 # ---- tensor-core engine ---------------------------------------------------------------------------------------------
 class TcWeights:
-    """Expanded int8 weights for the tensor-core engine (dabnn_tc_prepare_weights), with the filter geometry."""
+    """Expanded 4-bit (e2m1) weights for the tensor-core engine (dabnn_tc_prepare_weights), with the filter geometry."""
 
     def __init__(self, w_packed: torch.Tensor, C: int):
         w = _dev(w_packed, torch.int64, "w_packed")
@@ -371,7 +398,7 @@ class TcWeights:
         nbytes = int(lib().dabnn_tc_weights_bytes(self.O, C, self.kh, self.kw))
         if nbytes == 0:
             raise DabnnError("this filter bank is not covered by the tensor-core engine")
-        self.buf = torch.empty(nbytes, dtype=torch.uint8, device=w.device)
+        self.buf = _alloc((nbytes,), torch.uint8, w.device)
         _check(lib().dabnn_tc_prepare_weights(w.data_ptr(), self.O, C, self.kh, self.kw, self.buf.data_ptr(), _stream()))
 
 
@@ -394,7 +421,7 @@ def tc_bconv2d(a_packed, wt: TcWeights, stride=(1, 1), pad=(0, 0), pad_value: in
     a, N, H, W, OH, OW = _tc_geom(a_packed, wt, stride, pad)
     if out is None:
         shape = (N, OH, OW, wt.O) if out_layout == NHWC else (N, wt.O, OH, OW)
-        out = torch.empty(shape, dtype=torch.int32, device=a.device)
+        out = _alloc(shape, torch.int32, a.device)
     _check(lib().dabnn_tc_bconv2d(a.data_ptr(), Shape(N, wt.C, H, W), wt.buf.data_ptr(), wt.O,
                                   _conv(wt.kh, wt.kw, stride, pad, pad_value), out.data_ptr(), out_layout, _stream()))
     return out
@@ -406,7 +433,7 @@ def tc_bconv2d_bn_sign_pack(a_packed, wt: TcWeights, scale, shift, stride=(1, 1)
     a, N, H, W, OH, OW = _tc_geom(a_packed, wt, stride, pad)
     scale, shift = _dev(scale, torch.float32, "scale"), _dev(shift, torch.float32, "shift")
     if out is None:
-        out = torch.empty((N, OH, OW, words_per_pixel(wt.O)), dtype=torch.int64, device=a.device)
+        out = _alloc((N, OH, OW, words_per_pixel(wt.O)), torch.int64, a.device)
     _check(lib().dabnn_tc_bconv2d_bn_sign_pack(a.data_ptr(), Shape(N, wt.C, H, W), wt.buf.data_ptr(), wt.O,
                                                _conv(wt.kh, wt.kw, stride, pad, pad_value), scale.data_ptr(),
                                                shift.data_ptr(), out.data_ptr(), _stream()))
@@ -419,8 +446,8 @@ def tc_bconv2d_bn_add_sign_pack(a_packed, wt: TcWeights, scale, shift, residual,
     a, N, H, W, OH, OW = _tc_geom(a_packed, wt, stride, pad)
     scale, shift = _dev(scale, torch.float32, "scale"), _dev(shift, torch.float32, "shift")
     residual = _dev(residual, torch.float32, "residual")
-    y = torch.empty_like(residual)
-    bits = torch.empty((N, OH, OW, words_per_pixel(wt.O)), dtype=torch.int64, device=a.device) if want_bits else None
+    y = _alloc(residual.shape, torch.float32, a.device)
+    bits = _alloc((N, OH, OW, words_per_pixel(wt.O)), torch.int64, a.device) if want_bits else None
     _check(lib().dabnn_tc_bconv2d_bn_add_sign_pack(a.data_ptr(), Shape(N, wt.C, H, W), wt.buf.data_ptr(), wt.O,
                                                    _conv(wt.kh, wt.kw, stride, pad, pad_value), scale.data_ptr(),
                                                    shift.data_ptr(), residual.data_ptr(), y.data_ptr(),
@@ -435,6 +462,27 @@ def tc_set_max_ctas(max_ctas: int) -> int:
 
 def tc_error_flag() -> int:
     return int(lib().dabnn_tc_error_flag())
+
+
+def last_device_flag() -> int:
+    """dabnn_last_device_flag on the current stream: synchronises it, returns the device's error flag and clears it."""
+    return int(lib().dabnn_last_device_flag(_stream()))
+
+
+def stream_status() -> int:
+    """dabnn_stream_status on the current stream (0 = ok, ERR_TIMEOUT = a bounded wait inside a kernel ran out)."""
+    return int(lib().dabnn_stream_status(_stream()))
+
+
+def tc_wait_expiry_selftest(a_packed, wt: "TcWeights", stride=(1, 1), pad=(0, 0), pad_value: int = -1, wait_polls: int = 1000):
+    """dabnn_tc_wait_expiry_selftest: a launch whose first wait can never be satisfied and gives up after `wait_polls`
+    polls.  Returns the (undefined) output tensor."""
+    a, N, H, W, OH, OW = _tc_geom(a_packed, wt, stride, pad)
+    out = _alloc((N, OH, OW, wt.O), torch.int32, a.device)
+    _check(lib().dabnn_tc_wait_expiry_selftest(a.data_ptr(), Shape(N, wt.C, H, W), wt.buf.data_ptr(), wt.O,
+                                               _conv(wt.kh, wt.kw, stride, pad, pad_value), out.data_ptr(), int(wait_polls),
+                                               _stream()))
+    return out
 
 
 class Prepared:

@@ -32,13 +32,15 @@ dabnn_status launch_one(const BConvArgs& g, cudaStream_t st) {
   constexpr int THREADS = (BP / TP) * (BO / TO);
   constexpr size_t SMEM = (size_t)STAGES * (BP + BO) * PITCH * 4 + (size_t)BP * sizeof(RowInfo);
   auto kern = bconv_kernel<BP, BO, TP, TO, MINB, EPI, CSA, VEC16, STAGES>;
-  static bool configured = false;  // one attribute call per instantiation (idempotent if raced)
-  if (!configured) {
+  static bool configured[kMaxDevices] = {};  // one attribute call per instantiation and device (idempotent if raced)
+  const int dev = current_device();
+  if (dev < 0) return DABNN_ERR_CUDA;
+  if (!configured[dev]) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) {
       cudaGetLastError();
       return DABNN_ERR_CUDA;
     }
-    configured = true;
+    configured[dev] = true;
   }
   const long long gx = (g.M + BP - 1) / BP;
   const int ochan = (EPI == EPI_I32) ? g.O : g.Ow32 * 32;
@@ -112,16 +114,18 @@ dabnn_status fill_args(BConvArgs& g, const uint64_t* a, dabnn_shape in, const ui
 }  // namespace
 
 int sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, n = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+  static int cached[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
       cudaGetLastError();
       return 148;
     }
-    cached = n;
+    cached[dev] = n;
   }
-  return cached;
+  return cached[dev];
 }
 
 }  // namespace dabnn
@@ -158,6 +162,7 @@ extern "C" const char* dabnn_status_string(dabnn_status s) {
     case DABNN_ERR_ALIGNMENT: return "misaligned pointer";
     case DABNN_ERR_WORKSPACE: return "workspace too small";
     case DABNN_ERR_CUDA: return "CUDA launch error";
+    case DABNN_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out; the outputs of the launches since the flag was last read are undefined";
     case DABNN_ERR_STATIC_LIMIT: return "request exceeds the library's built-in scratch area (see DABNN_STATIC_MAX_BATCH)";
   }
   return "unknown status";

@@ -48,19 +48,14 @@ constexpr int TC_SMEM_MISC = 256 + 2 * TC_MAX_RES * 128 * 4;  // barriers, TMEM 
 constexpr int TC_WEIGHT_BUDGET = 147456;  // 144 KB of resident weights at most
 constexpr int TC_MAX_CW = 8;              // C <= 512
 constexpr int TC_MAX_SPT = 5;             // slots per producer thread: 2 for stride 1, up to 5 for stride 2
-constexpr int TC_TMEM_COLS = 512;         // 2 accumulators (<= 128 columns each) + the scale-factor columns
+constexpr int TC_TMEM_COLS = 512;         // the accumulators' columns + the scale-factor columns
+constexpr int TC_WAIT_POLLS = 1 << 20;    // polls of a barrier wait before it gives up (about a second)
 constexpr int TC_ACC_COLS = 384;          // columns [0, 384): up to four accumulators (three of 128 columns)
 constexpr int TC_SF_COL = 384;            // columns [384, 512) hold scale factors (all 1.0)
 constexpr int TC_MAX_BUFS = 4;            // accumulators / activation buffers in flight at most
 
-__device__ int g_tc_error = 0;  // 1: an mbarrier wait ran out
+__device__ int g_tc_error = 0;  // 1: an mbarrier wait ran out (one copy per device; cleared when read by dabnn_last_device_flag)
 int g_tc_max_ctas = 0;          // host: CTAs per launch at most (0: one per SM)
-#ifdef TC_TIMING
-__device__ unsigned long long g_tc_prof[24];
-#define TC_T(i) do { long long t_ = clock64(); prof[i] += t_ - tlast; tlast = t_; } while (0)
-#else
-#define TC_T(i) do {} while (0)
-#endif
 
 struct TcArgs {
   const uint64_t* a;
@@ -90,6 +85,8 @@ struct TcArgs {
   float* y_out;
   uint32_t* out_packed32;
   int Ow32;
+  int wait_polls;      // polls of a barrier wait before it gives up (TC_WAIT_POLLS; smaller only in the expiry self-test)
+  int extra_arrivals;  // 0; the expiry self-test makes `a_full` expect one arrival more than the producers make
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -107,8 +104,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 
 // Bounded wait for the given phase parity; false if it ran out, or if another role of this CTA has given up (`fail`,
 // looked at only now and then: shared-memory reads are slow while the tensor pipe streams its operands).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* fail) {
-  for (int tries = 0; tries < (1 << 20); tries++) {  // about a second at most, then give up
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* fail, int limit) {
+  for (int tries = 0; tries < limit; tries++) {  // about a microsecond per poll; then give up
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -123,8 +120,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 // The same with cluster-scope acquire: the arrivals may come from the peer CTA.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* fail) {
-  for (int tries = 0; tries < (1 << 20); tries++) {
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* fail, int limit) {
+  for (int tries = 0; tries < limit; tries++) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -293,7 +290,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     for (int i = 0; i < TC_MAX_BUFS; i++) {
       mbar_init(smem_u32(&bars[B_MMA_DONE + i]), 1);
       mbar_init(smem_u32(&bars[B_TMEM_FREE + i]), (g.epi2 ? 8 : 4) * PEERS);  // one arrival per epilogue warp
-      mbar_init(smem_u32(&bars[B_A_FULL + i]), 4 * PEERS);                     // one arrival per producer warp
+      mbar_init(smem_u32(&bars[B_A_FULL + i]), 4 * PEERS + (uint32_t)g.extra_arrivals);  // one arrival per producer warp
       mbar_init(smem_u32(&bars[B_A_FREE + i]), 1);
     }
     for (int i = 0; i < 3; i++) mbar_init(smem_u32(&bars[B_W_FULL + i]), TC_THREADS * PEERS);
@@ -439,16 +436,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
           asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
       };
       auto wait = [&](uint32_t bar, uint32_t parity) {
-        return PAIR ? mbar_wait_cluster(bar, parity, s_fail) : mbar_wait(bar, parity, s_fail);
+        return PAIR ? mbar_wait_cluster(bar, parity, s_fail, g.wait_polls) : mbar_wait(bar, parity, s_fail, g.wait_polls);
       };
       const bool k3 = g.kh == 3 && g.kw == 3;
       uint32_t off9[9];
 #pragma unroll
       for (int t = 0; t < 9; t++) off9[t] = k3 ? tap_offset(t / 3, t % 3) : 0u;
-#ifdef TC_TIMING
-      long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-      long long tlast = clock64();
-#endif
       // all MMAs of one tile and channel tile; KB = C / 64 as a compile-time constant, the 3x3 filter fully unrolled
       auto issue_tile = [&](uint32_t d_tmem, uint32_t a_lo0, uint32_t b_base, uint32_t a_stp, bool first, auto kbc) {
         constexpr int KB = decltype(kbc)::value;
@@ -482,9 +475,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       if (!ok) *s_fail = 1;
 #pragma unroll 1
       for (long long mt = mt_first; mt < mt_end && ok; mt += mt_step) {
-        TC_T(0);
         if (!wait(smem_u32(&bars[B_A_FULL + ab]), a_phase)) { *s_fail = 1; break; }  // rows written
-        TC_T(1);
         const uint32_t a_lo0 = a_lo_first + ab * a_buf_units;
         // (opaque to the compiler, so that it does not keep every tap's and K block's offset in a register of its own
         // across tiles: the sums are recomputed per tile, one add each)
@@ -510,12 +501,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
           if (++accb == (uint32_t)g.nacc) { accb = 0; acc_phase ^= 1u; }
         }
         commit(smem_u32(&bars[B_A_FREE + ab]));  // the tile's rows have been read: the A buffer may be refilled
-        TC_T(3);
         if (++ab == (uint32_t)g.abufs) { ab = 0; a_phase ^= 1u; }
       }
-#ifdef TC_TIMING
-      if (blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[16 + i] = prof[i]; }
-#endif
     }
   } else if (warp >= 4 && warp < 8) {
     // ================= producer warps: packed bits -> e2m1 rows ===================================================
@@ -590,10 +577,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     };
 
     int it = 0;
-#ifdef TC_TIMING
-    long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    long long tlast = clock64();
-#endif
     // Per tile: wait until the A buffer is free, expand the rows held in `cur`, hand them over, move the next tile's
     // bits (requested one tile ago, so they have landed) from `nxt` into `cur`, and request the tile after that into
     // `nxt`: registers that a load is still filling are never touched before the next iteration.
@@ -609,11 +592,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       uint32_t ab = 0, use_phase = 0;  // A buffer of this tile and the parity of the number of times it has been filled
 #pragma unroll 1
       for (; mt < mt_end; mt += mt_step, it++) {
-        TC_T(0);
         // its last reader: all MMAs of the tile that used it, signalled through `a_free` (in both CTAs of a pair)
         // (the verdict is taken by the warp as a whole, so that its lanes stay together for the warp-wide steps below)
-        if (it >= g.abufs && !__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&bars[B_A_FREE + ab]), use_phase ^ 1u, s_fail))) { *s_fail = 1; break; }
-        TC_T(1);
+        if (it >= g.abufs && !__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&bars[B_A_FREE + ab]), use_phase ^ 1u, s_fail, g.wait_polls))) { *s_fail = 1; break; }
         expand(cur, a_s + (size_t)ab * a_bytes, cwc);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
         __syncwarp();  // every lane's rows are written and fenced: one arrival stands for the warp
@@ -623,7 +604,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
           // share of the weights.
           weights_arrive();
         }
-        TC_T(2);
         if (TWO_SETS) {
 #pragma unroll
           for (int h = 0; h < SPT; h++) {
@@ -643,9 +623,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     else if (g.Cw <= 4) run(IntC<4>{});
     else if constexpr (PCW > 4) run(IntC<8>{});
     else prologue_sync();  // (not reached: the host launches this instance for C <= 256 only)
-#ifdef TC_TIMING
-    if (ptid == 0 && blockIdx.x == 0) { for (int i = 0; i < 8; i++) g_tc_prof[i] = prof[i]; g_tc_prof[15] = it; }
-#endif
   } else if (warp < 4 || g.epi2) {
     // ================= epilogue warps: TMEM accumulator -> output ===============================================
     uint32_t accb = 0, acc_phase = 0;  // accumulator of this round (one per tile and resident channel tile), parity of its uses
@@ -654,10 +631,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     // 32-column chunks, warps 8-11 the odd ones
     const int c_first = warp >= 8 ? 32 : 0;
     const int c_step = g.epi2 ? 64 : 32;
-#ifdef TC_TIMING
-    long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    long long tlast = clock64();
-#endif
     for (long long mt = mt_first; mt < mt_end && !failed; mt += mt_step) {
       const int row = 32 * (warp & 3) + lane;  // TMEM lane = slot row of the tile
       const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)row;
@@ -690,19 +663,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
         }
       };
       load_res(c_first);
-      TC_T(0);
-      if (!__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&bars[B_MMA_DONE + buf]), acc_phase, s_fail))) {
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&bars[B_MMA_DONE + buf]), acc_phase, s_fail, g.wait_polls))) {
         *s_fail = 1;
         failed = true;
         break;
       }
-      TC_T(1);
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const long long m = my_m;
 #pragma unroll 1
       for (int c0 = c_first; c0 < NT; c0 += c_step) {
         __syncwarp();  // the TMEM load is warp-wide: rejoin lanes that took different paths below
-        TC_T(4);
         float rc[32];
         if (EPI == EPI_BIREAL) {
 #pragma unroll
@@ -720,7 +690,6 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
               "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
             : "r"(taddr));
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        TC_T(3);
         const int o = nt * NT + c0;  // first of the 32 channels of this chunk; the lane owns them all for its row
         if (!my_valid) continue;
         const int nch = min(32, g.O - o);  // channels of this chunk that exist (<= 0: none)
@@ -812,12 +781,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       __syncwarp();  // (the tensor-memory loads were warp-wide; lanes may have parted since: rejoin, then one arrival per warp)
       if (lane == 0) arrive(bar_tmem_free0 + 8u * buf);
       if (++accb == (uint32_t)g.nacc) { accb = 0; acc_phase ^= 1u; }
-      TC_T(2);
       }
     }
-#ifdef TC_TIMING
-    if (tid == 0 && blockIdx.x == 0) { for (int i = 0; i < 6; i++) g_tc_prof[8 + i] = prof[i]; }
-#endif
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   if (PAIR) cluster_sync_all();  // neither CTA leaves, or frees tensor memory, while the other may still use it
@@ -884,9 +849,12 @@ int tc_n_ntiles(int O, int nt) { return ((O + 63) / 64 * 64 + nt - 1) / nt; }
 template <int NT, int EPI, int SPT, bool PAIR>
 dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
   auto kern = bconv_tc_kernel<NT, EPI, SPT, PAIR>;
-  static bool configured = false;
-  static int max_units = 0;  // CTAs (pairs) that can be resident at once
-  if (!configured) {
+  static bool configured[kMaxDevices] = {};
+  static int max_units_dev[kMaxDevices] = {};  // CTAs (pairs) that can be resident at once
+  const int dev = current_device();
+  if (dev < 0) return DABNN_ERR_CUDA;
+  int& max_units = max_units_dev[dev];
+  if (!configured[dev]) {
     // the largest shared-memory carve-out for every instance, whatever it needs: consecutive launches of different
     // instances then never make the SMs re-partition their L1 / shared memory
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, TC_SMEM_LIMIT) != cudaSuccess ||
@@ -911,7 +879,7 @@ dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
       }
       max_units = clusters < sm_count() / 2 ? clusters : sm_count() / 2;
     }
-    configured = true;
+    configured[dev] = true;
   }
   const long long m_units = PAIR ? (g.m_tiles + 1) / 2 : g.m_tiles;
   long long units = (long long)g.n_groups * m_units;
@@ -1046,6 +1014,7 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   g.pad_neg = cv.pad_value < 0;
   g.out = nullptr; g.out_nchw = 0; g.scale = g.shift = g.residual = nullptr; g.y_out = nullptr;
   g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64);
+  g.wait_polls = TC_WAIT_POLLS; g.extra_arrivals = 0;
   return DABNN_OK;
 }
 
@@ -1139,8 +1108,44 @@ extern "C" int dabnn_tc_error_flag(void) {
   return v;
 }
 
-#ifdef TC_TIMING
-extern "C" int dabnn_tc_debug_read(unsigned long long* out24) {
-  return cudaMemcpyFromSymbol(out24, g_tc_prof, 24 * sizeof(unsigned long long)) == cudaSuccess ? 0 : -1;
+extern "C" int dabnn_last_device_flag(void* stream) {
+  if (cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  if (v != 0) {
+    const int zero = 0;
+    if (cudaMemcpyToSymbol(g_tc_error, &zero, sizeof(int)) != cudaSuccess) {
+      cudaGetLastError();
+      return -1;
+    }
+  }
+  return v;
 }
-#endif
+
+extern "C" dabnn_status dabnn_stream_status(void* stream) {
+  const int v = dabnn_last_device_flag(stream);
+  if (v < 0) return DABNN_ERR_CUDA;
+  return v == 0 ? DABNN_OK : DABNN_ERR_TIMEOUT;
+}
+
+extern "C" dabnn_status dabnn_tc_wait_expiry_selftest(const uint64_t* a_packed, dabnn_shape in, const void* w_tc, int O,
+                                                      dabnn_conv cv, int32_t* out, int wait_polls, void* stream) {
+  TcArgs g;
+  dabnn_status s = tc_fill(g, a_packed, in, w_tc, O, cv);
+  if (s != DABNN_OK) return s;
+  if (!out) return DABNN_ERR_NULL;
+  if (!aligned(out, 4)) return DABNN_ERR_ALIGNMENT;
+  if (wait_polls < 1 || wait_polls > 4096) return DABNN_ERR_SHAPE;  // a few milliseconds at most
+  g.out = out;
+  g.out_nchw = 0;
+  g.wait_polls = wait_polls;
+  g.extra_arrivals = 1;  // `a_full` never completes: the MMA thread's first wait runs out, every other role follows
+  return tc_dispatch<EPI_I32>(g, as_stream(stream));
+}
+

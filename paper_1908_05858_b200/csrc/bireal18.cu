@@ -779,13 +779,15 @@ Workspace plan(int N) {
 
 dabnn_status launch_stem_8x8(const dabnn_bireal18_params* p, const float* images, int N, float* out, cudaStream_t st) {
   constexpr size_t SMEM = (size_t)(STEM_K * 64 + 2 * 3 * 37 * 2 * 20) * 4;
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0) return DABNN_ERR_CUDA;
+  if (!configured[dev]) {
     if (cudaFuncSetAttribute(stem_conv_bn_8x8, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) {
       cudaGetLastError();
       return DABNN_ERR_CUDA;
     }
-    configured = true;
+    configured[dev] = true;
   }
   const long long ntiles = (long long)N * 49, cap = 2LL * sm_count();
   stem_conv_bn_8x8<<<(unsigned)(ntiles < cap ? ntiles : cap), 256, SMEM, st>>>(images, p->stem_w, p->stem_scale,
@@ -798,13 +800,15 @@ dabnn_status launch_stem(const dabnn_bireal18_params* p, const float* images, in
   constexpr int PS = 2 * TS + 5, HALF = stem_half(PS);
   constexpr size_t SMEM = (size_t)(2 * STEM_K * 4 * CPT + 2 * 3 * PS * 2 * HALF) * 4;
   auto kern = stem_conv_bn<TS, PPT, CPT>;
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0) return DABNN_ERR_CUDA;
+  if (!configured[dev]) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) {
       cudaGetLastError();
       return DABNN_ERR_CUDA;
     }
-    configured = true;
+    configured[dev] = true;
   }
   const int tiles = (112 + TS - 1) / TS;
   const long long ntiles = (long long)N * tiles * tiles;
@@ -923,7 +927,6 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
 static __device__ __align__(256) unsigned char g_static_scratch[DABNN_STATIC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 void* g_static_addr[kMaxDevices] = {};  // device address of g_static_scratch, per device ordinal
 }  // namespace

@@ -52,7 +52,19 @@ inline void launch_chain(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t s
 }
 #endif
 
-// Number of SMs of the current device (cached per process; the library runs on one device at a time).
+// Per-device host caches (function attributes set, SM counts, symbol addresses) are arrays over the device ordinal.
+constexpr int kMaxDevices = 64;
+// Ordinal of the calling thread's current device, or -1 (no device, or an ordinal beyond kMaxDevices).
+inline int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return -1;
+  }
+  return (dev >= 0 && dev < kMaxDevices) ? dev : -1;
+}
+
+// Number of SMs of the current device (cached per device).
 int sm_count();
 
 }  // namespace dabnn

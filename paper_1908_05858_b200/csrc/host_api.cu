@@ -47,6 +47,7 @@ struct CopyLanes {
   cudaEvent_t ev[kEventRing];
   cudaEvent_t prev_compute;  // the kernels of the previous (uncaptured) call on this device are done
   bool has_prev = false;
+  const void* prev_ws = nullptr;  // workspace of that previous call
   int next = 0;
   bool ok = false;
 };
@@ -102,10 +103,13 @@ extern "C" dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape
   cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
   if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) return fail();
   const bool capturing = cap != cudaStreamCaptureStatusNone;
-  if (capturing) {
+  // A workspace that the previous call did not use may still be in use by whatever the caller's stream holds (another
+  // layer's call, or memory that the caller's allocator has just recycled): then, too, the copies wait for `st`.
+  if (capturing || !L->has_prev || L->prev_ws != workspace) {
     cudaEvent_t e_start = event();
     if (cudaEventRecord(e_start, st) != cudaSuccess || cudaStreamWaitEvent(L->in, e_start, 0) != cudaSuccess) return fail();
-  } else if (L->has_prev) {
+  }
+  if (!capturing && L->has_prev) {
     if (cudaStreamWaitEvent(L->in, L->prev_compute, 0) != cudaSuccess) return fail();
   }
   const int chunks = in.N < kHostChunks ? in.N : kHostChunks;
@@ -143,6 +147,7 @@ extern "C" dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape
   if (!capturing) {
     if (cudaEventRecord(L->prev_compute, st) != cudaSuccess) return fail();
     L->has_prev = true;
+    L->prev_ws = workspace;
   }
   // join: the caller's stream is done with this call when the last copy-out is
   if (cudaStreamWaitEvent(st, e_last_out, 0) != cudaSuccess) return fail();

@@ -186,9 +186,8 @@ def test_bireal_block_epilogue_matches_oracle(B, oracle_mod, case):
     scale_o, shift_o = o.bn_fold(*synth.bn_params(rng, O))
     acc = o.bconv_bits(o.pack(x), C, o.pack_weights(w), stride, pad, pv, o.NHWC)
     res = rng.standard_normal(acc.shape).astype(np.float32) * 20
-    # y = fmaf(acc, scale, shift) + r: fp64 product-sum is exact here, so rounding it once gives fmaf
-    y = (acc.astype(np.float64) * scale_o.astype(np.float64) + shift_o.astype(np.float64)).astype(np.float32) + res
-    want_bits = o.pack(y, o.NHWC)
+    y, want_bits = o.bn_add_sign_pack(acc, scale_o, shift_o, res)  # one fmaf, one rounded add, sign, pack
+    assert np.array_equal(want_bits, o.pack(y, o.NHWC))
     a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
     got_y, got_bits = B.bconv2d_bn_add_sign_pack(a, C, wp, dev(scale_o), dev(shift_o), dev(res), stride, pad, pv)
     assert np.array_equal(got_y.cpu().numpy().view(np.uint32), y.view(np.uint32))
@@ -201,6 +200,14 @@ def sample_coords(rng, N, O, OH, OW, n):
     # always include the corners and edges, where padding matters
     fixed = [(0, 0, 0, 0), (N - 1, O - 1, OH - 1, OW - 1), (N - 1, 0, 0, OW - 1), (0, O - 1, OH - 1, 0), (N // 2, O // 2, 0, OW // 2)]
     return np.concatenate([np.array(fixed), c]).astype(np.int32)
+
+
+def full_size_bn(C, N, O, K):
+    """Per-channel (scale, shift) whose thresholds spread over the attainable sums (standard deviation sqrt(K))."""
+    rng = np.random.default_rng(C + N + 1)
+    scale = rng.uniform(0.5, 1.5, O).astype(np.float32)
+    scale[::7] *= -1.0
+    return scale, rng.normal(0, 0.3 * np.sqrt(K), O).astype(np.float32)
 
 
 FULL = [(64, C, HW, C, 3, 1) for C, HW in synth.SWEEP_SHAPES] + [(256, 256, 28, 256, 3, 1), (256, 512, 14, 2048, 1, 0)]
@@ -222,7 +229,16 @@ def test_full_size_configs_on_sampled_outputs(B, oracle_mod, cfg):
     want = oracle_mod.bconv_pm1_at(x, w, coords, (1, 1), (pad, pad), -1)  # the definition, output by output
     assert np.array_equal(g[coords[:, 0], coords[:, 2], coords[:, 3], coords[:, 1]], want)
     # packed operands too, bit for bit
-    assert np.array_equal(u64(a), oracle_mod.pack(x))
+    ao, wo = oracle_mod.pack(x), oracle_mod.pack_weights(w)
+    assert np.array_equal(u64(a), ao)
+    # the whole tensor against Eq. 1 on the packed words
+    full = oracle_mod.bconv_bits(ao, C, wo, (1, 1), (pad, pad), -1, oracle_mod.NHWC)
+    assert np.array_equal(g, full)
+    del g
+    # and the whole packed output of the fused BN + sign + pack epilogue
+    scale, shift = full_size_bn(C, N, O, K)
+    bits = B.bconv2d_bn_sign_pack(a, C, wp, dev(scale), dev(shift), (1, 1), (pad, pad), -1)
+    assert np.array_equal(u64(bits), oracle_mod.bn_sign_pack(full, scale, shift))
 
 
 def test_full_size_pack_config(B, oracle_mod):
@@ -435,6 +451,34 @@ def test_bireal18_batch72_all_blocks_on_the_tensor_engine(B, oracle_mod):
     got_p = B.Bireal18(p, engine="popc").forward(dev(img)).cpu().numpy()
     assert np.array_equal(got_p.view(np.uint32), want.view(np.uint32))
     assert B.tc_error_flag() == 0
+
+
+def test_bireal18_batch128_matches_oracle(B, oracle_mod):
+    """The network configuration as stated (batch 128), in the launch configuration the benchmark times: logits against
+    the oracle within the stated tolerance, same argmax, and (pinned evaluation order) the same bits."""
+    p = synth.bireal18_params()
+    img = synth.bireal18_images(128)
+    want = oracle_mod.bireal18_forward(p, img, conv_form=1)
+    net = B.Bireal18(p)
+    logits = torch.empty((128, 1000), dtype=torch.float32, device="cuda")
+    got = net.forward(dev(img), logits).cpu().numpy()
+    assert np.max(np.abs(got - want)) <= 1e-3 * np.max(np.abs(want))
+    assert np.array_equal(got.argmax(axis=1), want.argmax(axis=1))
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert np.array_equal(got[:1], net.forward(dev(img[:1])).cpu().numpy())  # and batch 1 of the same configuration
+    assert B.last_device_flag() == 0
+
+
+def test_guard_bytes_catch_a_write_past_an_output(B, guard_outputs):
+    """The guarded allocator the GPU tests run under does notice an out-of-bounds write (made here with torch, on
+    purpose, one byte past an output)."""
+    t = B.pack(torch.zeros((1, 64, 2, 2), device="cuda"))
+    raw = guard_outputs.live[-1][0]
+    assert raw.numel() == 2 * 256 + t.numel() * 8
+    raw[256 + t.numel() * 8] = 0
+    with pytest.raises(AssertionError, match="after an output"):
+        guard_outputs.check()
+    assert guard_outputs.check() == 0
 
 
 @pytest.mark.parametrize("N,pinned", [(1, True), (3, True), (5, False), (9, True)])

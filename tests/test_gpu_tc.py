@@ -87,10 +87,10 @@ def test_tc_conv_and_epilogues_match_oracle(B, oracle_mod, case):
     assert np.array_equal(got_bits, want_bits)
     # Bi-Real block epilogue
     res = rng.standard_normal(acc.shape).astype(np.float32) * 20
-    y = (acc.astype(np.float64) * scale.astype(np.float64) + shift.astype(np.float64)).astype(np.float32) + res
+    y, want_ybits = o.bn_add_sign_pack(acc, scale, shift, res)
     got_y, got_ybits = B.tc_bconv2d_bn_add_sign_pack(a, wt, dev(scale), dev(shift), dev(res), st, (pad, pad), pv)
     assert np.array_equal(got_y.cpu().numpy().view(np.uint32), y.view(np.uint32))
-    assert np.array_equal(u64(got_ybits), o.pack(y, o.NHWC))
+    assert np.array_equal(u64(got_ybits), want_ybits)
     torch.cuda.synchronize()
     assert B.tc_error_flag() == 0
 
@@ -113,20 +113,23 @@ def test_tc_full_size_configs_on_sampled_outputs(B, oracle_mod, cfg):
     got = B.tc_bconv2d(a, B.TcWeights(wp, C), (1, 1), (pad, pad), -1, B.NHWC)
     K = C * k * k
     assert int(got.min()) >= -K and int(got.max()) <= K and bool(((got - K) % 2 == 0).all())
-    # the whole tensor against the xor/popcount kernel (itself checked against the oracle), and samples against the definition
-    assert bool((got == B.bconv2d(a, C, wp, (1, 1), (pad, pad), -1, B.NHWC)).all())
+    # the whole tensor against Eq. 1 on the packed words (the oracle), and samples against the definition
     g = got.cpu().numpy()
+    full = oracle_mod.bconv_bits(oracle_mod.pack(x), C, oracle_mod.pack_weights(w), (1, 1), (pad, pad), -1, oracle_mod.NHWC)
+    assert np.array_equal(g, full)
     rng = np.random.default_rng(C + N)
     coords = np.stack([rng.integers(0, N, 20000), rng.integers(0, O, 20000), rng.integers(0, HW, 20000), rng.integers(0, HW, 20000)], axis=1).astype(np.int32)
     want = oracle_mod.bconv_pm1_at(x, w, coords, (1, 1), (pad, pad), -1)
     assert np.array_equal(g[coords[:, 0], coords[:, 2], coords[:, 3], coords[:, 1]], want)
-    # the fused sign epilogue at full size: the whole tensor against the integer-pipe engine's fused kernel, and the
-    # oracle's fmaf + sign on the sampled pixels
+    # the fused sign epilogue at full size: the whole packed tensor against the oracle's fmaf + sign + pack of its own
+    # sums, and the definition on sampled pixels
     rng2 = np.random.default_rng(C + N + 1)
     scale = rng2.uniform(0.5, 1.5, O).astype(np.float32)
+    scale[::7] *= -1.0
     shift = rng2.normal(0, 0.3 * np.sqrt(K), O).astype(np.float32)
     bits = B.tc_bconv2d_bn_sign_pack(a, B.TcWeights(wp, C), dev(scale), dev(shift), (1, 1), (pad, pad), -1)
-    assert bool((bits == B.bconv2d_bn_sign_pack(a, C, wp, dev(scale), dev(shift), (1, 1), (pad, pad), -1)).all())
+    assert np.array_equal(u64(bits), oracle_mod.bn_sign_pack(full, scale, shift))
+    del full
     px = coords[:2000]
     acc_px = oracle_mod.bconv_pm1_at(x, w, np.stack([np.repeat(px[:, 0], O), np.tile(np.arange(O), len(px)), np.repeat(px[:, 2], O),
                                                      np.repeat(px[:, 3], O)], axis=1).astype(np.int32), (1, 1), (pad, pad), -1)
@@ -201,6 +204,36 @@ def test_asymmetric_filters_and_paddings_on_both_engines(B, oracle_mod, kh, kw, 
         assert np.array_equal(B.bconv2d(a, C, wp, (1, 1), (ph, pw), pv, B.NHWC).cpu().numpy(), want)
         assert np.array_equal(B.tc_bconv2d(a, B.TcWeights(wp, C), (1, 1), (ph, pw), pv, B.NHWC).cpu().numpy(), want)
     assert B.tc_error_flag() == 0
+
+
+def test_a_wait_that_runs_out_sets_the_flag_and_leaves_the_device_usable(B, oracle_mod):
+    """The failure path of the bounded waits, made to happen without any fault: a launch whose "rows ready" barrier expects
+    one arrival more than it gets, every wait limited to about a millisecond.  The kernel must return by itself, the
+    device flag must read 1 once (then 0 again), the call that reports it must say DABNN_ERR_TIMEOUT, and the next ordinary
+    launches must give the oracle's integers."""
+    import time
+    o = oracle_mod
+    for case in ((3, 128, 14, 14, 128, 3, 1), (100, 512, 7, 7, 512, 3, 1)):  # one CTA per tile; CTA pairs
+        N, C, H, W, O, k, pad = case
+        rng = np.random.default_rng(C)
+        x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+        w = rng.standard_normal((O, C, k, k)).astype(np.float32)
+        want = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (1, 1), (pad, pad), -1, o.NHWC)
+        a, wt = B.pack(dev(x)), B.TcWeights(B.pack_weights(dev(w)), C)
+        assert B.last_device_flag() == 0
+        t0 = time.perf_counter()
+        B.tc_wait_expiry_selftest(a, wt, (1, 1), (pad, pad), -1, wait_polls=1000)
+        assert B.last_device_flag() == 1          # synchronises: the kernel came back by itself
+        assert time.perf_counter() - t0 < 5.0
+        assert B.last_device_flag() == 0          # reading cleared it
+        B.tc_wait_expiry_selftest(a, wt, (1, 1), (pad, pad), -1, wait_polls=200)
+        assert B.stream_status() == B.ERR_TIMEOUT and B.stream_status() == 0
+        for _ in range(2):                        # tensor memory was freed, barriers start afresh: ordinary launches are exact
+            got = B.tc_bconv2d(a, wt, (1, 1), (pad, pad), -1, B.NHWC).cpu().numpy()
+            assert np.array_equal(got, want)
+        assert B.last_device_flag() == 0
+    with pytest.raises(B.DabnnError):
+        B.tc_wait_expiry_selftest(a, wt, (1, 1), (pad, pad), -1, wait_polls=1 << 20)  # limit beyond a few milliseconds: refused
 
 
 _FORCED_FORM_SCRIPT = r"""

@@ -24,8 +24,8 @@ def test_requests_beyond_the_built_in_scratch_are_refused():
     L = B.lib()
     fake = ctypes.c_void_p(0x1000)  # never dereferenced
     P = B.Bireal18Params()
-    assert L.dabnn_bireal18_forward_static(ctypes.byref(P), fake, B.STATIC_MAX_BATCH + 1, fake, None) == 7
-    assert b"built-in scratch" in L.dabnn_status_string(7)
+    assert L.dabnn_bireal18_forward_static(ctypes.byref(P), fake, B.STATIC_MAX_BATCH + 1, fake, None) == B.ERR_STATIC_LIMIT
+    assert b"built-in scratch" in L.dabnn_status_string(B.ERR_STATIC_LIMIT)
     assert L.dabnn_bireal18_forward_static(ctypes.byref(P), fake, 0, fake, None) == 2
     assert L.dabnn_bireal18_workspace_bytes(B.STATIC_MAX_BATCH) <= 8935424
 
