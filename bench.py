@@ -1,24 +1,28 @@
 #!/usr/bin/env python
 """Benchmark of the binarized-convolution hot path on B200.
 
-One "step" is one pass of the whole path over one batch of synthetic input: for each of the four
-ResNet-18 stage shapes (C = 64/128/256/512 at 56/28/14/7 pixels, 3x3, stride 1, pad 1 with value -1)
-at batch 64: binarize + pack the fp32 activations, binary convolution with int32 output, and binary
-convolution with the fused BN + sign + re-pack epilogue.  The headline value is the convolutions'
-bit-operations (2 per bit pair) divided by the time of the whole step.
+Workload: the large-batch configuration -- a binary 3x3 convolution (batch 256, 256 -> 256 channels, 28x28, stride 1,
+pad 1 with value -1) and a binary 1x1 convolution (batch 256, 512 -> 2048 channels, 14x14).  One "step" is one pass of
+the whole path over one batch of synthetic input, for each of the two layers: binarize + pack the fp32 activations,
+binary convolution with int32 output, and binary convolution with the fused BN + sign + re-pack epilogue (6 kernels).
+The headline value is the convolutions' bit-operations (2 per bit pair) divided by the time of the whole step, with the
+xor + popcount kernels (the paper's method, on the integer pipes); the same step on the tensor-core engine, the pack
+kernels' bandwidth and the Bi-Real Net 18 forward are reported in the same line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-extras]
+    python bench.py --case conv|fused|bireal_block|pack|bireal [--engine popc|tc] [--N ..] [--C ..] [--HW ..] [--O ..] [--k ..]
 
-Prints ONE JSON line (rank 0).  Under torchrun every rank runs the same per-GPU work on its own
-seeded batch (weak scaling, no data-path collective); the time is the maximum over ranks.
+Prints ONE JSON line (rank 0).  Under torchrun every rank runs the same per-GPU work on its own seeded batch (weak
+scaling, no data-path collective); times are the maximum over ranks.  `--case` runs one kernel case a few times (for
+profiler captures and quick timings) and prints one text line instead.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import re
 import statistics
-import subprocess
 import sys
 import time
 
@@ -30,10 +34,20 @@ import numpy as np  # noqa: E402
 
 from paper_1908_05858_b200 import synth  # noqa: E402
 
-BATCH = 64
-METRIC = "binary conv Gbit-ops/s"
+BATCH = 256
+# (name, C, HW, O, k, pad): the two layers of the large-batch configuration
+LAYERS = (("conv3x3_256", 256, 28, 256, 3, 1), ("conv1x1_512_2048", 512, 14, 2048, 1, 0))
+METRIC = "binary conv Gbit-ops/s (% of bit-op roofline); Bi-Real-18 images/s at batch 1/128"
 UNIT = "Gbit-ops/s"
-WORKLOAD = "binary 3x3 conv sweep, batch 64, (C,HW) in (64,56),(128,28),(256,14),(512,7): pack + bconv(int32) + bconv(bn,sign,pack)"
+WORKLOAD = ("large-batch binary convolutions, batch 256: 3x3 256->256 at 28x28 (stride 1, pad 1, pad value -1) and "
+            "1x1 512->2048 at 14x14; per layer pack + bconv(int32) + bconv(bn,sign,pack)")
+REGIONS = 50  # the K-step timed region is repeated this many times (median and minimum reported)
+
+
+def config_dict(world):
+    return {"workload": WORKLOAD, "batch_per_gpu": BATCH,
+            "l2": "inputs larger than L2: a step reads and writes 0.93 GB (L2 is 126 MB), no flush kernel",
+            "parallelism": "replicas" if world > 1 else "single GPU"}
 
 
 def conv_bitops(N, C, HW, O, k):
@@ -41,7 +55,14 @@ def conv_bitops(N, C, HW, O, k):
 
 
 def step_bitops(batch):
-    return sum(2 * conv_bitops(batch, C, HW, C, 3) for C, HW in synth.SWEEP_SHAPES)
+    return sum(2 * conv_bitops(batch, C, HW, O, k) for _, C, HW, O, k, _ in LAYERS)
+
+
+def conv_bytes(N, C, HW, O, k, fused):
+    """Algorithmic HBM bytes of one convolution launch: packed activations + packed weights + the output."""
+    cw = (C + 63) // 64
+    out = N * HW * HW * ((O + 63) // 64) * 8 if fused else 4 * N * HW * HW * O
+    return 8 * N * HW * HW * cw + 8 * O * k * k * cw + out
 
 
 def measured_peaks():
@@ -49,26 +70,31 @@ def measured_peaks():
     if os.path.exists(path):
         with open(path) as f:
             d = json.load(f)
-        return {"hbm_gbs": float(d["hbm_gbs"]), "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "source": "fallback"}
+        return {"hbm_gbs": float(d["hbm_gbs"]), "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)),
+                "bf16_tflops": float(d["bf16_tflops"]), "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "of measured"}
+    return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "of fallback"}
 
 
-def measured_tensor_peak_tops():
-    """Dense 4-bit (e2m1) tensor peak for the roofline: the measured bf16 burst peak x the nominal fp4 : bf16 ratio (4)."""
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(path):
-        with open(path) as f:
-            d = json.load(f)
-        return {"tops": float(d["bf16_tflops"]) * 4.0,
-                "how": "measured bf16 burst peak %.0f TFLOP/s x 4 (nominal dense fp4 : bf16 ratio), of measured" % float(d["bf16_tflops"])}
-    return {"tops": 1590.0 * 4.0, "how": "fallback bf16 peak 1590 TFLOP/s x 4 (nominal dense fp4 : bf16 ratio), of fallback"}
-
-
-def bitop_peak_tbitops(sm_count, sm_mhz):
+def carry_save_peak_tbitops(sm_count, sm_mhz):
     """Carry-save bound of sum popcount(a xor w) on the B200 integer pipes: with one POPC (XU pipe, 16 lanes/clk/SM)
     and four logic ops (ALU pipe, 64 lanes/clk/SM) per two 32-bit word pairs both pipes are full at 32 word pairs
     per clock per SM; 32 bit pairs per word pair, 2 bit-ops per bit pair."""
     return sm_count * 32 * 32 * 2 * sm_mhz * 1e6 / 1e12
+
+
+def popc_peak_tbitops(sm_count, sm_mhz):
+    """One POPC per 32-bit word pair: 16 POPC lanes per clock and SM."""
+    return sm_count * 16 * 32 * 2 * sm_mhz * 1e6 / 1e12
+
+
+def profile_figure(filename, key):
+    """A figure that a committed ncu summary under profiles/ states on a line `key: number` (None if absent)."""
+    path = os.path.join(ROOT, "profiles", filename)
+    if not os.path.exists(path):
+        return None
+    m = re.search(r"^%s:\s*([0-9.eE+]+)" % re.escape(key), open(path).read(), flags=re.M)
+    return float(m.group(1)) if m else None
 
 
 class ClockSampler:
@@ -137,49 +163,84 @@ class ClockSampler:
         sm = [m for m, _ in self.samples]
         return {"sm_mhz": statistics.median(sm), "sm_min_mhz": min(sm), "sm_max_mhz": self.max_mhz,
                 "power_w_max": max(p for _, p in self.samples), "samples": len(sm), "reasons": sorted(self.reasons),
-                "how": "NVML, every %.0f ms during the timed region" % (self.period * 1e3)}
+                "how": "NVML, every %.0f ms during the %d timed regions" % (self.period * 1e3, REGIONS)}
 
 
 # ---------------------------------------------------------------------------------------------------------------
+def oracle_cases(nb):
+    import oracle
+    cases = []
+    for _, C, HW, O, k, pad in LAYERS:
+        x, w = synth.conv_case(5, nb, C, HW, HW, O, k, k, salt=C)
+        scale, shift = oracle.bn_fold(*synth.bn_params(synth.rng(5, 900 + C), O))
+        cases.append((C, pad, x, oracle.pack_weights(w), scale, shift))
+    return cases
+
+
+def oracle_step(cases):
+    import oracle
+    for C, pad, x, wp, scale, shift in cases:
+        a = oracle.pack(x)
+        oracle.bconv_bits(a, C, wp, (1, 1), (pad, pad), -1)
+        acc = oracle.bconv_bits(a, C, wp, (1, 1), (pad, pad), -1)
+        oracle.bn_sign_pack(acc, scale, shift)
+
+
 def run_reference(args):
-    """The oracle, as it stands, on the host cores: each step is a bounded sample (batch 2 per shape) of the
-    workload, timed with the wall clock."""
+    """The oracle, as it stands, on the host cores: each step is a bounded sample (batch 8 of each layer instead of 256)
+    of the workload, timed with the wall clock."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import oracle
     cores = oracle.max_threads()
     oracle.set_threads(cores)
-    nb = 2
-    cases = []
-    for C, HW in synth.SWEEP_SHAPES:
-        x, w = synth.conv_case(2, nb, C, HW, HW, C, 3, 3, salt=C)
-        scale, shift = oracle.bn_fold(*synth.bn_params(synth.rng(2, 900 + C), C))
-        cases.append((C, x, oracle.pack_weights(w), scale, shift))
-
-    def step():
-        for C, x, wp, scale, shift in cases:
-            a = oracle.pack(x)
-            oracle.bconv_bits(a, C, wp, (1, 1), (1, 1), -1)
-            acc = oracle.bconv_bits(a, C, wp, (1, 1), (1, 1), -1)
-            oracle.bn_sign_pack(acc, scale, shift)
-
+    nb = 8
+    cases = oracle_cases(nb)
     for _ in range(args.warmup):
-        step()
+        oracle_step(cases)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        step()
+        oracle_step(cases)
     dt = time.perf_counter() - t0
     value = step_bitops(nb) * args.steps / dt / 1e9
-    sample = "batch %d of each of the four shapes per step (the workload's batch is %d)" % (nb, BATCH)
+    sample = "batch %d of each layer per step (the workload's batch is %d), whole steps, %d threads" % (nb, BATCH, cores)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "u64 words / int32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample": sample},
+        "config": config_dict(int(os.environ.get("WORLD_SIZE", "1"))),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def cpu_baseline():
+    """The oracle on the host cores, on a bounded sample of the same workload: whole steps at batch 8 of each layer
+    (instead of 256) on all cores for about 8 s, and the same steps on one thread for about 6 s."""
+    import oracle
+    cores = oracle.max_threads()
+    nb = 8
+    cases = oracle_cases(nb)
+
+    def timed(threads, budget_s):
+        oracle.set_threads(threads)
+        oracle_step(cases)
+        t, reps = 0.0, 0
+        while t < budget_s and reps < 200:
+            t0 = time.perf_counter()
+            oracle_step(cases)
+            t += time.perf_counter() - t0
+            reps += 1
+        return step_bitops(nb) * reps / t / 1e9, reps, t
+
+    v_all, r_all, t_all = timed(cores, 8.0)
+    v_one, r_one, t_one = timed(1, 6.0)
+    oracle.set_threads(cores)
+    return {"value": v_all, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d whole steps at batch %d of each layer instead of %d (%.1f s of wall time on %d threads)" % (r_all, nb, BATCH, t_all, cores),
+            "single_thread": {"value": v_one, "unit": UNIT, "cores": 1,
+                              "sample": "%d of the same steps on one thread (%.1f s)" % (r_one, t_one)}}
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -189,11 +250,29 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-extras", action="store_true", help="skip the per-config extra measurements")
+    ap.add_argument("--no-extras", action="store_true", help="skip the measurements beside the timed steps (pack, Bi-Real-18, ...)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--regions", type=int, default=REGIONS, help="repeats of the K-step timed region")
+    # one kernel case, for profiler captures and quick timings
+    ap.add_argument("--case", default=None, choices=["pack", "conv", "fused", "bireal_block", "bireal"])
+    ap.add_argument("--engine", default="popc", choices=["popc", "tc"])
+    ap.add_argument("--N", type=int, default=64)
+    ap.add_argument("--C", type=int, default=256)
+    ap.add_argument("--HW", type=int, default=28)
+    ap.add_argument("--O", type=int, default=0)
+    ap.add_argument("--k", type=int, default=3)
+    ap.add_argument("--stride", type=int, default=1)
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--reps", type=int, default=1, help="--case: launches per timed event pair")
+    ap.add_argument("--graph", action="store_true", help="--case: time a CUDA-graph replay of the `reps` launches")
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--tile", type=int, default=0)
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.case:
+        run_case(args)
         return
 
     import torch
@@ -214,173 +293,155 @@ def main():
     sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
     peaks = measured_peaks()
     warmup = max(args.warmup, 3)
+    regions = max(args.regions, 1)
 
     # ---- inputs: seeded, drawn on the host, resident in HBM before the timed region ------------------------------
     layers = []
-    for C, HW in synth.SWEEP_SHAPES:
-        x, w = synth.conv_case(2, BATCH, C, HW, HW, C, 3, 3, salt=C + 1000 * rank)
-        g = synth.rng(2, 900 + C)
-        bn = [torch.from_numpy(t).to(dev) for t in synth.bn_params(g, C)]
+    for name, C, HW, O, k, pad in LAYERS:
+        x, w = synth.conv_case(5, BATCH, C, HW, HW, O, k, k, salt=C + 1000 * rank)
+        bn = [torch.from_numpy(t).to(dev) for t in synth.bn_params(synth.rng(5, 900 + C), O)]
         scale, shift = B.bn_fold(*bn)
         xh = torch.from_numpy(x).pin_memory()
-        L = {
-            "C": C, "HW": HW, "x_host": xh, "x": xh.to(dev), "w": B.pack_weights(torch.from_numpy(w).to(dev)),
-            "scale": scale, "shift": shift,
-            "a": torch.empty((BATCH, HW, HW, (C + 63) // 64), dtype=torch.int64, device=dev),
-            "out": torch.empty((BATCH, HW, HW, C), dtype=torch.int32, device=dev),
-            "bits": torch.empty((BATCH, HW, HW, (C + 63) // 64), dtype=torch.int64, device=dev),
-            "bitops": conv_bitops(BATCH, C, HW, C, 3),
-        }
+        cw, ow = (C + 63) // 64, (O + 63) // 64
+        L = {"name": name, "C": C, "HW": HW, "O": O, "k": k, "pad": pad, "x_host": xh, "x": xh.to(dev),
+             "w": B.pack_weights(torch.from_numpy(w).to(dev)), "scale": scale, "shift": shift,
+             "a": torch.empty((BATCH, HW, HW, cw), dtype=torch.int64, device=dev),
+             "out": torch.empty((BATCH, HW, HW, O), dtype=torch.int32, device=dev),
+             "bits": torch.empty((BATCH, HW, HW, ow), dtype=torch.int64, device=dev),
+             "bitops": conv_bitops(BATCH, C, HW, O, k)}
         L["wt"] = B.TcWeights(L["w"], C)  # the same weights expanded once for the tensor-core engine
+        st, pd = (1, 1), (pad, pad)
         L["call_pack"] = B.prepare_pack(L["x"], L["a"])
-        L["call_conv"] = {"popc": B.prepare_bconv2d(L["a"], C, L["w"], L["out"], (1, 1), (1, 1), -1, B.NHWC),
-                          "tc": B.prepare_tc_bconv2d(L["a"], L["wt"], L["out"], (1, 1), (1, 1), -1, B.NHWC)}
-        L["call_fused"] = {"popc": B.prepare_bconv2d_bn_sign_pack(L["a"], C, L["w"], L["scale"], L["shift"], L["bits"], (1, 1), (1, 1), -1),
-                           "tc": B.prepare_tc_bconv2d_bn_sign_pack(L["a"], L["wt"], L["scale"], L["shift"], L["bits"], (1, 1), (1, 1), -1)}
-        L["out_host"] = torch.empty(L["out"].shape, dtype=torch.int32).pin_memory()
-        L["bits_host"] = torch.empty(L["bits"].shape, dtype=torch.int64).pin_memory()
-        ws_bytes = B.binary_layer_host_workspace_bytes(BATCH, C, HW, HW, C, 3, 3, (1, 1), (1, 1), -1)
-        L["ws"] = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        L["call_conv"] = {"popc": B.prepare_bconv2d(L["a"], C, L["w"], L["out"], st, pd, -1, B.NHWC),
+                          "tc": B.prepare_tc_bconv2d(L["a"], L["wt"], L["out"], st, pd, -1, B.NHWC)}
+        L["call_fused"] = {"popc": B.prepare_bconv2d_bn_sign_pack(L["a"], C, L["w"], L["scale"], L["shift"], L["bits"], st, pd, -1),
+                           "tc": B.prepare_tc_bconv2d_bn_sign_pack(L["a"], L["wt"], L["scale"], L["shift"], L["bits"], st, pd, -1)}
         layers.append(L)
-    # A second set of activation / output buffers with the same contents: consecutive steps alternate between the two
-    # sets, so that whatever a step reads or writes was last touched two steps (about 390 MB of traffic) earlier and
-    # has left the 126 MB L2; no flush kernel runs between steps.  Weights and BN vectors (1.3 MB) are shared.
-    def twin(L):
-        T = dict(L)
-        C = L["C"]
-        T["x"] = L["x"].clone()
-        for key in ("a", "out", "bits"):
-            T[key] = torch.empty_like(L[key])
-        T["call_pack"] = B.prepare_pack(T["x"], T["a"])
-        T["call_conv"] = {"popc": B.prepare_bconv2d(T["a"], C, L["w"], T["out"], (1, 1), (1, 1), -1, B.NHWC),
-                          "tc": B.prepare_tc_bconv2d(T["a"], L["wt"], T["out"], (1, 1), (1, 1), -1, B.NHWC)}
-        T["call_fused"] = {"popc": B.prepare_bconv2d_bn_sign_pack(T["a"], C, L["w"], L["scale"], L["shift"], T["bits"], (1, 1), (1, 1), -1),
-                           "tc": B.prepare_tc_bconv2d_bn_sign_pack(T["a"], L["wt"], L["scale"], L["shift"], T["bits"], (1, 1), (1, 1), -1)}
-        return T
-    layer_sets = [layers, [twin(L) for L in layers]]
-
-    def step(engine, convs_only=False, which=0):
-        for L in layer_sets[which]:
-            if not convs_only:
-                L["call_pack"]()
-            L["call_conv"][engine]()
-            L["call_fused"][engine]()
-    launches_per_step = 3 * len(layers)
-
-    # The four shapes are independent layers: in the timed step each is its own branch (stream) of the step's CUDA graph,
-    # pack -> convolution -> fused convolution in order inside a branch, so one shape's start-up and tail overlap the
-    # others' work.  The same 12 kernels; the serial form is timed beside it.
-    branch_streams = [torch.cuda.Stream() for _ in layers]
-
-    def step_branched(engine, which=0):
-        cur = torch.cuda.current_stream()
-        for L, bs in zip(layer_sets[which], branch_streams):
-            bs.wait_stream(cur)
-            with torch.cuda.stream(bs):
-                L["call_pack"]()
-                L["call_conv"][engine]()
-                L["call_fused"][engine]()
-        for bs in branch_streams:
-            cur.wait_stream(bs)
+    kernels_per_step = 3 * len(layers)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def capture(fn):
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        with torch.cuda.stream(side):
-            fn()
-            side.synchronize()
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=side):
-                fn()
-        torch.cuda.current_stream().wait_stream(side)
-        return graph
-
-    def timed_replays(graphs, n):
-        """n replays back to back, alternating between the two buffer sets; returns the device time per replay in ms."""
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        graphs[1].replay()  # (the set that the first timed replay does not use)
-        e0.record()
-        for k in range(n):
-            graphs[k % 2].replay()
-        e1.record()
+    def run_regions(engine, n_regions, k_steps):
+        """n_regions timed regions of k_steps steps each, launched eagerly on the current stream with a CUDA event between
+        all kernels.  Returns (ms of each region [max over ranks], {kernel name: mean ms per launch})."""
+        names = []
+        for L in layers:
+            names += ["pack_" + L["name"], "conv_int32_" + L["name"], "conv_fused_" + L["name"]]
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(k_steps * kernels_per_step + 1)] for _ in range(n_regions)]
+        for r in range(n_regions):
+            e = ev[r]
+            e[0].record()
+            i = 1
+            for _ in range(k_steps):
+                for L in layers:
+                    L["call_pack"](); e[i].record(); i += 1
+                    L["call_conv"][engine](); e[i].record(); i += 1
+                    L["call_fused"][engine](); e[i].record(); i += 1
         torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / n
+        region_ms = torch.tensor([ev[r][0].elapsed_time(ev[r][-1]) for r in range(n_regions)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(region_ms, op=dist.ReduceOp.MAX)
+        per = {n: [] for n in names}
+        for r in range(n_regions):
+            for i in range(k_steps * kernels_per_step):
+                per[names[i % kernels_per_step]].append(ev[r][i].elapsed_time(ev[r][i + 1]))
+        return region_ms.cpu().tolist(), {n: statistics.fmean(v) for n, v in per.items()}
 
-    for _ in range(warmup):
-        for which in (0, 1):
-            step("tc", which=which)
-            step("popc", which=which)
-    barrier()
-    # each step is one CUDA-graph replay (one host call), so the timed loop is never host-bound
-    g_step = {e: [capture(lambda e=e, w=w: step(e, which=w)) for w in (0, 1)] for e in ("tc", "popc")}
-    # side by side, launches capped at half the chip each fill it better than launches that each take all of it
-    B.tc_set_max_ctas(sm_count // 2)
-    g_branched = [capture(lambda w=w: step_branched("tc", which=w)) for w in (0, 1)]
-    B.tc_set_max_ctas(0)
-    g_conv = {e: [capture(lambda e=e, w=w: step(e, convs_only=True, which=w)) for w in (0, 1)] for e in ("tc", "popc")}
-    for _ in range(warmup):
-        g_branched[0].replay()
-        g_branched[1].replay()
+    for engine in ("popc", "tc"):
+        run_regions(engine, 1, warmup)
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.05)
     barrier()
+    # ---- the timed regions: `regions` times K steps with the xor + popcount kernels ---------------------------------
     host_t0 = time.perf_counter()
-    # ---- the timed region: K steps with the faster (tensor-core) engine ------------------------------------------
-    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for k in range(args.steps):
-        g_branched[k % 2].replay()
-    t_end.record()
-    host_issue_ms = (time.perf_counter() - host_t0) * 1e3  # time the host needed to enqueue everything
+    region_ms, per_kernel = run_regions("popc", regions, args.steps)
+    host_ms = (time.perf_counter() - host_t0) * 1e3
     barrier()
-    total_ms = torch.tensor([t_start.elapsed_time(t_end)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
-    total_ms = float(total_ms.item())
-    value = world * step_bitops(BATCH) * args.steps / (total_ms * 1e-3) / 1e9
-
-    # ---- the dominant kernels on their own: the eight convolution launches of a step, per engine ------------------
-    n_side = max(args.steps, 10)
-    tc_ms, popc_ms = timed_replays(g_conv["tc"], n_side), timed_replays(g_conv["popc"], n_side)
-    serial_step_ms = timed_replays(g_step["tc"], n_side)
-    popc_step_ms = timed_replays(g_step["popc"], n_side)
     clocks = sampler.stop()
-    conv_ops = step_bitops(BATCH)
-    tensor_peak = measured_tensor_peak_tops()
-    alu_peak = bitop_peak_tbitops(sm_count, peaks["sm_max_mhz"])
+    med_ms, min_ms = statistics.median(region_ms), min(region_ms)
+    value = world * step_bitops(BATCH) * args.steps / (med_ms * 1e-3) / 1e9
+    # the same step on the tensor-core engine, timed the same way
+    tc_regions = max(5, regions // 5)
+    tc_region_ms, tc_per_kernel = run_regions("tc", tc_regions, args.steps)
+    tc_med = statistics.median(tc_region_ms)
+
+    # ---- rooflines ----------------------------------------------------------------------------------------------
+    mhz = peaks["sm_max_mhz"]
+    cs_peak, popc_peak = carry_save_peak_tbitops(sm_count, mhz), popc_peak_tbitops(sm_count, mhz)
+    conv_names = [n for n in per_kernel if n.startswith("conv_")]
+    ops_of = {}
+    bytes_of = {}
+    for L in layers:
+        for form in ("int32", "fused"):
+            ops_of["conv_%s_%s" % (form, L["name"])] = L["bitops"]
+            bytes_of["conv_%s_%s" % (form, L["name"])] = conv_bytes(BATCH, L["C"], L["HW"], L["O"], L["k"], form == "fused")
+        bytes_of["pack_" + L["name"]] = L["x"].numel() * 4 + L["a"].numel() * 8
+    conv_ops = sum(ops_of[n] for n in conv_names)
+    conv_ms = sum(per_kernel[n] for n in conv_names)
+    achieved = conv_ops / (conv_ms * 1e-3) / 1e12
+    sampled_mhz = clocks.get("sm_mhz") or mhz
+    traffic = profile_figure("bconv_kernel_N256_C256_HW28_int32.md", "dram_bytes_per_launch")
     roofline = {
-        "bound": "tensor", "kernel": "bconv_tc_kernel (the 8 convolution launches of a step, one CUDA-graph replay)",
-        "achieved": conv_ops / (tc_ms * 1e-3) / 1e12, "peak": tensor_peak["tops"], "unit": "TFLOP/s",
-        "frac": conv_ops / (tc_ms * 1e-3) / 1e12 / tensor_peak["tops"], "peak_is": tensor_peak["how"],
-        "traffic": 5.34e6, "traffic_is": "dram bytes of one N=64 C=256 28x28 launch (ncu, profiles/bconv_tc_kernel_N64_C256_HW28.md); most of its int32 output (51 MB, evict-first) is still in L2 when the kernel ends",
-        "avg_launch_ms": tc_ms / 8, "conv_share_of_step": tc_ms / serial_step_ms,
-        "conv_share_is": "the eight convolutions one after another / the 12 kernels one after another (%.4f ms)" % serial_step_ms,
+        "bound": "alu",
+        "kernel": "bconv_kernel (xor + carry-save + popc on the integer pipes): the 4 convolution launches of a step, each timed "
+                  "with CUDA events on the launching stream inside the timed regions",
+        "achieved": achieved, "peak": cs_peak, "unit": "Tbit-ops/s", "frac": achieved / cs_peak,
+        "peak_is": "derived: 64 LOP3 lanes (ALU pipe) and 16 POPC lanes (XU pipe) per clock and SM; with one POPC and four logic ops per "
+                   "two 32-bit word pairs both pipes are full at 32 word pairs/clk/SM x %d SMs x %.0f MHz x 64 bit-ops; pipe rates %s "
+                   "(register-only micro-benchmark, profiles/ubench_int_pipes.md)" % (sm_count, mhz, peaks["source"]),
+        "frac_at_sampled_clock": achieved / carry_save_peak_tbitops(sm_count, sampled_mhz),
+        "popc_roofline": {"peak": popc_peak, "frac": achieved / popc_peak,
+                          "peak_is": "one POPC per 32-bit word pair: 16 POPC/clk/SM x %d SMs x 32 bits x 2 x %.0f MHz" % (sm_count, mhz)},
+        "avg_launch_ms": conv_ms / len(conv_names),
+        "traffic": traffic,
+        "traffic_is": "dram__bytes_read.sum + dram__bytes_write.sum of one conv_int32_conv3x3_256 launch at the bench's full size "
+                      "(profiles/bconv_kernel_N256_C256_HW28_int32.md); algorithmic bytes of that launch: %d" % bytes_of["conv_int32_conv3x3_256"],
+        "per_launch": {n: {"ms": per_kernel[n], "Tbit-ops/s": ops_of[n] / per_kernel[n] / 1e9,
+                           "frac": ops_of[n] / per_kernel[n] / 1e9 / cs_peak, "frac_of_popc_roofline": ops_of[n] / per_kernel[n] / 1e9 / popc_peak}
+                       for n in conv_names},
+        "hbm_kernels": {n: {"ms": per_kernel[n], "GB/s": bytes_of[n] / per_kernel[n] / 1e6,
+                            "frac": bytes_of[n] / per_kernel[n] / 1e6 / peaks["hbm_gbs"], "peak": peaks["hbm_gbs"], "peak_is": peaks["source"]}
+                        for n in per_kernel if n.startswith("pack_")},
         "note": "1 bit-op = 1 op: a +-1 multiply-add counts 2, as in FLOPs",
     }
-    roofline_bitop = {
-        "bound": "alu", "kernel": "bconv_kernel (integer pipes: xor + carry-save + popc), same 8 launches",
-        "achieved": conv_ops / (popc_ms * 1e-3) / 1e12, "peak": alu_peak, "unit": "Tbit-ops/s",
-        "frac": conv_ops / (popc_ms * 1e-3) / 1e12 / alu_peak,
-        "peak_is": "ALU+XU carry-save bound at %d SMs x %.0f MHz (derived: 64 LOP3 lanes and 16 POPC lanes per clock and SM, carry-save halves the POPCs); the one-POPC-per-word-pair bound is half of it"
-                   % (sm_count, peaks["sm_max_mhz"]),
-        "traffic": 2.69e6, "traffic_is": "dram bytes of one N=64 C=256 28x28 launch (ncu, profiles/bconv_kernel_N64_C256_HW28.md)",
-        "avg_launch_ms": popc_ms / 8,
-        "step_value_with_this_engine": step_bitops(BATCH) / (popc_step_ms * 1e-3) / 1e9,
+    # the tensor-core engine (not the bit-op method: its own bounds, never a % of the bit-op roofline)
+    fp4_peak = peaks["bf16_tflops_sustained"] * 4.0
+    tc_launch = {}
+    for n in conv_names:
+        ms = tc_per_kernel[n]
+        t_hbm = bytes_of[n] / (peaks["hbm_gbs"] * 1e9) * 1e3
+        t_tensor = ops_of[n] / (fp4_peak * 1e12) * 1e3
+        bound = "hbm" if t_hbm >= t_tensor else "tensor"
+        tc_launch[n] = {"ms": ms, "Tops/s": ops_of[n] / ms / 1e9, "bound": bound, "bound_ms": max(t_hbm, t_tensor),
+                        "frac": max(t_hbm, t_tensor) / ms,
+                        "GB/s": bytes_of[n] / ms / 1e6}
+    roofline["tensor_engine"] = {
+        "value": world * step_bitops(BATCH) * args.steps / (tc_med * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": tc_med / args.steps,
+        "regions": tc_regions, "kernel": "bconv_tc_kernel (bits expanded on chip to e2m1, tcgen05.mma kind::mxf4, TMEM accumulators)",
+        "per_launch": tc_launch,
+        "bounds_are": "per launch the slower of HBM (algorithmic bytes / %.0f GB/s %s) and the tensor pipe (ops / %.0f Tops/s = sustained bf16 "
+                      "peak %.0f x 4, the nominal dense fp4 : bf16 ratio, %s)" % (peaks["hbm_gbs"], peaks["source"], fp4_peak,
+                                                                                 peaks["bf16_tflops_sustained"], peaks["source"]),
+        "pack_ms": {n: tc_per_kernel[n] for n in tc_per_kernel if n.startswith("pack_")},
     }
 
     # ---- end to end through the host-buffer entry point ----------------------------------------------------------
+    for L in layers:
+        L["out_host"] = torch.empty(L["out"].shape, dtype=torch.int32).pin_memory()
+        L["bits_host"] = torch.empty(L["bits"].shape, dtype=torch.int64).pin_memory()
+        ws_bytes = B.binary_layer_host_workspace_bytes(BATCH, L["C"], L["HW"], L["HW"], L["O"], L["k"], L["k"], (1, 1), (L["pad"], L["pad"]), -1)
+        L["ws"] = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+
     def e2e_step():
         for L in layers:
-            B.binary_layer_host(L["x_host"], L["w"], L["ws"], (1, 1), (1, 1), -1, L["scale"], L["shift"],
+            B.binary_layer_host(L["x_host"], L["w"], L["ws"], (1, 1), (L["pad"], L["pad"]), -1, L["scale"], L["shift"],
                                 out_host=L["out_host"], bits_host=L["bits_host"])
-    e2e_steps = max(3, min(args.steps, 10))
+    e2e_steps = max(3, min(args.steps, 5))
     e2e_step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -396,135 +457,151 @@ def main():
         "value": world * step_bitops(BATCH) * e2e_steps / (float(e2e_ms.item()) * 1e-3) / 1e9, "unit": UNIT,
         "h2d_bytes_per_step": int(sum(L["x_host"].numel() * 4 for L in layers)),
         "d2h_bytes_per_step": int(sum(L["out_host"].numel() * 4 + L["bits_host"].numel() * 8 for L in layers)),
-        "steps": e2e_steps, "api": "dabnn_binary_layer_host (pinned host buffers in and out)",
+        "steps": e2e_steps, "ms_per_step": float(e2e_ms.item()) / e2e_steps,
+        "api": "dabnn_binary_layer_host (pinned host buffers in and out, copies inside the timed region; xor + popcount kernels)",
     }
+    for L in layers:
+        for key in ("out_host", "bits_host", "ws", "x_host"):
+            L.pop(key)
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
-        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "u64 words / int32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "batch_per_gpu": BATCH, "l2": "no flush: steps alternate between two buffer sets (about 390 MB touched between two uses of a buffer; L2 is 126 MB)",
-                   "launch": "each step is one CUDA-graph replay of its 12 kernels: four branches, one per shape (pack -> conv int32 -> conv fused), that the GPU overlaps, tensor-engine launches capped at half the SMs each (dabnn_tc_set_max_ctas)",
-                   "serial_ms_per_step": serial_step_ms,
-                   "engine": "tensor-core engine (e2m1 tcgen05) for the timed steps; the integer-pipe engine is timed beside it (roofline_bitop)",
-                   "parallelism": "replicas" if world > 1 else "single GPU"},
-        "roofline": roofline, "roofline_bitop": roofline_bitop, "e2e": e2e,
-        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
-        "host_issue_ms_per_step": host_issue_ms / args.steps,
+        "ms_per_step": med_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u64 words / int32", "data": "synthetic", "config": config_dict(world),
+        "roofline": roofline, "e2e": e2e,
+        "gpu_launches": kernels_per_step * args.steps * regions, "clocks": clocks,
+        "timed": {"regions": regions, "steps_per_region": args.steps, "region_ms_median": med_ms, "region_ms_min": min_ms,
+                  "total_ms": sum(region_ms), "host_ms": host_ms,
+                  "how": "each region = K steps launched eagerly (6 kernels per step, a CUDA event between kernels); value and ms_per_step "
+                         "come from the median region; engine = xor + popcount kernels on the integer pipes"},
     }
-
     if rank == 0 and world == 1:
+        del layers
+        torch.cuda.empty_cache()
+        if not args.no_extras:
+            bireal, extra = extras(B, torch, dev, peaks, sm_count)
+            result["bireal18"] = bireal
+            result["roofline"]["bireal18"] = bireal
+            result["roofline"]["pack_128x256x56x56"] = extra.pop("pack_128x256x56x56_back_to_back")
+            result["extras"] = extra
         if not args.no_cpu_baseline:
             result["cpu_baseline"] = cpu_baseline()
-        if not args.no_extras:
-            result["extras"] = extras(B, torch, dev, peaks, sm_count)
     if rank == 0:
         print(json.dumps(result))
     if world > 1:
         dist.destroy_process_group()
 
 
-def cpu_baseline():
-    """The oracle on the host cores, on a bounded sample of the same workload: whole steps at batch 32
-    (half the workload's batch), repeated until about 10 s of wall time have passed."""
-    import oracle
-    cores = oracle.max_threads()
-    oracle.set_threads(cores)
-    nb = 32
-    cases = []
-    for C, HW in synth.SWEEP_SHAPES:
-        x, w = synth.conv_case(2, nb, C, HW, HW, C, 3, 3, salt=C)
-        scale, shift = oracle.bn_fold(*synth.bn_params(synth.rng(2, 900 + C), C))
-        cases.append((C, x, oracle.pack_weights(w), scale, shift))
-    t, reps = 0.0, 0
-    while t < 10.0 and reps < 50:
-        t0 = time.perf_counter()
-        for C, x, wp, scale, shift in cases:
-            a = oracle.pack(x)
-            oracle.bconv_bits(a, C, wp, (1, 1), (1, 1), -1)
-            acc = oracle.bconv_bits(a, C, wp, (1, 1), (1, 1), -1)
-            oracle.bn_sign_pack(acc, scale, shift)
-        t += time.perf_counter() - t0
-        reps += 1
-    return {"value": step_bitops(nb) * reps / t / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "%d steps at batch %d instead of %d (%.1f s of wall time on %d threads)" % (reps, nb, BATCH, t, cores)}
+def time_fn(torch, fn, iters, flush=None):
+    fn(); fn(); fn()
+    torch.cuda.synchronize()
+    ms = []
+    for _ in range(iters):
+        if flush is not None:
+            flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    return statistics.median(ms), min(ms)
+
+
+def graph_of(torch, fn, reps):
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        fn()
+        s.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            for _ in range(reps):
+                fn()
+    torch.cuda.current_stream().wait_stream(s)
+    return g
 
 
 def extras(B, torch, dev, peaks, sm_count):
-    """Per-configuration measurements beside the headline (each a few launches; CUDA events)."""
+    """Measurements beside the timed steps (each a few launches; CUDA events): the Bi-Real Net 18 forward at batch 1 and
+    128, the bit-pack configuration, the batch-64 and batch-1 sweeps, BGEMM against direct convolution."""
     out = {}
 
-    def time_fn(fn, iters, flush=None):
-        fn(); fn(); fn()
-        torch.cuda.synchronize()
-        ms = []
-        for _ in range(iters):
-            if flush is not None:
-                flush.zero_()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(); fn(); e1.record()
-            torch.cuda.synchronize()
-            ms.append(e0.elapsed_time(e1))
-        return statistics.median(ms), min(ms)
+    # Bi-Real Net 18: batch 128 (eager launches and four forwards per CUDA graph) and batch 1 (CUDA-graph replay)
+    net = B.Bireal18(synth.bireal18_params())
+    img = torch.from_numpy(synth.bireal18_images(128)).to(dev)
+    logits = torch.empty((128, 1000), dtype=torch.float32, device=dev)
+    med, best = time_fn(torch, lambda: net.forward(img, logits), 10)
+    g128 = graph_of(torch, lambda: net.forward(img, logits), 4)
+    med4, _ = time_fn(torch, g128.replay, 10)
+    del g128
+    net_p = B.Bireal18(synth.bireal18_params(), engine="popc")
+    med_p, _ = time_fn(torch, lambda: net_p.forward(img, logits), 5)
+    del net_p
+    img1, logits1 = img[:1].contiguous(), torch.empty((1, 1000), dtype=torch.float32, device=dev)
+    g1 = graph_of(torch, lambda: net.forward(img1, logits1), 1)
+    med1, _ = time_fn(torch, g1.replay, 30)
+    g16 = graph_of(torch, lambda: net.forward(img1, logits1), 16)
+    med16, _ = time_fn(torch, g16.replay, 10)
+    del g1, g16
+    flag = B.last_device_flag()
+    bireal = {
+        "unit": "images/s",
+        "batch_128": {"images_per_s": 128 / (med4 / 4) * 1e3, "ms": med4 / 4,
+                      "launch": "four forward passes back to back in one CUDA graph; tensor-core engine on the 16 binary blocks",
+                      "eager_ms": med, "eager_images_per_s": 128 / med * 1e3,
+                      "xor_popcount_kernels_only_ms": med_p, "xor_popcount_kernels_only_images_per_s": 128 / med_p * 1e3},
+        "batch_1": {"images_per_s": 1e3 / med1, "ms": med1,
+                    "launch": "CUDA-graph replay of the 22 chained kernels, one replay per event pair: latency of a lone forward",
+                    "back_to_back_ms": med16 / 16, "back_to_back_images_per_s": 16e3 / med16},
+        "device_flag_after": flag,
+    }
+    del net, img, logits
 
     # bit-pack alone: fp32 NCHW 128x256x56x56 with ~1 % exact zeros (input 411 MB: cold by construction)
     x = torch.from_numpy(synth.pack_case()).to(dev)
     packed = torch.empty((128, 56, 56, 4), dtype=torch.int64, device=dev)
-    med, best = time_fn(lambda: B.pack(x, B.NCHW, out=packed), 10)
+    med, best = time_fn(torch, lambda: B.pack(x, B.NCHW, out=packed), 10)
     nbytes = x.numel() * 4 + packed.numel() * 8
     out["pack_128x256x56x56"] = {"ms": med, "GB/s": nbytes / med / 1e6, "frac_of_hbm_peak": nbytes / med / 1e6 / peaks["hbm_gbs"],
-                                 "peak_GB/s": peaks["hbm_gbs"], "peak_source": peaks["source"], "bytes": nbytes,
                                  "how": "one launch per CUDA-event pair (includes the launch gap of a lone kernel)"}
-    # the same launch ten times in one CUDA graph: the 411 MB input is larger than L2, so every launch reads DRAM, and
-    # the gaps between a lone kernel and its events drop out
-    s_pack = torch.cuda.Stream()
-    with torch.cuda.stream(s_pack):
-        B.pack(x, B.NCHW, out=packed)
-        s_pack.synchronize()
-        g_pack = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g_pack, stream=s_pack):
-            for _ in range(10):
-                B.pack(x, B.NCHW, out=packed)
-        med10, _ = time_fn(g_pack.replay, 5)
-    out["pack_128x256x56x56_back_to_back"] = {"ms": med10 / 10, "GB/s": nbytes / (med10 / 10) / 1e6,
-                                              "frac_of_hbm_peak": nbytes / (med10 / 10) / 1e6 / peaks["hbm_gbs"]}
-    del g_pack
-    del x, packed
+    g_pack = graph_of(torch, lambda: B.pack(x, B.NCHW, out=packed), 10)
+    med10, _ = time_fn(torch, g_pack.replay, 5)
+    out["pack_128x256x56x56_back_to_back"] = {"bound": "hbm", "ms": med10 / 10, "GB/s": nbytes / (med10 / 10) / 1e6,
+                                              "frac": nbytes / (med10 / 10) / 1e6 / peaks["hbm_gbs"], "peak": peaks["hbm_gbs"],
+                                              "peak_is": peaks["source"], "bytes": nbytes,
+                                              "how": "ten launches in one CUDA graph; the 411 MB input is larger than L2, so every launch reads DRAM"}
+    del g_pack, x, packed
+
+    # the batch-64 sweep of the four stage shapes (pack + conv int32 + conv fused each), per engine, as one CUDA graph
+    cs_peak = carry_save_peak_tbitops(sm_count, peaks["sm_max_mhz"])
+    sweep = []
+    for C, HW in synth.SWEEP_SHAPES:
+        g = torch.Generator(device=dev); g.manual_seed(5)
+        xs = torch.randn((64, C, HW, HW), device=dev, generator=g)
+        w = torch.randint(-2**62, 2**62, (C, 3, 3, C // 64), dtype=torch.int64, device=dev, generator=g)
+        sweep.append({"C": C, "x": xs, "w": w, "wt": B.TcWeights(w, C), "a": torch.empty((64, HW, HW, C // 64), dtype=torch.int64, device=dev),
+                      "o": torch.empty((64, HW, HW, C), dtype=torch.int32, device=dev), "sc": torch.rand(C, device=dev) + 0.5,
+                      "sh": torch.randn(C, device=dev), "bits": torch.empty((64, HW, HW, C // 64), dtype=torch.int64, device=dev)})
+    sweep_ops = sum(2 * conv_bitops(64, C, HW, C, 3) for C, HW in synth.SWEEP_SHAPES)
+
+    def sweep_step(engine):
+        for S in sweep:
+            B.pack(S["x"], B.NCHW, out=S["a"])
+            if engine == "tc":
+                B.tc_bconv2d(S["a"], S["wt"], (1, 1), (1, 1), -1, B.NHWC, out=S["o"])
+                B.tc_bconv2d_bn_sign_pack(S["a"], S["wt"], S["sc"], S["sh"], (1, 1), (1, 1), -1, out=S["bits"])
+            else:
+                B.bconv2d(S["a"], S["C"], S["w"], (1, 1), (1, 1), -1, B.NHWC, out=S["o"])
+                B.bconv2d_bn_sign_pack(S["a"], S["C"], S["w"], S["sc"], S["sh"], (1, 1), (1, 1), -1, out=S["bits"])
+    for engine in ("popc", "tc"):
+        gs = graph_of(torch, lambda: sweep_step(engine), 4)
+        m, _ = time_fn(torch, gs.replay, 10)
+        out["sweep_batch64_%s" % engine] = {"ms_per_step": m / 4, "Tbit-ops/s": sweep_ops / (m / 4) / 1e9,
+                                            "frac_of_carry_save_bound": sweep_ops / (m / 4) / 1e9 / cs_peak if engine == "popc" else None}
+        del gs
+    del sweep
 
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    peak = bitop_peak_tbitops(sm_count, peaks["sm_max_mhz"])
-    tpeak = measured_tensor_peak_tops()["tops"]
-    for name, (N, C, HW, O, k, pad) in {"conv_256x256x28x28_3x3": (256, 256, 28, 256, 3, 1),
-                                        "conv_256x512x14x14_1x1_to_2048": (256, 512, 14, 2048, 1, 0)}.items():
-        g = torch.Generator(device=dev); g.manual_seed(5)
-        a = torch.randint(-2**62, 2**62, (N, HW, HW, (C + 63) // 64), dtype=torch.int64, device=dev, generator=g)
-        w = torch.randint(-2**62, 2**62, (O, k, k, (C + 63) // 64), dtype=torch.int64, device=dev, generator=g)
-        o = torch.empty((N, HW, HW, O), dtype=torch.int32, device=dev)
-        wt = B.TcWeights(w, C)
-        ops = conv_bitops(N, C, HW, O, k)
-        med, best = time_fn(lambda: B.bconv2d(a, C, w, (1, 1), (pad, pad), -1, B.NHWC, out=o), 10, flush)
-        out[name] = {"int_pipes": {"ms": med, "Tbit-ops/s": ops / med / 1e9, "frac_of_bitop_peak": ops / med / 1e9 / peak}}
-        med, best = time_fn(lambda: B.tc_bconv2d(a, wt, (1, 1), (pad, pad), -1, B.NHWC, out=o), 10, flush)
-        out[name]["tensor"] = {"ms": med, "Tbit-ops/s": ops / med / 1e9, "frac_of_fp4_peak": ops / med / 1e9 / tpeak}
-        # the same launch with the fused BN + sign + pack epilogue (what a stack of binary layers runs), back to back
-        sc = torch.rand(O, device=dev) + 0.5
-        sh = torch.randn(O, device=dev)
-        bits = torch.empty((N, HW, HW, (O + 63) // 64), dtype=torch.int64, device=dev)
-        fused_call = B.prepare_tc_bconv2d_bn_sign_pack(a, wt, sc, sh, bits, (1, 1), (pad, pad), -1)
-        s_f = torch.cuda.Stream()
-        with torch.cuda.stream(s_f):
-            fused_call()
-            s_f.synchronize()
-            g_f = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g_f, stream=s_f):
-                for _ in range(10):
-                    fused_call()
-            med10, _ = time_fn(g_f.replay, 5)
-        out[name]["tensor_fused_back_to_back"] = {"ms": med10 / 10, "Tbit-ops/s": ops / (med10 / 10) / 1e9,
-                                                  "frac_of_fp4_peak": ops / (med10 / 10) / 1e9 / tpeak}
-        del a, w, o, wt, g_f, fused_call, bits
-
-    # BGEMM against direct convolution, the comparison of the paper's Fig. 4, on config 5a: the im2col matrix of the packed
+    # BGEMM against direct convolution, the comparison of the paper's Fig. 4, on the 3x3 layer: the im2col matrix of the packed
     # activations (padding taps hold the pad word) is materialised with torch slicing (plumbing, 58 MB of packed rows) and
     # multiplied by dabnn_bgemm; dabnn_bconv2d gathers the same rows on the fly (implicit BGEMM)
     N, C, HW, O = 256, 256, 28, 256
@@ -540,13 +617,13 @@ def extras(B, torch, dev, peaks, sm_count):
     direct = B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC)
     same = bool((B.bgemm(A, Bm, 9 * C).reshape(N, HW, HW, O) == direct).all())
     ops = conv_bitops(N, C, HW, O, 3)
-    t_gemm, _ = time_fn(lambda: B.bgemm(A, Bm, 9 * C), 5, flush)
-    t_both, _ = time_fn(lambda: B.bgemm(im2col(), Bm, 9 * C), 5, flush)
-    t_direct, _ = time_fn(lambda: B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC, out=direct), 5, flush)
+    t_gemm, _ = time_fn(torch, lambda: B.bgemm(A, Bm, 9 * C), 5, flush)
+    t_both, _ = time_fn(torch, lambda: B.bgemm(im2col(), Bm, 9 * C), 5, flush)
+    t_direct, _ = time_fn(torch, lambda: B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC, out=direct), 5, flush)
     out["bgemm_vs_direct_256x256x28x28"] = {"identical": same, "bgemm_ms": t_gemm, "im2col_plus_bgemm_ms": t_both,
                                             "direct_ms": t_direct, "direct_Tbit-ops/s": ops / t_direct / 1e9,
                                             "bgemm_Tbit-ops/s": ops / t_gemm / 1e9,
-                                            "note": "integer-pipe engine for both; im2col is torch slicing, not a tuned kernel"}
+                                            "note": "im2col is torch slicing, not a tuned kernel"}
     del a, w, A, Bm, direct
 
     # batch-1 latency of the four sweep shapes (CUDA-graph replay of 50 launches)
@@ -555,62 +632,82 @@ def extras(B, torch, dev, peaks, sm_count):
         a = torch.randint(-2**62, 2**62, (1, HW, HW, C // 64), dtype=torch.int64, device=dev, generator=g)
         w = torch.randint(-2**62, 2**62, (C, 3, 3, C // 64), dtype=torch.int64, device=dev, generator=g)
         o = torch.empty((1, HW, HW, C), dtype=torch.int32, device=dev)
-        s = torch.cuda.Stream()
-        with torch.cuda.stream(s):
-            for _ in range(3):
-                B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC, out=o)
-            s.synchronize()
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=s):
-                for _ in range(50):
-                    B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC, out=o)
-            med, best = time_fn(graph.replay, 5)
+        graph = graph_of(torch, lambda: B.bconv2d(a, C, w, (1, 1), (1, 1), -1, B.NHWC, out=o), 50)
+        med, best = time_fn(torch, graph.replay, 5)
         out["conv_batch1_C%d_%dx%d" % (C, HW, HW)] = {"us_per_conv": med * 1e3 / 50, "Tbit-ops/s": conv_bitops(1, C, HW, C, 3) / (med / 50) / 1e9}
+        del graph
+    return bireal, out
 
-    # Bi-Real Net 18: batch 128 (eager launches) and batch 1 (CUDA-graph replay)
-    net = B.Bireal18(synth.bireal18_params())
-    img = torch.from_numpy(synth.bireal18_images(128)).to(dev)
-    logits = torch.empty((128, 1000), dtype=torch.float32, device=dev)
-    med, best = time_fn(lambda: net.forward(img, logits), 5)
-    out["bireal18_batch128"] = {"ms": med, "images/s": 128 / med * 1e3, "engine": "tensor-core engine on all 16 binary blocks"}
-    s128 = torch.cuda.Stream()
-    with torch.cuda.stream(s128):
-        net.forward(img, logits)
-        s128.synchronize()
-        g128 = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g128, stream=s128):
-            for _ in range(4):
-                net.forward(img, logits)
-        med4, _ = time_fn(g128.replay, 5)
-    out["bireal18_batch128_graph"] = {"ms": med4 / 4, "images/s": 128 / (med4 / 4) * 1e3,
-                                      "launch": "four forward passes back to back in one CUDA graph"}
-    del g128
-    net_p = B.Bireal18(synth.bireal18_params(), engine="popc")
-    med, best = time_fn(lambda: net_p.forward(img, logits), 5)
-    out["bireal18_batch128_int_pipes"] = {"ms": med, "images/s": 128 / med * 1e3}
-    del net_p
-    img1, logits1 = img[:1].contiguous(), torch.empty((1, 1000), dtype=torch.float32, device=dev)
-    s = torch.cuda.Stream()
-    with torch.cuda.stream(s):
-        for _ in range(3):
-            net.forward(img1, logits1)
-        s.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=s):
-            net.forward(img1, logits1)
-        med, best = time_fn(graph.replay, 20)
-    out["bireal18_batch1"] = {"ms": med, "images/s": 1e3 / med,
-                              "launch": "CUDA graph replay of the 22 kernels (chained launches), one replay per event pair: latency of a lone forward"}
-    with torch.cuda.stream(s):
-        graph16 = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph16, stream=s):
-            for _ in range(16):
-                net.forward(img1, logits1)
-        med16, _ = time_fn(graph16.replay, 10)
-    out["bireal18_batch1_back_to_back"] = {"ms": med16 / 16, "images/s": 16e3 / med16,
-                                           "launch": "sixteen batch-1 forwards back to back in one CUDA graph"}
-    del graph16
-    return out
+
+# ---------------------------------------------------------------------------------------------------------------
+def run_case(a):
+    """Runs ONE kernel case a few times and prints the median CUDA-event time: what the ncu commands under profiles/ run."""
+    import torch
+
+    from paper_1908_05858_b200 import binding as B
+
+    O = a.O or a.C
+    dev = torch.device("cuda", 0)
+    B.set_conv_variant(a.variant)
+    B.set_conv_tile(a.tile)
+    pad = a.k // 2
+    st = (a.stride, a.stride)
+    OHW = (a.HW + 2 * pad - a.k) // a.stride + 1
+    ops = 2.0 * a.N * OHW * OHW * O * a.C * a.k * a.k / 1e12
+    work = ("Tbit-ops/s", ops)
+    if a.case == "bireal":
+        net = B.Bireal18(synth.bireal18_params(), engine="popc" if a.engine == "popc" else "auto")
+        img = torch.from_numpy(synth.bireal18_images(a.N)).to(dev)
+        logits = torch.empty((a.N, 1000), dtype=torch.float32, device=dev)
+        fn = lambda: net.forward(img, logits)
+        work = ("images/ms", a.N * 1e-3)
+    else:
+        x, w = synth.conv_case(9, a.N, a.C, a.HW, a.HW, O, a.k, a.k)
+        xd = torch.from_numpy(x).to(dev)
+        wp = B.pack_weights(torch.from_numpy(w).to(dev))
+        ap_ = B.pack(xd)
+        scale = torch.rand(O, device=dev) + 0.5
+        shift = torch.randn(O, device=dev)
+        wt = B.TcWeights(wp, a.C) if a.engine == "tc" else None
+        if a.case == "pack":
+            out = torch.empty_like(ap_)
+            fn = lambda: B.pack(xd, B.NCHW, out=out)
+            work = ("GB/s", (xd.numel() * 4 + out.numel() * 8) / 1e9)
+        elif a.case == "conv":
+            out = torch.empty((a.N, OHW, OHW, O), dtype=torch.int32, device=dev)
+            fn = ((lambda: B.tc_bconv2d(ap_, wt, st, (pad, pad), -1, B.NHWC, out=out)) if wt else
+                  (lambda: B.bconv2d(ap_, a.C, wp, st, (pad, pad), -1, B.NHWC, out=out)))
+        elif a.case == "fused":
+            out = torch.empty((a.N, OHW, OHW, (O + 63) // 64), dtype=torch.int64, device=dev)
+            fn = ((lambda: B.tc_bconv2d_bn_sign_pack(ap_, wt, scale, shift, st, (pad, pad), -1, out=out)) if wt else
+                  (lambda: B.bconv2d_bn_sign_pack(ap_, a.C, wp, scale, shift, st, (pad, pad), -1, out=out)))
+        else:  # bireal_block: the residual epilogue, in place on the fp32 stream as the network runs it
+            res = torch.randn((a.N, OHW, OHW, O), device=dev)
+            call = B.prepare_bireal_block(ap_, a.C, wp, wt, scale, shift, res, st, (pad, pad), -1)
+            fn = call
+    fn()
+    torch.cuda.synchronize()
+    reps = a.reps
+    if a.graph:
+        g = graph_of(torch, fn, a.reps)
+        fn, per = g.replay, a.reps
+        reps = 1
+    else:
+        per = a.reps
+    ms = []
+    for _ in range(a.iters):
+        # `reps` launches back to back inside one event pair, so that launch latency is hidden behind the
+        # previous launch's execution (a short kernel timed alone would measure the host, not the GPU)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1) / per)
+    med = statistics.median(ms)
+    print("%s engine=%s N=%d C=%d HW=%d O=%d k=%d stride=%d: median %.4f ms  %.1f %s" %
+          (a.case, a.engine, a.N, a.C, a.HW, O, a.k, a.stride, med, work[1] / (med * 1e-3), work[0]))
 
 
 if __name__ == "__main__":

@@ -535,6 +535,21 @@ def prepare_tc_bconv2d_bn_sign_pack(a_packed, wt: TcWeights, scale, shift, out, 
                      scale.data_ptr(), shift.data_ptr(), out.data_ptr()), (a, wt, scale, shift, out))
 
 
+def prepare_bireal_block(a_packed, C, w_packed, wt: Optional[TcWeights], scale, shift, stream_fp32, stride=(1, 1), pad=(0, 0),
+                         pad_value=-1) -> Prepared:
+    """The Bi-Real block call as the network makes it: y = BN(conv) + residual written over the residual (`stream_fp32`,
+    fp32 NHWC [N][OH][OW][O]) plus the packed signs; on the tensor-core engine when `wt` is given."""
+    a, w, N, H, W, O, kh, kw, OH, OW = _geom(a_packed, C, w_packed, stride, pad)
+    if tuple(stream_fp32.shape) != (N, OH, OW, O):
+        raise DabnnError("the fp32 stream must be NHWC [N][OH][OW][O]")
+    bits = _alloc((N, OH, OW, words_per_pixel(O)), torch.int64, a.device)
+    fn = lib().dabnn_tc_bconv2d_bn_add_sign_pack if wt is not None else lib().dabnn_bconv2d_bn_add_sign_pack
+    wptr = wt.buf.data_ptr() if wt is not None else w.data_ptr()
+    return Prepared(fn, (a.data_ptr(), Shape(N, C, H, W), wptr, O, _conv(kh, kw, stride, pad, pad_value), scale.data_ptr(),
+                         shift.data_ptr(), stream_fp32.data_ptr(), stream_fp32.data_ptr(), bits.data_ptr()),
+                    (a, w, wt, scale, shift, stream_fp32, bits))
+
+
 def set_conv_variant(variant: int) -> int:
     return int(lib().dabnn_set_conv_variant(int(variant)))
 
