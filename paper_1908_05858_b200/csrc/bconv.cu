@@ -27,11 +27,19 @@ namespace {
 int g_conv_variant = 0;
 int g_conv_tile = 0;
 
+// The mix of one- and two-level carry-save steps per K chunk (see bit_mac_pair), by register tile: tiles of up to 32
+// outputs per thread have room for the `twos` words.  Chosen by measurement (DABNN_L2MASK at build time overrides).
+#ifndef DABNN_L2MASK
+#define DABNN_L2MASK 0x00
+#endif
+template <int TP, int TO, bool CSA>
+constexpr int l2mask() { return (CSA && TP * TO <= 16) ? (DABNN_L2MASK) : 0; }
+
 template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16, int STAGES>
 dabnn_status launch_one(const BConvArgs& g, cudaStream_t st) {
   constexpr int THREADS = (BP / TP) * (BO / TO);
   constexpr size_t SMEM = (size_t)STAGES * (BP + BO) * PITCH * 4 + (size_t)BP * sizeof(RowInfo);
-  auto kern = bconv_kernel<BP, BO, TP, TO, MINB, EPI, CSA, VEC16, STAGES>;
+  auto kern = bconv_kernel<BP, BO, TP, TO, MINB, EPI, CSA, VEC16, STAGES, l2mask<TP, TO, CSA>()>;
   static bool configured[kMaxDevices] = {};  // one attribute call per instantiation and device (idempotent if raced)
   const int dev = current_device();
   if (dev < 0) return DABNN_ERR_CUDA;
@@ -68,9 +76,11 @@ dabnn_status launch_epi(const BConvArgs& g, cudaStream_t st) {
   auto ctas = [&](int bp, int bo) { return ((g.M + bp - 1) / bp) * ((ochan + bo - 1) / bo); };
   int tile = g_conv_tile;
   if (tile == 0) {
-    if (ochan > 64 && ctas(128, 128) >= 2LL * sms) tile = 1;
-    else if (ctas(128, 64) >= 4LL * sms) tile = 2;
-    else if (ctas(64, 64) >= 2LL * sms) tile = 3;
+    // Measured on B200 (batch 64 to 256, the ResNet-18 stage shapes and the 1x1 512 -> 2048 layer): 16 outputs per thread at
+    // four warps per scheduler beat the larger register tiles (which spill or leave two warps per scheduler) wherever K
+    // spans more than one chunk; short K (one chunk, nothing to pipeline inside a CTA) does better with 128 x 64.
+    if (g.K64 <= 12 && ctas(128, 64) >= 4LL * sms) tile = 2;
+    else if (ctas(64, 64) >= 4LL * sms) tile = 3;
     else if (ctas(32, 32) >= sms || g.K64 > 5 * KC64) tile = 4;
     else tile = 5;  // less than one wave of the smallest tile: latency is all that counts
   }
@@ -107,7 +117,9 @@ dabnn_status fill_args(BConvArgs& g, const uint64_t* a, dabnn_shape in, const ui
   g.pad_neg = cv.pad_value < 0;
   g.tail_mask = (in.C % 64 == 0) ? ~0ull : ((1ull << (in.C % 64)) - 1);
   g.out = nullptr; g.out_nchw = 0; g.scale = g.shift = g.residual = nullptr; g.y_out = nullptr;
-  g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64); g.one = 1;
+  g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64); g.one = 1; g.two = 2;
+  g.magic_cw = Cw == 1 ? 0ull : ~0ull / (unsigned long long)Cw + 1ull;
+  g.magic_kw = cv.kw == 1 ? 0ull : ~0ull / (unsigned long long)cv.kw + 1ull;
   return DABNN_OK;
 }
 

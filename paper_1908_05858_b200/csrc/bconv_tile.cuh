@@ -32,7 +32,8 @@ struct BConvArgs {
   float* y_out;
   uint32_t* out_packed32;  // packed output viewed as 32-bit halves
   int Ow32;                // 2*ceil(O/64)
-  int one;                 // the constant 1 (see bit_mac)
+  int one, two;            // the constants 1 and 2 (see bit_mac)
+  unsigned long long magic_cw, magic_kw;  // ceil(2^64 / Cw), ceil(2^64 / kw) (0 when the divisor is 1): see fast_div
 };
 
 struct RowInfo {
@@ -41,6 +42,10 @@ struct RowInfo {
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// floor(q / d) for q < 2^32 with magic = ceil(2^64 / d) (0 for d = 1): one 64-bit multiply-high instead of a division.
+__device__ __forceinline__ int fast_div(int q, unsigned long long magic) {
+  return magic == 0 ? q : (int)__umul64hi((unsigned long long)(uint32_t)q, magic);
+}
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
@@ -59,10 +64,14 @@ template <bool CSA>
 __device__ __forceinline__ void bit_mac(uint32_t a0, uint32_t a1, uint32_t w0, uint32_t w1, int& acc, uint32_t& ones,
                                         int one) {
   if (CSA) {
-    const uint32_t x1 = a0 ^ w0, x2 = a1 ^ w1;
-    uint32_t s, c;
-    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(s) : "r"(ones), "r"(x1), "r"(x2));  // sum bit
-    asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(c) : "r"(ones), "r"(x1), "r"(x2));  // carry bit (majority)
+    // Full adder of (ones, a0 ^ w0, a1 ^ w1) in three 3-input logic ops, the xors folded in:
+    //   t = ones ^ a0 ^ w0;  s = t ^ a1 ^ w1 (the sum bit);  carry = t ? ~s : ones
+    // (where ones and the first term differ, t = 1 and the majority is the second term, which is s ^ t = ~s; where
+    // they agree, t = 0 and the majority is their common value).
+    uint32_t t, s, c;
+    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(t) : "r"(ones), "r"(a0), "r"(w0));
+    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(s) : "r"(t), "r"(a1), "r"(w1));
+    asm("lop3.b32 %0, %1, %2, %3, 0x3A;" : "=r"(c) : "r"(t), "r"(s), "r"(ones));  // (t & ~s) | (~t & ones)
     ones = s;
     acc = __popc(c) * one + acc;
   } else {
@@ -71,9 +80,38 @@ __device__ __forceinline__ void bit_mac(uint32_t a0, uint32_t a1, uint32_t w0, u
   }
 }
 
+// Two 64-bit word pairs of one output (one 128-bit load of each operand).  L2 = false: two full adders into `ones`,
+// both carry words popcounted (6 logic ops, 2 POPC).  L2 = true: the two carry words go through a second full adder with a
+// running `twos` word and only ITS carry word (weight 4) is popcounted (8 logic ops, 1 POPC).  `acc` counts in units of 2.
+// POPC issues at a quarter of the logic rate, so the kernel mixes the two forms (L2MASK of bconv_tile) to load both pipes.
+template <bool L2>
+__device__ __forceinline__ void bit_mac_pair(const uint4 a, const uint4 w, int& acc, uint32_t& ones, uint32_t& twos,
+                                             int one, int two) {
+  uint32_t t, s, c0, c1;
+  asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(t) : "r"(ones), "r"(a.x), "r"(w.x));
+  asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(s) : "r"(t), "r"(a.y), "r"(w.y));
+  asm("lop3.b32 %0, %1, %2, %3, 0x3A;" : "=r"(c0) : "r"(t), "r"(s), "r"(ones));
+  ones = s;
+  asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(t) : "r"(ones), "r"(a.z), "r"(w.z));
+  asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(s) : "r"(t), "r"(a.w), "r"(w.w));
+  asm("lop3.b32 %0, %1, %2, %3, 0x3A;" : "=r"(c1) : "r"(t), "r"(s), "r"(ones));
+  ones = s;
+  if (L2) {
+    uint32_t s2, c4;
+    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(s2) : "r"(twos), "r"(c0), "r"(c1));
+    asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(c4) : "r"(twos), "r"(c0), "r"(c1));
+    twos = s2;
+    acc = __popc(c4) * two + acc;
+  } else {
+    acc = __popc(c0) * one + acc;
+    acc = __popc(c1) * one + acc;
+  }
+}
+
 // One tile: pixel tile `bx`, channel tile `by`, `smem` = STAGES * (BP + BO) * PITCH words + BP RowInfo.  All threads of
 // the CTA call it together.  CHAINED: the stand-alone kernel's hooks for chained launches (see common.cuh).
-template <int BP, int BO, int TP, int TO, int EPI, bool CSA, bool VEC16, int STAGES, bool CHAINED>
+// L2MASK (carry-save form only): bit u set = the u-th 128-bit step of a K chunk takes the two-level form of bit_mac_pair.
+template <int BP, int BO, int TP, int TO, int EPI, bool CSA, bool VEC16, int STAGES, bool CHAINED, int L2MASK = 0>
 __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long bx, const int by, uint32_t* smem) {
   constexpr int THREADS = (BP / TP) * (BO / TO);
   constexpr int UW = VEC16 ? 2 : 1;         // 64-bit words per copy unit
@@ -126,9 +164,9 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
     const bool k_live = k < g.K64;
     int tap = 0, cw = 0, ti = 0, tj = 0;
     if (k_live) {
-      tap = k / g.Cw;
+      tap = fast_div(k, g.magic_cw);
       cw = k - tap * g.Cw;
-      ti = tap / g.kw;
+      ti = fast_div(tap, g.magic_kw);
       tj = tap - ti * g.kw;
     }
     // activations: one im2col row per output pixel
@@ -149,7 +187,8 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
         if (UW == 2) *reinterpret_cast<ulonglong2*>(dst) = make_ulonglong2(p0, p1);
         else *reinterpret_cast<uint64_t*>(dst) = p0;
       } else {
-        const uint64_t* src = live ? g.a + ri.base + ((long long)ih * g.W + iw) * g.Cw + cw : g.a;
+        // (the offset inside one image fits 32 bits: checked on the host)
+        const uint64_t* src = live ? g.a + (ri.base + (long long)((ih * g.W + iw) * g.Cw + cw)) : g.a;
         if (UW == 2) cp_async16(smem_u32(dst), src, live ? 16 : 0);
         else cp_async8(smem_u32(dst), src, live ? 8 : 0);
       }
@@ -174,14 +213,18 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
   const int arow0 = wp * 8 * TP + pl;        // + 8*i
   const int wrow0 = wo * 4 * TO + ol * TO;   // + j
 
+  constexpr bool TWOS = CSA && L2MASK != 0;
+  const int two = g.two;
   int acc[TP][TO];
   uint32_t ones[TP][TO];
+  uint32_t twos[TWOS ? TP : 1][TWOS ? TO : 1];
 #pragma unroll
   for (int i = 0; i < TP; i++)
 #pragma unroll
     for (int j = 0; j < TO; j++) {
       acc[i][j] = 0;
       ones[i][j] = 0;
+      if (TWOS) twos[i][j] = 0;
     }
 
   float sc[TO], sf[TO], res[TP][TO];
@@ -240,20 +283,40 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
     const uint32_t* Ws = As + BP * PITCH;
     const int kvalid = min(KC64, g.K64 - chunk * KC64);  // 64-bit words in this chunk
     int k = 0;
+    if (TWOS) {
+      // the chunk's eight 128-bit steps unrolled, each in the form its bit of L2MASK selects
+#pragma unroll
+      for (int u = 0; u < KC64 / 2; u++) {
+        if (2 * u + 2 > kvalid) break;
+        uint4 w[TO];
+#pragma unroll
+        for (int j = 0; j < TO; j++) w[j] = *reinterpret_cast<const uint4*>(Ws + (wrow0 + j) * PITCH + 4 * u);
+#pragma unroll
+        for (int i = 0; i < TP; i++) {
+          const uint4 a = *reinterpret_cast<const uint4*>(As + (arow0 + 8 * i) * PITCH + 4 * u);
+#pragma unroll
+          for (int j = 0; j < TO; j++) {
+            if ((L2MASK >> u) & 1) bit_mac_pair<true>(a, w[j], acc[i][j], ones[i][j], twos[TWOS ? i : 0][TWOS ? j : 0], one, two);
+            else bit_mac_pair<false>(a, w[j], acc[i][j], ones[i][j], twos[TWOS ? i : 0][TWOS ? j : 0], one, two);
+          }
+        }
+        k = 2 * u + 2;
+      }
+    }
 #pragma unroll UNROLL_K
     for (; k + 2 <= kvalid; k += 2) {
-      uint4 a[TP], w[TO];
-#pragma unroll
-      for (int i = 0; i < TP; i++) a[i] = *reinterpret_cast<const uint4*>(As + (arow0 + 8 * i) * PITCH + 2 * k);
+      uint4 w[TO];
 #pragma unroll
       for (int j = 0; j < TO; j++) w[j] = *reinterpret_cast<const uint4*>(Ws + (wrow0 + j) * PITCH + 2 * k);
 #pragma unroll
-      for (int i = 0; i < TP; i++)
+      for (int i = 0; i < TP; i++) {  // (activation rows one at a time: a thread never holds all of them)
+        const uint4 a = *reinterpret_cast<const uint4*>(As + (arow0 + 8 * i) * PITCH + 2 * k);
 #pragma unroll
         for (int j = 0; j < TO; j++) {
-          bit_mac<CSA>(a[i].x, a[i].y, w[j].x, w[j].y, acc[i][j], ones[i][j], one);
-          bit_mac<CSA>(a[i].z, a[i].w, w[j].z, w[j].w, acc[i][j], ones[i][j], one);
+          bit_mac<CSA>(a.x, a.y, w[j].x, w[j].y, acc[i][j], ones[i][j], one);
+          bit_mac<CSA>(a.z, a.w, w[j].z, w[j].w, acc[i][j], ones[i][j], one);
         }
+      }
     }
     if (k < kvalid) {  // odd tail: one 64-bit word
       uint2 a[TP], w[TO];
@@ -279,7 +342,8 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
       int v[TO];
 #pragma unroll
       for (int j = 0; j < TO; j++) {
-        const int cnt = CSA ? 2 * acc[i][j] + __popc(ones[i][j]) : acc[i][j];
+        int cnt = CSA ? 2 * acc[i][j] + __popc(ones[i][j]) : acc[i][j];
+        if (TWOS) cnt += 2 * __popc(twos[i][j]);
         v[j] = g.Kbits - 2 * cnt;
       }
       const int o = o0 + wrow0;
@@ -327,7 +391,8 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
       float y[TO];
 #pragma unroll
       for (int j = 0; j < TO; j++) {
-        const int cnt = CSA ? 2 * acc[i][j] + __popc(ones[i][j]) : acc[i][j];
+        int cnt = CSA ? 2 * acc[i][j] + __popc(ones[i][j]) : acc[i][j];
+        if (TWOS) cnt += 2 * __popc(twos[i][j]);
         y[j] = __fmaf_rn((float)(g.Kbits - 2 * cnt), sc[j], sf[j]);
       }
       if (EPI == EPI_BIREAL) {
@@ -373,10 +438,10 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
   }
 }
 
-template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16, int STAGES>
+template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16, int STAGES, int L2MASK>
 __global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(const BConvArgs g) {
   extern __shared__ __align__(16) uint32_t bconv_smem[];
-  bconv_tile<BP, BO, TP, TO, EPI, CSA, VEC16, STAGES, true>(g, blockIdx.x, blockIdx.y, bconv_smem);
+  bconv_tile<BP, BO, TP, TO, EPI, CSA, VEC16, STAGES, true, L2MASK>(g, blockIdx.x, blockIdx.y, bconv_smem);
 }
 
 }  // namespace
