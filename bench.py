@@ -77,9 +77,9 @@ def measured_peaks():
 
 
 def carry_save_peak_tbitops(sm_count, sm_mhz):
-    """Carry-save bound of sum popcount(a xor w) on the B200 integer pipes: with one POPC (XU pipe, 16 lanes/clk/SM)
-    and four logic ops (ALU pipe, 64 lanes/clk/SM) per two 32-bit word pairs both pipes are full at 32 word pairs
-    per clock per SM; 32 bit pairs per word pair, 2 bit-ops per bit pair."""
+    """Carry-save bound of sum popcount(a xor w) on the B200 integer pipes: one POPC (XU pipe, 16 lanes/clk/SM) and
+    three logic ops (ALU pipe, 64 lanes/clk/SM) per two 32-bit word pairs fill the XU pipe at 32 word pairs per clock
+    per SM (ALU at 3/4); 32 bit pairs per word pair, 2 bit-ops per bit pair."""
     return sm_count * 32 * 32 * 2 * sm_mhz * 1e6 / 1e12
 
 
@@ -391,9 +391,9 @@ def main():
         "kernel": "bconv_kernel (xor + carry-save + popc on the integer pipes): the 4 convolution launches of a step, each timed "
                   "with CUDA events on the launching stream inside the timed regions",
         "achieved": achieved, "peak": cs_peak, "unit": "Tbit-ops/s", "frac": achieved / cs_peak,
-        "peak_is": "derived: 64 LOP3 lanes (ALU pipe) and 16 POPC lanes (XU pipe) per clock and SM; with one POPC and four logic ops per "
-                   "two 32-bit word pairs both pipes are full at 32 word pairs/clk/SM x %d SMs x %.0f MHz x 64 bit-ops; pipe rates %s "
-                   "(register-only micro-benchmark, profiles/ubench_int_pipes.md)" % (sm_count, mhz, peaks["source"]),
+        "peak_is": "derived: 16 POPC lanes (XU pipe) and 64 LOP3 lanes (ALU pipe) per clock and SM; the kernel's carry-save step is one POPC "
+                   "and three logic ops per two 32-bit word pairs, so the XU pipe is full at 32 word pairs/clk/SM x %d SMs x %.0f MHz x 64 "
+                   "bit-ops (ALU at 3/4); pipe rates %s (register-only micro-benchmark, profiles/ubench_int_pipes.md)" % (sm_count, mhz, peaks["source"]),
         "frac_at_sampled_clock": achieved / carry_save_peak_tbitops(sm_count, sampled_mhz),
         "popc_roofline": {"peak": popc_peak, "frac": achieved / popc_peak,
                           "peak_is": "one POPC per 32-bit word pair: 16 POPC/clk/SM x %d SMs x 32 bits x 2 x %.0f MHz" % (sm_count, mhz)},

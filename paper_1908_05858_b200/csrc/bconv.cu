@@ -11,10 +11,13 @@
 //
 // Pipes (measured on B200): POPC issues on the XU pipe at 16 lanes/clk/SM, LOP3 and IADD on the ALU
 // pipe at 64 lanes/clk/SM.  The plain loop (xor, popc, add per 32-bit word pair) is therefore
-// POPC-bound.  The carry-save loop feeds the two halves of a 64-bit word pair through a 3:2
-// compressor with a running "ones" word per output (2 xor + 2 lop3 per two word pairs) and
-// popcounts only the carry word: half the POPCs for twice the logic, which balances the two pipes.
+// POPC-bound.  The carry-save loop feeds the two halves of a 64-bit word pair through a full adder
+// with a running "ones" word per output -- three 3-input logic ops with the xors folded in, see
+// bit_mac -- and popcounts only the carry word: half the POPCs, so the bound doubles to 32 word
+// pairs/clk/SM (XU full, ALU at 3/4), and the accumulation is an IMAD on the FMA pipe.
 // Both give sum popcount(a xor w) exactly.
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "bconv_tile.cuh"
 
@@ -27,19 +30,11 @@ namespace {
 int g_conv_variant = 0;
 int g_conv_tile = 0;
 
-// The mix of one- and two-level carry-save steps per K chunk (see bit_mac_pair), by register tile: tiles of up to 32
-// outputs per thread have room for the `twos` words.  Chosen by measurement (DABNN_L2MASK at build time overrides).
-#ifndef DABNN_L2MASK
-#define DABNN_L2MASK 0x00
-#endif
-template <int TP, int TO, bool CSA>
-constexpr int l2mask() { return (CSA && TP * TO <= 16) ? (DABNN_L2MASK) : 0; }
-
 template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16, int STAGES>
 dabnn_status launch_one(const BConvArgs& g, cudaStream_t st) {
   constexpr int THREADS = (BP / TP) * (BO / TO);
   constexpr size_t SMEM = (size_t)STAGES * (BP + BO) * PITCH * 4 + (size_t)BP * sizeof(RowInfo);
-  auto kern = bconv_kernel<BP, BO, TP, TO, MINB, EPI, CSA, VEC16, STAGES, l2mask<TP, TO, CSA>()>;
+  auto kern = bconv_kernel<BP, BO, TP, TO, MINB, EPI, CSA, VEC16, STAGES>;
   static bool configured[kMaxDevices] = {};  // one attribute call per instantiation and device (idempotent if raced)
   const int dev = current_device();
   if (dev < 0) return DABNN_ERR_CUDA;
@@ -117,7 +112,7 @@ dabnn_status fill_args(BConvArgs& g, const uint64_t* a, dabnn_shape in, const ui
   g.pad_neg = cv.pad_value < 0;
   g.tail_mask = (in.C % 64 == 0) ? ~0ull : ((1ull << (in.C % 64)) - 1);
   g.out = nullptr; g.out_nchw = 0; g.scale = g.shift = g.residual = nullptr; g.y_out = nullptr;
-  g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64); g.one = 1; g.two = 2;
+  g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64); g.one = 1;
   g.magic_cw = Cw == 1 ? 0ull : ~0ull / (unsigned long long)Cw + 1ull;
   g.magic_kw = cv.kw == 1 ? 0ull : ~0ull / (unsigned long long)cv.kw + 1ull;
   return DABNN_OK;

@@ -32,7 +32,7 @@ struct BConvArgs {
   float* y_out;
   uint32_t* out_packed32;  // packed output viewed as 32-bit halves
   int Ow32;                // 2*ceil(O/64)
-  int one, two;            // the constants 1 and 2 (see bit_mac)
+  int one;                 // the constant 1 (see bit_mac)
   unsigned long long magic_cw, magic_kw;  // ceil(2^64 / Cw), ceil(2^64 / kw) (0 when the divisor is 1): see fast_div
 };
 
@@ -80,38 +80,9 @@ __device__ __forceinline__ void bit_mac(uint32_t a0, uint32_t a1, uint32_t w0, u
   }
 }
 
-// Two 64-bit word pairs of one output (one 128-bit load of each operand).  L2 = false: two full adders into `ones`,
-// both carry words popcounted (6 logic ops, 2 POPC).  L2 = true: the two carry words go through a second full adder with a
-// running `twos` word and only ITS carry word (weight 4) is popcounted (8 logic ops, 1 POPC).  `acc` counts in units of 2.
-// POPC issues at a quarter of the logic rate, so the kernel mixes the two forms (L2MASK of bconv_tile) to load both pipes.
-template <bool L2>
-__device__ __forceinline__ void bit_mac_pair(const uint4 a, const uint4 w, int& acc, uint32_t& ones, uint32_t& twos,
-                                             int one, int two) {
-  uint32_t t, s, c0, c1;
-  asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(t) : "r"(ones), "r"(a.x), "r"(w.x));
-  asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(s) : "r"(t), "r"(a.y), "r"(w.y));
-  asm("lop3.b32 %0, %1, %2, %3, 0x3A;" : "=r"(c0) : "r"(t), "r"(s), "r"(ones));
-  ones = s;
-  asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(t) : "r"(ones), "r"(a.z), "r"(w.z));
-  asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(s) : "r"(t), "r"(a.w), "r"(w.w));
-  asm("lop3.b32 %0, %1, %2, %3, 0x3A;" : "=r"(c1) : "r"(t), "r"(s), "r"(ones));
-  ones = s;
-  if (L2) {
-    uint32_t s2, c4;
-    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(s2) : "r"(twos), "r"(c0), "r"(c1));
-    asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(c4) : "r"(twos), "r"(c0), "r"(c1));
-    twos = s2;
-    acc = __popc(c4) * two + acc;
-  } else {
-    acc = __popc(c0) * one + acc;
-    acc = __popc(c1) * one + acc;
-  }
-}
-
 // One tile: pixel tile `bx`, channel tile `by`, `smem` = STAGES * (BP + BO) * PITCH words + BP RowInfo.  All threads of
 // the CTA call it together.  CHAINED: the stand-alone kernel's hooks for chained launches (see common.cuh).
-// L2MASK (carry-save form only): bit u set = the u-th 128-bit step of a K chunk takes the two-level form of bit_mac_pair.
-template <int BP, int BO, int TP, int TO, int EPI, bool CSA, bool VEC16, int STAGES, bool CHAINED, int L2MASK = 0>
+template <int BP, int BO, int TP, int TO, int EPI, bool CSA, bool VEC16, int STAGES, bool CHAINED>
 __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long bx, const int by, uint32_t* smem) {
   constexpr int THREADS = (BP / TP) * (BO / TO);
   constexpr int UW = VEC16 ? 2 : 1;         // 64-bit words per copy unit
@@ -213,18 +184,14 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
   const int arow0 = wp * 8 * TP + pl;        // + 8*i
   const int wrow0 = wo * 4 * TO + ol * TO;   // + j
 
-  constexpr bool TWOS = CSA && L2MASK != 0;
-  const int two = g.two;
   int acc[TP][TO];
   uint32_t ones[TP][TO];
-  uint32_t twos[TWOS ? TP : 1][TWOS ? TO : 1];
 #pragma unroll
   for (int i = 0; i < TP; i++)
 #pragma unroll
     for (int j = 0; j < TO; j++) {
       acc[i][j] = 0;
       ones[i][j] = 0;
-      if (TWOS) twos[i][j] = 0;
     }
 
   float sc[TO], sf[TO], res[TP][TO];
@@ -283,26 +250,6 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
     const uint32_t* Ws = As + BP * PITCH;
     const int kvalid = min(KC64, g.K64 - chunk * KC64);  // 64-bit words in this chunk
     int k = 0;
-    if (TWOS) {
-      // the chunk's eight 128-bit steps unrolled, each in the form its bit of L2MASK selects
-#pragma unroll
-      for (int u = 0; u < KC64 / 2; u++) {
-        if (2 * u + 2 > kvalid) break;
-        uint4 w[TO];
-#pragma unroll
-        for (int j = 0; j < TO; j++) w[j] = *reinterpret_cast<const uint4*>(Ws + (wrow0 + j) * PITCH + 4 * u);
-#pragma unroll
-        for (int i = 0; i < TP; i++) {
-          const uint4 a = *reinterpret_cast<const uint4*>(As + (arow0 + 8 * i) * PITCH + 4 * u);
-#pragma unroll
-          for (int j = 0; j < TO; j++) {
-            if ((L2MASK >> u) & 1) bit_mac_pair<true>(a, w[j], acc[i][j], ones[i][j], twos[TWOS ? i : 0][TWOS ? j : 0], one, two);
-            else bit_mac_pair<false>(a, w[j], acc[i][j], ones[i][j], twos[TWOS ? i : 0][TWOS ? j : 0], one, two);
-          }
-        }
-        k = 2 * u + 2;
-      }
-    }
 #pragma unroll UNROLL_K
     for (; k + 2 <= kvalid; k += 2) {
       uint4 w[TO];
@@ -342,8 +289,7 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
       int v[TO];
 #pragma unroll
       for (int j = 0; j < TO; j++) {
-        int cnt = CSA ? 2 * acc[i][j] + __popc(ones[i][j]) : acc[i][j];
-        if (TWOS) cnt += 2 * __popc(twos[i][j]);
+        const int cnt = CSA ? 2 * acc[i][j] + __popc(ones[i][j]) : acc[i][j];
         v[j] = g.Kbits - 2 * cnt;
       }
       const int o = o0 + wrow0;
@@ -391,8 +337,7 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
       float y[TO];
 #pragma unroll
       for (int j = 0; j < TO; j++) {
-        int cnt = CSA ? 2 * acc[i][j] + __popc(ones[i][j]) : acc[i][j];
-        if (TWOS) cnt += 2 * __popc(twos[i][j]);
+        const int cnt = CSA ? 2 * acc[i][j] + __popc(ones[i][j]) : acc[i][j];
         y[j] = __fmaf_rn((float)(g.Kbits - 2 * cnt), sc[j], sf[j]);
       }
       if (EPI == EPI_BIREAL) {
@@ -438,10 +383,10 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
   }
 }
 
-template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16, int STAGES, int L2MASK>
+template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16, int STAGES>
 __global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(const BConvArgs g) {
   extern __shared__ __align__(16) uint32_t bconv_smem[];
-  bconv_tile<BP, BO, TP, TO, EPI, CSA, VEC16, STAGES, true, L2MASK>(g, blockIdx.x, blockIdx.y, bconv_smem);
+  bconv_tile<BP, BO, TP, TO, EPI, CSA, VEC16, STAGES, true>(g, blockIdx.x, blockIdx.y, bconv_smem);
 }
 
 }  // namespace
