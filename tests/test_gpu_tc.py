@@ -236,6 +236,45 @@ def test_a_wait_that_runs_out_sets_the_flag_and_leaves_the_device_usable(B, orac
         B.tc_wait_expiry_selftest(a, wt, (1, 1), (pad, pad), -1, wait_polls=1 << 20)  # limit beyond a few milliseconds: refused
 
 
+def tc_matrix_cases():
+    """Channel words 1..8 x filter sizes 1, 2, 3, 4, 5, 7 x strides 1, 2: every count of K blocks per tap through the
+    unrolled 3x3 issue path and the runtime tap loops of the other filters, at a size with several tiles and a ragged
+    channel tile."""
+    return [(2, 64 * cw, 11, 10, 70, k, k // 2, -1 if (cw + k) % 2 else 1, st)
+            for cw in range(1, 9) for k in (1, 2, 3, 4, 5, 7) for st in (1, 2)]
+
+
+def run_tc_matrix(B, o):
+    """Returns (cases run, cases the engine declines); asserts bit equality with Eq. 1 on the packed words for the rest."""
+    ran = declined = 0
+    for N, C, H, W, O, k, pad, pv, st in tc_matrix_cases():
+        if not B.tc_supported(O, C, k, k, (st, st)):
+            declined += 1
+            continue
+        rng = np.random.default_rng(1000 * C + 10 * k + st)
+        x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+        w = rng.standard_normal((O, C, k, k)).astype(np.float32)
+        a = B.pack(torch.from_numpy(x).cuda())
+        wt = B.TcWeights(B.pack_weights(torch.from_numpy(w).cuda()), C)
+        try:
+            got = B.tc_bconv2d(a, wt, (st, st), (pad, pad), pv, B.NHWC).cpu().numpy()
+        except B.DabnnError as e:  # (stride 2 beyond 256 channels: declined at launch)
+            assert "supported" in str(e), (C, k, st, str(e))
+            declined += 1
+            continue
+        want = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (st, st), (pad, pad), pv, o.NHWC)
+        assert np.array_equal(got, want), (C, k, st)
+        ran += 1
+    torch.cuda.synchronize()
+    assert B.last_device_flag() == 0
+    return ran, declined
+
+
+def test_tc_matrix_of_channel_words_filters_and_strides(B, oracle_mod):
+    ran, declined = run_tc_matrix(B, oracle_mod)
+    assert ran >= 60 and ran + declined == 96, (ran, declined)
+
+
 _FORCED_FORM_SCRIPT = r"""
 import sys, numpy as np, torch
 from paper_1908_05858_b200 import binding as B
@@ -255,6 +294,10 @@ for N, C, H, W, O, k, pad, pv, st in cases:
     assert np.array_equal(bits, o.bn_sign_pack(want, sc.cpu().numpy(), sh.cpu().numpy())), (N, C, H, W, O, k)
 torch.cuda.synchronize()
 assert B.tc_error_flag() == 0
+sys.path.insert(0, "tests")
+import test_gpu_tc
+ran, declined = test_gpu_tc.run_tc_matrix(B, o)
+assert ran >= 50, (ran, declined)
 print("forced form ok")
 """
 
