@@ -601,6 +601,23 @@ def extras(B, torch, dev, peaks, sm_count):
     del sweep
 
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    # the paper's NC1HWC2 activation layout (C2 = 128 bits; Section 2.1.2, last paragraph) beside channel-packed NHWC words on
+    # the 3x3 layer: pack and convolution each, same kernels, same integers
+    xs, ws = synth.conv_case(5, 256, 256, 28, 28, 256, 3, 3, salt=256)
+    xd = torch.from_numpy(xs).to(dev)
+    wpk = B.pack_weights(torch.from_numpy(ws).to(dev))
+    lay = {}
+    outs = {}
+    for name, pl in (("nhwc_words", B.PACKED_NHWC), ("nc1hwc2", B.PACKED_NC1HWC2)):
+        ap = B.pack_as(xd, pl)
+        o32 = torch.empty((256, 28, 28, 256), dtype=torch.int32, device=dev)
+        t_pack, _ = time_fn(torch, lambda: B.pack_as(xd, pl, out=ap), 10)
+        t_conv, _ = time_fn(torch, lambda: B.bconv2d_from(ap, pl, 256, wpk, (1, 1), (1, 1), -1, B.NHWC, out=o32), 10, flush)
+        lay[name] = {"pack_ms": t_pack, "conv_ms": t_conv, "conv_Tbit-ops/s": conv_bitops(256, 256, 28, 256, 3) / t_conv / 1e9}
+        outs[name] = o32
+    lay["identical"] = bool((outs["nhwc_words"] == outs["nc1hwc2"]).all())
+    out["layout_nc1hwc2_vs_nhwc_words_256x256x28x28"] = lay
+    del xd, wpk, outs, ap, o32
     # BGEMM against direct convolution, the comparison of the paper's Fig. 4, on the 3x3 layer: the im2col matrix of the packed
     # activations (padding taps hold the pad word) is materialised with torch slicing (plumbing, 58 MB of packed rows) and
     # multiplied by dabnn_bgemm; dabnn_bconv2d gathers the same rows on the fly (implicit BGEMM)

@@ -76,6 +76,21 @@ dabnn_status dabnn_pack(const float* x, dabnn_layout in_layout, dabnn_shape s, u
  * errors as dabnn_pack; x must be 4-byte aligned (16-byte aligned input takes the vector path). */
 dabnn_status dabnn_pack_i32(const int32_t* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed, void* stream);
 
+/* Section 2.1.2, last paragraph / Fig. 3 -- the paper's NC1HWC2 activation layout, for comparison with the channel-packed
+ * NHWC words above.  C2 = 128 bits (the paper's vector register): uint64 [N][C1][H][W][2] with C1 = ceil(C/128); channel c
+ * lives in group c>>7, word (c>>6)&1, bit c&63; a last group of 64 channels or fewer has a zero second word.
+ *   dabnn_packed_words   64-bit words of a packed tensor in either layout (0 for an invalid shape or layout)
+ *   dabnn_pack_as        dabnn_pack into the chosen layout (packed: 16-byte aligned for NC1HWC2)
+ *   dabnn_bconv2d_from   dabnn_bconv2d reading activations in the chosen layout (weights stay [O][kh][kw][Cw]); the
+ *                        integers are the same whichever layout the activations are in. */
+typedef enum { DABNN_PACKED_NHWC = 0, DABNN_PACKED_NC1HWC2 = 1 } dabnn_packed_layout;
+size_t dabnn_packed_words(dabnn_shape s, dabnn_packed_layout packed_layout);
+dabnn_status dabnn_pack_as(const float* x, dabnn_layout in_layout, dabnn_shape s, dabnn_packed_layout packed_layout,
+                           uint64_t* packed, void* stream);
+dabnn_status dabnn_bconv2d_from(const uint64_t* a_packed, dabnn_packed_layout a_layout, dabnn_shape in,
+                                const uint64_t* w_packed, int O, dabnn_conv cv, int32_t* out, dabnn_layout out_layout,
+                                void* stream);
+
 /* Section 3 (weights are binarized and packed once, 32x smaller).
  * w_oihw: fp32 [O][C][kh][kw].  wpacked: uint64 [O][kh][kw][Cw], fully overwritten. */
 dabnn_status dabnn_pack_weights(const float* w_oihw, int O, int C, int kh, int kw, uint64_t* wpacked, void* stream);

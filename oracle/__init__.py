@@ -94,6 +94,33 @@ def pack(x: np.ndarray, layout: int = NCHW) -> np.ndarray:
     return P
 
 
+def pack_c2(x: np.ndarray, layout: int = NCHW) -> np.ndarray:
+    """Binarize and pack into the NC1HWC2 layout (Section 2.1.2, last paragraph): uint64 [N][ceil(C/128)][H][W][2]."""
+    x = _f32(x)
+    if layout == NCHW:
+        N, C, H, W = x.shape
+    else:
+        N, H, W, C = x.shape
+    P = np.empty((N, (C + 127) // 128, H, W, 2), dtype=np.uint64)
+    lib().oracle_pack_c2(_p(x), ctypes.c_int(layout), N, C, H, W, _p(P))
+    return P
+
+
+def bconv_bits_c2(A: np.ndarray, C: int, Wp: np.ndarray, stride=(1, 1), pad=(0, 0), pad_value=-1,
+                  out_layout=NHWC) -> np.ndarray:
+    """Eq. 1 with activations in the NC1HWC2 layout ([N][C1][H][W][2]); weights [O][kh][kw][Cw]."""
+    A = np.ascontiguousarray(A, dtype=np.uint64)
+    Wp = np.ascontiguousarray(Wp, dtype=np.uint64)
+    N, C1, H, W, two = A.shape
+    O, kh, kw, Cw = Wp.shape
+    assert two == 2 and C1 == (C + 127) // 128 and Cw == words_per_pixel(C)
+    OH, OW = out_dim(H, kh, stride[0], pad[0]), out_dim(W, kw, stride[1], pad[1])
+    out = np.empty(_out_shape(out_layout, N, O, OH, OW), dtype=np.int32)
+    lib().oracle_bconv_bits_c2(_p(A), N, C, H, W, _p(Wp), O, kh, kw, stride[0], stride[1], pad[0], pad[1],
+                               int(pad_value), _p(out), int(out_layout))
+    return out
+
+
 def pack_i32(x: np.ndarray, layout: int = NCHW) -> np.ndarray:
     """Pack the sign bits of int32 values (Section 2.1.1).  x: int32 NCHW or NHWC."""
     x = np.ascontiguousarray(x, dtype=np.int32)

@@ -8,6 +8,8 @@
  * the benchmark's CPU-baseline leg may load it.
  *
  * What each function follows:
+ *   oracle_pack_c2 / oracle_bconv_bits_c2   the same packer and Eq. 1 with the activations in the paper's NC1HWC2
+ *                                       layout (Section 2.1.2, last paragraph; Fig. 3), C2 = 128 bits.
  *   oracle_pack / oracle_pack_i32 / oracle_pack_weights
  *                                       Section 2.1.1 (bit-packing), the "naive" sequential
  *                                       packer the paper describes as the prior method:
@@ -111,6 +113,22 @@ void oracle_pack_i32(const int32_t* x, int layout, int N, int C, int H, int W, u
                                               : (((size_t)n * H + h) * W + w) * C + c;
           uint64_t bit = (x[xi] < 0) ? 1u : 0u;
           P[(((size_t)n * H + h) * W + w) * Cw + (size_t)(c >> 6)] |= bit << (c & 63);
+        }
+}
+
+/* Section 2.1.2, last paragraph (Fig. 3): the NC1HWC2 layout with C2 = 128 bits.  P is [N][C1][H][W][2] 64-bit words,
+   C1 = ceil(C/128); channel c sets bit c&63 of word (c>>6)&1 of group c>>7.  Same sequential packer. */
+void oracle_pack_c2(const float* x, int layout, int N, int C, int H, int W, uint64_t* P) {
+  size_t C1 = (size_t)((C + 127) / 128);
+  memset(P, 0, (size_t)N * C1 * H * W * 2 * sizeof(uint64_t));
+  for (int n = 0; n < N; n++)
+    for (int h = 0; h < H; h++)
+      for (int w = 0; w < W; w++)
+        for (int c = 0; c < C; c++) {
+          size_t xi = (layout == LAYOUT_NCHW) ? (((size_t)n * C + c) * H + h) * W + w
+                                              : (((size_t)n * H + h) * W + w) * C + c;
+          uint64_t bit = (binarize(x[xi]) == -1) ? 1u : 0u;
+          P[((((size_t)n * C1 + (size_t)(c >> 7)) * H + h) * W + w) * 2 + (size_t)((c >> 6) & 1)] |= bit << (c & 63);
         }
 }
 
@@ -228,6 +246,36 @@ void oracle_bconv_bits_at(const uint64_t* A, int N, int C, int H, int W, const u
   for (int64_t q = 0; q < ncoords; q++)
     vals[q] = bits_one(A, C, H, W, Wp, kh, kw, sh, sw, ph, pw, pad_value, coords[4 * q],
                        coords[4 * q + 1], coords[4 * q + 2], coords[4 * q + 3]);
+}
+
+/* Eq. 1 on activations in the NC1HWC2 layout (weights stay [O][kh][kw][Cw]): the same sum, words fetched from
+   [N][C1][H][W][2]. */
+void oracle_bconv_bits_c2(const uint64_t* A, int N, int C, int H, int W, const uint64_t* Wp, int O,
+                          int kh, int kw, int sh, int sw, int ph, int pw, int pad_value, int32_t* out,
+                          int out_layout) {
+  int OH = out_dim(H, kh, sh, ph), OW = out_dim(W, kw, sw, pw);
+  int Cw = (int)words_per_pixel(C), C1 = (C + 127) / 128, K = C * kh * kw;
+#pragma omp parallel for collapse(2) num_threads(g_threads) schedule(static)
+  for (int n = 0; n < N; n++)
+    for (int oh = 0; oh < OH; oh++)
+      for (int ow = 0; ow < OW; ow++)
+        for (int o = 0; o < O; o++) {
+          int agree = 0;
+          for (int i = 0; i < kh; i++)
+            for (int j = 0; j < kw; j++)
+              for (int cw = 0; cw < Cw; cw++) {
+                int ih = oh * sh + i - ph, iw = ow * sw + j - pw;
+                uint64_t a = (ih < 0 || ih >= H || iw < 0 || iw >= W)
+                                 ? pad_word(C, cw, pad_value)
+                                 : A[((((size_t)n * C1 + (size_t)(cw >> 1)) * H + ih) * W + iw) * 2 + (size_t)(cw & 1)];
+                uint64_t b = Wp[(((size_t)o * kh + i) * kw + j) * Cw + cw];
+                int valid = C - 64 * cw;
+                if (valid > 64) valid = 64;
+                uint64_t mask = (valid == 64) ? ~(uint64_t)0 : ((((uint64_t)1) << valid) - 1);
+                agree += popcount64(~(a ^ b) & mask);
+              }
+          out[out_index(out_layout, n, o, oh, ow, O, OH, OW)] = (int32_t)(2 * agree - K);
+        }
 }
 
 /* ---- BGEMM exactly as Eq. 1 prints it: C_ij = sum_k bitcount(xnor(A_ik, B_kj)) ------------------------

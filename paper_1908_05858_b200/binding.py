@@ -28,8 +28,11 @@ EXPORTS = (
     "dabnn_binary_layer_host_workspace_bytes", "dabnn_binary_layer_host", "dabnn_bireal18_forward_static", "dabnn_set_conv_tile",
     "dabnn_tc_set_max_ctas", "dabnn_tc_weights_bytes", "dabnn_tc_prepare_weights", "dabnn_tc_bconv2d", "dabnn_tc_bconv2d_bn_sign_pack",
     "dabnn_tc_bconv2d_bn_add_sign_pack", "dabnn_tc_error_flag", "dabnn_last_device_flag", "dabnn_stream_status",
-    "dabnn_tc_wait_expiry_selftest",
+    "dabnn_tc_wait_expiry_selftest", "dabnn_packed_words", "dabnn_pack_as", "dabnn_bconv2d_from",
 )
+
+PACKED_NHWC = 0
+PACKED_NC1HWC2 = 1
 
 ERR_TIMEOUT = 7
 ERR_STATIC_LIMIT = 8
@@ -108,6 +111,12 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).restype = ci
         L.dabnn_set_conv_tile.restype = ci
         L.dabnn_set_conv_tile.argtypes = [ci]
+        L.dabnn_packed_words.restype = ctypes.c_size_t
+        L.dabnn_packed_words.argtypes = [Shape, ci]
+        L.dabnn_pack_as.restype = ci
+        L.dabnn_pack_as.argtypes = [vp, ci, Shape, ci, vp, vp]
+        L.dabnn_bconv2d_from.restype = ci
+        L.dabnn_bconv2d_from.argtypes = [vp, ci, Shape, vp, ci, Conv, vp, ci, vp]
         L.dabnn_last_device_flag.restype = ci
         L.dabnn_last_device_flag.argtypes = [vp]
         L.dabnn_stream_status.restype = ci
@@ -179,6 +188,44 @@ def pack(x: torch.Tensor, layout: int = NCHW, out: Optional[torch.Tensor] = None
     if out is None:
         out = _alloc((N, H, W, words_per_pixel(C)), torch.int64, x.device)
     _check(lib().dabnn_pack(x.data_ptr(), layout, Shape(N, C, H, W), out.data_ptr(), _stream()))
+    return out
+
+
+def pack_as(x: torch.Tensor, packed_layout: int, layout: int = NCHW, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_pack_as: PACKED_NHWC gives int64 [N][H][W][Cw]; PACKED_NC1HWC2 gives int64 [N][C1][H][W][2] (Section 2.1.2)."""
+    x = _dev(x, torch.float32, "x")
+    N, C, H, W = x.shape if layout == NCHW else (x.shape[0], x.shape[3], x.shape[1], x.shape[2])
+    if out is None:
+        shape = (N, (C + 127) // 128, H, W, 2) if packed_layout == PACKED_NC1HWC2 else (N, H, W, words_per_pixel(C))
+        out = _alloc(shape, torch.int64, x.device)
+    if out.numel() != int(lib().dabnn_packed_words(Shape(N, C, H, W), packed_layout)):
+        raise DabnnError("packed tensor has the wrong size for this layout")
+    _check(lib().dabnn_pack_as(x.data_ptr(), layout, Shape(N, C, H, W), packed_layout, out.data_ptr(), _stream()))
+    return out
+
+
+def bconv2d_from(a_packed, packed_layout: int, C: int, w_packed, stride=(1, 1), pad=(0, 0), pad_value: int = -1,
+                 out_layout: int = NHWC, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_bconv2d_from: dabnn_bconv2d on activations in either packed layout."""
+    a = _dev(a_packed, torch.int64, "a_packed")
+    w = _dev(w_packed, torch.int64, "w_packed")
+    if packed_layout == PACKED_NC1HWC2:
+        N, C1, H, W, two = a.shape
+        if two != 2 or C1 != (C + 127) // 128:
+            raise DabnnError("NC1HWC2 activations must be [N][ceil(C/128)][H][W][2]")
+    else:
+        N, H, W, Cw = a.shape
+        if Cw != (C + 63) // 64:
+            raise DabnnError("packed word counts do not match C")
+    O, kh, kw, Cw2 = w.shape
+    if Cw2 != (C + 63) // 64:
+        raise DabnnError("packed word counts do not match C")
+    OH, OW = out_dim(H, kh, stride[0], pad[0]), out_dim(W, kw, stride[1], pad[1])
+    if out is None:
+        shape = (N, max(OH, 0), max(OW, 0), O) if out_layout == NHWC else (N, O, max(OH, 0), max(OW, 0))
+        out = _alloc(shape, torch.int32, a.device)
+    _check(lib().dabnn_bconv2d_from(a.data_ptr(), packed_layout, Shape(N, C, H, W), w.data_ptr(), O,
+                                    _conv(kh, kw, stride, pad, pad_value), out.data_ptr(), out_layout, _stream()))
     return out
 
 

@@ -90,7 +90,9 @@ dabnn_status launch_epi(const BConvArgs& g, cudaStream_t st) {
   }
 }
 
-dabnn_status fill_args(BConvArgs& g, const uint64_t* a, dabnn_shape in, const uint64_t* w, int O, dabnn_conv cv) {
+dabnn_status fill_args(BConvArgs& g, const uint64_t* a, dabnn_shape in, const uint64_t* w, int O, dabnn_conv cv,
+                       dabnn_packed_layout pl = DABNN_PACKED_NHWC) {
+  if (pl != DABNN_PACKED_NHWC && pl != DABNN_PACKED_NC1HWC2) return DABNN_ERR_SHAPE;
   if (!a || !w) return DABNN_ERR_NULL;
   if (in.N <= 0 || in.C <= 0 || in.H <= 0 || in.W <= 0 || O <= 0) return DABNN_ERR_SHAPE;
   if (cv.kh <= 0 || cv.kw <= 0 || cv.stride_h <= 0 || cv.stride_w <= 0 || cv.pad_h < 0 || cv.pad_w < 0)
@@ -113,6 +115,14 @@ dabnn_status fill_args(BConvArgs& g, const uint64_t* a, dabnn_shape in, const ui
   g.tail_mask = (in.C % 64 == 0) ? ~0ull : ((1ull << (in.C % 64)) - 1);
   g.out = nullptr; g.out_nchw = 0; g.scale = g.shift = g.residual = nullptr; g.y_out = nullptr;
   g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64); g.one = 1;
+  if (pl == DABNN_PACKED_NC1HWC2) {
+    const long long C1 = (in.C + 127) / 128;
+    if ((long long)in.H * in.W * C1 * 2 > 0x7FFFFFFF) return DABNN_ERR_UNSUPPORTED;
+    g.img_stride = C1 * in.H * in.W * 2; g.pix_stride = 2; g.pair_stride = 2 * in.H * in.W;
+    if (!aligned(a, 16)) return DABNN_ERR_ALIGNMENT;  // 128-bit vectors
+  } else {
+    g.img_stride = (long long)in.H * in.W * Cw; g.pix_stride = (int)Cw; g.pair_stride = 2;
+  }
   g.magic_cw = Cw == 1 ? 0ull : ~0ull / (unsigned long long)Cw + 1ull;
   g.magic_kw = cv.kw == 1 ? 0ull : ~0ull / (unsigned long long)cv.kw + 1ull;
   return DABNN_OK;
@@ -179,6 +189,20 @@ extern "C" dabnn_status dabnn_bconv2d(const uint64_t* a_packed, dabnn_shape in, 
                                       dabnn_conv cv, int32_t* out, dabnn_layout out_layout, void* stream) {
   BConvArgs g;
   dabnn_status s = fill_args(g, a_packed, in, w_packed, O, cv);
+  if (s != DABNN_OK) return s;
+  if (!out) return DABNN_ERR_NULL;
+  if (out_layout != DABNN_NCHW && out_layout != DABNN_NHWC) return DABNN_ERR_SHAPE;
+  if (!aligned(out, 4)) return DABNN_ERR_ALIGNMENT;
+  g.out = out;
+  g.out_nchw = out_layout == DABNN_NCHW;
+  return launch_epi<EPI_I32>(g, as_stream(stream));
+}
+
+extern "C" dabnn_status dabnn_bconv2d_from(const uint64_t* a_packed, dabnn_packed_layout a_layout, dabnn_shape in,
+                                           const uint64_t* w_packed, int O, dabnn_conv cv, int32_t* out,
+                                           dabnn_layout out_layout, void* stream) {
+  BConvArgs g;
+  dabnn_status s = fill_args(g, a_packed, in, w_packed, O, cv, a_layout);
   if (s != DABNN_OK) return s;
   if (!out) return DABNN_ERR_NULL;
   if (out_layout != DABNN_NCHW && out_layout != DABNN_NHWC) return DABNN_ERR_SHAPE;

@@ -34,6 +34,11 @@ struct BConvArgs {
   int Ow32;                // 2*ceil(O/64)
   int one;                 // the constant 1 (see bit_mac)
   unsigned long long magic_cw, magic_kw;  // ceil(2^64 / Cw), ceil(2^64 / kw) (0 when the divisor is 1): see fast_div
+  // Where word cw of pixel (ih, iw) of image n lives, in 64-bit words:  n * img_stride + (ih * W + iw) * pix_stride +
+  // (cw >> 1) * pair_stride + (cw & 1).  Channel-packed NHWC [N][H][W][Cw]: pix_stride = Cw, pair_stride = 2.
+  // NC1HWC2 with 128-bit vectors [N][C1][H][W][2] (Section 2.1.2, last paragraph): pix_stride = 2, pair_stride = 2*H*W.
+  long long img_stride;
+  int pix_stride, pair_stride;
 };
 
 struct RowInfo {
@@ -114,7 +119,7 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
       const long long t = m / g.OW;
       const int oh = (int)(t % g.OH);
       const long long n = t / g.OH;
-      ri.base = n * g.H * g.W * g.Cw;
+      ri.base = n * g.img_stride;
       ri.ih0 = oh * g.sh - g.ph;
       ri.iw0 = ow * g.sw - g.pw;
     } else {
@@ -159,7 +164,8 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
         else *reinterpret_cast<uint64_t*>(dst) = p0;
       } else {
         // (the offset inside one image fits 32 bits: checked on the host)
-        const uint64_t* src = live ? g.a + (ri.base + (long long)((ih * g.W + iw) * g.Cw + cw)) : g.a;
+        const uint64_t* src =
+            live ? g.a + (ri.base + (long long)((ih * g.W + iw) * g.pix_stride + (cw >> 1) * g.pair_stride + (cw & 1))) : g.a;
         if (UW == 2) cp_async16(smem_u32(dst), src, live ? 16 : 0);
         else cp_async8(smem_u32(dst), src, live ? 8 : 0);
       }

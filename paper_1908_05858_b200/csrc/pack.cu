@@ -38,7 +38,9 @@ __device__ __forceinline__ unsigned neg(int32_t v) { return (unsigned)(v < 0); }
 // channels.  Each lane owns 4 consecutive pixels (one float4 per channel); the four warps split every word's 64
 // channels into quarters of 16, so a thread has 16 independent 16-byte loads in flight per word, and the 16-bit
 // quarters are placed side by side in shared memory, which assembles the 64-bit words without any exchange.
-template <typename T>
+// C2: the words leave in the NC1HWC2 layout instead ([N][C1][H][W][2]: 128-bit vectors of one channel group, pixel after
+// pixel; an odd last word gets a zero partner).
+template <typename T, bool C2>
 __global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const T* __restrict__ x, int C, int HW, int Cw,
                                                                uint64_t* __restrict__ packed) {
   extern __shared__ __align__(16) uint64_t s_words[];  // [128][Cw]
@@ -87,6 +89,16 @@ __global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const T* __restri
   // contiguous in global memory: pixels pix0 .. pix0+npix-1, all words
   const int npix = min(128, HW - pix0);
   if (npix <= 0) return;
+  if (C2) {
+    const int C1 = (Cw + 1) / 2;
+    ulonglong2* d2 = reinterpret_cast<ulonglong2*>(packed);  // 16-byte aligned: checked on the host
+    for (int i = threadIdx.x; i < C1 * npix; i += kPackThreads) {
+      const int grp = i / npix, px = i - grp * npix;  // consecutive threads: consecutive pixels of one channel group
+      const uint64_t lo = s_words[px * Cw + 2 * grp], hi = (2 * grp + 1 < Cw) ? s_words[px * Cw + 2 * grp + 1] : 0ull;
+      d2[((size_t)n * C1 + grp) * HW + pix0 + px] = make_ulonglong2(lo, hi);
+    }
+    return;
+  }
   uint64_t* dst = packed + ((size_t)n * HW + pix0) * Cw;
   const int total = npix * Cw;
   if ((((size_t)n * HW + pix0) * Cw) % 2 == 0 && (reinterpret_cast<uintptr_t>(packed) & 15) == 0) {
@@ -131,10 +143,11 @@ __global__ void __launch_bounds__(256) pack_nchw_tile(const T* __restrict__ x, i
   }
 }
 
-// Any layout, any shape: one thread per output word.
+// Any layout, any shape: one thread per output word (c2: the word goes to its place in the NC1HWC2 layout, and the
+// thread of an odd last word also writes the zero partner).
 template <typename T>
 __global__ void pack_generic(const T* __restrict__ x, int nhwc, int C, int HW, int Cw, long long total_words,
-                             uint64_t* __restrict__ packed) {
+                             uint64_t* __restrict__ packed, int c2) {
   long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= total_words) return;
   const int cw = (int)(t % Cw);
@@ -149,7 +162,15 @@ __global__ void pack_generic(const T* __restrict__ x, int nhwc, int C, int HW, i
     const T* src = x + ((size_t)n * C + c0) * HW + hw;
     for (int c = 0; c < cn; c++) w |= (uint64_t)neg(src[(size_t)c * HW]) << c;
   }
-  packed[t] = w;
+  if (c2) {
+    const long long n = pix / HW, hw = pix % HW;
+    const int C1 = (Cw + 1) / 2;
+    uint64_t* v = packed + (((size_t)n * C1 + (cw >> 1)) * HW + hw) * 2;
+    v[cw & 1] = w;
+    if (cw == Cw - 1 && (cw & 1) == 0) v[1] = 0;
+  } else {
+    packed[t] = w;
+  }
 }
 
 // NHWC with C a multiple of 64 and 16-byte aligned input: 16 lanes share one word; each lane tests 4
@@ -204,11 +225,14 @@ __global__ void pack_weights_kernel(const float* __restrict__ w, int O, int C, i
 using namespace dabnn;
 
 template <typename T>
-dabnn_status pack_any(const T* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed, void* stream) {
+dabnn_status pack_any(const T* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed, void* stream,
+                      dabnn_packed_layout pl = DABNN_PACKED_NHWC) {
   if (!x || !packed) return DABNN_ERR_NULL;
   if (s.N <= 0 || s.C <= 0 || s.H <= 0 || s.W <= 0) return DABNN_ERR_SHAPE;
   if (in_layout != DABNN_NCHW && in_layout != DABNN_NHWC) return DABNN_ERR_SHAPE;
-  if (!aligned(x, 4) || !aligned(packed, 8)) return DABNN_ERR_ALIGNMENT;
+  if (pl != DABNN_PACKED_NHWC && pl != DABNN_PACKED_NC1HWC2) return DABNN_ERR_SHAPE;
+  const bool c2 = pl == DABNN_PACKED_NC1HWC2;
+  if (!aligned(x, 4) || !aligned(packed, c2 ? 16 : 8)) return DABNN_ERR_ALIGNMENT;
   const long long HW = (long long)s.H * s.W;
   const long long Cw = (s.C + 63) / 64;
   if (HW > 0x7FFFFFFF || (long long)s.N * HW > 0x7FFFFFFFFFFLL) return DABNN_ERR_UNSUPPORTED;
@@ -216,11 +240,12 @@ dabnn_status pack_any(const T* x, dabnn_layout in_layout, dabnn_shape s, uint64_
   cudaStream_t st = as_stream(stream);
   if (in_layout == DABNN_NCHW && HW % 4 == 0 && aligned(x, 16) && s.N <= 65535 && Cw * 128 * 8 <= 48 * 1024) {
     dim3 grid(ceil_div(HW, 128), s.N);
-    pack_nchw_vec4<T><<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, packed);
-  } else if (in_layout == DABNN_NCHW && s.N <= 65535 && Cw <= 65535) {
+    if (c2) pack_nchw_vec4<T, true><<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, packed);
+    else pack_nchw_vec4<T, false><<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, packed);
+  } else if (!c2 && in_layout == DABNN_NCHW && s.N <= 65535 && Cw <= 65535) {
     dim3 grid(ceil_div(HW, 128), s.N, (unsigned)Cw);
     pack_nchw_tile<T><<<grid, 256, 0, st>>>(x, s.C, (int)HW, (int)Cw, packed);
-  } else if (in_layout == DABNN_NHWC && s.C % 64 == 0 && aligned(x, 16)) {
+  } else if (!c2 && in_layout == DABNN_NHWC && s.C % 64 == 0 && aligned(x, 16)) {
     const long long warps_needed = (total_words + 7) / 8;
     long long blocks = (warps_needed + 7) / 8;
     const long long cap = (long long)sm_count() * 16;
@@ -230,7 +255,7 @@ dabnn_status pack_any(const T* x, dabnn_layout in_layout, dabnn_shape s, uint64_
     const long long blocks = (total_words + 255) / 256;
     if (blocks > 0x7FFFFFFF) return DABNN_ERR_UNSUPPORTED;
     pack_generic<T><<<(unsigned)blocks, 256, 0, st>>>(x, in_layout == DABNN_NHWC, s.C, (int)HW, (int)Cw, total_words,
-                                                   packed);
+                                                   packed, c2 ? 1 : 0);
   }
   return launch_status();
 }
@@ -238,6 +263,18 @@ dabnn_status pack_any(const T* x, dabnn_layout in_layout, dabnn_shape s, uint64_
 extern "C" dabnn_status dabnn_pack(const float* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed,
                                    void* stream) {
   return pack_any<float>(x, in_layout, s, packed, stream);
+}
+
+extern "C" dabnn_status dabnn_pack_as(const float* x, dabnn_layout in_layout, dabnn_shape s, dabnn_packed_layout packed_layout,
+                                      uint64_t* packed, void* stream) {
+  return pack_any<float>(x, in_layout, s, packed, stream, packed_layout);
+}
+
+extern "C" size_t dabnn_packed_words(dabnn_shape s, dabnn_packed_layout packed_layout) {
+  if (s.N <= 0 || s.C <= 0 || s.H <= 0 || s.W <= 0) return 0;
+  const size_t pix = (size_t)s.N * s.H * s.W;
+  if (packed_layout == DABNN_PACKED_NC1HWC2) return pix * 2 * (size_t)((s.C + 127) / 128);
+  return packed_layout == DABNN_PACKED_NHWC ? pix * (size_t)((s.C + 63) / 64) : 0;
 }
 
 extern "C" dabnn_status dabnn_pack_i32(const int32_t* x, dabnn_layout in_layout, dabnn_shape s, uint64_t* packed,

@@ -194,6 +194,44 @@ def test_bireal_block_epilogue_matches_oracle(B, oracle_mod, case):
     assert np.array_equal(u64(got_bits), want_bits)
 
 
+# ---- the paper's NC1HWC2 activation layout (Section 2.1.2, last paragraph) ---------------------------------------------
+@pytest.mark.parametrize("shape", [(2, 256, 28, 28), (3, 64, 7, 5), (2, 130, 9, 8), (1, 300, 12, 12), (2, 128, 6, 7), (1, 2100, 3, 3)])
+def test_pack_nc1hwc2(B, oracle_mod, shape):
+    rng = np.random.default_rng(sum(shape) + 4)
+    x = rng.standard_normal(shape).astype(np.float32)
+    x[rng.random(shape) < 0.01] = 0.0
+    got = u64(B.pack_as(dev(x), B.PACKED_NC1HWC2))
+    assert np.array_equal(got, oracle_mod.pack_c2(x))
+    xt = np.ascontiguousarray(x.transpose(0, 2, 3, 1))
+    assert np.array_equal(u64(B.pack_as(dev(xt), B.PACKED_NC1HWC2, B.NHWC)), oracle_mod.pack_c2(x))
+    assert np.array_equal(u64(B.pack_as(dev(x), B.PACKED_NHWC)), oracle_mod.pack(x))
+
+
+@pytest.mark.parametrize("case", [CONV_CASES[0], CONV_CASES[1], CONV_CASES[3], CONV_CASES[4], CONV_CASES[8], CONV_CASES[9],
+                                  CONV_CASES[11], CONV_CASES[12], (2, 300, 10, 9, 40, 3, 3, (1, 1), (1, 1), +1)])
+def test_bconv2d_from_nc1hwc2_matches_oracle(B, oracle_mod, case):
+    N, C, H, W, O, kh, kw, stride, pad, pv = case
+    x, w = conv_inputs(case)
+    o = oracle_mod
+    want = o.bconv_bits_c2(o.pack_c2(x), C, o.pack_weights(w), stride, pad, pv, o.NHWC)
+    a2, wp = B.pack_as(dev(x), B.PACKED_NC1HWC2), B.pack_weights(dev(w))
+    got = B.bconv2d_from(a2, B.PACKED_NC1HWC2, C, wp, stride, pad, pv, B.NHWC).cpu().numpy()
+    assert np.array_equal(got, want)
+    assert np.array_equal(B.bconv2d_from(a2, B.PACKED_NC1HWC2, C, wp, stride, pad, pv, B.NCHW).cpu().numpy(), want.transpose(0, 3, 1, 2))
+    # the same integers from the channel-packed NHWC words
+    assert np.array_equal(B.bconv2d_from(B.pack(dev(x)), B.PACKED_NHWC, C, wp, stride, pad, pv, B.NHWC).cpu().numpy(), want)
+
+
+def test_nc1hwc2_full_size_3x3_layer(B, oracle_mod):
+    """The large-batch 3x3 layer (batch 256, 256 channels, 28x28) from NC1HWC2 activations: the whole tensor against Eq. 1."""
+    x, w = synth.conv_case(5, 256, 256, 28, 28, 256, 3, 3, salt=256)
+    a2, wp = B.pack_as(dev(x), B.PACKED_NC1HWC2), B.pack_weights(dev(w))
+    assert np.array_equal(u64(a2), oracle_mod.pack_c2(x))
+    got = B.bconv2d_from(a2, B.PACKED_NC1HWC2, 256, wp, (1, 1), (1, 1), -1, B.NHWC).cpu().numpy()
+    want = oracle_mod.bconv_bits(oracle_mod.pack(x), 256, oracle_mod.pack_weights(w), (1, 1), (1, 1), -1, oracle_mod.NHWC)
+    assert np.array_equal(got, want)
+
+
 # ---- full-size configurations, sampled ---------------------------------------------------------------------
 def sample_coords(rng, N, O, OH, OW, n):
     c = np.stack([rng.integers(0, N, n), rng.integers(0, O, n), rng.integers(0, OH, n), rng.integers(0, OW, n)], axis=1)

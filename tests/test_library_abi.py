@@ -70,6 +70,11 @@ def test_argument_errors_are_reported_before_any_launch(L):
     assert L.dabnn_bn_fold(fake, fake, fake, fake, 1e-5, 0, fake, fake, None) == 2
     assert L.dabnn_bireal18_forward(None, fake, 1, fake, fake, 1 << 30, None) == 1
     assert L.dabnn_set_conv_variant(0) in (0, 1, 2)
+    assert L.dabnn_pack_as(fake, 0, s, 2, fake, None) == 2            # unknown packed layout
+    assert L.dabnn_pack_as(fake, 0, s, 1, ctypes.c_void_p(0x1008), None) == 4  # NC1HWC2 wants 16-byte aligned vectors
+    assert L.dabnn_bconv2d_from(fake, 3, s, fake, 8, cv, fake, 1, None) == 2
+    assert L.dabnn_packed_words(Shape(2, 130, 3, 4), 0) == 2 * 3 * 4 * 3 and L.dabnn_packed_words(Shape(2, 130, 3, 4), 1) == 2 * 3 * 4 * 4
+    assert L.dabnn_packed_words(Shape(2, 130, 3, 4), 5) == 0
     assert L.dabnn_tc_wait_expiry_selftest(fake, Shape(1, 64, 8, 8), fake, 64, cv, None, 100, None) == 1
     assert L.dabnn_tc_wait_expiry_selftest(fake, Shape(1, 64, 8, 8), fake, 64, cv, fake, 0, None) == 2
     assert b"wait" in L.dabnn_status_string(7) and b"built-in scratch" in L.dabnn_status_string(8)

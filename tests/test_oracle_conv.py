@@ -213,3 +213,20 @@ def test_bgemm_xnor_counts_against_brute_force_and_the_dot_product(oracle_mod):
     # the worked example, by hand: 0x46^0xD3 = 0x95 (4 differ, 4 agree); 0x46^0x87 = 0xC1 (3 differ, 5 agree);
     # 0x8F^0xD3 = 0x5C (4 differ, 4 agree); 0x8F^0x87 = 0x08 (1 differs, 7 agree)
     assert o.bgemm_xnor(np.array([[0x46], [0x8F]], dtype=np.uint64), np.array([[0xD3], [0x87]], dtype=np.uint64), 8).tolist() == [[4, 5], [4, 7]]
+
+
+@pytest.mark.parametrize("case", [(2, 64, 5, 6, 7, 3, 1, 1, -1), (1, 130, 6, 5, 9, 3, 2, 1, +1), (2, 256, 4, 4, 5, 1, 1, 0, -1),
+                                  (1, 300, 7, 6, 4, 5, 1, 2, -1)])
+def test_eq1_on_the_nc1hwc2_layout_equals_the_definition(oracle_mod, case):
+    """Eq. 1 reading activations from the NC1HWC2 layout (Section 2.1.2, last paragraph) gives the convolution of the
+    +-1 tensors as defined, for odd and even word counts, channel tails, both pad values and stride 2."""
+    o = oracle_mod
+    N, C, H, W, O, k, st, pad, pv = case
+    rng = np.random.default_rng(C + k)
+    x = rng.standard_normal((N, C, H, W)).astype(np.float32)
+    w = rng.standard_normal((O, C, k, k)).astype(np.float32)
+    want = o.bconv_pm1(x, w, (st, st), (pad, pad), pv, o.NHWC)
+    got = o.bconv_bits_c2(o.pack_c2(x), C, o.pack_weights(w), (st, st), (pad, pad), pv, o.NHWC)
+    assert np.array_equal(got, want)
+    assert np.array_equal(o.bconv_bits_c2(o.pack_c2(x), C, o.pack_weights(w), (st, st), (pad, pad), pv, o.NCHW),
+                          want.transpose(0, 3, 1, 2))

@@ -96,3 +96,36 @@ def test_pack_weights_layout(oracle_mod):
     bits, tail = unpack_words(Wp, 70)
     assert np.array_equal(bits, (np.transpose(w, (0, 2, 3, 1)) < 0).astype(np.uint8))
     assert not tail.any()
+
+
+def test_nc1hwc2_layout_places_every_channel_bit(oracle_mod):
+    """The NC1HWC2 layout (Section 2.1.2, last paragraph; C2 = 128 bits): channel c is bit c&63 of word (c>>6)&1 of the
+    128-bit vector of group c>>7, one vector per pixel and group.  Checked by unpacking every bit independently."""
+    o = oracle_mod
+    rng = np.random.default_rng(21)
+    for shape in ((2, 300, 3, 5), (1, 64, 4, 4), (3, 128, 2, 3), (1, 130, 1, 2)):
+        N, C, H, W = shape
+        x = rng.standard_normal(shape).astype(np.float32)
+        x.reshape(-1)[:4] = [0.0, -0.0, np.nan, -1e-45]
+        P = o.pack_c2(x, o.NCHW)
+        C1 = (C + 127) // 128
+        assert P.shape == (N, C1, H, W, 2) and P.dtype == np.uint64
+        bits = np.zeros((N, C1 * 128, H, W), dtype=np.uint8)
+        for g in range(C1):
+            for j in range(2):
+                for b in range(64):
+                    bits[:, 128 * g + 64 * j + b] = ((P[:, g, :, :, j] >> np.uint64(b)) & np.uint64(1)).astype(np.uint8)
+        assert np.array_equal(bits[:, :C], (x < 0).astype(np.uint8))
+        assert not bits[:, C:].any()  # tail bits, and the zero partner word of an odd last group
+        # the NHWC-input form packs the same bits
+        assert np.array_equal(o.pack_c2(np.ascontiguousarray(x.transpose(0, 2, 3, 1)), o.NHWC), P)
+        # and the two packed layouts hold the same words, rearranged
+        Q = o.pack(x, o.NCHW)  # [N][H][W][Cw]
+        for cw in range(Q.shape[-1]):
+            assert np.array_equal(P[:, cw >> 1, :, :, cw & 1], Q[..., cw])
+
+
+def test_nc1hwc2_hand_vector(oracle_mod):
+    x = -np.ones((1, 130, 1, 1), dtype=np.float32)
+    P = oracle_mod.pack_c2(x)
+    assert P.reshape(-1).tolist() == [2**64 - 1, 2**64 - 1, 3, 0]
