@@ -264,6 +264,9 @@ class _Bireal18Params(ctypes.Structure):
         ("fc_b", ctypes.c_void_p),
         ("bn_eps", ctypes.c_double),
         ("conv_form", ctypes.c_int),
+        ("use_stem_module", ctypes.c_int),
+        ("sm_w", ctypes.c_void_p * 4),
+        ("sm_bn", (ctypes.c_void_p * 4) * 4),
     ]
 
 
@@ -271,14 +274,16 @@ STAGE_C = (64, 128, 256, 512)
 STAGE_HW = (56, 28, 14, 7)
 
 
-def bireal18_forward(params: dict, images: np.ndarray, conv_form: int = 1, want_taps: bool = False):
+def bireal18_forward(params: dict, images: np.ndarray, conv_form: int = 1, want_taps: bool = False,
+                     stem_module: bool = False):
     """Bi-Real Net 18 forward (Section 2.3).
 
     ``params`` holds fp32 numpy arrays: ``stem_w`` [64,3,7,7]; ``stem_bn`` = (gamma, beta,
     mean, var); ``block_w[b]`` [O,C,3,3]; ``block_bn[b]``; ``down_w[d]`` [O,C];
     ``down_bn[d]``; ``fc_w`` [1000,512]; ``fc_b`` [1000].  ``conv_form`` 0 uses the +-1
     products, 1 uses Eq. 1 on packed words (identical integers).  Returns logits [N,1000]
-    (and, if asked, the 17 intermediate activations as fp32 NCHW arrays).
+    (and, if asked, the 17 intermediate activations as fp32 NCHW arrays).  ``stem_module``: the STEM module of
+    Section 2.3 (a reading of the missing Fig. 6, see oracle.c) in place of the 7x7 convolution and the max-pool.
     """
     keep = []
 
@@ -303,6 +308,12 @@ def bireal18_forward(params: dict, images: np.ndarray, conv_form: int = 1, want_
     P.fc_b = ptr(params["fc_b"])
     P.bn_eps = float(params.get("bn_eps", 1e-5))
     P.conv_form = int(conv_form)
+    P.use_stem_module = 1 if stem_module else 0
+    if stem_module:  # params["stem_module"] = {"w": [4 arrays OIHW], "bn": [4 x (gamma, beta, mean, var)]} (Section 2.3)
+        for i in range(4):
+            P.sm_w[i] = ptr(params["stem_module"]["w"][i])
+            for j in range(4):
+                P.sm_bn[i][j] = ptr(params["stem_module"]["bn"][i][j])
     images = _f32(images)
     N = images.shape[0]
     assert images.shape[1:] == (3, 224, 224)

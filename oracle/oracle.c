@@ -39,7 +39,9 @@
  *     stated order (see oracle_bireal18_forward), so the result is single-valued.
  *
  * Parity of oracle_bireal18_forward's TOPOLOGY is unpinned by the paper (it only names
- * the network); its arithmetic is pinned by the tests against fp64 library routines.
+ * the network); its arithmetic is pinned by the tests against fp64 library routines.  The same holds
+ * for the STEM module variant (Section 2.3): its figure is missing from the paper's text, so the
+ * module's structure is a reading (see stem_module): PARITY UNPINNED by the paper.
  *
  * Build: gcc -O2 -mfma -mpopcnt -ffp-contract=off -fopenmp -shared -fPIC oracle.c -lm
  * (-ffp-contract=off: the only fused multiply-adds are the explicit fmaf calls.)
@@ -351,7 +353,73 @@ typedef struct {
   const float* fc_b;                         /* [1000] */
   double bn_eps;
   int conv_form;                             /* 0: +-1 products (definition), 1: Eq. 1 on packed words */
+  int use_stem_module;                       /* 0: 7x7 stem conv + max-pool; 1: the STEM module below (Section 2.3, Fig. 6) */
+  const float* sm_w[4];                      /* [32][3][3][3], [16][32][1][1], [32][16][3][3], [64][64][1][1] */
+  const float* sm_bn[4][4];                  /* gamma, beta, mean, var of the BN after each of the four convolutions */
 } oracle_bireal18_params;
+
+/* One fp32 convolution of the STEM module, NCHW, zero padding, no bias, in the pinned order (c, kh, kw ascending, taps
+   outside the image skipped), then y = fmaf(acc, scale, shift) and, if relu, y = (y > 0) ? y : +0. */
+static void conv_bn_fp32(const float* x, int N, int C, int H, int W, const float* w, int O, int k, int stride, int pad,
+                         const float* scale, const float* shift, int relu, float* y) {
+  int OH = out_dim(H, k, stride, pad), OW = out_dim(W, k, stride, pad);
+#pragma omp parallel for collapse(2) num_threads(g_threads) schedule(static)
+  for (int n = 0; n < N; n++)
+    for (int o = 0; o < O; o++)
+      for (int oh = 0; oh < OH; oh++)
+        for (int ow = 0; ow < OW; ow++) {
+          float a = 0.0f;
+          for (int c = 0; c < C; c++)
+            for (int i = 0; i < k; i++)
+              for (int j = 0; j < k; j++) {
+                int ih = oh * stride + i - pad, iw = ow * stride + j - pad;
+                if (ih < 0 || ih >= H || iw < 0 || iw >= W) continue;
+                a = fmaf(x[(((size_t)n * C + c) * H + ih) * W + iw], w[(((size_t)o * C + c) * k + i) * k + j], a);
+              }
+          float v = fmaf(a, scale[o], shift[o]);
+          if (relu) v = (v > 0.0f) ? v : 0.0f;
+          y[(((size_t)n * O + o) * OH + oh) * OW + ow] = v;
+        }
+}
+
+/* The STEM module that replaces the 7x7 convolution and the max-pool (Section 2.3, Fig. 6; the figure is not in the
+   paper's text, so this is a READING, after the stem block of PeleeNet that the paper cites: PARITY UNPINNED BY THE PAPER):
+     s1  = relu(BN(conv3x3/2, pad 1, 3 -> 32))(image)            224 -> 112
+     a   = relu(BN(conv1x1, 32 -> 16))(s1)
+     a   = relu(BN(conv3x3/2, pad 1, 16 -> 32))(a)               112 -> 56
+     b   = maxpool2x2/2(s1)                                      112 -> 56
+     out = BN(conv1x1, 64 -> 64)(concat(a, b))                   no activation: the binary blocks take its sign
+   out is fp32 NCHW [N][64][56][56]. */
+static void stem_module(const oracle_bireal18_params* p, const float* images, int N, float* out) {
+  float scale[64], shift[64];
+  float* s1 = (float*)malloc((size_t)N * 32 * 112 * 112 * sizeof(float));
+  float* a1 = (float*)malloc((size_t)N * 16 * 112 * 112 * sizeof(float));
+  float* cat = (float*)malloc((size_t)N * 64 * 56 * 56 * sizeof(float));
+  float* a2 = (float*)malloc((size_t)N * 32 * 56 * 56 * sizeof(float));
+  oracle_bn_fold(p->sm_bn[0][0], p->sm_bn[0][1], p->sm_bn[0][2], p->sm_bn[0][3], p->bn_eps, 32, scale, shift);
+  conv_bn_fp32(images, N, 3, 224, 224, p->sm_w[0], 32, 3, 2, 1, scale, shift, 1, s1);
+  oracle_bn_fold(p->sm_bn[1][0], p->sm_bn[1][1], p->sm_bn[1][2], p->sm_bn[1][3], p->bn_eps, 16, scale, shift);
+  conv_bn_fp32(s1, N, 32, 112, 112, p->sm_w[1], 16, 1, 1, 0, scale, shift, 1, a1);
+  oracle_bn_fold(p->sm_bn[2][0], p->sm_bn[2][1], p->sm_bn[2][2], p->sm_bn[2][3], p->bn_eps, 32, scale, shift);
+  conv_bn_fp32(a1, N, 16, 112, 112, p->sm_w[2], 32, 3, 2, 1, scale, shift, 1, a2);
+  for (int n = 0; n < N; n++) {
+    /* channels 0..31: the convolution branch; 32..63: the pooled branch */
+    memcpy(cat + (size_t)n * 64 * 56 * 56, a2 + (size_t)n * 32 * 56 * 56, (size_t)32 * 56 * 56 * sizeof(float));
+    for (int c = 0; c < 32; c++)
+      for (int oh = 0; oh < 56; oh++)
+        for (int ow = 0; ow < 56; ow++) {
+          const float* q = s1 + (((size_t)n * 32 + c) * 112 + 2 * oh) * 112 + 2 * ow;
+          float m = q[0];
+          if (q[1] > m) m = q[1];
+          if (q[112] > m) m = q[112];
+          if (q[113] > m) m = q[113];
+          cat[(((size_t)n * 64 + 32 + c) * 56 + oh) * 56 + ow] = m;
+        }
+  }
+  oracle_bn_fold(p->sm_bn[3][0], p->sm_bn[3][1], p->sm_bn[3][2], p->sm_bn[3][3], p->bn_eps, 64, scale, shift);
+  conv_bn_fp32(cat, N, 64, 56, 56, p->sm_w[3], 64, 1, 1, 0, scale, shift, 0, out);
+  free(s1); free(a1); free(cat); free(a2);
+}
 
 static const int kStageC[4] = {64, 128, 256, 512};
 static const int kStageHW[4] = {56, 28, 14, 7};
@@ -373,6 +441,10 @@ void oracle_bireal18_forward(const oracle_bireal18_params* p, const float* image
   uint64_t* pa = (uint64_t*)malloc((size_t)N * 56 * 56 * 8 * sizeof(uint64_t));
   uint64_t* pw = (uint64_t*)malloc((size_t)512 * 9 * 8 * sizeof(uint64_t));
 
+  if (p->use_stem_module) {
+    stem_module(p, images, N, cur);
+    goto blocks;
+  }
   /* 1. stem: conv 7x7, 3 -> 64, stride 2, zero pad 3, no bias; then BN */
   oracle_bn_fold(p->stem_bn[0], p->stem_bn[1], p->stem_bn[2], p->stem_bn[3], p->bn_eps, 64, scale, shift);
 #pragma omp parallel for collapse(2) num_threads(g_threads) schedule(static)
@@ -407,6 +479,7 @@ void oracle_bireal18_forward(const oracle_bireal18_params* p, const float* image
             }
           cur[(((size_t)n * 64 + c) * 56 + oh) * 56 + ow] = m;
         }
+blocks:
   if (taps && taps[0]) memcpy(taps[0], cur, (size_t)N * 64 * 56 * 56 * sizeof(float));
 
   /* 2. sixteen blocks: out = BN(bconv3x3(sign(x))) + shortcut(x) */

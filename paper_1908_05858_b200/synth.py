@@ -79,6 +79,15 @@ def bireal18_params(config_id: int = 4) -> dict:
     return p
 
 
+def stem_module_params(config_id: int = 4) -> dict:
+    """Random-init parameters of the STEM module (Section 2.3): four fp32 convolutions (OIHW, N(0,1)/sqrt(fan_in)) with a
+    BN each: 3x3/2 3->32, 1x1 32->16, 3x3/2 16->32, 1x1 64->64."""
+    g = rng(config_id, 2)
+    shapes = ((32, 3, 3, 3), (16, 32, 1, 1), (32, 16, 3, 3), (64, 64, 1, 1))
+    w = [(g.standard_normal(size=sh) / np.sqrt(float(sh[1] * sh[2] * sh[3]))).astype(np.float32) for sh in shapes]
+    return {"w": w, "bn": [bn_params(g, sh[0]) for sh in shapes]}
+
+
 def bireal18_images(N: int, config_id: int = 4) -> np.ndarray:
     """fp32 NCHW N x 3 x 224 x 224, N(0,1); image n is the same for every N (drawn one by one)."""
     out = np.empty((N, 3, 224, 224), dtype=np.float32)

@@ -76,3 +76,29 @@ def test_both_conv_forms_give_identical_logits(oracle_mod, run):
     p, img, logits, _ = run
     l0 = oracle_mod.bireal18_forward(p, img[:1], conv_form=0)
     assert np.array_equal(l0, logits[:1])  # bitwise, and batch-independent
+
+
+def test_stem_module_against_fp64(oracle_mod):
+    """The STEM module variant (Section 2.3; structure = a reading of the missing figure): its output against the same
+    structure built from fp64 library routines, and the blocks after it unchanged (same code path as the 7x7 variant)."""
+    p = dict(synth.bireal18_params())
+    p["stem_module"] = synth.stem_module_params()
+    img = synth.bireal18_images(2)
+    logits, taps = oracle_mod.bireal18_forward(p, img, conv_form=1, want_taps=True, stem_module=True)
+    sm = p["stem_module"]
+    x = torch.from_numpy(img).double()
+    w = [torch.from_numpy(t).double() for t in sm["w"]]
+    s1 = F.relu(bn64(F.conv2d(x, w[0], stride=2, padding=1), sm["bn"][0], p["bn_eps"]))
+    a = F.relu(bn64(F.conv2d(s1, w[1]), sm["bn"][1], p["bn_eps"]))
+    a = F.relu(bn64(F.conv2d(a, w[2], stride=2, padding=1), sm["bn"][2], p["bn_eps"]))
+    b = F.max_pool2d(s1, 2, stride=2)
+    y = bn64(F.conv2d(torch.cat([a, b], dim=1), w[3]), sm["bn"][3], p["bn_eps"])
+    assert taps[0].shape == (2, 64, 56, 56)
+    assert close(taps[0], y.numpy())
+    assert (taps[0] < 0).mean() > 0.2 and (taps[0] > 0).mean() > 0.2  # a signed stream: the binary blocks see both signs
+    # the head still follows from the last block
+    g = torch.from_numpy(taps[16]).double().mean(dim=(2, 3))
+    want = g @ torch.from_numpy(p["fc_w"]).double().t() + torch.from_numpy(p["fc_b"]).double()
+    assert close(logits, want.numpy())
+    # and it is a different network from the 7x7 one
+    assert not np.array_equal(logits, oracle_mod.bireal18_forward(p, img, conv_form=1))
