@@ -163,6 +163,23 @@ size_t dabnn_bireal18_workspace_bytes(int N);
 dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float* images, int N, float* logits,
                                     void* workspace, size_t workspace_bytes, void* stream);
 
+/* Section 2.3 / Fig. 6 / Table 2, second row -- Bi-Real Net 18 with the STEM module in place of the 7x7 convolution and
+ * the max-pool.  The module's figure is not in the paper's text; the structure here is a reading after the stem block of
+ * the network the paper cites for it (so its parity is pinned to this library's oracle only, not to the paper):
+ *   s1 = relu(BN(conv3x3/2 pad 1, 3 -> 32))(image); a = relu(BN(conv1x1, 32 -> 16))(s1); a = relu(BN(conv3x3/2 pad 1, 16 -> 32))(a);
+ *   b = maxpool2x2/2(s1); out = BN(conv1x1, 64 -> 64)(concat(a, b)), fp32 [N][56][56][64], which feeds the sixteen blocks.
+ * w[i]: fp32 OIHW weights of the four convolutions ([32][3][3][3], [16][32][1][1], [32][16][3][3], [64][64][1][1]);
+ * scale[i], shift[i]: their folded BN vectors.  p's stem_w / stem_scale / stem_shift are not used (may be NULL).
+ * Workspace: dabnn_bireal18_workspace_bytes(N), as for dabnn_bireal18_forward; everything else as there. */
+typedef struct {
+  const float* w[4];
+  const float* scale[4];
+  const float* shift[4];
+} dabnn_stem_module_params;
+dabnn_status dabnn_bireal18_forward_stem_module(const dabnn_bireal18_params* p, const dabnn_stem_module_params* sm,
+                                                const float* images, int N, float* logits, void* workspace,
+                                                size_t workspace_bytes, void* stream);
+
 /* (No counterpart in the paper: a packaging convenience of this library.)
  * dabnn_bireal18_forward for callers that must not allocate device memory.  Some hosts of this library cannot call
  * cudaMalloc: a plug-in inside a server whose framework has reserved the whole device for its own pool, a

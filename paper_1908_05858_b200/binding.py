@@ -29,6 +29,7 @@ EXPORTS = (
     "dabnn_tc_set_max_ctas", "dabnn_tc_weights_bytes", "dabnn_tc_prepare_weights", "dabnn_tc_bconv2d", "dabnn_tc_bconv2d_bn_sign_pack",
     "dabnn_tc_bconv2d_bn_add_sign_pack", "dabnn_tc_error_flag", "dabnn_last_device_flag", "dabnn_stream_status",
     "dabnn_tc_wait_expiry_selftest", "dabnn_packed_words", "dabnn_pack_as", "dabnn_bconv2d_from",
+    "dabnn_bireal18_forward_stem_module",
 )
 
 PACKED_NHWC = 0
@@ -59,6 +60,10 @@ class Bireal18Params(ctypes.Structure):
         ("fc_w", ctypes.c_void_p), ("fc_b", ctypes.c_void_p),
         ("block_w_tc", ctypes.c_void_p * 16),
     ]
+
+
+class StemModuleParams(ctypes.Structure):
+    _fields_ = [("w", ctypes.c_void_p * 4), ("scale", ctypes.c_void_p * 4), ("shift", ctypes.c_void_p * 4)]
 
 
 _lib: Optional[ctypes.CDLL] = None
@@ -111,6 +116,9 @@ def lib() -> ctypes.CDLL:
             getattr(L, name).restype = ci
         L.dabnn_set_conv_tile.restype = ci
         L.dabnn_set_conv_tile.argtypes = [ci]
+        L.dabnn_bireal18_forward_stem_module.restype = ci
+        L.dabnn_bireal18_forward_stem_module.argtypes = [ctypes.POINTER(Bireal18Params), ctypes.POINTER(StemModuleParams), vp, ci, vp, vp,
+                                                         ctypes.c_size_t, vp]
         L.dabnn_packed_words.restype = ctypes.c_size_t
         L.dabnn_packed_words.argtypes = [Shape, ci]
         L.dabnn_pack_as.restype = ci
@@ -372,6 +380,15 @@ class Bireal18:
         self.P = P
         self.device = dev
         self._ws = None
+        self.SM = None
+        if "stem_module" in params:  # Section 2.3: the STEM module variant (forward_stem_module)
+            SM = StemModuleParams()
+            for i in range(4):
+                w = up(params["stem_module"]["w"][i])
+                sc, sh = bn_fold(*[up(t) for t in params["stem_module"]["bn"][i]], eps=eps)
+                self.keep += [w, sc, sh]
+                SM.w[i], SM.scale[i], SM.shift[i] = w.data_ptr(), sc.data_ptr(), sh.data_ptr()
+            self.SM = SM
 
     def workspace(self, N: int) -> torch.Tensor:
         need = bireal18_workspace_bytes(N)
@@ -391,6 +408,22 @@ class Bireal18:
         _check(lib().dabnn_bireal18_forward(ctypes.byref(self.P), images.data_ptr(), N, logits.data_ptr(),
                                             ws.data_ptr(), ws.numel(), _stream()))
         return logits
+
+
+def bireal18_forward_stem_module(net: "Bireal18", images: torch.Tensor, logits: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """dabnn_bireal18_forward_stem_module: the forward pass with the STEM module (the net's params held "stem_module")."""
+    if net.SM is None:
+        raise DabnnError("this network was built without STEM module parameters")
+    images = _dev(images, torch.float32, "images")
+    N = images.shape[0]
+    if tuple(images.shape[1:]) != (3, 224, 224):
+        raise DabnnError("images must be [N][3][224][224]")
+    ws = net.workspace(N)
+    if logits is None:
+        logits = _alloc((N, 1000), torch.float32, images.device)
+    _check(lib().dabnn_bireal18_forward_stem_module(ctypes.byref(net.P), ctypes.byref(net.SM), images.data_ptr(), N,
+                                                    logits.data_ptr(), ws.data_ptr(), ws.numel(), _stream()))
+    return logits
 
 
 def binary_layer_host_workspace_bytes(N, C, H, W, O, kh, kw, stride=(1, 1), pad=(0, 0), pad_value=-1) -> int:

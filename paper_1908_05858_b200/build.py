@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdabnn_b200.so")
-SOURCES = ["pack.cu", "bconv.cu", "bconv_tc.cu", "bireal18.cu", "host_api.cu"]
+SOURCES = ["pack.cu", "bconv.cu", "bconv_tc.cu", "bireal18.cu", "stem_module.cu", "host_api.cu"]
 # -fmad=false: no implicit contraction of fp32 mul+add; every fused multiply-add is an explicit fmaf.
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-fmad=false",

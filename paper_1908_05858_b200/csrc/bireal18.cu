@@ -834,11 +834,12 @@ extern "C" dabnn_status dabnn_bn_fold(const float* gamma, const float* beta, con
 
 extern "C" size_t dabnn_bireal18_workspace_bytes(int N) { return N <= 0 ? 0 : plan(N).total; }
 
-extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float* images, int N,
-                                               float* logits, void* workspace, size_t workspace_bytes, void* stream) {
+// sm == nullptr: the 7x7 stem and the max-pool; else the STEM module in their place.
+static dabnn_status forward_impl(const dabnn_bireal18_params* p, const dabnn_stem_module_params* sm, const float* images,
+                                 int N, float* logits, void* workspace, size_t workspace_bytes, void* stream) {
   if (!p || !images || !logits || !workspace) return DABNN_ERR_NULL;
   if (N <= 0 || N > 65535) return DABNN_ERR_SHAPE;
-  if (!p->stem_w || !p->stem_scale || !p->stem_shift || !p->fc_w || !p->fc_b) return DABNN_ERR_NULL;
+  if ((!sm && (!p->stem_w || !p->stem_scale || !p->stem_shift)) || !p->fc_w || !p->fc_b) return DABNN_ERR_NULL;
   for (int b = 0; b < 16; b++)
     if (!p->block_w[b] || !p->block_scale[b] || !p->block_shift[b]) return DABNN_ERR_NULL;
   for (int d = 0; d < 3; d++)
@@ -862,11 +863,19 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
   uint64_t* bits_in = reinterpret_cast<uint64_t*>(base + ws.bits_a);
   uint64_t* bits_out = reinterpret_cast<uint64_t*>(base + ws.bits_b);
 
-  dabnn_status s = (N * 49 >= 2 * sm_count()) ? launch_stem_8x8(p, images, N, stem_out, st)
-                                               : (N == 1 ? launch_stem<8, 2, 8>(p, images, N, stem_out, st)  // one image: 392 half-tile CTAs
-                                                          : launch_stem<8, 2, 16>(p, images, N, stem_out, st));
-  if (s != DABNN_OK) return s;
-  {
+  dabnn_status s;
+  if (sm) {
+    // the stem output area holds the module's three scratch tensors: s1 (half of it), a1 and the concatenation (a quarter each)
+    float* a1 = stem_out + (size_t)N * 112 * 112 * 32;
+    float* cat = a1 + (size_t)N * 112 * 112 * 16;
+    if ((s = launch_stem_module(sm, images, N, stem_out, a1, cat, cur, bits_in, st)) != DABNN_OK) return s;
+  } else {
+    s = (N * 49 >= 2 * sm_count()) ? launch_stem_8x8(p, images, N, stem_out, st)
+                                   : (N == 1 ? launch_stem<8, 2, 8>(p, images, N, stem_out, st)  // one image: 392 half-tile CTAs
+                                              : launch_stem<8, 2, 16>(p, images, N, stem_out, st));
+    if (s != DABNN_OK) return s;
+  }
+  if (!sm) {
     const long long npix = (long long)N * 56 * 56;
     launch_chain(maxpool_pack, dim3(ceil_div(npix * 16, 256)), dim3(256), (size_t)0, st, stem_out, npix, cur, bits_in);
     if ((s = launch_status()) != DABNN_OK) return s;
@@ -919,6 +928,18 @@ extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, c
     else fc_batched<<<dim3(ceil_div(1000, 64), ceil_div(N, 8)), 64, 0, st>>>(gbuf, N, p->fc_w, p->fc_b, logits);
   }
   return launch_status();
+}
+
+extern "C" dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float* images, int N,
+                                               float* logits, void* workspace, size_t workspace_bytes, void* stream) {
+  return forward_impl(p, nullptr, images, N, logits, workspace, workspace_bytes, stream);
+}
+
+extern "C" dabnn_status dabnn_bireal18_forward_stem_module(const dabnn_bireal18_params* p, const dabnn_stem_module_params* sm,
+                                                           const float* images, int N, float* logits, void* workspace,
+                                                           size_t workspace_bytes, void* stream) {
+  if (!sm) return DABNN_ERR_NULL;
+  return forward_impl(p, sm, images, N, logits, workspace, workspace_bytes, stream);
 }
 
 // ---- allocation-free variant ---------------------------------------------------------------------------

@@ -52,6 +52,10 @@ inline void launch_chain(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t s
 }
 #endif
 
+// The STEM module front end of Bi-Real Net 18 (stem_module.cu): fp32 [N][56][56][64] and its packed signs from the images.
+dabnn_status launch_stem_module(const dabnn_stem_module_params* sm, const float* images, int N, float* s1, float* a1,
+                                float* cat, float* out, uint64_t* bits, cudaStream_t st);
+
 // Per-device host caches (function attributes set, SM counts, symbol addresses) are arrays over the device ordinal.
 constexpr int kMaxDevices = 64;
 // Ordinal of the calling thread's current device, or -1 (no device, or an ordinal beyond kMaxDevices).

@@ -507,6 +507,26 @@ def test_bireal18_batch128_matches_oracle(B, oracle_mod):
     assert B.last_device_flag() == 0
 
 
+@pytest.mark.parametrize("N", [1, 3, 9, 72])
+def test_bireal18_with_stem_module_matches_oracle(B, oracle_mod, N):
+    """The STEM module variant (Section 2.3; the module's structure is a reading of the missing figure, so this pins the
+    CUDA path to the oracle's reading, not to the paper): logits bit for bit, at batch sizes that take the chained
+    launches (1, 3), the ordinary order (9) and the tensor-core engine on every block (72)."""
+    p = dict(synth.bireal18_params())
+    p["stem_module"] = synth.stem_module_params()
+    img = synth.bireal18_images(N)
+    want = oracle_mod.bireal18_forward(p, img, conv_form=1, stem_module=True)
+    net = B.Bireal18(p)
+    got = B.bireal18_forward_stem_module(net, dev(img)).cpu().numpy()
+    assert np.max(np.abs(got - want)) <= 1e-3 * np.max(np.abs(want))
+    assert np.array_equal(got.argmax(axis=1), want.argmax(axis=1))
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    # the 7x7 variant of the same object still gives its own logits
+    assert np.array_equal(net.forward(dev(img[:1])).cpu().numpy().view(np.uint32),
+                          oracle_mod.bireal18_forward(p, img[:1], conv_form=1).view(np.uint32))
+    assert B.last_device_flag() == 0
+
+
 def test_guard_bytes_catch_a_write_past_an_output(B, guard_outputs):
     """The guarded allocator the GPU tests run under does notice an out-of-bounds write (made here with torch, on
     purpose, one byte past an output)."""
