@@ -227,7 +227,8 @@ dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const 
  * The same convolutions (Section 2.1.2, Eq. 1 read as a +-1 dot product) computed on the tcgen05 tensor cores with
  * 4-bit {+1,-1} operands (e2m1, block scale 1.0, fp32 accumulation: exact) expanded on chip from the packed bits.
  * Results are identical to dabnn_bconv2d* bit for bit.
- * Covered: stride 1 or 2 (both axes alike), C a multiple of 64 and at most 512 (256 for stride 2), images narrow enough
+ * Covered: stride 1 or 2 (both axes alike), C at most 512 (256 for stride 2; channels beyond C in the last 64-channel word
+ * are given zero weights, which is what the zero tail bits of the packed words mean in Eq. 1), images narrow enough
  * that the 128 + (kh-1)*SP + kw-1 slots a tile reads fit its activation buffer of 640 rows (SP = W + pad_w slots per
  * image row at stride 1, so W + pad_w <= 255 for a 3x3 filter; wider still at C <= 256, where a thread holds five rows),
  * filters whose expanded weights fit the resident budget (dabnn_tc_weights_bytes returns 0 otherwise); other cases
@@ -265,6 +266,9 @@ dabnn_status dabnn_tc_bconv2d_bn_sign_pack(const uint64_t* a_packed, dabnn_shape
 dabnn_status dabnn_tc_bconv2d_bn_add_sign_pack(const uint64_t* a_packed, dabnn_shape in, const void* w_tc, int O,
                                                dabnn_conv cv, const float* scale, const float* shift, const float* residual,
                                                float* y_out, uint64_t* out_packed, void* stream);
+/* Eq. 1 (BGEMM) on the tensor-core engine: dabnn_bgemm with B expanded once by
+ * dabnn_tc_prepare_weights(B, N, Kbits, 1, 1, b_tc) (dabnn_tc_weights_bytes(N, Kbits, 1, 1) bytes; Kbits <= 512).  Same integers. */
+dabnn_status dabnn_tc_bgemm(const uint64_t* A, int M, const void* b_tc, int N, int Kbits, int32_t* C, void* stream);
 int dabnn_tc_error_flag(void);
 int dabnn_last_device_flag(void* stream);
 dabnn_status dabnn_stream_status(void* stream);

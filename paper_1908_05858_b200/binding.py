@@ -29,7 +29,7 @@ EXPORTS = (
     "dabnn_tc_set_max_ctas", "dabnn_tc_weights_bytes", "dabnn_tc_prepare_weights", "dabnn_tc_bconv2d", "dabnn_tc_bconv2d_bn_sign_pack",
     "dabnn_tc_bconv2d_bn_add_sign_pack", "dabnn_tc_error_flag", "dabnn_last_device_flag", "dabnn_stream_status",
     "dabnn_tc_wait_expiry_selftest", "dabnn_packed_words", "dabnn_pack_as", "dabnn_bconv2d_from",
-    "dabnn_bireal18_forward_stem_module",
+    "dabnn_bireal18_forward_stem_module", "dabnn_tc_bgemm",
 )
 
 PACKED_NHWC = 0
@@ -119,6 +119,8 @@ def lib() -> ctypes.CDLL:
         L.dabnn_bireal18_forward_stem_module.restype = ci
         L.dabnn_bireal18_forward_stem_module.argtypes = [ctypes.POINTER(Bireal18Params), ctypes.POINTER(StemModuleParams), vp, ci, vp, vp,
                                                          ctypes.c_size_t, vp]
+        L.dabnn_tc_bgemm.restype = ci
+        L.dabnn_tc_bgemm.argtypes = [vp, ci, vp, ci, ci, vp, vp]
         L.dabnn_packed_words.restype = ctypes.c_size_t
         L.dabnn_packed_words.argtypes = [Shape, ci]
         L.dabnn_pack_as.restype = ci
@@ -533,6 +535,17 @@ def tc_bconv2d_bn_add_sign_pack(a_packed, wt: TcWeights, scale, shift, residual,
                                                    shift.data_ptr(), residual.data_ptr(), y.data_ptr(),
                                                    bits.data_ptr() if want_bits else None, _stream()))
     return y, bits
+
+
+def tc_bgemm(A: torch.Tensor, Bt: "TcWeights", Kbits: int) -> torch.Tensor:
+    """dabnn_tc_bgemm: A int64 [M][Kw] times the rows of B (a TcWeights built from B viewed as [N][1][1][Kw]) -> int32 [M][N]."""
+    A = _dev(A, torch.int64, "A")
+    M, Kw = A.shape
+    if Kw != (Kbits + 63) // 64 or Bt.C != Kbits or Bt.kh != 1 or Bt.kw != 1:
+        raise DabnnError("operands do not match Kbits")
+    out = _alloc((M, Bt.O), torch.int32, A.device)
+    _check(lib().dabnn_tc_bgemm(A.data_ptr(), M, Bt.buf.data_ptr(), Bt.O, int(Kbits), out.data_ptr(), _stream()))
+    return out
 
 
 def tc_set_max_ctas(max_ctas: int) -> int:

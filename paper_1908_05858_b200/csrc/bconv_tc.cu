@@ -800,7 +800,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 
 // Weights: packed bits [O][taps][Cw] -> e2m1 [blocks of 32 output channels][taps][C/32][32][16 bytes = 32 channels];
 // the blocks cover O rounded up to 128, rows beyond O are zero (e2m1 0.0: they contribute nothing).
-__global__ void tc_prepare_weights_kernel(const uint64_t* __restrict__ wp, int O, int taps, int Cw, int cgroups,
+// Channels beyond C in the last 64-channel word (C not a multiple of 64) get 0.0 as well: whatever the activation rows
+// hold there, the product is 0 -- exactly as the zero tail bits of the packed words contribute nothing to Eq. 1.
+__global__ void tc_prepare_weights_kernel(const uint64_t* __restrict__ wp, int O, int C, int taps, int Cw, int cgroups,
                                           long long units, uint4* __restrict__ out) {
   const long long u = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (u >= units) return;
@@ -814,6 +816,15 @@ __global__ void tc_prepare_weights_kernel(const uint64_t* __restrict__ wp, int O
   if (o < O) {
     const uint32_t half = (uint32_t)(wp[((long long)o * taps + tap) * Cw + (grp >> 1)] >> (32 * (grp & 1)));
     bytes = expand32(half);
+    const int live = C - 32 * grp;  // channels of this group that exist
+    if (live < 32) {
+      // the validity bits go through the same expansion (and so the same channel order): 0xA marks a live nibble
+      const uint4 v = expand32(live <= 0 ? 0u : (1u << live) - 1u);
+      bytes.x &= ((v.x >> 3) & 0x11111111u) * 0xFu;
+      bytes.y &= ((v.y >> 3) & 0x11111111u) * 0xFu;
+      bytes.z &= ((v.z >> 3) & 0x11111111u) * 0xFu;
+      bytes.w &= ((v.w >> 3) & 0x11111111u) * 0xFu;
+    }
   }
   out[u] = bytes;
 }
@@ -827,14 +838,17 @@ int tc_mode() {
   return mode;
 }
 
+// C rounded up to whole 64-channel words: what the operand layouts are sized for
+int tc_cpad(int C) { return (C + 63) / 64 * 64; }
+
 bool tc_covers(int O, int C, int taps) {
-  return O > 0 && C > 0 && C % 64 == 0 && C <= 64 * TC_MAX_CW && 32LL * (C / 2) * taps <= TC_WEIGHT_BUDGET;
+  return O > 0 && C > 0 && tc_cpad(C) <= 64 * TC_MAX_CW && 32LL * (tc_cpad(C) / 2) * taps <= TC_WEIGHT_BUDGET;
 }
 
 // Channels per MMA for a launch: the widest of 128 / 64 / 32 whose rows (half of them per CTA of a pair) fit the
 // resident budget, without padding a small O to a wide tile.
 int tc_ntile(int O, int C, int taps, bool pair) {
-  const long long Kb = (long long)C / 2 * taps;  // bytes per weight row
+  const long long Kb = (long long)tc_cpad(C) / 2 * taps;  // bytes per weight row
   for (int nt = 128; nt >= (pair ? 64 : 32); nt >>= 1) {
     if ((pair ? nt / 2 : nt) * Kb > TC_WEIGHT_BUDGET) continue;
     if (nt > 32 && nt / 2 >= O) continue;
@@ -950,7 +964,7 @@ dabnn_status tc_dispatch(TcArgs& g, cudaStream_t st) {
 // Launch form for a problem: CTA pairs when there are enough tiles to fill the chip with pairs, and as many channel
 // tiles resident per CTA (pair) as fit while every CTA (pair) still gets work.
 void tc_plan(TcArgs& g, int O, int C, int taps) {
-  const long long Kb = (long long)C / 2 * taps;
+  const long long Kb = (long long)tc_cpad(C) / 2 * taps;
   const int mode = tc_mode();
   const int units1 = sm_count(), units2 = sm_count() / 2;
   const int nt2 = tc_ntile(O, C, taps, true);
@@ -985,10 +999,10 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   const int OH = dabnn_out_dim(in.H, cv.kh, cv.stride_h, cv.pad_h), OW = dabnn_out_dim(in.W, cv.kw, cv.stride_w, cv.pad_w);
   if (OH <= 0 || OW <= 0) return DABNN_ERR_SHAPE;
   // what this engine covers; everything else is served by the xor/popcount kernel
-  if (cv.stride_h != cv.stride_w || cv.stride_h > 2 || in.C % 64 != 0) return DABNN_ERR_UNSUPPORTED;
+  if (cv.stride_h != cv.stride_w || cv.stride_h > 2) return DABNN_ERR_UNSUPPORTED;
   if (!tc_covers(O, in.C, cv.kh * cv.kw)) return DABNN_ERR_UNSUPPORTED;
   g.a = a; g.w_tc = static_cast<const uint8_t*>(w_tc);
-  g.N = in.N; g.H = in.H; g.W = in.W; g.Cw = (in.C + 63) / 64; g.C = in.C;
+  g.N = in.N; g.H = in.H; g.W = in.W; g.Cw = (in.C + 63) / 64; g.C = tc_cpad(in.C);  // (the kernel sizes everything by whole words; see tc_prepare_weights_kernel)
   g.O = O; g.kh = cv.kh; g.kw = cv.kw; g.ph = cv.pad_h; g.pw = cv.pad_w; g.OH = OH; g.OW = OW;
   g.S = cv.stride_h;
   // Stride 1 with pad <= k - 1: the slot grid keeps only the left and top padding of each image.  A tap that reaches the
@@ -1036,7 +1050,7 @@ using namespace dabnn;
 
 extern "C" size_t dabnn_tc_weights_bytes(int O, int C, int kh, int kw) {
   if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0 || !tc_covers(O, C, kh * kw)) return 0;
-  return (size_t)((O + 127) / 128 * 128) * kh * kw * (C / 2);
+  return (size_t)((O + 127) / 128 * 128) * kh * kw * (tc_cpad(C) / 2);
 }
 
 extern "C" dabnn_status dabnn_tc_prepare_weights(const uint64_t* w_packed, int O, int C, int kh, int kw, void* w_tc,
@@ -1045,9 +1059,9 @@ extern "C" dabnn_status dabnn_tc_prepare_weights(const uint64_t* w_packed, int O
   if (O <= 0 || C <= 0 || kh <= 0 || kw <= 0) return DABNN_ERR_SHAPE;
   if (!tc_covers(O, C, kh * kw)) return DABNN_ERR_UNSUPPORTED;
   if (!aligned(w_packed, 8) || !aligned(w_tc, 16)) return DABNN_ERR_ALIGNMENT;
-  const int taps = kh * kw, cgroups = C / 32;
+  const int taps = kh * kw, cgroups = tc_cpad(C) / 32;
   const long long units = (long long)((O + 127) / 128 * 128) * taps * cgroups;
-  tc_prepare_weights_kernel<<<ceil_div(units, 256), 256, 0, as_stream(stream)>>>(w_packed, O, taps, (C + 63) / 64, cgroups,
+  tc_prepare_weights_kernel<<<ceil_div(units, 256), 256, 0, as_stream(stream)>>>(w_packed, O, C, taps, (C + 63) / 64, cgroups,
                                                                                  units, static_cast<uint4*>(w_tc));
   return launch_status();
 }
@@ -1091,6 +1105,15 @@ extern "C" dabnn_status dabnn_tc_bconv2d_bn_add_sign_pack(const uint64_t* a_pack
   g.scale = scale; g.shift = shift; g.residual = residual; g.y_out = y_out;
   g.out_packed32 = reinterpret_cast<uint32_t*>(out_packed);
   return tc_dispatch<EPI_BIREAL>(g, as_stream(stream));
+}
+
+extern "C" dabnn_status dabnn_tc_bgemm(const uint64_t* A, int M, const void* b_tc, int N, int Kbits, int32_t* C, void* stream) {
+  // rows of A are the "pixels" of a 1x1 image batch, rows of B the "filters" (expanded by dabnn_tc_prepare_weights with
+  // O = N, C = Kbits, kh = kw = 1): a 1x1 convolution over Kbits channels
+  if (M <= 0 || N <= 0 || Kbits <= 0) return DABNN_ERR_SHAPE;
+  const dabnn_shape in = {M, Kbits, 1, 1};
+  const dabnn_conv cv = {1, 1, 1, 1, 0, 0, -1};
+  return dabnn_tc_bconv2d(A, in, b_tc, N, cv, C, DABNN_NHWC, stream);
 }
 
 extern "C" int dabnn_tc_set_max_ctas(int max_ctas) {

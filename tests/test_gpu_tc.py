@@ -27,6 +27,11 @@ def u64(t):
 
 
 TC_CASES = [
+    (2, 70, 7, 5, 9, 3, 1, -1),         # channel tail in the only word, tiny O
+    (3, 96, 9, 10, 40, 3, 1, +1),       # C = 96: half of the second word
+    (2, 130, 9, 8, 37, 3, 1, -1, 2),    # two live channels in the third word, stride 2
+    (2, 500, 6, 6, 70, 1, 0, -1),       # 1x1 with a tail in the eighth word
+    (2, 3, 12, 12, 5, 5, 2, -1),        # three channels
     # N, C, H, W, O, k, pad, pad_value[, stride]
     (1, 64, 14, 14, 64, 3, 1, -1),      # BASELINE config 1
     (2, 128, 9, 11, 100, 3, 1, +1),     # O not a multiple of 16, pad +1
@@ -95,9 +100,23 @@ def test_tc_conv_and_epilogues_match_oracle(B, oracle_mod, case):
     assert B.tc_error_flag() == 0
 
 
+@pytest.mark.parametrize("shape", [(300, 260, 512), (129, 65, 64), (70, 33, 150), (1000, 2048, 500)])
+def test_tc_bgemm_matches_eq1(B, oracle_mod, shape):
+    M, N, K = shape
+    rng = np.random.default_rng(M + N + K)
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    b = rng.standard_normal((N, K)).astype(np.float32)
+    A = B.pack(dev(a.reshape(M, K, 1, 1))).reshape(M, -1)
+    Bp = B.pack(dev(b.reshape(N, K, 1, 1)))  # [N][1][1][Kw]: the layout of packed 1x1 weights
+    got = B.tc_bgemm(A, B.TcWeights(Bp, K), K).cpu().numpy()
+    counts = oracle_mod.bgemm_xnor(u64(A), u64(Bp).reshape(N, -1), K)  # Eq. 1 as printed: agreeing positions
+    assert np.array_equal(got, 2 * counts - K)
+    assert np.array_equal(got, B.bgemm(A, Bp.reshape(N, -1), K).cpu().numpy())
+
+
 def test_tc_declines_what_it_does_not_cover(B):
     assert not B.tc_supported(64, 64, 3, 3, stride=(3, 3))
-    assert not B.tc_supported(64, 96, 3, 3)          # C not a multiple of 64
+    assert not B.tc_supported(64, 576, 3, 3)         # more than 512 channels
     assert not B.tc_supported(64, 2048, 7, 7)        # expanded weights larger than the resident budget
     a = torch.zeros((1, 8, 8, 1), dtype=torch.int64, device="cuda")
     wt = B.TcWeights(torch.zeros((64, 3, 3, 1), dtype=torch.int64, device="cuda"), 64)
@@ -240,8 +259,8 @@ def tc_matrix_cases():
     """Channel words 1..8 x filter sizes 1, 2, 3, 4, 5, 7 x strides 1, 2: every count of K blocks per tap through the
     unrolled 3x3 issue path and the runtime tap loops of the other filters, at a size with several tiles and a ragged
     channel tile."""
-    return [(2, 64 * cw, 11, 10, 70, k, k // 2, -1 if (cw + k) % 2 else 1, st)
-            for cw in range(1, 9) for k in (1, 2, 3, 4, 5, 7) for st in (1, 2)]
+    return [(2, 64 * cw - (17 if (cw + k) % 3 == 0 else 0), 11, 10, 70, k, k // 2, -1 if (cw + k) % 2 else 1, st)
+            for cw in range(1, 9) for k in (1, 2, 3, 4, 5, 7) for st in (1, 2)]  # (a third of the cases with a channel tail)
 
 
 def run_tc_matrix(B, o):
