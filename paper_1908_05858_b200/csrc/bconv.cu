@@ -123,6 +123,10 @@ dabnn_status fill_args(BConvArgs& g, const uint64_t* a, dabnn_shape in, const ui
   } else {
     g.img_stride = (long long)in.H * in.W * Cw; g.pix_stride = (int)Cw; g.pair_stride = 2;
   }
+  g.magic_ow = OW == 1 ? 0ull : ~0ull / (unsigned long long)OW + 1ull;
+  g.magic_oh = OH == 1 ? 0ull : ~0ull / (unsigned long long)OH + 1ull;
+  g.pointwise = (pl == DABNN_PACKED_NHWC && cv.kh == 1 && cv.kw == 1 && cv.stride_h == 1 && cv.stride_w == 1 && cv.pad_h == 0 &&
+                 cv.pad_w == 0) ? 1 : 0;
   g.magic_cw = Cw == 1 ? 0ull : ~0ull / (unsigned long long)Cw + 1ull;
   g.magic_kw = cv.kw == 1 ? 0ull : ~0ull / (unsigned long long)cv.kw + 1ull;
   return DABNN_OK;

@@ -39,6 +39,9 @@ struct BConvArgs {
   // NC1HWC2 with 128-bit vectors [N][C1][H][W][2] (Section 2.1.2, last paragraph): pix_stride = 2, pair_stride = 2*H*W.
   long long img_stride;
   int pix_stride, pair_stride;
+  unsigned long long magic_ow, magic_oh;  // ceil(2^64 / OW), ceil(2^64 / OH) (0 for 1), used when M < 2^31
+  int pointwise;  // 1x1 filter, stride 1, no padding, channel-packed NHWC words: the im2col row of output pixel m is
+                  // simply pixel m's words, so the loader needs no per-row table and no bounds tests
 };
 
 struct RowInfo {
@@ -111,14 +114,24 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
   const long long m0 = bx * BP;
   const int o0 = by * BO;
 
-  for (int r = tid; r < BP; r += THREADS) {
+  for (int r = tid; r < (g.pointwise ? 0 : BP); r += THREADS) {
     const long long m = m0 + r;
     RowInfo ri;
     if (m < g.M) {
-      const int ow = (int)(m % g.OW);
-      const long long t = m / g.OW;
-      const int oh = (int)(t % g.OH);
-      const long long n = t / g.OH;
+      int ow, oh;
+      long long n;
+      if (g.M < (1LL << 31)) {  // the usual case: 32-bit coordinates, multiply-high instead of 64-bit divisions
+        const int t = fast_div((int)m, g.magic_ow);
+        ow = (int)m - t * g.OW;
+        const int nn = fast_div(t, g.magic_oh);
+        oh = t - nn * g.OH;
+        n = nn;
+      } else {
+        ow = (int)(m % g.OW);
+        const long long t = m / g.OW;
+        oh = (int)(t % g.OH);
+        n = t / g.OH;
+      }
       ri.base = n * g.img_stride;
       ri.ih0 = oh * g.sh - g.ph;
       ri.iw0 = ow * g.sw - g.pw;
@@ -149,8 +162,15 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
 #pragma unroll
     for (int it = 0; it < (want_a ? BP / ROWS_PER_PASS : 0); it++) {
       const int r = row_first + it * ROWS_PER_PASS;
-      const RowInfo ri = rows[r];
       uint32_t* dst = As + r * PITCH + unit * UW * 2;
+      if (g.pointwise) {  // (uniform) pixel m's words are the row: k counts channel words
+        const bool live = k_live && m0 + r < g.M;
+        const uint64_t* src = live ? g.a + ((m0 + r) * g.Cw + k) : g.a;
+        if (UW == 2) cp_async16(smem_u32(dst), src, live ? 16 : 0);
+        else cp_async8(smem_u32(dst), src, live ? 8 : 0);
+        continue;
+      }
+      const RowInfo ri = rows[r];
       const int ih = ri.ih0 + ti, iw = ri.iw0 + tj;
       const bool live = k_live && ri.base >= 0;
       if (live && (ih < 0 || ih >= g.H || iw < 0 || iw >= g.W)) {
