@@ -265,6 +265,7 @@ def main():
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--reps", type=int, default=1, help="--case: launches per timed event pair")
     ap.add_argument("--graph", action="store_true", help="--case: time a CUDA-graph replay of the `reps` launches")
+    ap.add_argument("--stem-module", action="store_true", help="--case bireal: the STEM module variant of the network")
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--tile", type=int, default=0)
     args = ap.parse_args()
@@ -685,10 +686,13 @@ def run_case(a):
     ops = 2.0 * a.N * OHW * OHW * O * a.C * a.k * a.k / 1e12
     work = ("Tbit-ops/s", ops)
     if a.case == "bireal":
-        net = B.Bireal18(synth.bireal18_params(), engine="popc" if a.engine == "popc" else "auto")
+        params = dict(synth.bireal18_params())
+        if a.stem_module:
+            params["stem_module"] = synth.stem_module_params()
+        net = B.Bireal18(params, engine="popc" if a.engine == "popc" else "auto")
         img = torch.from_numpy(synth.bireal18_images(a.N)).to(dev)
         logits = torch.empty((a.N, 1000), dtype=torch.float32, device=dev)
-        fn = lambda: net.forward(img, logits)
+        fn = (lambda: B.bireal18_forward_stem_module(net, img, logits)) if a.stem_module else (lambda: net.forward(img, logits))
         work = ("images/ms", a.N * 1e-3)
     else:
         x, w = synth.conv_case(9, a.N, a.C, a.HW, a.HW, O, a.k, a.k)

@@ -14,89 +14,115 @@ namespace dabnn {
 
 namespace {
 
-// Direct fp32 convolution, zero padding, then y = fmaf(acc, scale, shift) and an optional ReLU.  A thread owns two
-// neighbouring output pixels x CO output channels; the CO filters of the CTA (blockIdx.y) sit in shared memory as
-// [c][kh][kw][CO], read as broadcast 128-bit loads.  Taps outside the image multiply a zero: fmaf(0, w, acc) = acc.
+// Direct fp32 convolution, zero padding, then y = fmaf(acc, scale, shift) and an optional ReLU, as a register-tiled product
+// with a fixed summation order.  A CTA of 256 threads owns 128 consecutive output pixels x BN output channels; K = CIN * k * k
+// is walked in chunks of CG channels x all taps (k index = c * taps + tap ascending: the pinned order).  Per chunk the
+// im2col values of the CTA's pixels go to shared memory k-major ([k][pixel]: a thread later reads its 4 pixels as one
+// 128-bit load) and the filters as [k][channel] (broadcast reads); thread (tx, ty) keeps 4 pixels x TN = BN / 8 channels.
+// The loader thread of pixel p fetches CG consecutive channels of a tap with one vector load (NHWC input) or walks the
+// channels (NCHW input, lanes along the image row).  Taps outside the image are zeros: fmaf(0, w, acc) = acc.
 // x: NCHW (IN_NCHW) or NHWC with CIN channels per pixel; y: NHWC with y_stride channels per pixel, written at channel y_off.
-template <int K, int S, int PAD, int CIN, int CO, bool IN_NCHW, bool RELU>
-__global__ void __launch_bounds__(128) conv_fp32_pinned(const float* __restrict__ x, int N, int H, int W, int OH, int OW,
+template <int K, int S, int PAD, int CIN, int BN, int CG, bool IN_NCHW, bool RELU>
+__global__ void __launch_bounds__(256) conv_fp32_pinned(const float* __restrict__ x, int N, int H, int W, int OH, int OW,
                                                         const float* __restrict__ w_oihw, const float* __restrict__ scale,
                                                         const float* __restrict__ shift, float* __restrict__ y,
                                                         int y_stride, int y_off) {
-  __shared__ __align__(16) float ws[CIN * K * K * CO];
-  const int o0 = blockIdx.y * CO;
-  for (int idx = threadIdx.x; idx < CIN * K * K * CO; idx += 128) {
-    const int o = idx % CO, k = idx / CO;
-    ws[idx] = w_oihw[(size_t)(o0 + o) * (CIN * K * K) + k];
+  constexpr int BM = 128, T = K * K, KC = CG * T, TN = BN / 8, AP = BM + 4, WP = BN + 4;
+  static_assert(CIN % CG == 0 && BN % 16 == 0 && (IN_NCHW || (K == 1 ? CG % 8 == 0 : CG == 4)), "tile");
+  __shared__ __align__(16) float a_s[KC * AP];
+  __shared__ __align__(16) float w_s[KC * WP];
+  const int tid = threadIdx.x;
+  const long long npix = (long long)N * OH * OW;
+  const long long p0 = (long long)blockIdx.x * BM;
+  const int o0 = blockIdx.y * BN;
+  // loader role: pixel lp, and one half of the chunk's taps (or channels, for a single tap)
+  const int lp = tid & (BM - 1), lhalf = tid >> 7;
+  const long long pl = p0 + lp;
+  int ih0 = 0, iw0 = 0;
+  long long xn = -1;  // offset of image n in x, or -1 for a pixel beyond the end
+  if (pl < npix) {
+    const int ow = (int)(pl % OW), oh = (int)((pl / OW) % OH);
+    const long long n = pl / ((long long)OW * OH);
+    ih0 = oh * S - PAD;
+    iw0 = ow * S - PAD;
+    xn = n * (long long)CIN * H * W;
   }
-  __syncthreads();
-  const int pairs_per_row = (OW + 1) / 2;
-  const long long pp = (long long)blockIdx.x * 128 + threadIdx.x;
-  if (pp >= (long long)N * OH * pairs_per_row) return;
-  const int pw = (int)(pp % pairs_per_row);
-  const int oh = (int)((pp / pairs_per_row) % OH);
-  const long long n = pp / ((long long)pairs_per_row * OH);
-  const int ow0 = 2 * pw;
-  const bool second = ow0 + 1 < OW;
+  const int tx = tid & 31, ty = tid >> 5;
+  float acc[4][TN];
+#pragma unroll
+  for (int i = 0; i < 4; i++)
+#pragma unroll
+    for (int j = 0; j < TN; j++) acc[i][j] = 0.0f;
 
-  // per tap: offset of the input value of channel 0 and whether the tap lies inside the image, for both pixels
-  long long off[2][K * K];
-  bool in[2][K * K];
+  for (int c0 = 0; c0 < CIN; c0 += CG) {
+    // filters of this chunk: w_s[k][o] = w[o0 + o][c0 * T + k]
+    for (int idx = tid; idx < KC * BN; idx += 256) {
+      const int o = idx / KC, k = idx - o * KC;  // consecutive threads: consecutive k of one filter (contiguous in OIHW)
+      w_s[k * WP + o] = w_oihw[(size_t)(o0 + o) * (CIN * T) + c0 * T + k];
+    }
+    // im2col values of this chunk
+    if (IN_NCHW) {
 #pragma unroll
-  for (int q = 0; q < 2; q++)
-#pragma unroll
-    for (int i = 0; i < K; i++)
-#pragma unroll
-      for (int j = 0; j < K; j++) {
-        const int ih = oh * S + i - PAD, iw = (ow0 + q) * S + j - PAD;
-        const bool ok = ih >= 0 && ih < H && iw >= 0 && iw < W && (q == 0 || second);
-        in[q][i * K + j] = ok;
-        off[q][i * K + j] = !ok ? 0 : IN_NCHW ? ((n * CIN) * H + ih) * (long long)W + iw : ((n * H + ih) * W + iw) * (long long)CIN;
+      for (int k = 0; k < KC; k++) {
+        if ((k & 1) != lhalf) continue;
+        const int cc = k / T, t = k % T, ih = ih0 + t / K, iw = iw0 + t % K;
+        float v = 0.0f;
+        if (xn >= 0 && ih >= 0 && ih < H && iw >= 0 && iw < W) v = __ldg(x + xn + ((long long)(c0 + cc) * H + ih) * W + iw);
+        a_s[k * AP + lp] = v;
       }
-  constexpr long long CSTEP_NHWC = 1;
-  const long long cstep = IN_NCHW ? (long long)H * W : CSTEP_NHWC;
-
-  float acc[2][CO];
+    } else if (T == 1) {
+      // one tap: the two loader threads of a pixel take half of the chunk's channels each
 #pragma unroll
-  for (int q = 0; q < 2; q++)
+      for (int q = 0; q < CG / 8; q++) {
+        const int cc = lhalf * (CG / 2) + 4 * q;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (xn >= 0) v = __ldg(reinterpret_cast<const float4*>(x + xn + ((long long)ih0 * W + iw0) * CIN + c0 + cc));
+        a_s[(cc + 0) * AP + lp] = v.x; a_s[(cc + 1) * AP + lp] = v.y; a_s[(cc + 2) * AP + lp] = v.z; a_s[(cc + 3) * AP + lp] = v.w;
+      }
+    } else {
 #pragma unroll
-    for (int o = 0; o < CO; o++) acc[q][o] = 0.0f;
-#pragma unroll 2
-  for (int c = 0; c < CIN; c++) {
-#pragma unroll
-    for (int t = 0; t < K * K; t++) {
-      const float x0 = in[0][t] ? __ldg(x + off[0][t] + c * cstep) : 0.0f;
-      const float x1 = in[1][t] ? __ldg(x + off[1][t] + c * cstep) : 0.0f;
-      const float4* wv = reinterpret_cast<const float4*>(ws + (c * K * K + t) * CO);
-#pragma unroll
-      for (int o4 = 0; o4 < CO / 4; o4++) {
-        const float4 w4 = wv[o4];
-        acc[0][4 * o4] = __fmaf_rn(x0, w4.x, acc[0][4 * o4]);
-        acc[0][4 * o4 + 1] = __fmaf_rn(x0, w4.y, acc[0][4 * o4 + 1]);
-        acc[0][4 * o4 + 2] = __fmaf_rn(x0, w4.z, acc[0][4 * o4 + 2]);
-        acc[0][4 * o4 + 3] = __fmaf_rn(x0, w4.w, acc[0][4 * o4 + 3]);
-        acc[1][4 * o4] = __fmaf_rn(x1, w4.x, acc[1][4 * o4]);
-        acc[1][4 * o4 + 1] = __fmaf_rn(x1, w4.y, acc[1][4 * o4 + 1]);
-        acc[1][4 * o4 + 2] = __fmaf_rn(x1, w4.z, acc[1][4 * o4 + 2]);
-        acc[1][4 * o4 + 3] = __fmaf_rn(x1, w4.w, acc[1][4 * o4 + 3]);
+      for (int t = 0; t < T; t++) {
+        if ((t & 1) != lhalf) continue;
+        const int ih = ih0 + t / K, iw = iw0 + t % K;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (xn >= 0 && ih >= 0 && ih < H && iw >= 0 && iw < W) v = __ldg(reinterpret_cast<const float4*>(x + xn + ((long long)ih * W + iw) * CIN + c0));
+        a_s[(0 * T + t) * AP + lp] = v.x; a_s[(1 * T + t) * AP + lp] = v.y; a_s[(2 * T + t) * AP + lp] = v.z; a_s[(3 * T + t) * AP + lp] = v.w;
       }
     }
-  }
+    __syncthreads();
+#pragma unroll 4
+    for (int k = 0; k < KC; k++) {
+      const float4 a = *reinterpret_cast<const float4*>(a_s + k * AP + 4 * tx);
+      float wv[TN];
 #pragma unroll
-  for (int q = 0; q < 2; q++) {
-    if (q == 1 && !second) break;
-    float* dst = y + ((n * OH + oh) * (long long)OW + ow0 + q) * y_stride + y_off + o0;
-#pragma unroll
-    for (int o4 = 0; o4 < CO / 4; o4++) {
-      float v[4];
-#pragma unroll
-      for (int e = 0; e < 4; e++) {
-        const int o = 4 * o4 + e;
-        float r = __fmaf_rn(acc[q][o], __ldg(scale + o0 + o), __ldg(shift + o0 + o));
-        if (RELU) r = (r > 0.0f) ? r : 0.0f;
-        v[e] = r;
+      for (int j = 0; j < TN; j += 2) {
+        const float2 w2 = *reinterpret_cast<const float2*>(w_s + k * WP + ty * TN + j);
+        wv[j] = w2.x; wv[j + 1] = w2.y;
       }
-      *reinterpret_cast<float4*>(dst + 4 * o4) = make_float4(v[0], v[1], v[2], v[3]);
+#pragma unroll
+      for (int j = 0; j < TN; j++) {
+        acc[0][j] = __fmaf_rn(a.x, wv[j], acc[0][j]);
+        acc[1][j] = __fmaf_rn(a.y, wv[j], acc[1][j]);
+        acc[2][j] = __fmaf_rn(a.z, wv[j], acc[2][j]);
+        acc[3][j] = __fmaf_rn(a.w, wv[j], acc[3][j]);
+      }
+    }
+    __syncthreads();
+  }
+  const int o = o0 + ty * TN;
+  float sc[TN], sf[TN];
+#pragma unroll
+  for (int j = 0; j < TN; j++) { sc[j] = __ldg(scale + o + j); sf[j] = __ldg(shift + o + j); }
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    const long long pp = p0 + 4 * tx + i;
+    if (pp >= npix) continue;
+    float* dst = y + pp * y_stride + y_off + o;
+#pragma unroll
+    for (int j = 0; j < TN; j += 2) {
+      float r0 = __fmaf_rn(acc[i][j], sc[j], sf[j]), r1 = __fmaf_rn(acc[i][j + 1], sc[j + 1], sf[j + 1]);
+      if (RELU) { r0 = (r0 > 0.0f) ? r0 : 0.0f; r1 = (r1 > 0.0f) ? r1 : 0.0f; }
+      *reinterpret_cast<float2*>(dst + j) = make_float2(r0, r1);
     }
   }
 }
@@ -128,16 +154,16 @@ dabnn_status launch_stem_module(const dabnn_stem_module_params* sm, const float*
                                 float* cat, float* out, uint64_t* bits, cudaStream_t st) {
   for (int i = 0; i < 4; i++)
     if (!sm->w[i] || !sm->scale[i] || !sm->shift[i]) return DABNN_ERR_NULL;
-  const long long p112 = (long long)N * 112 * 56, p56 = (long long)N * 56 * 28;  // pixel pairs
-  conv_fp32_pinned<3, 2, 1, 3, 16, true, true><<<dim3(ceil_div(p112, 128), 2), 128, 0, st>>>(
+  const long long p112 = (long long)N * 112 * 112, p56 = (long long)N * 56 * 56;  // output pixels
+  conv_fp32_pinned<3, 2, 1, 3, 32, 3, true, true><<<dim3(ceil_div(p112, 128), 1), 256, 0, st>>>(
       images, N, 224, 224, 112, 112, sm->w[0], sm->scale[0], sm->shift[0], s1, 32, 0);
-  conv_fp32_pinned<1, 1, 0, 32, 16, false, true><<<dim3(ceil_div(p112, 128), 1), 128, 0, st>>>(
+  conv_fp32_pinned<1, 1, 0, 32, 16, 16, false, true><<<dim3(ceil_div(p112, 128), 1), 256, 0, st>>>(
       s1, N, 112, 112, 112, 112, sm->w[1], sm->scale[1], sm->shift[1], a1, 16, 0);
-  conv_fp32_pinned<3, 2, 1, 16, 16, false, true><<<dim3(ceil_div(p56, 128), 2), 128, 0, st>>>(
+  conv_fp32_pinned<3, 2, 1, 16, 32, 4, false, true><<<dim3(ceil_div(p56, 128), 1), 256, 0, st>>>(
       a1, N, 112, 112, 56, 56, sm->w[2], sm->scale[2], sm->shift[2], cat, 64, 0);
   const long long npix = (long long)N * 56 * 56;
   stem_pool_concat<<<ceil_div(npix * 8, 256), 256, 0, st>>>(s1, npix, cat);
-  conv_fp32_pinned<1, 1, 0, 64, 16, false, false><<<dim3(ceil_div(p56, 128), 4), 128, 0, st>>>(
+  conv_fp32_pinned<1, 1, 0, 64, 64, 16, false, false><<<dim3(ceil_div(p56, 128), 1), 256, 0, st>>>(
       cat, N, 56, 56, 56, 56, sm->w[3], sm->scale[3], sm->shift[3], out, 64, 0);
   dabnn_status s = launch_status();
   if (s != DABNN_OK) return s;
