@@ -71,10 +71,10 @@ dabnn_status launch_epi(const BConvArgs& g, cudaStream_t st) {
   auto ctas = [&](int bp, int bo) { return ((g.M + bp - 1) / bp) * ((ochan + bo - 1) / bo); };
   int tile = g_conv_tile;
   if (tile == 0) {
-    // Measured on B200 (batch 64 to 256, the ResNet-18 stage shapes and the 1x1 512 -> 2048 layer): 16 outputs per thread at
-    // four warps per scheduler beat the larger register tiles (which spill or leave two warps per scheduler) wherever K
-    // spans more than one chunk; short K (one chunk, nothing to pipeline inside a CTA) does better with 128 x 64.
-    if (g.K64 <= 12 && ctas(128, 64) >= 4LL * sms) tile = 2;
+    // Measured on B200 (batch 64 to 256, the ResNet-18 stage shapes and the 1x1 512 -> 2048 layer): 32 outputs per thread
+    // (128 x 64, two CTAs = 16 warps per SM) where that still gives four waves of CTAs, else 16 outputs per thread (64 x 64);
+    // the 8 x 8 register tile of 128 x 128 spills at 255 registers, leaves two warps per scheduler and is slower everywhere.
+    if (ctas(128, 64) >= 4LL * sms) tile = 2;
     else if (ctas(64, 64) >= 4LL * sms) tile = 3;
     else if (ctas(32, 32) >= sms || g.K64 > 5 * KC64) tile = 4;
     else tile = 5;  // less than one wave of the smallest tile: latency is all that counts
