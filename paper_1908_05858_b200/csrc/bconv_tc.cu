@@ -186,15 +186,19 @@ __device__ __forceinline__ void st_global_v8(void* p, uint32_t a, uint32_t b, ui
                "r"(f), "r"(g2), "r"(h)
                : "memory");
 }
-// The same with an evict-first policy in L2: for output that nothing in this library reads back (the int32 sums), so that
-// it drains to DRAM as it is produced instead of displacing the weights and activations that the next launches read.
-__device__ __forceinline__ void st_global_v8_stream(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e,
+// The same with an evict-first policy in L2 (made once per thread): for output that nothing in this library reads back (the
+// int32 sums), so that it drains to DRAM as it is produced instead of displacing the weights and activations that the
+// next launches read.
+__device__ __forceinline__ uint64_t evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void st_global_v8_stream(void* p, uint64_t pol, uint32_t a, uint32_t b, uint32_t c, uint32_t d, uint32_t e,
                                                     uint32_t f, uint32_t g2, uint32_t h) {
-  asm volatile(
-      "{\n\t.reg .b64 pol;\n\tcreatepolicy.fractional.L2::evict_first.b64 pol, 1.0;\n\t"
-      "st.global.L2::cache_hint.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8}, pol;\n\t}" ::"l"(p),
-      "r"(a), "r"(b), "r"(c), "r"(d), "r"(e), "r"(f), "r"(g2), "r"(h)
-      : "memory");
+  asm volatile("st.global.L2::cache_hint.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8}, %9;" ::"l"(p), "r"(a), "r"(b), "r"(c),
+               "r"(d), "r"(e), "r"(f), "r"(g2), "r"(h), "l"(pol)
+               : "memory");
 }
 __device__ __forceinline__ void ld_global_v8(const void* p, float (&r)[8]) {
   asm volatile("ld.global.L1::no_allocate.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
@@ -631,6 +635,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     // 32-column chunks, warps 8-11 the odd ones
     const int c_first = warp >= 8 ? 32 : 0;
     const int c_step = g.epi2 ? 64 : 32;
+    const uint64_t pol_stream = EPI == EPI_I32 ? evict_first_policy() : 0ull;  // (made once, not per store)
     for (long long mt = mt_first; mt < mt_end && !failed; mt += mt_step) {
       const int row = 32 * (warp & 3) + lane;  // TMEM lane = slot row of the tile
       const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)row;
@@ -700,7 +705,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #pragma unroll
             for (int q = 0; q < 4; q++)
               if (8 * q < nch)  // nch is a multiple of 8 here
-                st_global_v8_stream(dst + 8 * q, acc_to_int(v[8 * q]),
+                st_global_v8_stream(dst + 8 * q, pol_stream, acc_to_int(v[8 * q]),
                              acc_to_int(v[8 * q + 1]),
                              acc_to_int(v[8 * q + 2]),
                              acc_to_int(v[8 * q + 3]),
@@ -957,7 +962,11 @@ dabnn_status tc_dispatch(TcArgs& g, cudaStream_t st) {
   // output row; elsewhere the extra warps only add contention.
   // (environment DABNN_TC_EPI2 = 0 / 1 overrides, for measurements)
   static const int epi_env = [] { const char* e = getenv("DABNN_TC_EPI2"); return e ? atoi(e) : -1; }();
-  g.epi2 = epi_env >= 0 ? (epi_env != 0) : (EPI == EPI_BIREAL);
+  // ... and for short-K layers with many output channels (a 1x1 layer: a handful of MMAs per 128 x 128 accumulator, several
+  // accumulators per activation tile), where the epilogue is most of the work: +4 % with int32 output, +10 % with sign words
+  // on the 1x1 512 -> 2048 layer; 3x3 layers measured the same or slightly slower with it.
+  const bool short_k = g.kh * g.kw * g.Cw <= 8 && g.nres >= 2;
+  g.epi2 = epi_env >= 0 ? (epi_env != 0) : (EPI == EPI_BIREAL || short_k);
   return g.pair ? tc_dispatch_mode<EPI, true>(g, st) : tc_dispatch_mode<EPI, false>(g, st);
 }
 
