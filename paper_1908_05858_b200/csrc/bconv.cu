@@ -53,6 +53,30 @@ dabnn_status launch_one(const BConvArgs& g, cudaStream_t st) {
   return launch_status();
 }
 
+// The several-tiles-per-CTA form for short-K pointwise layers (bconv_pointwise_tiles), 128 x 64 tiles.
+template <int EPI, bool VEC16>
+dabnn_status launch_pointwise(const BConvArgs& g, cudaStream_t st) {
+  constexpr int BP = 128, BO = 64, TP = 8, TO = 4, NSUB = 4, THREADS = (BP / TP) * (BO / TO);
+  constexpr size_t SMEM = (size_t)(BO + 3 * BP) * PITCH * 4 + (size_t)BP * (BO / 32) * 4;
+  auto kern = bconv_pointwise_kernel<BP, BO, TP, TO, 2, EPI, VEC16, NSUB>;
+  static bool configured[kMaxDevices] = {};
+  const int dev = current_device();
+  if (dev < 0) return DABNN_ERR_CUDA;
+  if (!configured[dev]) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) {
+      cudaGetLastError();
+      return DABNN_ERR_CUDA;
+    }
+    configured[dev] = true;
+  }
+  const int ochan = (EPI == EPI_I32) ? g.O : g.Ow32 * 32;
+  const long long gx = ((g.M + BP - 1) / BP + NSUB - 1) / NSUB;
+  const int gy = (ochan + BO - 1) / BO;
+  if (gx > 0x7FFFFFFF || gy > 65535) return DABNN_ERR_UNSUPPORTED;
+  kern<<<dim3((unsigned)gx, (unsigned)gy), THREADS, SMEM, st>>>(g);
+  return launch_status();
+}
+
 template <int BP, int BO, int TP, int TO, int MINB, int EPI, int STAGES = STAGES_DEFAULT>
 dabnn_status launch_tile(const BConvArgs& g, bool csa, cudaStream_t st) {
   const bool vec16 = (g.Cw % 2 == 0) && aligned(g.a, 16) && aligned(g.w, 16);
@@ -78,6 +102,14 @@ dabnn_status launch_epi(const BConvArgs& g, cudaStream_t st) {
     else if (ctas(64, 64) >= 4LL * sms) tile = 3;
     else if (ctas(32, 32) >= sms || g.K64 > 5 * KC64) tile = 4;
     else tile = 5;  // less than one wave of the smallest tile: latency is all that counts
+  }
+  if constexpr (EPI != EPI_BIREAL) {
+    // short-K pointwise layers with at least four waves of four-tile CTAs (DABNN_CONV_POINTWISE=0 in the environment, read
+    // once, keeps the one-tile form, for measurements)
+    static const bool pw_off = [] { const char* e = getenv("DABNN_CONV_POINTWISE"); return e && atoi(e) == 0; }();
+    if (g.pointwise && csa && !pw_off && !g_chain_launch && g.K64 <= KC64 && (g_conv_tile == 0 || g_conv_tile == 2) &&
+        ctas(128, 64) >= 16LL * sms)
+      return ((g.Cw % 2 == 0) && aligned(g.a, 16) && aligned(g.w, 16)) ? launch_pointwise<EPI, true>(g, st) : launch_pointwise<EPI, false>(g, st);
   }
   switch (tile) {
     case 1: return launch_tile<128, 128, 8, 8, 1, EPI>(g, csa, st);

@@ -429,6 +429,174 @@ __device__ __forceinline__ void bconv_tile(const BConvArgs& g, const long long b
   }
 }
 
+// ---- short-K pointwise layers: several pixel tiles per CTA -----------------------------------------------------
+// An unpadded 1x1 stride-1 layer whose K fits one chunk (C <= 1024) has no K loop to pipeline: a one-tile CTA is set-up,
+// one round of loads, 256 word-pair steps per thread and an epilogue, and a third of its instructions are the fixed part.
+// Here a CTA keeps its BO weight rows in shared memory and walks over NSUB consecutive pixel tiles, whose activation rows
+// run through the ring: the loads of tile s + 2 are in flight while tile s is multiplied and written.
+template <int BP, int BO, int TP, int TO, int EPI, bool VEC16, int NSUB>
+__device__ __forceinline__ void bconv_pointwise_tiles(const BConvArgs& g, uint32_t* smem) {
+  static_assert(EPI == EPI_I32 || EPI == EPI_BNPACK, "output form");
+  constexpr int THREADS = (BP / TP) * (BO / TO);
+  constexpr int STAGES = 3;
+  constexpr int UW = VEC16 ? 2 : 1;
+  constexpr int UNITS = KC64 / UW;
+  constexpr int ROWS_PER_PASS = THREADS / UNITS;
+  static_assert(THREADS % UNITS == 0 && BP % ROWS_PER_PASS == 0 && BO % ROWS_PER_PASS == 0, "loader passes");
+  constexpr int WPN = BP / (8 * TP);
+  constexpr int BW = BO / 32;
+  uint32_t* Ws = smem;                         // [BO][PITCH]
+  uint32_t* ring = smem + BO * PITCH;          // [STAGES][BP][PITCH]
+  uint32_t* sbits = ring + STAGES * BP * PITCH;  // [BP][BW]
+
+  const int tid = threadIdx.x;
+  const int o0 = blockIdx.y * BO;
+  const long long n_bx = (g.M + BP - 1) / BP;
+  const long long t_first = (long long)blockIdx.x * NSUB;
+  const int nsub = (int)min((long long)NSUB, n_bx - t_first);
+  const int unit = tid % UNITS, row_first = tid / UNITS;
+  const int k = unit * UW;
+  const bool k_live = k < g.K64;
+
+  auto load_a = [&](int sidx, int stage) {
+    uint32_t* As = ring + stage * BP * PITCH;
+    const long long m0 = (t_first + sidx) * BP;
+#pragma unroll
+    for (int it = 0; it < BP / ROWS_PER_PASS; it++) {
+      const int r = row_first + it * ROWS_PER_PASS;
+      const bool live = k_live && m0 + r < g.M;
+      const uint64_t* src = live ? g.a + ((m0 + r) * g.Cw + k) : g.a;
+      if (UW == 2) cp_async16(smem_u32(As + r * PITCH + unit * UW * 2), src, live ? 16 : 0);
+      else cp_async8(smem_u32(As + r * PITCH + unit * UW * 2), src, live ? 8 : 0);
+    }
+  };
+#pragma unroll
+  for (int it = 0; it < BO / ROWS_PER_PASS; it++) {  // the CTA's weight rows, once
+    const int r = row_first + it * ROWS_PER_PASS;
+    const bool live = k_live && o0 + r < g.O;
+    const uint64_t* src = live ? g.w + (long long)(o0 + r) * g.K64 + k : g.w;
+    if (UW == 2) cp_async16(smem_u32(Ws + r * PITCH + unit * UW * 2), src, live ? 16 : 0);
+    else cp_async8(smem_u32(Ws + r * PITCH + unit * UW * 2), src, live ? 8 : 0);
+  }
+#pragma unroll
+  for (int s = 0; s < STAGES - 1; s++) {
+    if (s < nsub) load_a(s, s);
+    cp_async_commit();
+  }
+
+  const int lane = tid & 31, wid = tid >> 5;
+  const int pl = lane & 7, ol = lane >> 3;
+  const int wp = wid % WPN, wo = wid / WPN;
+  const int arow0 = wp * 8 * TP + pl;
+  const int wrow0 = wo * 4 * TO + ol * TO;
+  const int o = o0 + wrow0;
+  const int one = g.one;
+  float sc[TO], sf[TO];
+  if (EPI == EPI_BNPACK) {
+#pragma unroll
+    for (int j = 0; j < TO; j++) {
+      sc[j] = (o + j < g.O) ? g.scale[o + j] : 0.f;
+      sf[j] = (o + j < g.O) ? g.shift[o + j] : 0.f;
+    }
+  }
+  int acc[TP][TO];
+  uint32_t ones[TP][TO];
+  for (int s = 0; s < nsub; s++) {
+#pragma unroll
+    for (int i = 0; i < TP; i++)
+#pragma unroll
+      for (int j = 0; j < TO; j++) {
+        acc[i][j] = 0;
+        ones[i][j] = 0;
+      }
+    cp_async_wait<STAGES - 2>();
+    __syncthreads();  // tile s (and the weights) visible to all; everyone is done with the stage about to be refilled
+    if (s + STAGES - 1 < nsub) load_a(s + STAGES - 1, (s + STAGES - 1) % STAGES);
+    cp_async_commit();
+    const uint32_t* As = ring + (s % STAGES) * BP * PITCH;
+    int kk = 0;
+    for (; kk + 2 <= g.K64; kk += 2) {
+      uint4 w[TO];
+#pragma unroll
+      for (int j = 0; j < TO; j++) w[j] = *reinterpret_cast<const uint4*>(Ws + (wrow0 + j) * PITCH + 2 * kk);
+#pragma unroll
+      for (int i = 0; i < TP; i++) {
+        const uint4 a = *reinterpret_cast<const uint4*>(As + (arow0 + 8 * i) * PITCH + 2 * kk);
+#pragma unroll
+        for (int j = 0; j < TO; j++) bit_mac_pair(a, w[j], acc[i][j], ones[i][j]);
+      }
+    }
+    if (kk < g.K64) {  // odd tail: one 64-bit word
+      uint2 w[TO];
+#pragma unroll
+      for (int j = 0; j < TO; j++) w[j] = *reinterpret_cast<const uint2*>(Ws + (wrow0 + j) * PITCH + 2 * kk);
+#pragma unroll
+      for (int i = 0; i < TP; i++) {
+        const uint2 a = *reinterpret_cast<const uint2*>(As + (arow0 + 8 * i) * PITCH + 2 * kk);
+#pragma unroll
+        for (int j = 0; j < TO; j++) bit_mac<true>(a.x, a.y, w[j].x, w[j].y, acc[i][j], ones[i][j], one);
+      }
+    }
+    const long long m0 = (t_first + s) * BP;
+    if (EPI == EPI_I32) {
+#pragma unroll
+      for (int i = 0; i < TP; i++) {
+        const long long m = m0 + arow0 + 8 * i;
+        if (m >= g.M) continue;
+        int v[TO];
+#pragma unroll
+        for (int j = 0; j < TO; j++) v[j] = g.Kbits - 2 * (2 * acc[i][j] + __popc(ones[i][j]));
+        if (!g.out_nchw) {
+          int32_t* dst = g.out + m * g.O + o;
+          if (TO % 4 == 0 && o + TO <= g.O && (g.O & 3) == 0 && (reinterpret_cast<uintptr_t>(g.out) & 15) == 0) {
+#pragma unroll
+            for (int j = 0; j < TO; j += 4) __stcs(reinterpret_cast<int4*>(dst + j), make_int4(v[j], v[j + 1], v[j + 2], v[j + 3]));
+          } else {
+#pragma unroll
+            for (int j = 0; j < TO; j++)
+              if (o + j < g.O) __stcs(dst + j, v[j]);
+          }
+        } else {
+          const long long ohw = (long long)g.OH * g.OW;
+          const long long n = m / ohw, q = m % ohw;
+#pragma unroll
+          for (int j = 0; j < TO; j++)
+            if (o + j < g.O) __stcs(g.out + (n * g.O + o + j) * ohw + q, v[j]);
+        }
+      }
+    } else {
+      for (int t = tid; t < BP * BW; t += THREADS) sbits[t] = 0;  // (the previous tile's readers passed this tile's barrier)
+      __syncthreads();
+#pragma unroll
+      for (int i = 0; i < TP; i++) {
+        const long long m = m0 + arow0 + 8 * i;
+        if (m >= g.M) continue;
+        uint32_t field = 0;
+#pragma unroll
+        for (int j = 0; j < TO; j++) {
+          const float y = __fmaf_rn((float)(g.Kbits - 2 * (2 * acc[i][j] + __popc(ones[i][j]))), sc[j], sf[j]);
+          field |= (uint32_t)((o + j < g.O) && (y < 0.0f)) << j;
+        }
+        if (field) atomicOr(&sbits[(arow0 + 8 * i) * BW + (wrow0 >> 5)], field << (wrow0 & 31));
+      }
+      __syncthreads();
+      const int wbase = o0 >> 5;
+      for (int t = tid; t < BP * BW; t += THREADS) {
+        const int r = t / BW, q = t - r * BW;
+        const long long m = m0 + r;
+        if (m < g.M && wbase + q < g.Ow32) g.out_packed32[m * g.Ow32 + wbase + q] = sbits[t];
+      }
+    }
+  }
+  cp_async_wait<0>();
+}
+
+template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool VEC16, int NSUB>
+__global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_pointwise_kernel(const BConvArgs g) {
+  extern __shared__ __align__(16) uint32_t bconv_smem[];
+  bconv_pointwise_tiles<BP, BO, TP, TO, EPI, VEC16, NSUB>(g, bconv_smem);
+}
+
 template <int BP, int BO, int TP, int TO, int MINB, int EPI, bool CSA, bool VEC16, int STAGES>
 __global__ void __launch_bounds__((BP / TP) * (BO / TO), MINB) bconv_kernel(const BConvArgs g) {
   extern __shared__ __align__(16) uint32_t bconv_smem[];

@@ -123,6 +123,8 @@ CONV_CASES = [
     (1, 64, 56, 56, 64, 3, 3, (1, 1), (1, 1), -1),
     (4, 64, 30, 30, 128, 7, 7, (2, 2), (3, 3), -1),     # 49 taps
     (40, 192, 20, 20, 192, 3, 3, (1, 1), (1, 1), -1),   # large enough for the 128x128 tile
+    (130, 192, 13, 13, 1000, 1, 1, (1, 1), (0, 0), -1),  # 1x1, enough tiles for the several-tiles-per-CTA form; odd word count,
+    (131, 128, 13, 13, 1000, 1, 1, (1, 1), (0, 0), +1),  # ragged last CTA (173 pixel tiles), ragged channel tile; 16-byte units
 ]
 
 
