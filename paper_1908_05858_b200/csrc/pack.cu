@@ -34,30 +34,32 @@ template <> struct Vec4<int32_t> { using type = int4; };
 __device__ __forceinline__ unsigned neg(float v) { return (unsigned)(v < 0.0f); }
 __device__ __forceinline__ unsigned neg(int32_t v) { return (unsigned)(v < 0); }
 
-// NCHW, H*W a multiple of 4, 16-byte aligned input.  A CTA covers 128 consecutive pixels of one image and all
-// channels.  Each lane owns 4 consecutive pixels (one float4 per channel); the four warps split every word's 64
-// channels into quarters of 16, so a thread has 16 independent 16-byte loads in flight per word, and the 16-bit
+// NCHW, H*W a multiple of 4, 16-byte aligned input.  A CTA covers 128 consecutive pixels of the batch (images follow one
+// another in the pixel count: a tile may span two or more images, so small images leave no ragged tile per image) and all
+// channels.  Each lane owns 4 consecutive pixels of one image (one float4 per channel); the four warps split every word's
+// 64 channels into quarters of 16, so a thread has 16 independent 16-byte loads in flight per word, and the 16-bit
 // quarters are placed side by side in shared memory, which assembles the 64-bit words without any exchange.
 // C2: the words leave in the NC1HWC2 layout instead ([N][C1][H][W][2]: 128-bit vectors of one channel group, pixel after
 // pixel; an odd last word gets a zero partner).
 template <typename T, bool C2>
-__global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const T* __restrict__ x, int C, int HW, int Cw,
+__global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const T* __restrict__ x, int C, int HW, int Cw, long long npix,
                                                                uint64_t* __restrict__ packed) {
   extern __shared__ __align__(16) uint64_t s_words[];  // [128][Cw]
   uint16_t* s_q = reinterpret_cast<uint16_t*>(s_words);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n = blockIdx.y;
-  const int pix0 = blockIdx.x * 128;
-  const int p = pix0 + lane * 4;  // first of this lane's 4 pixels
-  const bool live = p < HW;       // HW % 4 == 0, so all 4 pixels are live together
+  const long long pix0 = (long long)blockIdx.x * 128;  // in pixels of the whole batch
+  const long long p = pix0 + lane * 4;                 // first of this lane's 4 pixels
+  const bool live = p < npix;                          // HW % 4 == 0, so all 4 pixels are live together and in one image
   using V4 = typename Vec4<T>::type;
-  const T* xn = x + (size_t)n * C * HW;
+  const long long n = live ? p / HW : 0;
+  const int hw = live ? (int)(p - n * HW) : 0;
+  const T* xn = x + (size_t)n * C * HW + hw;
   const size_t cstride = (size_t)HW / 4;
   for (int cw = 0; cw < Cw; cw++) {
     const int c0 = cw * 64 + warp * 16;
     unsigned b0 = 0, b1 = 0, b2 = 0, b3 = 0;  // 16 channels of each of the 4 pixels
     if (live && c0 < C) {
-      const V4* src = reinterpret_cast<const V4*>(xn + (size_t)c0 * HW + p);
+      const V4* src = reinterpret_cast<const V4*>(xn + (size_t)c0 * HW);
       if (c0 + 16 <= C) {
         V4 v[16];
 #pragma unroll
@@ -86,22 +88,23 @@ __global__ void __launch_bounds__(kPackThreads) pack_nchw_vec4(const T* __restri
     s_q[((lp + 3) * Cw + cw) * 4 + warp] = (uint16_t)b3;
   }
   __syncthreads();
-  // contiguous in global memory: pixels pix0 .. pix0+npix-1, all words
-  const int npix = min(128, HW - pix0);
-  if (npix <= 0) return;
+  const int npx = (int)min((long long)128, npix - pix0);
+  if (npx <= 0) return;
   if (C2) {
     const int C1 = (Cw + 1) / 2;
     ulonglong2* d2 = reinterpret_cast<ulonglong2*>(packed);  // 16-byte aligned: checked on the host
-    for (int i = threadIdx.x; i < C1 * npix; i += kPackThreads) {
-      const int grp = i / npix, px = i - grp * npix;  // consecutive threads: consecutive pixels of one channel group
+    for (int i = threadIdx.x; i < C1 * npx; i += kPackThreads) {
+      const int grp = i / npx, px = i - grp * npx;  // consecutive threads: consecutive pixels of one channel group
+      const long long pp = pix0 + px, nn = pp / HW, hh = pp - nn * HW;
       const uint64_t lo = s_words[px * Cw + 2 * grp], hi = (2 * grp + 1 < Cw) ? s_words[px * Cw + 2 * grp + 1] : 0ull;
-      d2[((size_t)n * C1 + grp) * HW + pix0 + px] = make_ulonglong2(lo, hi);
+      d2[((size_t)nn * C1 + grp) * HW + hh] = make_ulonglong2(lo, hi);
     }
     return;
   }
-  uint64_t* dst = packed + ((size_t)n * HW + pix0) * Cw;
-  const int total = npix * Cw;
-  if ((((size_t)n * HW + pix0) * Cw) % 2 == 0 && (reinterpret_cast<uintptr_t>(packed) & 15) == 0) {
+  // contiguous in global memory: pixels pix0 .. pix0+npx-1 of the batch, all words
+  uint64_t* dst = packed + (size_t)pix0 * Cw;
+  const int total = npx * Cw;
+  if (((size_t)pix0 * Cw) % 2 == 0 && (reinterpret_cast<uintptr_t>(packed) & 15) == 0) {
     const int pairs = total / 2;
     const ulonglong2* s2 = reinterpret_cast<const ulonglong2*>(s_words);
     ulonglong2* d2 = reinterpret_cast<ulonglong2*>(dst);
@@ -238,10 +241,12 @@ dabnn_status pack_any(const T* x, dabnn_layout in_layout, dabnn_shape s, uint64_
   if (HW > 0x7FFFFFFF || (long long)s.N * HW > 0x7FFFFFFFFFFLL) return DABNN_ERR_UNSUPPORTED;
   const long long total_words = (long long)s.N * HW * Cw;
   cudaStream_t st = as_stream(stream);
-  if (in_layout == DABNN_NCHW && HW % 4 == 0 && aligned(x, 16) && s.N <= 65535 && Cw * 128 * 8 <= 48 * 1024) {
-    dim3 grid(ceil_div(HW, 128), s.N);
-    if (c2) pack_nchw_vec4<T, true><<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, packed);
-    else pack_nchw_vec4<T, false><<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, packed);
+  if (in_layout == DABNN_NCHW && HW % 4 == 0 && aligned(x, 16) && Cw * 128 * 8 <= 48 * 1024 &&
+      (long long)s.N * HW <= 128LL * 0x7FFFFFFF) {
+    const long long npix = (long long)s.N * HW;
+    const unsigned grid = (unsigned)((npix + 127) / 128);
+    if (c2) pack_nchw_vec4<T, true><<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, npix, packed);
+    else pack_nchw_vec4<T, false><<<grid, kPackThreads, (size_t)128 * Cw * 8, st>>>(x, s.C, (int)HW, (int)Cw, npix, packed);
   } else if (!c2 && in_layout == DABNN_NCHW && s.N <= 65535 && Cw <= 65535) {
     dim3 grid(ceil_div(HW, 128), s.N, (unsigned)Cw);
     pack_nchw_tile<T><<<grid, 256, 0, st>>>(x, s.C, (int)HW, (int)Cw, packed);
