@@ -154,10 +154,11 @@ size_t dabnn_bireal18_workspace_bytes(int N);
 /* p: HOST struct of device pointers.  images: fp32 NCHW [N][3][224][224].  logits: fp32 [N][1000].
  * workspace: device memory, 256-byte aligned, at least dabnn_bireal18_workspace_bytes(N) bytes; its contents
  * are scratch (activations between layers) and are undefined afterwards.
- * Kernels are chosen by batch size (results are the same bits whichever runs).  For one to four images the launches are
- * chained with programmatic stream serialization: a kernel may begin its set-up while its predecessor finishes and waits
- * for it before it reads any activation; on the stream the call as a whole is ordered like any other work, and it can
- * be captured into a CUDA graph.  DABNN_NO_CHAIN=1 in the environment (read once) gives ordinary launches.
+ * Kernels are chosen by batch size (results are the same bits whichever runs).  The launches are chained with programmatic
+ * stream serialization: a kernel may begin its set-up (for the tensor-engine blocks also the copy of its weights and BN
+ * vectors, which must therefore not be written by work still pending on the stream) while its predecessor finishes, and
+ * waits for it before it reads any activation; on the stream the call as a whole is ordered like any other work, and it
+ * can be captured into a CUDA graph.  DABNN_NO_CHAIN=1 in the environment (read once) gives ordinary launches.
  * Where blocks run on the tensor-core engine, a wait that ran out inside one of its kernels leaves the logits undefined
  * while this call has long returned DABNN_OK: after synchronising, check dabnn_stream_status(stream). */
 dabnn_status dabnn_bireal18_forward(const dabnn_bireal18_params* p, const float* images, int N, float* logits,

@@ -85,6 +85,9 @@ struct TcArgs {
   float* y_out;
   uint32_t* out_packed32;
   int Ow32;
+  int chained;         // 1: launched with programmatic stream serialization by the Bi-Real forward, whose weights and BN
+                       // vectors are constants: the kernel starts while its predecessor's last CTAs still run, sets up
+                       // (tensor memory, barriers, thresholds, the weight copy) and only then waits for the predecessor
   int wait_polls;      // polls of a barrier wait before it gives up (TC_WAIT_POLLS; smaller only in the expiry self-test)
   int extra_arrivals;  // 0; the expiry self-test makes `a_full` expect one arrival more than the producers make
 };
@@ -251,6 +254,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   // a pair runs while its leader has a tile (the peer's last tile may lie beyond the end: pad rows, nothing stored)
   const long long mt_end = PAIR ? (g.m_tiles + 1) / 2 * 2 : g.m_tiles;
 
+  if (g.chained) chain_trigger();  // the successor may start as CTAs of this launch leave (it waits for all of them itself)
   if (EPI == EPI_BIREAL) {
     for (int i = tid; i < nres_here * NT; i += TC_THREADS) {
       const int o = (ng * g.nres + i / NT) * NT + (i % NT);
@@ -367,6 +371,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     arrive(bar_w_full + 16u);
   };
+  // (chained launches: nothing above reads or writes what the previous kernel of the stream produces or still reads; the
+  // activation bits, the residual and every output come after this point.  A no-op in an ordinary launch.)
+  chain_wait();
   if (!is_producer) {
     prologue_sync();
     tmem_base = *tmem_slot;
@@ -911,19 +918,28 @@ dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
   const long long cap = (long long)avail / g.n_groups * g.n_groups;
   if (cap <= 0) return DABNN_ERR_UNSUPPORTED;
   if (units > cap) units = cap;
-  if (!PAIR) {
+  if (!PAIR && !g.chained) {
     kern<<<(unsigned)units, TC_THREADS, smem, st>>>(g);
     return launch_status();
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(2 * units));
+  cfg.gridDim = dim3((unsigned)((PAIR ? 2 : 1) * units));
   cfg.blockDim = dim3(TC_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute at;
-  at.id = cudaLaunchAttributeClusterDimension;
-  at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
-  cfg.attrs = &at; cfg.numAttrs = 1;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (PAIR) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = 2; at[na].val.clusterDim.y = 1; at[na].val.clusterDim.z = 1;
+    na++;
+  }
+  if (g.chained) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    na++;
+  }
+  cfg.attrs = at; cfg.numAttrs = na;
   if (cudaLaunchKernelEx(&cfg, kern, g) != cudaSuccess) {
     cudaGetLastError();
     return DABNN_ERR_CUDA;
@@ -1037,7 +1053,7 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   g.pad_neg = cv.pad_value < 0;
   g.out = nullptr; g.out_nchw = 0; g.scale = g.shift = g.residual = nullptr; g.y_out = nullptr;
   g.out_packed32 = nullptr; g.Ow32 = 2 * ((O + 63) / 64);
-  g.wait_polls = TC_WAIT_POLLS; g.extra_arrivals = 0;
+  g.wait_polls = TC_WAIT_POLLS; g.extra_arrivals = 0; g.chained = 0;
   return DABNN_OK;
 }
 
@@ -1100,6 +1116,23 @@ extern "C" dabnn_status dabnn_tc_bconv2d_bn_sign_pack(const uint64_t* a_packed, 
   g.out_packed32 = reinterpret_cast<uint32_t*>(out_packed);
   return tc_dispatch<EPI_BNPACK>(g, as_stream(stream));
 }
+
+namespace dabnn {
+dabnn_status tc_bireal_block(const uint64_t* a_packed, dabnn_shape in, const void* w_tc, int O, dabnn_conv cv,
+                             const float* scale, const float* shift, const float* residual, float* y_out,
+                             uint64_t* out_packed, bool chained, cudaStream_t st) {
+  TcArgs g;
+  dabnn_status s = tc_fill(g, a_packed, in, w_tc, O, cv);
+  if (s != DABNN_OK) return s;
+  if (!scale || !shift || !residual || !y_out) return DABNN_ERR_NULL;
+  if (!aligned(scale, 4) || !aligned(shift, 4) || !aligned(residual, 4) || !aligned(y_out, 4) || !aligned(out_packed, 8))
+    return DABNN_ERR_ALIGNMENT;
+  g.scale = scale; g.shift = shift; g.residual = residual; g.y_out = y_out;
+  g.out_packed32 = reinterpret_cast<uint32_t*>(out_packed);
+  g.chained = chained ? 1 : 0;
+  return tc_dispatch<EPI_BIREAL>(g, st);
+}
+}  // namespace dabnn
 
 extern "C" dabnn_status dabnn_tc_bconv2d_bn_add_sign_pack(const uint64_t* a_packed, dabnn_shape in, const void* w_tc,
                                                           int O, dabnn_conv cv, const float* scale, const float* shift,

@@ -184,6 +184,7 @@ __global__ void __launch_bounds__(256, 2) stem_conv_bn_8x8(const float* __restri
                                                            const float* __restrict__ scale,
                                                            const float* __restrict__ shift, int N,
                                                            float* __restrict__ out /*[N][112][112][64]*/) {
+  chain_trigger();  // (a chained successor may set itself up as this grid drains; it waits for all of it before reading)
   constexpr int TS = 16, IH = 224, IW = 224, OHW = 112;
   constexpr int PS = 2 * TS + 5;         // 37
   constexpr int HALF = 20;               // columns per parity (19 / 18 used), a multiple of 4
@@ -333,6 +334,7 @@ __global__ void __launch_bounds__(256, BM == 128 ? 2 : 3) shortcut_down(const fl
                                                      const float* __restrict__ w /*[O][C]*/, int O,
                                                      const float* __restrict__ scale, const float* __restrict__ shift,
                                                      long long npix_out, float* __restrict__ y /*[N][HW/2][HW/2][O]*/) {
+  chain_trigger();  // (as in the stem: lets a chained tensor-engine block start its set-up under this grid's tail)
   constexpr int PV = BM * SC_BK / 256;   // pooled values a thread forms per chunk: 8 or 4 consecutive c of one pixel
   constexpr int TYP = BM / 16;           // pixels per thread in the register tile
   static_assert(BM == 128 || BM == 64, "pixel tile");
@@ -849,13 +851,15 @@ static dabnn_status forward_impl(const dabnn_bireal18_params* p, const dabnn_ste
   const Workspace ws = plan(N);
   if (workspace_bytes < ws.total) return DABNN_ERR_WORKSPACE;
   cudaStream_t st = as_stream(stream);
-  // One to four images: a chain of 22 short launches, each allowed to start its set-up while its predecessor finishes
-  // (see launch_chain; DABNN_NO_CHAIN=1 in the environment keeps the ordinary stream order, for measurements).
+  // The launches are chained: each kernel that takes part may start its set-up while its predecessor finishes (see
+  // launch_chain; DABNN_NO_CHAIN=1 in the environment keeps the ordinary stream order, for measurements).  For one to four
+  // images that is a chain of 22 launches shorter than a launch takes; for large batches it hides the start-up of the
+  // persistent tensor-engine kernels (tensor memory, barriers, 144 KB of weights per CTA) under the previous kernel's tail.
   static const bool chain_off = getenv("DABNN_NO_CHAIN") != nullptr;
   struct ChainScope {
     explicit ChainScope(bool on) { g_chain_launch = on; }
     ~ChainScope() { g_chain_launch = false; }
-  } chain_scope(N <= 4 && !chain_off);
+  } chain_scope(!chain_off);
   char* base = static_cast<char*>(workspace);
   float* stem_out = reinterpret_cast<float*>(base + ws.stem_out);
   float* cur = reinterpret_cast<float*>(base + ws.res_a);
@@ -880,6 +884,8 @@ static dabnn_status forward_impl(const dabnn_bireal18_params* p, const dabnn_ste
     launch_chain(maxpool_pack, dim3(ceil_div(npix * 16, 256)), dim3(256), (size_t)0, st, stem_out, npix, cur, bits_in);
     if ((s = launch_status()) != DABNN_OK) return s;
   }
+  // consecutive tensor-engine blocks are chained (DABNN_NO_CHAIN=1 keeps the ordinary stream order)
+  const bool tc_chain = !chain_off;
   int C = 64, HW = 56;
   for (int b = 0; b < 16; b++) {
     const int stage = b / 4, O = kStageC[stage], OHW = kStageHW[stage];
@@ -907,8 +913,8 @@ static dabnn_status forward_impl(const dabnn_bireal18_params* p, const dabnn_ste
     const dabnn_conv cv = {3, 3, stride, stride, 1, 1, -1};
     s = DABNN_ERR_UNSUPPORTED;
     if (p->block_w_tc[b] != nullptr && tc_worthwhile(in, O, cv))  // tensor-core engine where it covers the layer and pays
-      s = dabnn_tc_bconv2d_bn_add_sign_pack(bits_in, in, p->block_w_tc[b], O, cv, p->block_scale[b], p->block_shift[b], cur,
-                                            cur, b == 15 ? nullptr : bits_out, st);
+      s = tc_bireal_block(bits_in, in, p->block_w_tc[b], O, cv, p->block_scale[b], p->block_shift[b], cur, cur,
+                          b == 15 ? nullptr : bits_out, tc_chain, st);
     if (s == DABNN_ERR_UNSUPPORTED)
       s = dabnn_bconv2d_bn_add_sign_pack(bits_in, in, p->block_w[b], O, cv, p->block_scale[b], p->block_shift[b], cur, cur,
                                          b == 15 ? nullptr : bits_out, st);

@@ -21,6 +21,12 @@ inline int ceil_div(long long a, long long b) { return static_cast<int>((a + b -
 // (below that the integer-pipe kernel, which spreads small problems over many small CTAs, is faster).
 bool tc_worthwhile(dabnn_shape in, int O, dabnn_conv cv);
 
+// The Bi-Real block on the tensor-core engine as the forward launches it.  chained: with programmatic stream serialization
+// (the kernel sets itself up under its predecessor's tail; its weights and BN vectors must be constants of the stream).
+dabnn_status tc_bireal_block(const uint64_t* a_packed, dabnn_shape in, const void* w_tc, int O, dabnn_conv cv,
+                             const float* scale, const float* shift, const float* residual, float* y_out,
+                             uint64_t* out_packed, bool chained, cudaStream_t st);
+
 // Chained launches for forwards of a few images, where every kernel is shorter than the time it takes to start one.  A
 // kernel started by launch_chain() while g_chain_launch is set may begin before its predecessor in the stream has
 // finished: it may do what does not depend on the predecessor (index set-up, fetching weights) and must call
