@@ -209,6 +209,14 @@ __device__ __forceinline__ void ld_global_v8(const void* p, float (&r)[8]) {
                : "l"(p));
 }
 
+// Read-only-path load of activation bits.  Volatile asm, not __ldg: the compiler treats __ldg as an invariant load that it
+// may move anywhere, also above the wait of a chained launch, before which the previous kernel may not have written the bits.
+__device__ __forceinline__ uint64_t ld_nc_u64(const uint64_t* p) {
+  uint64_t v;
+  asm volatile("ld.global.nc.b64 %0, [%1];" : "=l"(v) : "l"(p));
+  return v;
+}
+
 // The fp32 accumulator holds an exact integer of magnitude <= K < 2^22: adding 1.5 * 2^23 leaves it in the low mantissa
 // bits (two full-rate instructions instead of a conversion).
 __device__ __forceinline__ uint32_t acc_to_int(uint32_t acc_bits) {
@@ -559,7 +567,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
             const uint64_t* src = g.a + (((long long)co_n[h] * g.H + ih) * g.W + iw) * g.Cw;
 #pragma unroll
             for (int cw = 0; cw < CW; cw++)
-              if (cw < g.Cw) R.words[h][cw] = __ldg(src + cw);  // (CW is g.Cw rounded up to 1, 2, 4 or 8)
+              if (cw < g.Cw) R.words[h][cw] = ld_nc_u64(src + cw);  // (CW is g.Cw rounded up to 1, 2, 4 or 8)
           }
           co_c[h] += dc;
           if (co_c[h] >= g.SP) { co_c[h] -= g.SP; co_r[h]++; }

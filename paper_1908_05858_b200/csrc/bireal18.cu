@@ -288,9 +288,13 @@ __global__ void __launch_bounds__(256, 2) stem_conv_bn_8x8(const float* __restri
   asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
+// In the kernels that take part in chained launches, the pointer to the ACTIVATIONS (what the previous kernel of the stream
+// wrote) is deliberately neither __restrict__ nor read with __ldg: such loads count as invariant and the compiler may move
+// them above the wait for the previous kernel (seen in a trial that chained the fc kernel: it read pooled values before
+// they were written).  Where the read-only path matters, ld_nc_f4 (volatile asm) keeps the load behind the wait.
 // ---- maxpool 3x3 / 2, pad 1 (64 channels) -> fp32 residual stream + packed signs -------------------
 // A thread handles 4 channels of one output pixel; 16 lanes make one 64-bit word.
-__global__ void __launch_bounds__(256) maxpool_pack(const float* __restrict__ x /*[N][112][112][64]*/, long long npix,
+__global__ void __launch_bounds__(256) maxpool_pack(const float* x /*[N][112][112][64]*/, long long npix,
                                                     float* __restrict__ y /*[N][56][56][64]*/,
                                                     uint64_t* __restrict__ bits /*[N][56][56][1]*/) {
   const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -310,7 +314,7 @@ __global__ void __launch_bounds__(256) maxpool_pack(const float* __restrict__ x 
       for (int j = 0; j < 3; j++) {
         const int ih = 2 * oh + i - 1, iw = 2 * ow + j - 1;
         if (ih < 0 || ih >= 112 || iw < 0 || iw >= 112) continue;
-        const float4 v = *reinterpret_cast<const float4*>(x + ((n * 112 + ih) * 112 + iw) * 64 + c4 * 4);
+        const float4 v = ld_nc_f4(x + ((n * 112 + ih) * 112 + iw) * 64 + c4 * 4);
         m.x = fmaxf(m.x, v.x); m.y = fmaxf(m.y, v.y); m.z = fmaxf(m.z, v.z); m.w = fmaxf(m.w, v.w);
       }
     *reinterpret_cast<float4*>(y + pix * 64 + c4 * 4) = m;
@@ -623,7 +627,7 @@ __global__ void __launch_bounds__(512) gap_small(const float* __restrict__ x /*[
 // One to four images: pooling and fc in one launch.  A 512-thread CTA takes 8 logits of one image: it pools the image's
 // 7x7x512 map itself (thread c owns channel c; same sum order and division as gap_small) while its 8 weight rows are in
 // flight, then 8 threads run the 8 fmaf chains out of shared memory.
-__global__ void __launch_bounds__(512) head_small(const float* __restrict__ x /*[N][7][7][512]*/,
+__global__ void __launch_bounds__(512) head_small(const float* x /*[N][7][7][512]*/,
                                                   const float* __restrict__ fw, const float* __restrict__ fb,
                                                   float* __restrict__ logits) {
   constexpr int PITCH = 516;

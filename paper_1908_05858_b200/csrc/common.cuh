@@ -38,6 +38,15 @@ extern thread_local bool g_chain_launch;  // per host thread: set by a forward c
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void chain_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Read-only-path 16-byte load for data that the PREVIOUS kernel of a chain wrote.  Volatile asm, so that it stays behind
+// chain_wait(): __ldg and loads through const __restrict__ pointers count as invariant, and the compiler may move those
+// above the wait, before which the data may not have been written.
+__device__ __forceinline__ float4 ld_nc_f4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+
 template <typename... KArgs, typename... Args>
 inline void launch_chain(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
   if (!g_chain_launch) {
