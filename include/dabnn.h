@@ -239,7 +239,11 @@ dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const 
  * cannot keep 128 output channels of weights resident: C = 512 with a 3x3 filter).  Both give the same bits.
  * The int32 output is written with a streaming (evict-first) cache policy.
  * Environment, read once, for measurements only: DABNN_TC_MODE = 1 (never pairs) or 2 (pairs wherever possible);
- * DABNN_TC_EPI2 = 0 / 1 (second group of epilogue warps off / on).
+ * DABNN_TC_EPI2 = 0 / 1 (second group of epilogue warps off / on); DABNN_TC_RES_RING = 0 (residual of the Bi-Real epilogue
+ * read with ordinary loads everywhere) or 2..4 (chunks per epilogue warp in flight where bulk tensor copies fetch it).
+ * The Bi-Real epilogue of a long stride-1 launch whose rows are whole 128-byte chunks (O a multiple of 32, residual and
+ * y_out 32-byte aligned) fetches the residual with bulk tensor copies; the library then encodes a tensor map on the host
+ * in the call (cuTensorMapEncodeTiled, looked up through the runtime; if it is not there, ordinary loads are used).
  *   dabnn_tc_weights_bytes    bytes of the expanded weight buffer for a filter bank (0 = not covered): O rounded up to
  *                             128 rows of C*kh*kw/2 bytes, the same buffer for every launch form
  *   dabnn_tc_prepare_weights  w_packed [O][kh][kw][Cw] -> w_tc (device, 16-byte aligned, that many bytes); once per model

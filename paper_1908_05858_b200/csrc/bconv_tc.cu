@@ -35,6 +35,8 @@
 // Every wait on an mbarrier is bounded: on expiry the kernel records an error flag, stops, frees its TMEM and returns.
 #include "common.cuh"
 
+#include <cuda.h>  // the tensor-map type and enums only: the one driver function used is looked up at run time
+
 namespace dabnn {
 
 namespace {
@@ -44,7 +46,10 @@ enum { EPI_I32 = 0, EPI_BNPACK = 1, EPI_BIREAL = 2 };
 constexpr int TC_THREADS = 416;           // warps 0-3 and (optionally) 8-11: epilogue, 4-7: producers, 12: MMA issue
 constexpr int TC_SMEM_LIMIT = 232448;     // 227 KB opt-in maximum per CTA
 constexpr int TC_MAX_RES = 4;              // channel tiles resident per CTA (pair) at most
-constexpr int TC_SMEM_MISC = 256 + 2 * TC_MAX_RES * 128 * 4;  // barriers, TMEM base, flags; this CTA's scale / shift
+constexpr int TC_SMEM_HDR = 512;           // barriers, TMEM base, flags
+constexpr int TC_SMEM_MISC = TC_SMEM_HDR + 2 * TC_MAX_RES * 128 * 4;  // ... and this CTA's scale / shift
+constexpr int TC_RING_MAX = 4;             // residual chunks in flight per epilogue warp at most
+constexpr int TC_RING_CHUNK = 4096;        // one chunk: 32 rows x 32 fp32 channels
 constexpr int TC_WEIGHT_BUDGET = 147456;  // 144 KB of resident weights at most
 constexpr int TC_MAX_CW = 8;              // C <= 512
 constexpr int TC_MAX_SPT = 5;             // slots per producer thread: 2 for stride 1, up to 5 for stride 2
@@ -90,6 +95,9 @@ struct TcArgs {
                        // (tensor memory, barriers, thresholds, the weight copy) and only then waits for the predecessor
   int wait_polls;      // polls of a barrier wait before it gives up (TC_WAIT_POLLS; smaller only in the expiry self-test)
   int extra_arrivals;  // 0; the expiry self-test makes `a_full` expect one arrival more than the producers make
+  int res_ring;        // > 0: the residual reaches the epilogue warps as bulk tensor copies into a ring of this many
+                       // 4 KB chunks per warp (res_map: [pixels][O] fp32, boxes of 32 rows x 32 channels, 128-byte swizzle)
+  alignas(64) CUtensorMap res_map;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -231,8 +239,8 @@ __device__ __forceinline__ uint32_t fast_div(uint32_t q, unsigned long long magi
   return magic == 0 ? q : (uint32_t)__umul64hi((unsigned long long)q, magic);
 }
 
-template <int NT, int EPI, int SPT, bool PAIR>
-__global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g) {
+template <int NT, int EPI, int SPT, bool PAIR, bool RES_TMA = false>
+__global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_constant__ TcArgs g) {
   extern __shared__ __align__(1024) uint8_t smem[];
   constexpr int WR = PAIR ? NT / 2 : NT;  // weight rows (output channels) of one channel tile held by this CTA
   constexpr uint32_t PEERS = PAIR ? 2 : 1;
@@ -249,7 +257,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
   constexpr int B_MMA_DONE = 0, B_TMEM_FREE = 4, B_A_FULL = 8, B_A_FREE = 12, B_W_FULL = 16;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 160);
   volatile int* s_fail = reinterpret_cast<volatile int*>(misc + 168);
-  float* s_scale = reinterpret_cast<float*>(misc + 256);     // [nres][NT] this CTA's channels
+  // [32 + 4 * e ..]: `res_full` of epilogue warp e's ring of residual chunks
+  constexpr int B_RES_FULL = 32;
+  float* s_scale = reinterpret_cast<float*>(misc + TC_SMEM_HDR);  // [nres][NT] this CTA's channels
   float* s_shift = s_scale + TC_MAX_RES * NT;                // [nres][NT]
 
   // work: CTA (pair) `unit` takes channel-tile group `ng` and every `unit_step`-th tile (pair of tiles) of 128 slots
@@ -310,6 +320,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       mbar_init(smem_u32(&bars[B_A_FREE + i]), 1);
     }
     for (int i = 0; i < 3; i++) mbar_init(smem_u32(&bars[B_W_FULL + i]), TC_THREADS * PEERS);
+    if (RES_TMA)
+      for (int i = 0; i < 8 * TC_RING_MAX; i++) mbar_init(smem_u32(&bars[B_RES_FULL + i]), 1);  // the warp's issuing lane
     *s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -651,6 +663,47 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
     const int c_first = warp >= 8 ? 32 : 0;
     const int c_step = g.epi2 ? 64 : 32;
     const uint64_t pol_stream = EPI == EPI_I32 ? evict_first_policy() : 0ull;  // (made once, not per store)
+    // The residual as bulk tensor copies (g.res_ring > 0): every epilogue warp owns a ring of 4 KB chunks (32 rows x 32
+    // channels) and its lane 0 requests the chunks in the order the warp will use them, `res_ring` chunks ahead -- across
+    // tiles, which register prefetch cannot afford.  The valid slots of a warp's 32 rows are consecutive output pixels,
+    // so a chunk is the box (first channel, first valid pixel) of the [pixels][O] tensor; rows of the box beyond the
+    // warp's pixels (or beyond the tensor: zero fill) are read and ignored.  128-byte swizzle: lane = row reads its 16-byte
+    // piece j at (j ^ (row & 7)), free of bank conflicts.
+    constexpr bool tma_res = RES_TMA;
+    const int ew = warp < 4 ? warp : warp - 4;  // epilogue warp 0..7
+    const uint32_t ring0 = ((smem_u32(misc) + (uint32_t)TC_SMEM_MISC + 1023u) & ~1023u) + (uint32_t)(ew * g.res_ring) * TC_RING_CHUNK;
+    const uint32_t rbar0 = smem_u32(&bars[B_RES_FULL + ew * TC_RING_MAX]);
+    long long mt_i = mt_first;                 // the next chunk to request: tile, resident channel tile, first channel
+    int r_i = 0, c0_i = warp >= 8 ? 32 : 0;
+    uint32_t slot_i = 0, slot_u = 0, phase_u = 0, in_flight = 0;
+    auto issue_next = [&]() {  // (warp-uniform state; lane 0 issues)
+      if (mt_i >= mt_end) return;
+      if (lane == 0) {
+        // output pixels before the warp's first slot = the pixel index of its first valid row
+        const uint32_t Q0 = (uint32_t)mt_i * 128u + 32u * (uint32_t)(warp & 3);
+        const uint32_t rr0 = fast_div(Q0, g.magic_sp);
+        const uint32_t col0 = Q0 - rr0 * (uint32_t)g.SP;
+        const uint32_t n0 = fast_div(rr0, g.magic_hp);
+        const uint32_t r0 = rr0 - n0 * (uint32_t)g.HP;
+        uint32_t m0 = (n0 * (uint32_t)g.OH + min(r0, (uint32_t)g.OH)) * (uint32_t)g.OW + (r0 < (uint32_t)g.OH ? min(col0, (uint32_t)g.OW) : 0u);
+        if (n0 >= (uint32_t)g.N) m0 = (uint32_t)g.N * (uint32_t)g.OH * (uint32_t)g.OW;  // beyond the batch: an all-zero box
+        const uint32_t bar = rbar0 + 8u * slot_i, dst = ring0 + slot_i * TC_RING_CHUNK;
+        const uint32_t ch = (uint32_t)((ng * g.nres + r_i) * NT + c0_i);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)TC_RING_CHUNK) : "memory");
+        asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+                     "l"(reinterpret_cast<uint64_t>(&g.res_map)), "r"(ch), "r"(m0), "r"(bar)
+                     : "memory");
+      }
+      in_flight++;
+      if (++slot_i == (uint32_t)g.res_ring) slot_i = 0;
+      c0_i += g.epi2 ? 64 : 32;
+      if (c0_i >= NT) {
+        c0_i = warp >= 8 ? 32 : 0;
+        if (++r_i >= nres_here) { r_i = 0; mt_i += mt_step; }
+      }
+    };
+    if (tma_res)
+      for (int i = 0; i < g.res_ring; i++) issue_next();
     for (long long mt = mt_first; mt < mt_end && !failed; mt += mt_step) {
       const int row = 32 * (warp & 3) + lane;  // TMEM lane = slot row of the tile
       const uint32_t Q = (uint32_t)mt * 128u + (uint32_t)row;
@@ -660,6 +713,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       const int r = (int)(rr - n * (uint32_t)g.HP);
       const int my_valid = (n < (uint32_t)g.N && r < g.OH && col < g.OW) ? 1 : 0;
       const int my_m = (int)((n * (uint32_t)g.OH + (uint32_t)r) * (uint32_t)g.OW + (uint32_t)col);  // < 2^31 (host check)
+      // row of this lane's pixel in the warp's residual chunks: its rank among the warp's valid rows
+      const uint32_t srow = tma_res ? (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, my_valid != 0) & ((1u << lane) - 1u)) : 0u;
       // wide outputs: 256-bit accesses when rows are 32-byte multiples at 32-byte aligned addresses
       const bool wide_i32 = EPI == EPI_I32 && !g.out_nchw && (g.O & 7) == 0 && (reinterpret_cast<uintptr_t>(g.out) & 31) == 0;
       const bool wide_y = EPI == EPI_BIREAL && (g.O & 7) == 0 &&
@@ -673,7 +728,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
       // every later chunk one chunk ahead of its use.
       float rpre[32];
       auto load_res = [&](int c0) {
-        if (EPI == EPI_BIREAL && wide_y && my_valid) {
+        if (EPI == EPI_BIREAL && wide_y && my_valid && !tma_res) {
           const int o = nt * NT + c0;
           const int nch = min(32, g.O - o);
           const float* rs = g.residual + (long long)my_m * g.O + o;
@@ -693,8 +748,67 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
 #pragma unroll 1
       for (int c0 = c_first; c0 < NT; c0 += c_step) {
         __syncwarp();  // the TMEM load is warp-wide: rejoin lanes that took different paths below
+        if constexpr (tma_res) {
+          // this chunk has landed (requested `res_ring` chunks ago)
+          if (!__all_sync(0xFFFFFFFFu, mbar_wait(rbar0 + 8u * slot_u, phase_u, s_fail, g.wait_polls))) {
+            *s_fail = 1;
+            failed = true;
+            break;
+          }
+          in_flight--;
+          uint32_t v[32];
+          const uint32_t taddr = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16) + (uint32_t)(buf * NT + c0);
+          asm volatile(
+              "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+              "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+              : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+                "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+                "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+              : "r"(taddr));
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          const int o = nt * NT + c0;
+          if (my_valid && o < g.O) {  // (O is a multiple of 32 on this path: a chunk exists whole or not at all)
+            const uint32_t src = ring0 + slot_u * TC_RING_CHUNK + srow * 128u;
+            float* yd = g.y_out + m * g.O + o;
+            uint32_t word = 0;
+#pragma unroll
+            for (int q = 0; q < 4; q++) {
+              float rc[8], y[8];
+#pragma unroll
+              for (int h = 0; h < 2; h++) {
+                const uint32_t ad = src + ((((uint32_t)(2 * q + h)) ^ (srow & 7u)) << 4);
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(rc[4 * h]), "=f"(rc[4 * h + 1]), "=f"(rc[4 * h + 2]), "=f"(rc[4 * h + 3])
+                             : "r"(ad));
+                const float4 sc = *reinterpret_cast<const float4*>(r_scale + c0 + 8 * q + 4 * h);
+                const float4 sh = *reinterpret_cast<const float4*>(r_shift + c0 + 8 * q + 4 * h);
+                y[4 * h] = __fmaf_rn(__uint_as_float(v[8 * q + 4 * h]), sc.x, sh.x);
+                y[4 * h + 1] = __fmaf_rn(__uint_as_float(v[8 * q + 4 * h + 1]), sc.y, sh.y);
+                y[4 * h + 2] = __fmaf_rn(__uint_as_float(v[8 * q + 4 * h + 2]), sc.z, sh.z);
+                y[4 * h + 3] = __fmaf_rn(__uint_as_float(v[8 * q + 4 * h + 3]), sc.w, sh.w);
+              }
+#pragma unroll
+              for (int j = 0; j < 8; j++) {
+                y[j] = __fadd_rn(y[j], rc[j]);
+                word |= (uint32_t)(y[j] < 0.0f) << (8 * q + j);
+              }
+              st_global_v8(yd + 8 * q, __float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]), __float_as_uint(y[3]),
+                           __float_as_uint(y[4]), __float_as_uint(y[5]), __float_as_uint(y[6]), __float_as_uint(y[7]));
+            }
+            if (g.out_packed32 != nullptr) g.out_packed32[m * g.Ow32 + (o >> 5)] = word;
+          } else if (my_valid && o < g.Ow32 * 32 && g.out_packed32 != nullptr) {
+            g.out_packed32[m * g.Ow32 + (o >> 5)] = 0u;  // sign words are written whole: the half beyond O holds zeros
+          }
+          // the chunk is in registers (or stored): its buffer takes the next request
+          if (++slot_u == (uint32_t)g.res_ring) { slot_u = 0; phase_u ^= 1u; }
+          __syncwarp();
+          issue_next();
+          continue;
+        }
         float rc[32];
-        if (EPI == EPI_BIREAL) {
+        if (false) {
+        } else if (EPI == EPI_BIREAL) {
 #pragma unroll
           for (int j = 0; j < 32; j++) rc[j] = rpre[j];
           if (c0 + c_step < NT) load_res(c0 + c_step);
@@ -796,12 +910,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const TcArgs g)
           }
         }
       }
+      if (failed) break;
       // this accumulator buffer may be overwritten by the tile after next
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();  // (the tensor-memory loads were warp-wide; lanes may have parted since: rejoin, then one arrival per warp)
       if (lane == 0) arrive(bar_tmem_free0 + 8u * buf);
       if (++accb == (uint32_t)g.nacc) { accb = 0; acc_phase ^= 1u; }
       }
+    }
+    // (only after a wait ran out:) chunks still on their way must land before the CTA gives up its shared memory
+    while (tma_res && in_flight > 0) {
+      __all_sync(0xFFFFFFFFu, mbar_wait(rbar0 + 8u * slot_u, phase_u, s_fail, g.wait_polls));
+      in_flight--;
+      if (++slot_u == (uint32_t)g.res_ring) { slot_u = 0; phase_u ^= 1u; }
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -880,9 +1001,9 @@ int tc_ntile(int O, int C, int taps, bool pair) {
 // Channel tiles cover O rounded up to whole 64-bit sign words (rows beyond O hold zero weights).
 int tc_n_ntiles(int O, int nt) { return ((O + 63) / 64 * 64 + nt - 1) / nt; }
 
-template <int NT, int EPI, int SPT, bool PAIR>
+template <int NT, int EPI, int SPT, bool PAIR, bool RES_TMA = false>
 dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
-  auto kern = bconv_tc_kernel<NT, EPI, SPT, PAIR>;
+  auto kern = bconv_tc_kernel<NT, EPI, SPT, PAIR, RES_TMA>;
   static bool configured[kMaxDevices] = {};
   static int max_units_dev[kMaxDevices] = {};  // CTAs (pairs) that can be resident at once
   const int dev = current_device();
@@ -955,6 +1076,36 @@ dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
   return launch_status();
 }
 
+// cuTensorMapEncodeTiled, looked up through the runtime (the library does not link against the driver library)
+typedef CUresult (*tc_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+tc_encode_fn tc_encoder() {
+  static const tc_encode_fn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      p = nullptr;
+    }
+    return reinterpret_cast<tc_encode_fn>(p);
+  }();
+  return fn;
+}
+
+// The residual of a Bi-Real block as a tensor [pixels][O] of fp32, fetched in boxes of 32 rows x 32 channels (128 bytes,
+// 128-byte swizzle); rows beyond the tensor read as zero.
+bool tc_residual_map(CUtensorMap* map, const float* residual, long long pixels, int O) {
+  const tc_encode_fn enc = tc_encoder();
+  if (enc == nullptr) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)O, (cuuint64_t)pixels};
+  const cuuint64_t strides[1] = {(cuuint64_t)O * 4};
+  const cuuint32_t box[2] = {32, 32}, estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(residual), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int EPI, bool PAIR>
 dabnn_status tc_dispatch_mode(TcArgs& g, cudaStream_t st) {
   const size_t wr = (size_t)g.ntile / (PAIR ? 2 : 1);
@@ -962,8 +1113,32 @@ dabnn_status tc_dispatch_mode(TcArgs& g, cudaStream_t st) {
   g.abufs = 1;
   while (g.abufs < TC_MAX_BUFS && wbytes + (size_t)(g.abufs + 1) * abytes + TC_SMEM_MISC <= (size_t)TC_SMEM_LIMIT) g.abufs++;
   g.nacc = TC_ACC_COLS / g.ntile < TC_MAX_BUFS ? TC_ACC_COLS / g.ntile : TC_MAX_BUFS;
-  const size_t smem = wbytes + g.abufs * abytes + TC_SMEM_MISC;
+  size_t smem = wbytes + g.abufs * abytes + TC_SMEM_MISC;
   if (smem > (size_t)TC_SMEM_LIMIT) return DABNN_ERR_UNSUPPORTED;
+  g.res_ring = 0;
+  if (EPI == EPI_BIREAL) {
+    // The residual through a ring of bulk tensor copies, where shared memory has room for it beside every activation
+    // buffer and the launch is long enough for the prefetch distance to matter (environment DABNN_TC_RES_RING = 0 turns
+    // it off, = n asks for n chunks per warp; read once, for measurements).
+    static const int ring_env = [] { const char* e = getenv("DABNN_TC_RES_RING"); return e ? atoi(e) : -1; }();
+    const bool wide = (g.O & 31) == 0 && ((reinterpret_cast<uintptr_t>(g.residual) | reinterpret_cast<uintptr_t>(g.y_out)) & 31) == 0;
+    if (!PAIR && g.slots <= 256 && g.ntile >= 64 && wide && ring_env != 0 && g.m_tiles >= 2LL * sm_count()) {
+      const int warps = g.epi2 ? 8 : 4;
+      int ring = ring_env > 0 ? (ring_env < TC_RING_MAX ? ring_env : TC_RING_MAX) : 2;
+      for (; ring >= 2; ring--)
+        if (smem + 1024 + (size_t)warps * ring * TC_RING_CHUNK <= (size_t)TC_SMEM_LIMIT) break;
+      if (ring >= 2 && tc_residual_map(&g.res_map, g.residual, (long long)g.N * g.OH * g.OW, g.O)) {
+        g.res_ring = ring;
+        smem += 1024 + (size_t)warps * ring * TC_RING_CHUNK;
+      }
+    }
+  }
+  if constexpr (EPI == EPI_BIREAL && !PAIR) {
+    if (g.res_ring > 0) {
+      if (g.ntile == 128) return tc_launch<128, EPI, 2, false, true>(g, smem, st);
+      return tc_launch<64, EPI, 2, false, true>(g, smem, st);
+    }
+  }
   if (g.slots <= 256) {
     switch (g.ntile) {
       case 128: return tc_launch<128, EPI, 2, PAIR>(g, smem, st);

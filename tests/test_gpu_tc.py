@@ -100,6 +100,45 @@ def test_tc_conv_and_epilogues_match_oracle(B, oracle_mod, case):
     assert B.tc_error_flag() == 0
 
 
+# Launches long enough for the form of the Bi-Real epilogue that fetches the residual with bulk tensor copies (a ring of
+# 32-row x 32-channel chunks per epilogue warp): ragged slot rows, a channel tile that reaches beyond O, several images per
+# tile, and the in-place call the network makes (y written over the residual).
+RING_CASES = [
+    (16, 64, 56, 56, 64, 3, 1, -1),
+    (48, 128, 28, 28, 128, 3, 1, +1),
+    (50, 64, 30, 27, 96, 3, 1, -1),
+    (700, 128, 7, 9, 160, 1, 0, -1),
+]
+
+
+@pytest.mark.parametrize("case", RING_CASES)
+def test_tc_bireal_epilogue_with_the_residual_through_bulk_copies(B, oracle_mod, case):
+    N, C, H, W, O, k, pad, pv = case
+    x, w = inputs(case)
+    o = oracle_mod
+    acc = o.bconv_bits(o.pack(x), C, o.pack_weights(w), (1, 1), (pad, pad), pv, o.NHWC)
+    rng = np.random.default_rng(O + N)
+    gamma, beta, mean, var = synth.bn_params(rng, O)
+    gamma[::3] *= -1.0
+    scale, shift = o.bn_fold(gamma, beta, mean, var)
+    res = (rng.standard_normal(acc.shape) * 15).astype(np.float32)
+    y, want_bits = o.bn_add_sign_pack(acc, scale, shift, res)
+    a, wp = B.pack(dev(x)), B.pack_weights(dev(w))
+    wt = B.TcWeights(wp, C)
+    got_y, got_bits = B.tc_bconv2d_bn_add_sign_pack(a, wt, dev(scale), dev(shift), dev(res), (1, 1), (pad, pad), pv)
+    assert np.array_equal(got_y.cpu().numpy().view(np.uint32), y.view(np.uint32))
+    assert np.array_equal(u64(got_bits), want_bits)
+    # in place, twice in a row from the same input (the second call must not see anything of the first)
+    for _ in range(2):
+        stream = dev(res)
+        call = B.prepare_bireal_block(a, C, wp, wt, dev(scale), dev(shift), stream, (1, 1), (pad, pad), pv)
+        call()
+        torch.cuda.synchronize()
+        assert np.array_equal(stream.cpu().numpy().view(np.uint32), y.view(np.uint32))
+        assert np.array_equal(u64(call.keep[-1]), want_bits)
+    assert B.tc_error_flag() == 0
+
+
 @pytest.mark.parametrize("shape", [(300, 260, 512), (129, 65, 64), (70, 33, 150), (1000, 2048, 500)])
 def test_tc_bgemm_matches_eq1(B, oracle_mod, shape):
     M, N, K = shape
