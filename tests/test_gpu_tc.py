@@ -369,3 +369,27 @@ def test_both_launch_forms_in_a_child_process(mode):
     env = dict(os.environ, DABNN_TC_MODE=mode, PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
     r = subprocess.run([sys.executable, "-c", _FORCED_FORM_SCRIPT], env=env, cwd=root, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and "forced form ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+_RING_SCRIPT = r"""
+import sys
+sys.path.insert(0, "tests")
+import oracle as o
+o.set_threads(o.max_threads())
+from paper_1908_05858_b200 import binding as B
+import test_gpu_tc
+for case in test_gpu_tc.RING_CASES:
+    test_gpu_tc.test_tc_bireal_epilogue_with_the_residual_through_bulk_copies(B, o, case)
+print("ring ok")
+"""
+
+
+@pytest.mark.parametrize("ring", ["0", "4"])
+def test_residual_ring_depths_in_a_child_process(ring):
+    """DABNN_TC_RES_RING (read once per process): 0 = the epilogue warps load the residual themselves, 4 = the deepest ring
+    of bulk copies.  Both must give the oracle's bits on the cases of the default depth."""
+    import os, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, DABNN_TC_RES_RING=ring, PYTHONPATH=root + os.pathsep + os.environ.get("PYTHONPATH", ""))
+    r = subprocess.run([sys.executable, "-c", _RING_SCRIPT], env=env, cwd=root, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "ring ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
