@@ -228,11 +228,14 @@ dabnn_status dabnn_binary_layer_host(const float* x_host, dabnn_shape in, const 
  * The same convolutions (Section 2.1.2, Eq. 1 read as a +-1 dot product) computed on the tcgen05 tensor cores with
  * 4-bit {+1,-1} operands (e2m1, block scale 1.0, fp32 accumulation: exact) expanded on chip from the packed bits.
  * Results are identical to dabnn_bconv2d* bit for bit.
- * Covered: stride 1 or 2 (both axes alike), C at most 512 (256 for stride 2; channels beyond C in the last 64-channel word
- * are given zero weights, which is what the zero tail bits of the packed words mean in Eq. 1), images narrow enough
+ * Covered: stride 1 or 2 (both axes alike); any C whose expanded weights fit (below) -- up to 512 channels (256 at stride 2)
+ * a tile's activations are expanded at once, more pass through the activation buffers in groups of 512 (256) channels
+ * while the tile's sums stay in one accumulator (channels beyond C in the last 64-channel word
+ * are given zero weights, which is what the zero tail bits of the packed words mean in Eq. 1); images narrow enough
  * that the 128 + (kh-1)*SP + kw-1 slots a tile reads fit its activation buffer of 640 rows (SP = W + pad_w slots per
  * image row at stride 1, so W + pad_w <= 255 for a 3x3 filter; wider still at C <= 256, where a thread holds five rows),
- * filters whose expanded weights fit the resident budget (dabnn_tc_weights_bytes returns 0 otherwise); other cases
+ * filters whose expanded weights fit the resident budget: 32 output channels x kh*kw*C/2 bytes <= 144 KB, i.e. C <= 1024 for
+ * a 3x3 filter and <= 9216 for 1x1 (dabnn_tc_weights_bytes returns 0 otherwise); C*kh*kw < 2^22; other cases
  * return DABNN_ERR_UNSUPPORTED and are served by dabnn_bconv2d*.
  * A launch takes one of two forms, chosen by the library from the problem size: one CTA per tile of 128 output
  * positions, or pairs of CTAs of a thread-block cluster that share every tensor-core instruction (used where one CTA

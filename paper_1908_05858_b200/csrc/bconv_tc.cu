@@ -51,7 +51,7 @@ constexpr int TC_SMEM_MISC = TC_SMEM_HDR + 2 * TC_MAX_RES * 128 * 4;  // ... and
 constexpr int TC_RING_MAX = 4;             // residual chunks in flight per epilogue warp at most
 constexpr int TC_RING_CHUNK = 4096;        // one chunk: 32 rows x 32 fp32 channels
 constexpr int TC_WEIGHT_BUDGET = 147456;  // 144 KB of resident weights at most
-constexpr int TC_MAX_CW = 8;              // C <= 512
+constexpr int TC_MAX_CW = 8;              // words of a row that a producer thread holds: 512 channels per channel group
 constexpr int TC_MAX_SPT = 5;             // slots per producer thread: 2 for stride 1, up to 5 for stride 2
 constexpr int TC_TMEM_COLS = 512;         // the accumulators' columns + the scale-factor columns
 constexpr int TC_WAIT_POLLS = 1 << 20;    // polls of a barrier wait before it gives up (about a second)
@@ -95,6 +95,8 @@ struct TcArgs {
                        // (tensor memory, barriers, thresholds, the weight copy) and only then waits for the predecessor
   int wait_polls;      // polls of a barrier wait before it gives up (TC_WAIT_POLLS; smaller only in the expiry self-test)
   int extra_arrivals;  // 0; the expiry self-test makes `a_full` expect one arrival more than the producers make
+  int kgroups, gw;     // channel groups of `gw` 64-bit words (8, or 4 where a thread holds five rows) that a tile's channels
+                       // pass through the activation buffers in; 1 group = all channels at once (C <= 512 / 256)
   int res_ring;        // > 0: the residual reaches the epilogue warps as bulk tensor copies into a ring of this many
                        // 4 KB chunks per warp (res_map: [pixels][O] fp32, boxes of 32 rows x 32 channels, 128-byte swizzle)
   alignas(64) CUtensorMap res_map;
@@ -239,7 +241,10 @@ __device__ __forceinline__ uint32_t fast_div(uint32_t q, unsigned long long magi
   return magic == 0 ? q : (uint32_t)__umul64hi((unsigned long long)q, magic);
 }
 
-template <int NT, int EPI, int SPT, bool PAIR, bool RES_TMA = false>
+// KG: more channels than one activation buffer takes (C > 512, or > 256 at stride 2).  The weights stay resident; the
+// activations of a tile pass through the ring of activation buffers one channel group (g.gw words per row) at a time and
+// the MMAs of all groups add up in the same accumulator.  One channel tile per CTA, no CTA pairs.
+template <int NT, int EPI, int SPT, bool PAIR, bool RES_TMA = false, bool KG = false>
 __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_constant__ TcArgs g) {
   extern __shared__ __align__(1024) uint8_t smem[];
   constexpr int WR = PAIR ? NT / 2 : NT;  // weight rows (output channels) of one channel tile held by this CTA
@@ -247,7 +252,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_co
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // 0: the CTA that issues the pair's MMAs
   const int Kb = g.kh * g.kw * (g.C >> 1);               // bytes per weight row
-  const int a_bytes = g.slots * (g.C >> 1);              // bytes of one A buffer
+  const int a_bytes = KG ? g.slots * g.gw * 32 : g.slots * (g.C >> 1);  // bytes of one A buffer (one channel group)
   uint8_t* w_s = smem;                                   // [nres][taps][C/32][WR][16]
   uint8_t* a_s = smem + (size_t)g.nres * WR * Kb;        // [abufs][C/32][slots][16]
   uint8_t* misc = a_s + (size_t)g.abufs * a_bytes;
@@ -474,26 +479,29 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_co
 #pragma unroll
       for (int t = 0; t < 9; t++) off9[t] = k3 ? tap_offset(t / 3, t % 3) : 0u;
       // all MMAs of one tile and channel tile; KB = C / 64 as a compile-time constant, the 3x3 filter fully unrolled
-      auto issue_tile = [&](uint32_t d_tmem, uint32_t a_lo0, uint32_t b_base, uint32_t a_stp, bool first, auto kbc) {
+      // (KG: `more` = 1 for every channel group after a tile's first: its MMAs add to what the groups before left; the
+      // weights of a tap are g.Cw K blocks apart, of which this group's KB start at b_base)
+      auto issue_tile = [&](uint32_t d_tmem, uint32_t a_lo0, uint32_t b_base, uint32_t a_stp, bool first, uint32_t more, auto kbc) {
         constexpr int KB = decltype(kbc)::value;
+        const uint32_t tap_blocks = KG ? (uint32_t)g.Cw : (uint32_t)KB;
         if (k3) {
 #pragma unroll
           for (int t = 0; t < 9; t++) {
-            if (first && (t == 3 || t == 6) && !wait(smem_u32(&bars[B_W_FULL + t / 3]), 0)) *s_fail = 1;  // that row of taps
+            if (!KG && first && (t == 3 || t == 6) && !wait(smem_u32(&bars[B_W_FULL + t / 3]), 0)) *s_fail = 1;  // that row of taps
             const uint32_t a_lo = a_lo0 + off9[t];
 #pragma unroll
             for (int kb = 0; kb < KB; kb++)
-              mma(d_tmem, a_lo + (uint32_t)kb * a_stp, b_base + (uint32_t)(t * KB + kb) * b_step, (t | kb) ? 1u : 0u);
+              mma(d_tmem, a_lo + (uint32_t)kb * a_stp, b_base + ((uint32_t)t * tap_blocks + (uint32_t)kb) * b_step, (t | kb) ? 1u : more);
           }
         } else {
-          if (first && !(wait(smem_u32(&bars[B_W_FULL + 1]), 0) && wait(smem_u32(&bars[B_W_FULL + 2]), 0))) *s_fail = 1;
-          uint32_t b_lo = b_base, accumulate = 0;
+          if (!KG && first && !(wait(smem_u32(&bars[B_W_FULL + 1]), 0) && wait(smem_u32(&bars[B_W_FULL + 2]), 0))) *s_fail = 1;
+          uint32_t b_tap = b_base, accumulate = more;
           for (int ti = 0; ti < g.kh; ti++)
-            for (int tj = 0; tj < g.kw; tj++) {
+            for (int tj = 0; tj < g.kw; tj++, b_tap += tap_blocks * b_step) {
               const uint32_t a_lo = a_lo0 + tap_offset(ti, tj);
 #pragma unroll
-              for (int kb = 0; kb < KB; kb++, b_lo += b_step) {
-                mma(d_tmem, a_lo + (uint32_t)kb * a_stp, b_lo, accumulate);
+              for (int kb = 0; kb < KB; kb++) {
+                mma(d_tmem, a_lo + (uint32_t)kb * a_stp, b_tap + (uint32_t)kb * b_step, accumulate);
                 accumulate = 1;
               }
             }
@@ -503,7 +511,40 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_co
       uint32_t accb = 0, acc_phase = 0;  // accumulator of this round and the parity of its uses so far
       int ar = 0;                    // accumulator rounds so far: one per (tile, resident channel tile)
       bool ok = wait(smem_u32(&bars[B_W_FULL]), 0);  // first third of the resident weights, and the scale factors
+      if (KG) ok = ok && wait(smem_u32(&bars[B_W_FULL + 1]), 0) && wait(smem_u32(&bars[B_W_FULL + 2]), 0);  // ... all of them
       if (!ok) *s_fail = 1;
+      if constexpr (KG) {
+#pragma unroll 1
+        for (long long mt = mt_first; mt < mt_end && ok; mt += mt_step, ar++) {
+          if (ar >= g.nacc && !wait(smem_u32(&bars[B_TMEM_FREE + accb]), acc_phase ^ 1u)) { *s_fail = 1; break; }  // accumulator drained
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t d_tmem = tmem_base + accb * (uint32_t)NT;
+#pragma unroll 1
+          for (int grp = 0; grp < g.kgroups; grp++) {
+            if (!wait(smem_u32(&bars[B_A_FULL + ab]), a_phase)) { *s_fail = 1; ok = false; break; }  // this group's rows written
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_lo0 = a_lo_first + ab * a_buf_units;
+            const uint32_t b_base = b_lo0 + (uint32_t)(grp * g.gw) * b_step;
+            const int kbs = min(g.gw, g.Cw - grp * g.gw);  // K blocks of this group
+            const uint32_t more = grp ? 1u : 0u;
+            switch (kbs) {
+              case 1: issue_tile(d_tmem, a_lo0, b_base, a_step, false, more, IntC<1>{}); break;
+              case 2: issue_tile(d_tmem, a_lo0, b_base, a_step, false, more, IntC<2>{}); break;
+              case 3: issue_tile(d_tmem, a_lo0, b_base, a_step, false, more, IntC<3>{}); break;
+              case 4: issue_tile(d_tmem, a_lo0, b_base, a_step, false, more, IntC<4>{}); break;
+              case 5: issue_tile(d_tmem, a_lo0, b_base, a_step, false, more, IntC<5>{}); break;
+              case 6: issue_tile(d_tmem, a_lo0, b_base, a_step, false, more, IntC<6>{}); break;
+              case 7: issue_tile(d_tmem, a_lo0, b_base, a_step, false, more, IntC<7>{}); break;
+              default: issue_tile(d_tmem, a_lo0, b_base, a_step, false, more, IntC<8>{}); break;
+            }
+            commit(smem_u32(&bars[B_A_FREE + ab]));  // the group's rows have been read: the A buffer may be refilled
+            if (++ab == (uint32_t)g.abufs) { ab = 0; a_phase ^= 1u; }
+          }
+          if (!ok) break;
+          commit(smem_u32(&bars[B_MMA_DONE + accb]));
+          if (++accb == (uint32_t)g.nacc) { accb = 0; acc_phase ^= 1u; }
+        }
+      } else
 #pragma unroll 1
       for (long long mt = mt_first; mt < mt_end && ok; mt += mt_step) {
         if (!wait(smem_u32(&bars[B_A_FULL + ab]), a_phase)) { *s_fail = 1; break; }  // rows written
@@ -519,14 +560,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_co
           const uint32_t d_tmem = tmem_base + accb * (uint32_t)NT;
           const uint32_t b_base = b_lo0 + (uint32_t)r * b_tile;
           switch (g.Cw) {  // C / 64 = 1..8
-            case 1: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<1>{}); break;
-            case 2: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<2>{}); break;
-            case 3: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<3>{}); break;
-            case 4: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<4>{}); break;
-            case 5: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<5>{}); break;
-            case 6: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<6>{}); break;
-            case 7: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<7>{}); break;
-            default: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, IntC<8>{}); break;
+            case 1: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, 0u, IntC<1>{}); break;
+            case 2: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, 0u, IntC<2>{}); break;
+            case 3: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, 0u, IntC<3>{}); break;
+            case 4: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, 0u, IntC<4>{}); break;
+            case 5: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, 0u, IntC<5>{}); break;
+            case 6: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, 0u, IntC<6>{}); break;
+            case 7: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, 0u, IntC<7>{}); break;
+            default: issue_tile(d_tmem, a_lo0, b_base, a_step_t, ar == 0, 0u, IntC<8>{}); break;
           }
           commit(smem_u32(&bars[B_MMA_DONE + accb]));
           if (++accb == (uint32_t)g.nacc) { accb = 0; acc_phase ^= 1u; }
@@ -565,9 +606,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_co
       co_n[h] = (int)n;
       co_plane[h] = plane;
     }
+    int pf_grp = 0;  // (KG) channel group of the next request; the slot coordinates move on after a tile's last group
     auto prefetch = [&](SlotRegs& R, auto cwc) {
       constexpr int CW = decltype(cwc)::value;
       const int sshift = g.S - 1;  // stride 1 or 2
+      const int w0 = KG ? pf_grp * CW : 0;            // first word of the group
+      const int wn = KG ? g.Cw - w0 : g.Cw;           // words from there on (CW of them are taken at most)
+      const bool move_on = !KG || pf_grp + 1 == g.kgroups;
 #pragma unroll
       for (int h = 0; h < SPT; h++) {
 #pragma unroll
@@ -576,21 +621,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_co
           const int ih = (co_r[h] << sshift) + (co_plane[h] >> sshift) - g.ph;  // un-padded input coordinates
           const int iw = (co_c[h] << sshift) + (co_plane[h] & sshift) - g.pw;
           if (co_n[h] < g.N && ih >= 0 && ih < g.H && iw >= 0 && iw < g.W) {
-            const uint64_t* src = g.a + (((long long)co_n[h] * g.H + ih) * g.W + iw) * g.Cw;
+            const uint64_t* src = g.a + (((long long)co_n[h] * g.H + ih) * g.W + iw) * g.Cw + w0;
 #pragma unroll
             for (int cw = 0; cw < CW; cw++)
-              if (cw < g.Cw) R.words[h][cw] = ld_nc_u64(src + cw);  // (CW is g.Cw rounded up to 1, 2, 4 or 8)
+              if (cw < wn) R.words[h][cw] = ld_nc_u64(src + cw);  // (CW is g.Cw rounded up to 1, 2, 4 or 8)
           }
-          co_c[h] += dc;
-          if (co_c[h] >= g.SP) { co_c[h] -= g.SP; co_r[h]++; }
-          co_r[h] += dr;
-          if (co_r[h] >= g.HP) { co_r[h] -= g.HP; co_n[h]++; }
-          co_n[h] += dn;
+          if (move_on) {
+            co_c[h] += dc;
+            if (co_c[h] >= g.SP) { co_c[h] -= g.SP; co_r[h]++; }
+            co_r[h] += dr;
+            if (co_r[h] >= g.HP) { co_r[h] -= g.HP; co_n[h]++; }
+            co_n[h] += dn;
+          }
         }
       }
+      if (KG && ++pf_grp == g.kgroups) pf_grp = 0;
     };
+    int ex_grp = 0;  // (KG) channel group of the rows expanded next
     auto expand = [&](const SlotRegs& R, uint8_t* abuf, auto cwc) {
       constexpr int CW = decltype(cwc)::value;
+      const int wn = KG ? g.Cw - ex_grp * CW : g.Cw;  // words of this group (CW of them at most)
+      if (KG && ++ex_grp == g.kgroups) ex_grp = 0;
 #pragma unroll
       for (int h = 0; h < SPT; h++) {
         const int s = ptid + 128 * h;
@@ -599,7 +650,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_co
         const size_t gstride = (size_t)g.slots * 16;  // bytes between consecutive 32-channel groups
 #pragma unroll
         for (int cw = 0; cw < CW; cw++) {
-          if (cw >= g.Cw) break;  // warp-uniform
+          if (cw >= wn) break;  // warp-uniform
           const uint4 lo = expand32((uint32_t)R.words[h][cw]), hi = expand32((uint32_t)(R.words[h][cw] >> 32));
           *reinterpret_cast<uint4*>(dst + (size_t)(2 * cw) * gstride) = lo;
           *reinterpret_cast<uint4*>(dst + (size_t)(2 * cw + 1) * gstride) = hi;
@@ -621,11 +672,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_co
       if (TWO_SETS) prefetch(nxt, cwc);
       prologue_sync();
       uint32_t ab = 0, use_phase = 0;  // A buffer of this tile and the parity of the number of times it has been filled
+      bool stop = false;
 #pragma unroll 1
-      for (; mt < mt_end; mt += mt_step, it++) {
+      for (; mt < mt_end && !stop; mt += mt_step)
+#pragma unroll 1
+      for (int grp = 0; grp < (KG ? g.kgroups : 1); grp++, it++) {  // (KG: a tile's channel groups, one A buffer each)
         // its last reader: all MMAs of the tile that used it, signalled through `a_free` (in both CTAs of a pair)
-        // (the verdict is taken by the warp as a whole, so that its lanes stay together for the warp-wide steps below)
-        if (it >= g.abufs && !__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&bars[B_A_FREE + ab]), use_phase ^ 1u, s_fail, g.wait_polls))) { *s_fail = 1; break; }
+        // (the decision is taken by the warp as a whole, so that its lanes stay together for the warp-wide steps below)
+        if (it >= g.abufs && !__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&bars[B_A_FREE + ab]), use_phase ^ 1u, s_fail, g.wait_polls))) { *s_fail = 1; stop = true; break; }
         expand(cur, a_s + (size_t)ab * a_bytes, cwc);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
         __syncwarp();  // every lane's rows are written and fenced: one arrival stands for the warp
@@ -649,7 +703,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) bconv_tc_kernel(const __grid_co
       }
     };
     // C is a multiple of 64 up to 512: 1..8 words; the common counts get their own straight-line code
-    if (g.Cw == 1) run(IntC<1>{});
+    if constexpr (KG) run(IntC<PCW>{});  // groups of 8 words (4 where a thread holds five rows): g.gw == PCW
+    else if (g.Cw == 1) run(IntC<1>{});
     else if (g.Cw == 2) run(IntC<2>{});
     else if (g.Cw <= 4) run(IntC<4>{});
     else if constexpr (PCW > 4) run(IntC<8>{});
@@ -982,8 +1037,9 @@ int tc_mode() {
 // C rounded up to whole 64-channel words: what the operand layouts are sized for
 int tc_cpad(int C) { return (C + 63) / 64 * 64; }
 
+// (any C whose expanded weights fit: more than 512 channels pass through the activation buffers in groups)
 bool tc_covers(int O, int C, int taps) {
-  return O > 0 && C > 0 && tc_cpad(C) <= 64 * TC_MAX_CW && 32LL * (tc_cpad(C) / 2) * taps <= TC_WEIGHT_BUDGET;
+  return O > 0 && C > 0 && 32LL * (tc_cpad(C) / 2) * taps <= TC_WEIGHT_BUDGET;
 }
 
 // Channels per MMA for a launch: the widest of 128 / 64 / 32 whose rows (half of them per CTA of a pair) fit the
@@ -1001,9 +1057,9 @@ int tc_ntile(int O, int C, int taps, bool pair) {
 // Channel tiles cover O rounded up to whole 64-bit sign words (rows beyond O hold zero weights).
 int tc_n_ntiles(int O, int nt) { return ((O + 63) / 64 * 64 + nt - 1) / nt; }
 
-template <int NT, int EPI, int SPT, bool PAIR, bool RES_TMA = false>
+template <int NT, int EPI, int SPT, bool PAIR, bool RES_TMA = false, bool KG = false>
 dabnn_status tc_launch(const TcArgs& g, size_t smem, cudaStream_t st) {
-  auto kern = bconv_tc_kernel<NT, EPI, SPT, PAIR, RES_TMA>;
+  auto kern = bconv_tc_kernel<NT, EPI, SPT, PAIR, RES_TMA, KG>;
   static bool configured[kMaxDevices] = {};
   static int max_units_dev[kMaxDevices] = {};  // CTAs (pairs) that can be resident at once
   const int dev = current_device();
@@ -1109,7 +1165,8 @@ bool tc_residual_map(CUtensorMap* map, const float* residual, long long pixels, 
 template <int EPI, bool PAIR>
 dabnn_status tc_dispatch_mode(TcArgs& g, cudaStream_t st) {
   const size_t wr = (size_t)g.ntile / (PAIR ? 2 : 1);
-  const size_t wbytes = (size_t)g.nres * wr * g.kh * g.kw * (g.C / 2), abytes = (size_t)g.slots * (g.C / 2);
+  const size_t wbytes = (size_t)g.nres * wr * g.kh * g.kw * (g.C / 2);
+  const size_t abytes = g.kgroups > 1 ? (size_t)g.slots * g.gw * 32 : (size_t)g.slots * (g.C / 2);
   g.abufs = 1;
   while (g.abufs < TC_MAX_BUFS && wbytes + (size_t)(g.abufs + 1) * abytes + TC_SMEM_MISC <= (size_t)TC_SMEM_LIMIT) g.abufs++;
   g.nacc = TC_ACC_COLS / g.ntile < TC_MAX_BUFS ? TC_ACC_COLS / g.ntile : TC_MAX_BUFS;
@@ -1122,7 +1179,7 @@ dabnn_status tc_dispatch_mode(TcArgs& g, cudaStream_t st) {
     // it off, = n asks for n chunks per warp; read once, for measurements).
     static const int ring_env = [] { const char* e = getenv("DABNN_TC_RES_RING"); return e ? atoi(e) : -1; }();
     const bool wide = (g.O & 31) == 0 && ((reinterpret_cast<uintptr_t>(g.residual) | reinterpret_cast<uintptr_t>(g.y_out)) & 31) == 0;
-    if (!PAIR && g.slots <= 256 && g.ntile >= 64 && wide && ring_env != 0 && g.m_tiles >= 2LL * sm_count()) {
+    if (!PAIR && g.kgroups == 1 && g.slots <= 256 && g.ntile >= 64 && wide && ring_env != 0 && g.m_tiles >= 2LL * sm_count()) {
       const int warps = g.epi2 ? 8 : 4;
       int ring = ring_env > 0 ? (ring_env < TC_RING_MAX ? ring_env : TC_RING_MAX) : 2;
       for (; ring >= 2; ring--)
@@ -1138,6 +1195,24 @@ dabnn_status tc_dispatch_mode(TcArgs& g, cudaStream_t st) {
       if (g.ntile == 128) return tc_launch<128, EPI, 2, false, true>(g, smem, st);
       return tc_launch<64, EPI, 2, false, true>(g, smem, st);
     }
+  }
+  if constexpr (!PAIR) {
+    if (g.kgroups > 1) {
+      if (g.slots <= 256) {
+        switch (g.ntile) {
+          case 128: return tc_launch<128, EPI, 2, false, false, true>(g, smem, st);
+          case 64: return tc_launch<64, EPI, 2, false, false, true>(g, smem, st);
+          default: return tc_launch<32, EPI, 2, false, false, true>(g, smem, st);
+        }
+      }
+      switch (g.ntile) {
+        case 128: return tc_launch<128, EPI, TC_MAX_SPT, false, false, true>(g, smem, st);
+        case 64: return tc_launch<64, EPI, TC_MAX_SPT, false, false, true>(g, smem, st);
+        default: return tc_launch<32, EPI, TC_MAX_SPT, false, false, true>(g, smem, st);
+      }
+    }
+  } else if (g.kgroups > 1) {
+    return DABNN_ERR_UNSUPPORTED;  // (not reached: tc_plan never pairs CTAs for grouped channels)
   }
   if (g.slots <= 256) {
     switch (g.ntile) {
@@ -1176,7 +1251,7 @@ void tc_plan(TcArgs& g, int O, int C, int taps) {
   const int mode = tc_mode();
   const int units1 = sm_count(), units2 = sm_count() / 2;
   const int nt2 = tc_ntile(O, C, taps, true);
-  bool pair = nt2 != 0 && mode != 1;
+  bool pair = nt2 != 0 && mode != 1 && g.kgroups == 1;
   if (pair && mode == 0) {
     // Measured: pairs win where one CTA cannot keep a 128-channel tile resident (C = 512 at 3x3) and there are
     // enough double tiles to go round; elsewhere the one-CTA form is as fast or faster.
@@ -1193,6 +1268,7 @@ void tc_plan(TcArgs& g, int O, int C, int taps) {
   if (nres > g.n_ntiles) nres = g.n_ntiles;
   const long long m_units = pair ? (g.m_tiles + 1) / 2 : g.m_tiles;
   while (nres > 1 && (g.n_ntiles + nres - 1) / nres * m_units < (pair ? units2 : units1)) nres--;
+  if (g.kgroups > 1) nres = 1;  // (the groups of a tile add up in one accumulator)
   g.nres = (int)nres;
   g.n_groups = (g.n_ntiles + g.nres - 1) / g.nres;
 }
@@ -1227,9 +1303,11 @@ dabnn_status tc_fill(TcArgs& g, const uint64_t* a, dabnn_shape in, const void* w
   g.slots_p = (128 + ((cv.kh - 1) / g.S) * g.SP + (cv.kw - 1) / g.S + 7) / 8 * 8;
   g.slots = g.S * g.S * g.slots_p;
   if ((long long)in.C * cv.kh * cv.kw >= (1LL << 22)) return DABNN_ERR_UNSUPPORTED;  // exact fp32 sums and acc_to_int
-  if (g.slots > 128 * TC_MAX_SPT || g.Cw > TC_MAX_CW || g.total_q + 512 >= (1LL << 31))
-    return DABNN_ERR_UNSUPPORTED;
+  if (g.slots > 128 * TC_MAX_SPT || g.total_q + 512 >= (1LL << 31)) return DABNN_ERR_UNSUPPORTED;
   g.m_tiles = (g.total_q + 127) / 128;
+  // words per row that a producer thread holds: 8 (4 where it holds five rows, stride 2); more channels go in groups
+  g.gw = g.slots <= 256 ? TC_MAX_CW : 4;
+  g.kgroups = (g.Cw + g.gw - 1) / g.gw;
   tc_plan(g, O, in.C, cv.kh * cv.kw);
   if (g.ntile == 0) return DABNN_ERR_UNSUPPORTED;
   if ((long long)in.N * OH * OW >= (1LL << 31) || (long long)in.N * OH * OW * O > (1LL << 40)) return DABNN_ERR_UNSUPPORTED;

@@ -55,6 +55,14 @@ TC_CASES = [
     (40, 256, 14, 14, 256, 3, 1, -1),   # enough tiles for CTA pairs with two resident channel tiles
     (33, 512, 7, 7, 512, 3, 1, +1),     # pairs, odd number of tiles, four channel-tile groups
     (70, 128, 28, 28, 128, 3, 1, -1, 2),  # pairs, stride 2
+    # more channels than one activation buffer takes: a tile's channels pass through the buffers in groups
+    (3, 576, 9, 9, 70, 3, 1, -1),         # nine words: a group of eight and a group of one
+    (2, 1000, 8, 7, 40, 3, 1, +1),        # sixteen words with a channel tail, weights of 32 channels per CTA
+    (5, 2048, 6, 6, 200, 1, 0, -1),       # 1x1 over 2048 channels: four groups
+    (3, 1500, 5, 5, 96, 1, 0, -1),        # 24 words: three groups, the last with a tail
+    (2, 320, 20, 20, 64, 3, 1, -1, 2),    # stride 2 with five words: groups of four
+    (4, 512, 14, 14, 128, 3, 1, -1, 2),   # stride 2, C = 512: two groups of four
+    (2, 640, 12, 12, 64, 1, 0, +1, 2),    # 1x1 stride 2, ten words
 ]
 
 
@@ -139,7 +147,7 @@ def test_tc_bireal_epilogue_with_the_residual_through_bulk_copies(B, oracle_mod,
     assert B.tc_error_flag() == 0
 
 
-@pytest.mark.parametrize("shape", [(300, 260, 512), (129, 65, 64), (70, 33, 150), (1000, 2048, 500)])
+@pytest.mark.parametrize("shape", [(300, 260, 512), (129, 65, 64), (70, 33, 150), (1000, 2048, 500), (700, 300, 4096), (260, 100, 9000)])
 def test_tc_bgemm_matches_eq1(B, oracle_mod, shape):
     M, N, K = shape
     rng = np.random.default_rng(M + N + K)
@@ -155,7 +163,8 @@ def test_tc_bgemm_matches_eq1(B, oracle_mod, shape):
 
 def test_tc_declines_what_it_does_not_cover(B):
     assert not B.tc_supported(64, 64, 3, 3, stride=(3, 3))
-    assert not B.tc_supported(64, 576, 3, 3)         # more than 512 channels
+    assert B.tc_supported(64, 576, 3, 3)             # more than 512 channels: in groups
+    assert not B.tc_supported(64, 1100, 3, 3)        # ... while the weights of 32 output channels still fit the resident budget
     assert not B.tc_supported(64, 2048, 7, 7)        # expanded weights larger than the resident budget
     a = torch.zeros((1, 8, 8, 1), dtype=torch.int64, device="cuda")
     wt = B.TcWeights(torch.zeros((64, 3, 3, 1), dtype=torch.int64, device="cuda"), 64)
