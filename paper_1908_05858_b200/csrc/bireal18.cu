@@ -713,7 +713,7 @@ __global__ void __launch_bounds__(64) fc_mid(const float* __restrict__ g /*[N][5
 __global__ void __launch_bounds__(64) fc_batched(const float* __restrict__ g /*[N][512]*/, int N, const float* __restrict__ fw,
                                                  const float* __restrict__ fb, float* __restrict__ logits) {
   __shared__ __align__(16) float gs[8][512];
-  __shared__ float ws[64][33];
+  __shared__ __align__(16) float ws[64][36];  // (pitch 36: 128-bit rows in and 128-bit columns out, both free of bank conflicts)
   const int tid = threadIdx.x;
   const int n0 = blockIdx.y * 8, nimg = min(8, N - n0);
   for (int t = tid; t < 8 * 128; t += 64) {
@@ -735,7 +735,7 @@ __global__ void __launch_bounds__(64) fc_batched(const float* __restrict__ g /*[
 #pragma unroll
     for (int u = 0; u < 8; u++) {
       const int idx = tid + 64 * u, row = idx >> 3, q = idx & 7;
-      ws[row][4 * q] = wreg[u].x; ws[row][4 * q + 1] = wreg[u].y; ws[row][4 * q + 2] = wreg[u].z; ws[row][4 * q + 3] = wreg[u].w;
+      *reinterpret_cast<float4*>(&ws[row][4 * q]) = wreg[u];
     }
   };
   float a[8];
@@ -747,11 +747,17 @@ __global__ void __launch_bounds__(64) fc_batched(const float* __restrict__ g /*[
     w_store();
     __syncthreads();
     if (k0 + 32 < 512) w_load(k0 + 32);
-#pragma unroll 8
-    for (int kk = 0; kk < 32; kk++) {
-      const float wv = ws[tid][kk];
+#pragma unroll 2
+    for (int kk = 0; kk < 32; kk += 4) {  // four inputs per 128-bit load; each chain still takes them in ascending order
+      const float4 wv = *reinterpret_cast<const float4*>(&ws[tid][kk]);
 #pragma unroll
-      for (int im = 0; im < 8; im++) a[im] = __fmaf_rn(gs[im][k0 + kk], wv, a[im]);
+      for (int im = 0; im < 8; im++) {
+        const float4 gv = *reinterpret_cast<const float4*>(&gs[im][k0 + kk]);
+        a[im] = __fmaf_rn(gv.x, wv.x, a[im]);
+        a[im] = __fmaf_rn(gv.y, wv.y, a[im]);
+        a[im] = __fmaf_rn(gv.z, wv.z, a[im]);
+        a[im] = __fmaf_rn(gv.w, wv.w, a[im]);
+      }
     }
   }
   if (j >= 1000) return;
