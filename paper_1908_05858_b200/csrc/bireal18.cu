@@ -432,16 +432,17 @@ __global__ void __launch_bounds__(256, BM == 128 ? 2 : 3) shortcut_down(const fl
       w_load((ch + 1) * SC_BK);
     }
     const int cn = min(SC_BK, C - ch * SC_BK);
-#pragma unroll 4
-    for (int cc = 0; cc < cn; cc++) {
+    const float* pb = &p_s[st][0][ty * TYP];
+    const float* wbse = &w_s[st][0][tx * 4];
+    auto mac = [&](int cc) {  // one input channel of the chunk for the thread's whole register tile
       float pv[TYP];
 #pragma unroll
       for (int i = 0; i < TYP; i += 4) {
-        const float4 pa = *reinterpret_cast<const float4*>(&p_s[st][cc][ty * TYP + i]);
+        const float4 pa = *reinterpret_cast<const float4*>(pb + cc * (BM + 4) + i);
         pv[i] = pa.x; pv[i + 1] = pa.y; pv[i + 2] = pa.z; pv[i + 3] = pa.w;
       }
-      const float4 wa = *reinterpret_cast<const float4*>(&w_s[st][cc][tx * 4]);
-      const float4 wb = *reinterpret_cast<const float4*>(&w_s[st][cc][64 + tx * 4]);
+      const float4 wa = *reinterpret_cast<const float4*>(wbse + cc * (SC_BN + 4));
+      const float4 wb = *reinterpret_cast<const float4*>(wbse + cc * (SC_BN + 4) + 64);
       const unsigned long long w2[4] = {pack_f32x2(wa.x, wa.y), pack_f32x2(wa.z, wa.w), pack_f32x2(wb.x, wb.y),
                                         pack_f32x2(wb.z, wb.w)};
 #pragma unroll
@@ -450,6 +451,12 @@ __global__ void __launch_bounds__(256, BM == 128 ? 2 : 3) shortcut_down(const fl
 #pragma unroll
         for (int j = 0; j < 4; j++) fma_f32x2(acc2[i][j], p2, w2[j]);
       }
+    };
+    if (cn == SC_BK) {  // a whole chunk: straight-line code, every address an immediate offset
+#pragma unroll
+      for (int cc = 0; cc < SC_BK; cc++) mac(cc);
+    } else {
+      for (int cc = 0; cc < cn; cc++) mac(cc);
     }
     if (ch + 1 < nchunks) {
       pool_store(st ^ 1);
