@@ -294,7 +294,9 @@ int dabnn_tc_set_max_ctas(int max_ctas);
 int dabnn_set_conv_variant(int variant);
 /* Forces the convolution's CTA tile for measurement runs: 0 = automatic (default), 1 = 128 pixels x 128 channels,
  * 2 = 128 x 64, 3 = 64 x 64, 4 = 32 x 32, 5 = 16 x 32 with all of K in flight (the choice for launches of less than
- * one wave).  All give identical results.  Returns the previous setting. */
+ * one wave).  All give identical results.  Returns the previous setting.
+ * (Environment, read once, for measurements: DABNN_CONV_POINTWISE=0 keeps long unpadded 1x1 stride-1 layers on the
+ * one-tile-per-CTA kernel instead of the form that walks four pixel tiles with the weight rows resident.) */
 int dabnn_set_conv_tile(int tile);
 
 #ifdef __cplusplus
